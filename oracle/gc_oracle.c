@@ -1,0 +1,234 @@
+/*
+ * CPU oracle for the Gradient Cache "Step 2" computation (arXiv 2101.06983, Section 3.3):
+ * the in-batch-negative contrastive loss over all B query and N passage representations and
+ * its exact gradients with respect to every representation.
+ *
+ * THIS IS TEST INFRASTRUCTURE, not the product.  It is deliberately plain and slow: double
+ * precision, the whole B x N logit matrix S stored explicitly, an explicit softmax, ordinary
+ * loops, no blocking, no BLAS.  It shares no code with the CUDA library and is only executed
+ * by the tests, the smoke check and the benchmark's CPU-baseline leg.
+ *
+ * Parity pins (see tests/test_oracle_pins.py): central finite differences of the loss, row
+ * sums of softmax-minus-onehot, closed forms for identical representations and for the 1x2
+ * logistic case, scale and permutation symmetries, and the paper's exactness claim on a linear
+ * encoder.  No function here is "parity unpinned".
+ *
+ * Notation (paper, Section 3.1-3.2): Q row i is f(s_i), P row j is g(t_j), pos_idx[i] is r_i,
+ * tau the temperature, S_ij = <f(s_i), g(t_j)> / tau.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define GCO_MASK_NONE 0
+#define GCO_MASK_SELF 1
+
+/* Mask reading (not in the paper, which has no mask): with GCO_MASK_SELF the pair (i, i) is
+ * removed from the denominator of Eq. 1 altogether, so p_ii = 0 exactly. */
+static int allowed(int mask_mode, int64_t i, int64_t j) {
+    return !(mask_mode == GCO_MASK_SELF && i == j);
+}
+
+int gco_num_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+static int check_args(const int32_t* pos_idx, int64_t B, int64_t N, int64_t d, double tau,
+                      int mask_mode) {
+    if (B <= 0 || N <= 0 || d <= 0) return 1;
+    if (!(tau > 0.0) || !isfinite(tau)) return 2;
+    if (mask_mode != GCO_MASK_NONE && mask_mode != GCO_MASK_SELF) return 3;
+    for (int64_t i = 0; i < B; ++i) {
+        if (pos_idx[i] < 0 || pos_idx[i] >= N) return 4;
+        if (!allowed(mask_mode, i, pos_idx[i])) return 5;
+    }
+    return 0;
+}
+
+/* Logits of one query row: S_ij = (sum_k Q_ik P_jk) / tau  (exponent of Eq. 1). */
+static void logits_row(const double* Q, const double* P, int64_t i, int64_t N, int64_t d,
+                       double tau, double* S_row) {
+    const double* q = Q + i * d;
+    for (int64_t j = 0; j < N; ++j) {
+        const double* p = P + j * d;
+        double acc = 0.0;
+        for (int64_t k = 0; k < d; ++k) acc += q[k] * p[k];
+        S_row[j] = acc / tau;
+    }
+}
+
+/* Natural-log logsumexp of one row over the allowed columns (denominator of Eq. 1 / Eq. 4). */
+static double lse_row(const double* S_row, int64_t i, int64_t N, int mask_mode) {
+    double m = -INFINITY;
+    for (int64_t j = 0; j < N; ++j)
+        if (allowed(mask_mode, i, j) && S_row[j] > m) m = S_row[j];
+    double sum = 0.0;
+    for (int64_t j = 0; j < N; ++j)
+        if (allowed(mask_mode, i, j)) sum += exp(S_row[j] - m);
+    return m + log(sum);
+}
+
+/*
+ * Full computation with S and G stored explicitly.
+ *   loss      : Eq. 1, mean over the B queries of (lse_i - S_{i, r_i})
+ *   row_lse   : [B]  lse_i
+ *   pos_logit : [B]  S_{i, r_i}
+ *   dQ        : [B x d]  Eq. 5 (generalised to any tau: the exact derivative of Eq. 1)
+ *   dP        : [N x d]  Eq. 6-7, with eps_j read as the SUM of f(s_k) over all k with r_k = j
+ * Any output pointer may be NULL except that gradients need nothing else.
+ * Returns 0 on success, a positive code for bad arguments, -1 when out of memory.
+ */
+int gco_build_cache(const double* Q, const double* P, const int32_t* pos_idx, int64_t B,
+                    int64_t N, int64_t d, double tau, int mask_mode, double* loss,
+                    double* row_lse, double* pos_logit, double* dQ, double* dP) {
+    int rc = check_args(pos_idx, B, N, d, tau, mask_mode);
+    if (rc) return rc;
+    double* S = (double*)malloc(sizeof(double) * (size_t)B * (size_t)N);
+    double* lse = (double*)malloc(sizeof(double) * (size_t)B);
+    if (!S || !lse) { free(S); free(lse); return -1; }
+
+    /* S = Q P^T / tau */
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < B; ++i) logits_row(Q, P, i, N, d, tau, S + i * N);
+
+    /* lse_i, and the loss of Eq. 1 */
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < B; ++i) lse[i] = lse_row(S + i * N, i, N, mask_mode);
+    double total = 0.0;
+    for (int64_t i = 0; i < B; ++i) total += lse[i] - S[i * N + pos_idx[i]];
+    if (loss) *loss = total / (double)B;
+    if (row_lse) memcpy(row_lse, lse, sizeof(double) * (size_t)B);
+    if (pos_logit)
+        for (int64_t i = 0; i < B; ++i) pos_logit[i] = S[i * N + pos_idx[i]];
+
+    if (dQ || dP) {
+        /* G_ij = (p_ij - [j == r_i]) / B, with p_ij of Eq. 4 (0 where masked); in place of S */
+#pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < B; ++i) {
+            double* row = S + i * N;
+            for (int64_t j = 0; j < N; ++j) {
+                double p = allowed(mask_mode, i, j) ? exp(row[j] - lse[i]) : 0.0;
+                double onehot = (j == pos_idx[i]) ? 1.0 : 0.0;
+                row[j] = (p - onehot) / (double)B;
+            }
+        }
+        const double* G = S;
+        if (dQ) {
+            /* Eq. 5: dL/df(s_i) = (1/tau) sum_j G_ij g(t_j) */
+#pragma omp parallel for schedule(static)
+            for (int64_t i = 0; i < B; ++i) {
+                double* out = dQ + i * d;
+                for (int64_t k = 0; k < d; ++k) out[k] = 0.0;
+                for (int64_t j = 0; j < N; ++j) {
+                    double g = G[i * N + j];
+                    const double* p = P + j * d;
+                    for (int64_t k = 0; k < d; ++k) out[k] += g * p[k];
+                }
+                for (int64_t k = 0; k < d; ++k) out[k] /= tau;
+            }
+        }
+        if (dP) {
+            /* Eq. 6-7: dL/dg(t_j) = (1/tau) sum_i G_ij f(s_i) */
+#pragma omp parallel for schedule(static)
+            for (int64_t j = 0; j < N; ++j) {
+                double* out = dP + j * d;
+                for (int64_t k = 0; k < d; ++k) out[k] = 0.0;
+                for (int64_t i = 0; i < B; ++i) {
+                    double g = G[i * N + j];
+                    const double* q = Q + i * d;
+                    for (int64_t k = 0; k < d; ++k) out[k] += g * q[k];
+                }
+                for (int64_t k = 0; k < d; ++k) out[k] /= tau;
+            }
+        }
+    }
+    free(S);
+    free(lse);
+    return 0;
+}
+
+/*
+ * Row-sampled variant for sizes where B x N doubles do not fit: for each listed query row i
+ * (n_rows of them) compute lse_i, S_{i,r_i} and (optionally) row i of dQ.  Each row needs only
+ * its own row of S, held in a per-thread buffer; the arithmetic is the same as above.
+ * dQ_rows is [n_rows x d].
+ */
+int gco_query_rows(const double* Q, const double* P, const int32_t* pos_idx, int64_t B, int64_t N,
+                   int64_t d, double tau, int mask_mode, const int64_t* rows, int64_t n_rows,
+                   double* row_lse, double* pos_logit, double* dQ_rows) {
+    int rc = check_args(pos_idx, B, N, d, tau, mask_mode);
+    if (rc) return rc;
+    for (int64_t r = 0; r < n_rows; ++r)
+        if (rows[r] < 0 || rows[r] >= B) return 6;
+    int failed = 0;
+#pragma omp parallel
+    {
+        double* S_row = (double*)malloc(sizeof(double) * (size_t)N);
+        if (!S_row) {
+#pragma omp atomic write
+            failed = 1;
+        }
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t r = 0; r < n_rows; ++r) {
+            if (!S_row) continue;
+            int64_t i = rows[r];
+            logits_row(Q, P, i, N, d, tau, S_row);
+            double lse = lse_row(S_row, i, N, mask_mode);
+            if (row_lse) row_lse[r] = lse;
+            if (pos_logit) pos_logit[r] = S_row[pos_idx[i]];
+            if (dQ_rows) {
+                double* out = dQ_rows + r * d;
+                for (int64_t k = 0; k < d; ++k) out[k] = 0.0;
+                for (int64_t j = 0; j < N; ++j) {
+                    double p = allowed(mask_mode, i, j) ? exp(S_row[j] - lse) : 0.0;
+                    double g = (p - ((j == pos_idx[i]) ? 1.0 : 0.0)) / (double)B;
+                    const double* pj = P + j * d;
+                    for (int64_t k = 0; k < d; ++k) out[k] += g * pj[k];
+                }
+                for (int64_t k = 0; k < d; ++k) out[k] /= tau;
+            }
+        }
+        free(S_row);
+    }
+    return failed ? -1 : 0;
+}
+
+/*
+ * Row-sampled dP: for each listed passage row j compute row j of dP (Eq. 6-7) given lse_i for
+ * ALL queries (row_lse, length B, from gco_build_cache or gco_query_rows over every row).
+ * dP_rows is [n_rows x d].
+ */
+int gco_passage_rows(const double* Q, const double* P, const int32_t* pos_idx, int64_t B,
+                     int64_t N, int64_t d, double tau, int mask_mode, const double* row_lse,
+                     const int64_t* rows, int64_t n_rows, double* dP_rows) {
+    int rc = check_args(pos_idx, B, N, d, tau, mask_mode);
+    if (rc) return rc;
+    for (int64_t r = 0; r < n_rows; ++r)
+        if (rows[r] < 0 || rows[r] >= N) return 6;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t r = 0; r < n_rows; ++r) {
+        int64_t j = rows[r];
+        const double* pj = P + j * d;
+        double* out = dP_rows + r * d;
+        for (int64_t k = 0; k < d; ++k) out[k] = 0.0;
+        for (int64_t i = 0; i < B; ++i) {
+            const double* q = Q + i * d;
+            double s = 0.0;
+            for (int64_t k = 0; k < d; ++k) s += q[k] * pj[k];
+            s /= tau;
+            double p = allowed(mask_mode, i, j) ? exp(s - row_lse[i]) : 0.0;
+            double g = (p - ((j == pos_idx[i]) ? 1.0 : 0.0)) / (double)B;
+            for (int64_t k = 0; k < d; ++k) out[k] += g * q[k];
+        }
+        for (int64_t k = 0; k < d; ++k) out[k] /= tau;
+    }
+    return 0;
+}
