@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of gc_build_cache (Step 2 of Gradient Cache: loss + representation gradients).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config I]
+
+One "step" is one gc_build_cache call over one synthetic batch.  The default workload is the
+headline configuration B = 4096, N = 8192, d = 768, bf16 inputs.  The metric is useful TFLOP/s
+counting 3 GEMMs of 2 B N d each.  With N > 1 (torchrun) every rank runs an independent replica
+of the same batch shape; there is no collective on the data path.
+
+Prints ONE JSON line on rank 0.  `--impl reference` times the CPU oracle instead (a deliberately
+plain program; see oracle/).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "gc_build_cache TFLOP/s (3 GEMMs of 2*B*N*d) at B=4096,N=8192,d=768"
+UNIT = "TFLOP/s"
+NOMINAL_BF16_TFLOPS = 2250.0      # public dense bf16 figure for B200, context only
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            pk = json.load(fh)
+        return dict(hbm=float(pk["hbm_gbs"]), tf_burst=float(pk["bf16_tflops"]),
+                    tf_sustained=float(pk.get("bf16_tflops_sustained", pk["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm=6650.0, tf_burst=1590.0, tf_sustained=1400.0, source="fallback")
+
+
+def useful_flop(B, N, d):
+    return 3.0 * 2.0 * B * N * d
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs
+    (read-only queries)."""
+
+    def __init__(self, index: int, period: float = 0.05):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self.stop_flag = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:          # NVML missing: report nulls
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+            nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+            nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+            nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap",
+            nv.nvmlClocksThrottleReasonHwPowerBrakeSlowdown: "hw_power_brake",
+        }
+        while not self.stop_flag.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def result(self):
+        self.stop_flag.set()
+        if self.is_alive():
+            self.join(timeout=2.0)
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": []}
+        s = sorted(self.samples)
+        return {"sm_mhz": s[len(s) // 2], "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(s)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except (ValueError, IndexError):
+            return local_rank
+    return local_rank
+
+
+def make_problem(index: int, rank: int):
+    from paper_2101_06983_b200 import inputs
+    if rank == 0:
+        return inputs.config(index)
+    # other replicas: same recipe, different seed
+    base = inputs.config  # noqa: F841
+    if index == 3:
+        return inputs.simclr_batch(4096, 128, "bf16", seed=inputs.BASE_SEED + 3 + 100 * rank)
+    B = {0: 64, 1: 128, 2: 4096, 4: 65536}[index]
+    return inputs.dpr_batch(B, 768, "f32" if index == 0 else "bf16",
+                            seed=inputs.BASE_SEED + index + 100 * rank)
+
+
+def run_reference(args, rank, world):
+    """CPU oracle timed as it stands on a bounded sample of the workload."""
+    if rank != 0:
+        return
+    import oracle
+    from paper_2101_06983_b200 import inputs
+    prob = inputs.config(args.config)
+    rows = max(1, min(prob.B, args.ref_rows, int(2.6e10 / (prob.N * prob.d))))
+    Q, pos = prob.Q[:rows], prob.pos_idx[:rows]
+    flop = useful_flop(rows, prob.N, prob.d)
+    for _ in range(args.warmup):
+        oracle.build_cache(Q, prob.P, pos, prob.tau, prob.mask_mode)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.build_cache(Q, prob.P, pos, prob.tau, prob.mask_mode)
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    value = flop / dt / 1e12
+    sample = (f"first {rows} of {prob.B} query rows against all {prob.N} passages "
+              f"(loss, dQ rows, dP contributions), double precision, per step")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": prob.name, "B": prob.B, "N": prob.N, "d": prob.d,
+                   "sample_rows": rows},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, rank, local_rank, world):
+    import torch
+    import torch.distributed as dist
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2101_06983_b200 import binding
+
+    prob = make_problem(args.config, rank)
+    B, N, d = prob.B, prob.N, prob.d
+    code = binding.GC_BF16 if prob.dtype == "bf16" else binding.GC_F32
+    Q, P, pos = binding.problem_tensors(prob, dev)
+    out = binding.Outputs(B, N, d, code, dev)
+    flop = useful_flop(B, N, d)
+    plan = binding.gc_plan_name(binding.GC_OP_BUILD, B, N, d, code)
+    launches = binding.gc_kernel_launches(binding.GC_OP_BUILD, B, N, d, code)
+
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # larger than the 126 MB L2
+
+    def step():
+        binding.gc_build_cache(Q, P, pos, prob.tau, prob.mask_mode, out.loss, out.row_lse,
+                               out.dQ, out.dP, out.pos_logit, out.ws, out.dev_status)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing: every step starts with a cold L2 ---------------------------
+    for _ in range(max(args.warmup, 3)):
+        flush.fill_(1)
+        step()
+    barrier()
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler.start()
+    binding.gc_profile_enable(True)
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+          for _ in range(args.steps)]
+    kern = [0.0, 0.0, 0.0]
+    for a, b in ev:
+        flush.fill_(1)
+        a.record()
+        step()
+        b.record()
+        ms = binding.gc_profile_read()          # waits for this step's kernels
+        for k in range(3):
+            kern[k] += ms[k]
+    barrier()
+    binding.gc_profile_enable(False)
+    total_ms = sum(a.elapsed_time(b) for a, b in ev)
+    clocks = sampler.result()
+
+    # ---- back-to-back timing (inputs and outputs stay in L2, as right after an encoder) -------
+    barrier()
+    a = torch.cuda.Event(enable_timing=True)
+    b = torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        step()
+    b.record()
+    barrier()
+    warm_ms = a.elapsed_time(b) / args.steps
+
+    # ---- end to end through the C ABI with host buffers ------------------------------------------
+    hQ = Q.cpu().pin_memory()
+    hP = hQ if prob.shared else P.cpu().pin_memory()
+    hpos = pos.cpu().pin_memory()
+    hdQ = torch.empty(out.dQ.shape, dtype=torch.float32).pin_memory()
+    hdP = torch.empty(out.dP.shape, dtype=torch.float32).pin_memory()
+    hloss = torch.empty(1, dtype=torch.float32).pin_memory()
+    dQin = torch.empty_like(Q)
+    dPin = dQin if prob.shared else torch.empty_like(P)
+    dpos = torch.empty_like(pos)
+
+    def e2e_step():
+        dQin.copy_(hQ, non_blocking=True)
+        if not prob.shared:
+            dPin.copy_(hP, non_blocking=True)
+        dpos.copy_(hpos, non_blocking=True)
+        binding.gc_build_cache(dQin, dPin, dpos, prob.tau, prob.mask_mode, out.loss, out.row_lse,
+                               out.dQ, out.dP, out.pos_logit, out.ws, out.dev_status)
+        hdQ.copy_(out.dQ, non_blocking=True)
+        hdP.copy_(out.dP, non_blocking=True)
+        hloss.copy_(out.loss, non_blocking=True)
+
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(2):
+        e2e_step()
+    barrier()
+    a.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    b.record()
+    barrier()
+    e2e_ms = a.elapsed_time(b) / e2e_steps
+    h2d = hQ.numel() * hQ.element_size() + (0 if prob.shared else hP.numel() * hP.element_size()) \
+        + hpos.numel() * 4
+    d2h = (hdQ.numel() + hdP.numel() + 1) * 4
+    status = int(out.dev_status.item())
+
+    # ---- max over ranks ------------------------------------------------------------------------------
+    vals = torch.tensor([total_ms, warm_ms, e2e_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
+    total_ms, warm_ms, e2e_ms = (float(x) for x in vals.tolist())
+    ms_per_step = total_ms / args.steps
+
+    if rank == 0:
+        pk = load_peaks()
+        # dominant kernel: the gradient sweep (two launches per step: dQ and dP), each of which
+        # delivers one useful GEMM of 2 B N d
+        sweep_ms = (kern[1] + kern[2]) / (2 * args.steps)
+        achieved = (2.0 * B * N * d) / (sweep_ms * 1e-3) / 1e12 if sweep_ms > 0 else 0.0
+        value = world * flop / (ms_per_step * 1e-3) / 1e12
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16" if prob.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": prob.name, "B": B, "N": N, "d": d, "tau": prob.tau,
+                       "mask": "self" if prob.mask_mode else "none", "plan": plan,
+                       "l2": "flushed before every timed step (256 MiB write)",
+                       "parallelism": f"{world} independent replica(s)"},
+            "rows_per_s": world * (B + N) / (ms_per_step * 1e-3),
+            "pct_of_bf16_peak": {"burst_measured": 100 * value / world / pk["tf_burst"],
+                                 "sustained_measured": 100 * value / world / pk["tf_sustained"],
+                                 "nominal_dense": 100 * value / world / NOMINAL_BF16_TFLOPS,
+                                 "peaks": pk["source"]},
+            "warm_l2": {"ms_per_step": warm_ms,
+                        "value": world * flop / (warm_ms * 1e-3) / 1e12, "unit": UNIT},
+            "kernel_ms": {"fwd_sweep": kern[0] / args.steps, "dq_sweep": kern[1] / args.steps,
+                          "dp_sweep": kern[2] / args.steps},
+            "roofline": {"bound": "tensor", "kernel": f"{plan} gradient sweep (dQ and dP launches)",
+                         "achieved": achieved, "peak": pk["tf_burst"], "unit": "TFLOP/s",
+                         "frac": achieved / pk["tf_burst"], "peak_source": pk["source"],
+                         "traffic": None},
+            "e2e": {"value": world * flop / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+                    "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+            "gpu_launches": launches * args.steps,
+            "clocks": clocks, "dev_status": status, "loss": float(out.loss.item()),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            rows = max(1, min(B, args.ref_rows, int(2.6e10 / (N * d))))   # about 10-30 s
+            t0 = time.perf_counter()
+            ref = oracle.build_cache(prob.Q[:rows], prob.P, prob.pos_idx[:rows], prob.tau,
+                                     prob.mask_mode)
+            dt = time.perf_counter() - t0
+            line["cpu_baseline"] = {
+                "value": useful_flop(rows, N, d) / dt / 1e12, "unit": UNIT,
+                "cores": oracle.num_threads(), "kind": "oracle", "seconds": dt,
+                "sample": f"first {rows} of {B} query rows against all {N} passages, one pass, "
+                          f"double precision"}
+            if rows == B:
+                line["loss_rel_err_vs_oracle"] = abs(line["loss"] - ref["loss"]) / abs(ref["loss"])
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", type=int, default=2, help="workload index 0..4 (2 = headline)")
+    ap.add_argument("--ref-rows", type=int, default=None,
+                    help="query rows in the CPU sample (default: whole batch for ours' "
+                         "cpu_baseline, 512 for --impl reference)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        if args.ref_rows is None:
+            args.ref_rows = 512
+        run_reference(args, rank, world)
+        return
+    if args.ref_rows is None:
+        args.ref_rows = 4096
+    run_ours(args, rank, local_rank, world)
+
+
+if __name__ == "__main__":
+    main()

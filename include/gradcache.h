@@ -1,0 +1,123 @@
+/*
+ * gradcache.h - C ABI of the B200 (sm_100a) library that fills the Representation Gradient
+ * Cache of Gradient Cache (arXiv 2101.06983, Section 3.3, "Step 2").
+ *
+ * Given the numerical representations Q (B x d, row i = f(s_i)) and P (N x d, row j = g(t_j))
+ * and the relevance map pos_idx (r_i, Section 3.1), the library computes
+ *
+ *   S_ij     = <Q_i, P_j> / tau                                   (exponent of Eq. 1)
+ *   lse_i    = log sum_{allowed j} exp(S_ij)                      (denominator of Eq. 1 / Eq. 4)
+ *   loss     = (1/B) sum_i (lse_i - S_{i, r_i})                   (Eq. 1)
+ *   G_ij     = (exp(S_ij - lse_i) - [j == r_i]) / B               (Eq. 4; 0 where masked)
+ *   dQ_i     = (1/tau) sum_j G_ij P_j                             (Eq. 5)
+ *   dP_j     = (1/tau) sum_i G_ij Q_i                             (Eq. 6-7)
+ *
+ * dQ and dP together are the cache [u_1..u_B, v_1..v_N] of (B + N) d floats (Section 3.3).
+ * The paper fixes tau = 1 and has no mask; for general tau these are the exact derivatives of
+ * Eq. 1, and eps_j of Eq. 7 is the sum of f(s_k) over every k with r_k = j.  The B x N matrix
+ * S is never written to memory.
+ *
+ * Conventions shared by all calls
+ *   - Every pointer is a DEVICE pointer (including loss and dev_status) unless stated; the
+ *     caller owns all buffers, including the workspace.  The library allocates nothing.
+ *   - Matrices are row-major with unit stride along d; ldq/ldp/lddq/lddp are leading
+ *     dimensions in ELEMENTS.  Q/P rows must start on 16-byte boundaries (base address and
+ *     ld * element size multiples of 16), dQ/dP likewise; otherwise GC_ERR_ALIGN.
+ *   - Q and P may be the same buffer (symmetric loss); dQ/dP are then the derivatives with
+ *     respect to each role and the caller adds them.  Outputs may not alias inputs.
+ *   - dtype is the element type of Q and P; all outputs are float, accumulation is float.
+ *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t, may be NULL for the default
+ *     stream) and return a gc_status for host-detectable errors only.
+ *   - Data-dependent errors are OR-ed into *dev_status (may be NULL) on the device:
+ *     GC_DEV_POS_RANGE for pos_idx[i] outside [0, N), GC_DEV_POS_MASKED for pos_idx[i] equal
+ *     to the masked column.  Such a row contributes pos_logit = 0 and no one-hot term; nothing
+ *     is read out of bounds and nothing traps.  GC_DEV_WAIT_LIMIT means a bounded on-chip wait
+ *     gave up; outputs are then undefined.  The caller zeroes *dev_status beforehand.
+ *   - Results are deterministic: no floating-point atomics, fixed reduction order.
+ */
+#ifndef GRADCACHE_H_
+#define GRADCACHE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GC_OK = 0,
+    GC_ERR_NULL = 1,      /* a required pointer is NULL */
+    GC_ERR_SHAPE = 2,     /* B, N or d <= 0, ld < d, tau not finite or <= 0 */
+    GC_ERR_DTYPE = 3,     /* unknown dtype */
+    GC_ERR_MASK = 4,      /* unknown mask mode, or GC_MASK_SELF with N < 2 */
+    GC_ERR_ALIGN = 5,     /* a row does not start on a 16-byte boundary */
+    GC_ERR_WORKSPACE = 6, /* workspace NULL, misaligned (256 bytes) or too small */
+    GC_ERR_CUDA = 7,      /* a CUDA call or launch failed */
+    GC_ERR_ARCH = 8       /* the current device is not compute capability 10.x */
+} gc_status;
+
+typedef enum { GC_F32 = 0, GC_BF16 = 1 } gc_dtype;
+typedef enum { GC_MASK_NONE = 0, GC_MASK_SELF = 1 } gc_mask; /* SELF: drop the pair (i, i) */
+typedef enum { GC_OP_FWD = 0, GC_OP_BWD = 1, GC_OP_BUILD = 2 } gc_op;
+
+enum { GC_DEV_POS_RANGE = 1, GC_DEV_POS_MASKED = 2, GC_DEV_WAIT_LIMIT = 4 };
+
+/* Bytes of workspace the given call needs for these sizes on the current device (a multiple
+ * of 256; O((B + N) d), never O(B N)).  Returns 0 for invalid arguments. */
+size_t gc_workspace_bytes(int op, int64_t B, int64_t N, int d, int dtype);
+
+/* Name of the kernel plan the library will use for these sizes: "tcgen05" (TMA + tcgen05 MMA
+ * with TMEM accumulators; bf16, d a multiple of 64 up to 768) or "simt" (fp32 FMA tiles; every
+ * other case, including all fp32 inputs).  Static string. */
+const char* gc_plan_name(int op, int64_t B, int64_t N, int d, int dtype);
+
+/* Number of kernels one call launches for these sizes (for launch accounting). */
+int gc_kernel_launches(int op, int64_t B, int64_t N, int d, int dtype);
+
+/*
+ * Forward: Eq. 1.  Writes loss[1], row_lse[B] (natural log) and, if non-NULL, pos_logit[B]
+ * (S_{i, r_i}).  An online row maximum / sum runs over passage tiles (Section 3.2, Eq. 4's
+ * denominator); the positive logit is picked out of the tile that holds column r_i.
+ */
+int gc_loss_fwd(const void* Q, int64_t ldq, const void* P, int64_t ldp, const int32_t* pos_idx,
+                int64_t B, int64_t N, int d, float tau, int mask_mode, int dtype,
+                float* loss, float* row_lse, float* pos_logit,
+                void* ws, size_t ws_bytes, int* dev_status, void* cuda_stream);
+
+/*
+ * Backward: Eq. 5-7 given row_lse[B] from the forward.  Overwrites dQ[B x d] and dP[N x d]
+ * (either may be NULL to skip it).  S tiles are recomputed; G is formed in registers.
+ */
+int gc_loss_bwd(const void* Q, int64_t ldq, const void* P, int64_t ldp, const int32_t* pos_idx,
+                int64_t B, int64_t N, int d, float tau, int mask_mode, int dtype,
+                const float* row_lse, float* dQ, int64_t lddq, float* dP, int64_t lddp,
+                void* ws, size_t ws_bytes, int* dev_status, void* cuda_stream);
+
+/*
+ * Step 2 of Section 3.3 in one call: loss, row_lse, (pos_logit) and the cache dQ, dP.
+ */
+int gc_build_cache(const void* Q, int64_t ldq, const void* P, int64_t ldp, const int32_t* pos_idx,
+                   int64_t B, int64_t N, int d, float tau, int mask_mode, int dtype,
+                   float* loss, float* row_lse, float* pos_logit,
+                   float* dQ, int64_t lddq, float* dP, int64_t lddp,
+                   void* ws, size_t ws_bytes, int* dev_status, void* cuda_stream);
+
+/*
+ * Measurement aid (not part of the paper's method).  After gc_profile_enable(1) every call
+ * brackets its three main kernels - the forward sweep, the dQ sweep (Eq. 5) and the dP sweep
+ * (Eq. 6-7) - with CUDA events recorded on the call's own stream.  gc_profile_read waits for
+ * the most recent call's events and returns each kernel's duration in milliseconds (0 for a
+ * kernel that call did not launch).  Host pointers.  One set of events per process: enable it
+ * for single-stream measurement runs only.  Events are created on the first enable.
+ */
+int gc_profile_enable(int on);
+int gc_profile_read(float* ms_fwd, float* ms_dq, float* ms_dp);
+
+/* Human-readable name of a gc_status value.  Static string. */
+const char* gc_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GRADCACHE_H_ */

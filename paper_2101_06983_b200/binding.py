@@ -1,0 +1,209 @@
+"""Thin ctypes binding over libgradcache.so (include/gradcache.h).
+
+Argument marshalling only: torch tensors supply device memory and the current CUDA stream;
+every numerical step runs inside the library's kernels.  There is no CPU fallback: if the
+shared library is missing the import fails, and the calls need a CUDA device.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+from . import _build
+
+GC_F32, GC_BF16 = 0, 1
+GC_MASK_NONE, GC_MASK_SELF = 0, 1
+GC_OP_FWD, GC_OP_BWD, GC_OP_BUILD = 0, 1, 2
+GC_DEV_POS_RANGE, GC_DEV_POS_MASKED, GC_DEV_WAIT_LIMIT = 1, 2, 4
+
+EXPORTS = ("gc_workspace_bytes", "gc_plan_name", "gc_kernel_launches", "gc_loss_fwd",
+           "gc_loss_bwd", "gc_build_cache", "gc_status_string", "gc_profile_enable",
+           "gc_profile_read")
+
+
+class GradCacheError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (gc_status {status})")
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.LIB
+    if not os.path.exists(path):
+        raise ImportError(
+            f"{path} is missing: build it with `python -m paper_2101_06983_b200._build` "
+            "(there is no fallback implementation)")
+    lib = ctypes.CDLL(path)
+    vp, i64, i32, f32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float
+    common = [vp, i64, vp, i64, vp, i64, i64, i32, f32, i32, i32]
+    lib.gc_workspace_bytes.restype = ctypes.c_size_t
+    lib.gc_workspace_bytes.argtypes = [i32, i64, i64, i32, i32]
+    lib.gc_plan_name.restype = ctypes.c_char_p
+    lib.gc_plan_name.argtypes = [i32, i64, i64, i32, i32]
+    lib.gc_kernel_launches.restype = i32
+    lib.gc_kernel_launches.argtypes = [i32, i64, i64, i32, i32]
+    lib.gc_status_string.restype = ctypes.c_char_p
+    lib.gc_status_string.argtypes = [i32]
+    lib.gc_loss_fwd.restype = i32
+    lib.gc_loss_fwd.argtypes = common + [vp, vp, vp, vp, ctypes.c_size_t, vp, vp]
+    lib.gc_loss_bwd.restype = i32
+    lib.gc_loss_bwd.argtypes = common + [vp, vp, i64, vp, i64, vp, ctypes.c_size_t, vp, vp]
+    lib.gc_build_cache.restype = i32
+    lib.gc_build_cache.argtypes = common + [vp, vp, vp, vp, i64, vp, i64, vp, ctypes.c_size_t,
+                                            vp, vp]
+    lib.gc_profile_enable.restype = i32
+    lib.gc_profile_enable.argtypes = [i32]
+    lib.gc_profile_read.restype = i32
+    lib.gc_profile_read.argtypes = [ctypes.POINTER(f32)] * 3
+    return lib
+
+
+_lib = _load()
+
+
+def status_string(status: int) -> str:
+    return _lib.gc_status_string(int(status)).decode()
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return GC_F32
+    if t.dtype == torch.bfloat16:
+        return GC_BF16
+    raise TypeError(f"Q/P must be float32 or bfloat16, got {t.dtype}")
+
+
+def gc_workspace_bytes(op: int, B: int, N: int, d: int, dtype: int) -> int:
+    return int(_lib.gc_workspace_bytes(op, B, N, d, dtype))
+
+
+def gc_plan_name(op: int, B: int, N: int, d: int, dtype: int) -> str:
+    return _lib.gc_plan_name(op, B, N, d, dtype).decode()
+
+
+def gc_kernel_launches(op: int, B: int, N: int, d: int, dtype: int) -> int:
+    return int(_lib.gc_kernel_launches(op, B, N, d, dtype))
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _common(Q, P, pos_idx, tau, mask_mode):
+    if Q.dim() != 2 or P.dim() != 2 or Q.stride(1) != 1 or P.stride(1) != 1:
+        raise ValueError("Q and P must be 2-D with unit stride along d")
+    if pos_idx.dtype != torch.int32 or not pos_idx.is_contiguous():
+        raise TypeError("pos_idx must be a contiguous int32 tensor")
+    if P.dtype != Q.dtype or P.shape[1] != Q.shape[1]:
+        raise ValueError("Q and P must share dtype and width")
+    B, d = Q.shape
+    N = P.shape[0]
+    code = _dtype_code(Q)
+    args = [_ptr(Q), Q.stride(0), _ptr(P), P.stride(0), _ptr(pos_idx), B, N, d, float(tau),
+            int(mask_mode), code]
+    return args, B, N, d, code
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def alloc_workspace(op: int, B: int, N: int, d: int, dtype: int, device) -> torch.Tensor:
+    """A workspace tensor of the size gc_workspace_bytes reports (torch memory is 512-byte
+    aligned, which covers the 256-byte requirement)."""
+    n = max(gc_workspace_bytes(op, B, N, d, dtype), 256)
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def gc_loss_fwd(Q, P, pos_idx, tau, mask_mode, loss, row_lse, pos_logit=None, ws=None,
+                dev_status=None):
+    """Eq. 1: writes loss[1], row_lse[B] and optionally pos_logit[B] (all float32 on device)."""
+    args, B, N, d, code = _common(Q, P, pos_idx, tau, mask_mode)
+    if ws is None:
+        ws = alloc_workspace(GC_OP_FWD, B, N, d, code, Q.device)
+    rc = _lib.gc_loss_fwd(*args, _ptr(loss), _ptr(row_lse), _ptr(pos_logit), _ptr(ws),
+                          ws.numel(), _ptr(dev_status), _stream())
+    if rc != 0:
+        raise GradCacheError(rc, "gc_loss_fwd")
+
+
+def gc_loss_bwd(Q, P, pos_idx, tau, mask_mode, row_lse, dQ, dP, ws=None, dev_status=None):
+    """Eq. 5-7 given row_lse: overwrites dQ[B x d] and dP[N x d] (either may be None)."""
+    args, B, N, d, code = _common(Q, P, pos_idx, tau, mask_mode)
+    if ws is None:
+        ws = alloc_workspace(GC_OP_BWD, B, N, d, code, Q.device)
+    rc = _lib.gc_loss_bwd(*args, _ptr(row_lse), _ptr(dQ), 0 if dQ is None else dQ.stride(0),
+                          _ptr(dP), 0 if dP is None else dP.stride(0), _ptr(ws), ws.numel(),
+                          _ptr(dev_status), _stream())
+    if rc != 0:
+        raise GradCacheError(rc, "gc_loss_bwd")
+
+
+def gc_build_cache(Q, P, pos_idx, tau, mask_mode, loss, row_lse, dQ, dP, pos_logit=None,
+                   ws=None, dev_status=None):
+    """Step 2 of Section 3.3: loss, row_lse and the representation gradient cache dQ, dP."""
+    args, B, N, d, code = _common(Q, P, pos_idx, tau, mask_mode)
+    if ws is None:
+        ws = alloc_workspace(GC_OP_BUILD, B, N, d, code, Q.device)
+    rc = _lib.gc_build_cache(*args, _ptr(loss), _ptr(row_lse), _ptr(pos_logit), _ptr(dQ),
+                             dQ.stride(0), _ptr(dP), dP.stride(0), _ptr(ws), ws.numel(),
+                             _ptr(dev_status), _stream())
+    if rc != 0:
+        raise GradCacheError(rc, "gc_build_cache")
+
+
+def gc_profile_enable(on: bool) -> None:
+    rc = _lib.gc_profile_enable(1 if on else 0)
+    if rc != 0:
+        raise GradCacheError(rc, "gc_profile_enable")
+
+
+def gc_profile_read() -> tuple[float, float, float]:
+    """Milliseconds of the last call's forward sweep, dQ sweep and dP sweep kernels."""
+    a, b, c = ctypes.c_float(), ctypes.c_float(), ctypes.c_float()
+    rc = _lib.gc_profile_read(ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
+    if rc != 0:
+        raise GradCacheError(rc, "gc_profile_read")
+    return a.value, b.value, c.value
+
+
+def problem_tensors(prob, device="cuda"):
+    """(Q, P, pos_idx) device tensors for an inputs.Problem, in its dtype.  Shared rows stay one
+    buffer (Q is P)."""
+    import numpy as np
+    if prob.dtype == "bf16":
+        Q = torch.from_numpy(prob.Q_bits.view(np.int16)).view(torch.bfloat16).to(device)
+        P = Q if prob.shared else torch.from_numpy(prob.P_bits.view(np.int16)).view(
+            torch.bfloat16).to(device)
+    else:
+        Q = torch.from_numpy(prob.Q).to(device)
+        P = Q if prob.shared else torch.from_numpy(prob.P).to(device)
+    return Q, P, torch.from_numpy(prob.pos_idx).to(device)
+
+
+class Outputs:
+    """Device buffers for one problem size, allocated once and reused across calls."""
+
+    def __init__(self, B: int, N: int, d: int, dtype: int, device="cuda"):
+        f = dict(dtype=torch.float32, device=device)
+        self.loss = torch.zeros(1, **f)
+        self.row_lse = torch.empty(B, **f)
+        self.pos_logit = torch.empty(B, **f)
+        self.dQ = torch.empty(B, d, **f)
+        self.dP = torch.empty(N, d, **f)
+        self.dev_status = torch.zeros(1, dtype=torch.int32, device=device)
+        self.ws = alloc_workspace(GC_OP_BUILD, B, N, d, dtype, device)
+
+
+def build_cache(Q, P, pos_idx, tau=1.0, mask_mode=GC_MASK_NONE, out: Outputs | None = None):
+    """Convenience wrapper: allocates outputs (or reuses `out`) and calls gc_build_cache."""
+    B, d = Q.shape
+    N = P.shape[0]
+    if out is None:
+        out = Outputs(B, N, d, _dtype_code(Q), Q.device)
+    out.dev_status.zero_()
+    gc_build_cache(Q, P, pos_idx, tau, mask_mode, out.loss, out.row_lse, out.dQ, out.dP,
+                   out.pos_logit, out.ws, out.dev_status)
+    return out

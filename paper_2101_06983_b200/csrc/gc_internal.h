@@ -1,0 +1,94 @@
+// Internal declarations shared by the translation units of libgradcache (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "gradcache.h"
+
+namespace gc {
+
+// One problem instance as the entry points receive it.
+struct Problem {
+    const void* Q;
+    const void* P;
+    const int32_t* pos_idx;
+    int64_t ldq, ldp;
+    int64_t B, N;
+    int d;
+    float tau;
+    int mask_mode;
+    int dtype;
+};
+
+// The two tile sweeps share one shape: a stationary row tile X, a streamed row tile Y,
+// S_xy = <X_x, Y_y> / tau, a weight W_xy derived from S, and acc_x += sum_y W_xy Y_y.
+//   SWEEP_DQ: x = query i,   y = passage j, W = exp(S - lse[x]) - [y == pos[x]]   (Eq. 5)
+//   SWEEP_DP: x = passage j, y = query i,   W = exp(S - lse[y]) - [x == pos[y]]   (Eq. 6-7)
+// In both, W = 0 for the masked pair (query index == passage index under GC_MASK_SELF).
+enum SweepMode { SWEEP_DQ = 0, SWEEP_DP = 1 };
+
+struct SweepArgs {
+    const void* X;          // stationary rows  [nx x d]
+    const void* Y;          // streamed rows    [ny x d]
+    int64_t ldx, ldy;
+    int64_t nx, ny;
+    int d;
+    int mode;               // SweepMode
+    int mask_mode;
+    int dtype;
+    float inv_tau;
+    float out_scale;        // 1 / (B * tau), applied where the final value is written
+    const float* row_lse;   // [B], indexed by the query index
+    const int32_t* pos_idx; // [B], indexed by the query index
+    float* out;             // [nx x d] final output (used when groups == 1)
+    int64_t ldo;
+    float* partial;         // [groups x nx x d] unscaled partial sums (used when groups > 1)
+    int groups;             // the y range is split into this many contiguous parts
+};
+
+struct FwdArgs {
+    Problem p;
+    float* part_m;          // [groups x B] running maximum of each part
+    float* part_l;          // [groups x B] sum of exp(S - m) of each part
+    float* pos_logit;       // [B] written only by the owner of column pos_idx[i]
+    int groups;
+};
+
+// How one call is carried out for given sizes on the current device.
+struct Plan {
+    int tc;                 // 1: tcgen05 kernels, 0: SIMT kernels
+    int g_fwd, g_dq, g_dp;  // split factors of the streamed range
+    size_t off_m, off_l, off_pos, off_accq, off_accp;
+    size_t total;           // workspace bytes (multiple of 256)
+    int launches_fwd, launches_bwd;
+};
+
+int sm_count();
+Plan make_plan(int64_t B, int64_t N, int d, int dtype);
+
+// gc_combine.cu
+cudaError_t launch_lse_combine(const float* part_m, const float* part_l, const float* pos_ws,
+                               const int32_t* pos_idx, int groups, int64_t B, int64_t N,
+                               int mask_mode, float* row_lse, float* pos_logit, float* loss,
+                               int* dev_status, cudaStream_t st);
+cudaError_t launch_pos_check(const int32_t* pos_idx, int64_t B, int64_t N, int mask_mode,
+                             int* dev_status, cudaStream_t st);
+cudaError_t launch_partial_reduce(const float* partial, int groups, int64_t rows, int d,
+                                  float scale, float* out, int64_t ldo, cudaStream_t st);
+
+// gc_simt.cu
+cudaError_t simt_launch_fwd(const FwdArgs& a, cudaStream_t st);
+cudaError_t simt_launch_sweep(const SweepArgs& a, cudaStream_t st);
+int simt_fwd_groups(int64_t B, int64_t N);
+int simt_sweep_groups(int64_t nx, int64_t ny, int d);
+
+// gc_tc.cu
+bool tc_supported(int64_t B, int64_t N, int d, int dtype);
+cudaError_t tc_launch_fwd(const FwdArgs& a, cudaStream_t st);
+cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st);
+int tc_fwd_groups(int64_t B, int64_t N, int d);
+int tc_sweep_groups(int64_t nx, int64_t ny, int d);
+
+}  // namespace gc
