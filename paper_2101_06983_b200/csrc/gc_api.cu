@@ -135,6 +135,7 @@ int run_fwd(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_
     fa.part_l = reinterpret_cast<float*>(ws + pl.off_l);
     fa.pos_logit = reinterpret_cast<float*>(ws + pl.off_pos);
     fa.groups = pl.g_fwd;
+    fa.dev_status = dev_status;
     cudaError_t e;
     {
         KernelTimer t(0, st);
@@ -147,7 +148,7 @@ int run_fwd(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_
 }
 
 int run_sweep(const Problem& p, const Plan& pl, char* ws, int mode, const float* row_lse,
-              float* out, int64_t ldo, cudaStream_t st) {
+              float* out, int64_t ldo, int* dev_status, cudaStream_t st) {
     SweepArgs sa;
     const bool dq = (mode == SWEEP_DQ);
     sa.X = dq ? p.Q : p.P;   sa.ldx = dq ? p.ldq : p.ldp;   sa.nx = dq ? p.B : p.N;
@@ -164,6 +165,7 @@ int run_sweep(const Problem& p, const Plan& pl, char* ws, int mode, const float*
     sa.ldo = ldo;
     sa.groups = dq ? pl.g_dq : pl.g_dp;
     sa.partial = reinterpret_cast<float*>(ws + (dq ? pl.off_accq : pl.off_accp));
+    sa.dev_status = dev_status;
     cudaError_t e;
     {
         KernelTimer t(dq ? 1 : 2, st);
@@ -237,8 +239,8 @@ int gc_loss_bwd(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
     if (dev_status && launch_pos_check(pos_idx, B, N, mask_mode, dev_status, st) != cudaSuccess)
         return GC_ERR_CUDA;
     char* w = static_cast<char*>(ws);
-    if (dQ && (rc = run_sweep(p, pl, w, SWEEP_DQ, row_lse, dQ, lddq, st))) return rc;
-    if (dP && (rc = run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, st))) return rc;
+    if (dQ && (rc = run_sweep(p, pl, w, SWEEP_DQ, row_lse, dQ, lddq, dev_status, st))) return rc;
+    if (dP && (rc = run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, dev_status, st))) return rc;
     return GC_OK;
 }
 
@@ -258,8 +260,8 @@ int gc_build_cache(const void* Q, int64_t ldq, const void* P, int64_t ldp, const
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
     char* w = static_cast<char*>(ws);
     if ((rc = run_fwd(p, pl, w, loss, row_lse, pos_logit, dev_status, st))) return rc;
-    if ((rc = run_sweep(p, pl, w, SWEEP_DQ, row_lse, dQ, lddq, st))) return rc;
-    if ((rc = run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, st))) return rc;
+    if ((rc = run_sweep(p, pl, w, SWEEP_DQ, row_lse, dQ, lddq, dev_status, st))) return rc;
+    if ((rc = run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, dev_status, st))) return rc;
     return GC_OK;
 }
 

@@ -46,6 +46,7 @@ struct SweepArgs {
     int64_t ldo;
     float* partial;         // [groups x nx x d] unscaled partial sums (used when groups > 1)
     int groups;             // the y range is split into this many contiguous parts
+    int* dev_status;        // may be NULL
 };
 
 struct FwdArgs {
@@ -54,6 +55,7 @@ struct FwdArgs {
     float* part_l;          // [groups x B] sum of exp(S - m) of each part
     float* pos_logit;       // [B] written only by the owner of column pos_idx[i]
     int groups;
+    int* dev_status;        // may be NULL
 };
 
 // How one call is carried out for given sizes on the current device.

@@ -1,9 +1,720 @@
-// placeholder until the tensor-core plan lands
+// Tensor-core plan for bf16 inputs with d a multiple of 64 (up to 768): TMA-staged tiles in
+// 128-byte-swizzled shared memory, tcgen05 MMAs with fp32 accumulators in tensor memory, the
+// softmax arithmetic in registers.  One kernel template serves three sweeps:
+//
+//   FWD  (Eq. 1)    x = 128 queries,  y streams passages: S = X Y^T, online row max / sum.
+//   DQ   (Eq. 5)    x = 128 queries,  y streams passages: W = exp(S - lse_x) - onehot, acc += W Y
+//   DP   (Eq. 6-7)  x = 128 passages, y streams queries:  W = exp(S - lse_y) - onehot, acc += W Y
+//
+// The stationary tile X (128 x d) stays resident in shared memory; Y arrives in (SN x 64)
+// chunks through an mbarrier ring.  S tiles (128 x SN, fp32) are double buffered in tensor
+// memory so the MMAs of step t+1 run while the softmax warps work on step t.  W is written
+// back over its S buffer as packed bf16 and used as the A operand (from tensor memory) of the
+// second MMA, whose B operand is the same Y chunk read MN-major.  An accumulator of 128 x 768
+// fp32 does not fit the 512 tensor-memory columns, so wide rows are split into column parts
+// (at most 384 columns each), one CTA per part.  S is never written to global memory.
+//
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer (and tensor-memory
+// allocator), warps 2..5 = softmax / epilogue, one thread per tile row.
+// Every wait is bounded: on a timeout the CTA raises GC_DEV_WAIT_LIMIT, drains and exits.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <math.h>
+
 #include "gc_internal.h"
+
 namespace gc {
-bool tc_supported(int64_t, int64_t, int, int) { return false; }
-cudaError_t tc_launch_fwd(const FwdArgs&, cudaStream_t) { return cudaErrorNotSupported; }
-cudaError_t tc_launch_sweep(const SweepArgs&, cudaStream_t) { return cudaErrorNotSupported; }
-int tc_fwd_groups(int64_t, int64_t, int) { return 1; }
-int tc_sweep_groups(int64_t, int64_t, int) { return 1; }
+
+namespace {
+
+constexpr int XROWS = 128;                 // rows of the stationary tile = MMA M
+constexpr int CHUNK_BYTES_PER_ROW = 128;   // 64 bf16 = one swizzle row
+constexpr uint32_t X_CHUNK_BYTES = XROWS * CHUNK_BYTES_PER_ROW;
+constexpr int NTHREADS = 192;
+constexpr int MAX_STAGES = 8;
+constexpr int TMEM_COLS = 512;
+constexpr int MAX_D = 768;
+constexpr int MAX_PART_CHUNKS = 6;         // 384 accumulator columns
+constexpr size_t SMEM_LIMIT = 232448;      // 227 KB per block
+constexpr size_t SMEM_STATIC_RESERVE = 2048;
+constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
+
+enum { MODE_FWD = 0, MODE_DQ = 1, MODE_DP = 2 };
+
+struct TcParams {
+    int64_t nx, ny;
+    int64_t nq;               // number of queries B (pitch of the forward partial arrays)
+    int kc;                   // d / 64
+    int dparts, dpc;          // accumulator column parts and chunks per part
+    int groups;
+    int nstage;
+    int mask_mode;
+    float c1;                 // log2(e) / tau
+    float inv_tau;
+    float out_scale;
+    const float* row_lse;
+    const int32_t* pos_idx;
+    float* out;
+    int64_t ldo;
+    float* partial;
+    float* part_m;
+    float* part_l;
+    float* pos_logit;
+    int* dev_status;
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+    return (uint32_t)__cvta_generic_to_shared(p);
 }
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false when the CTA is aborting or the time limit passed.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try(bar, parity)) return true;
+    uint64_t t0 = global_ns();
+    uint32_t spins = 0;
+    while (true) {
+        if (mbar_try(bar, parity)) return true;
+        if ((++spins & 127u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > WAIT_LIMIT_NS) {
+                *abort_flag = 1;
+                return false;
+            }
+        }
+    }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1,
+                                            uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                 ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                       uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// D[tmem] (+)= A[tmem] * B[smem]
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
+                                       uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
+          "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
+          "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]),
+          "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]),
+          "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() {
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]),
+          "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]),
+          "r"(v[14]), "r"(v[15])
+        : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() {
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Shared-memory matrix descriptor for 128-byte-swizzled tiles whose rows are 128 bytes:
+// start address and stride-between-8-row-groups (1024 bytes) in 16-byte units, descriptor
+// version 1, layout type 2 (SWIZZLE_128B).  K-major operands step 32 bytes per K = 16 inside the
+// swizzle row; MN-major operands step 16 rows (2048 bytes) per K = 16.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFF);
+    d |= (uint64_t)(1024 >> 4) << 16;     // leading byte offset (next 64-element MN atom; unused)
+    d |= (uint64_t)(1024 >> 4) << 32;     // stride byte offset: 8 rows x 128 bytes
+    d |= (uint64_t)1 << 46;               // descriptor version
+    d |= (uint64_t)2 << 61;               // SWIZZLE_128B
+    return d;
+}
+// Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, M = 128.
+__device__ __forceinline__ uint32_t instr_desc(int n, bool b_mn_major) {
+    uint32_t d = 0;
+    d |= 1u << 4;                          // D format f32
+    d |= 1u << 7;                          // A format bf16
+    d |= 1u << 10;                         // B format bf16
+    d |= (b_mn_major ? 1u : 0u) << 16;     // B major
+    d |= (uint32_t)(n >> 3) << 17;
+    d |= (uint32_t)(XROWS >> 4) << 24;
+    return d;
+}
+
+__device__ __forceinline__ void part_range(int64_t steps, int groups, int g, int64_t* lo,
+                                           int64_t* hi) {
+    int64_t base = steps / groups, rem = steps % groups;
+    *lo = g * base + (g < rem ? g : rem);
+    *hi = *lo + base + (g < rem ? 1 : 0);
+}
+
+struct Bars {
+    uint64_t x_full;
+    uint64_t y_full[MAX_STAGES];
+    uint64_t y_empty[MAX_STAGES];
+    uint64_t s_full[2];
+    uint64_t w_full[2];
+    uint64_t acc_full;
+};
+
+// ---------------------------------------------------------------------------------------------
+// The sweep kernel
+// ---------------------------------------------------------------------------------------------
+template <int MODE, int SN>
+__global__ void __launch_bounds__(NTHREADS, 1)
+tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
+          const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) Bars bars;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ int abort_s;
+    volatile int* abort_flag = &abort_s;
+
+    constexpr uint32_t STAGE_BYTES = SN * CHUNK_BYTES_PER_ROW;
+    constexpr uint32_t S_COL0 = TMEM_COLS - 2 * SN;     // S buffers sit at the top columns
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // work item: (x tile, column part, part of the streamed range)
+    int unit = blockIdx.x;
+    const int g = unit % p.groups;
+    unit /= p.groups;
+    const int dp = unit % p.dparts;
+    const int64_t xt = unit / p.dparts;
+    const int64_t x0 = xt * XROWS;
+    const int c_begin = dp * p.dpc;
+    const int c_count = (MODE == MODE_FWD) ? 0 : min(p.dpc, p.kc - c_begin);
+
+    int64_t lo, hi;
+    part_range((p.ny + SN - 1) / SN, p.groups, g, &lo, &hi);
+    const int T = (int)(hi - lo);
+
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t x_smem = base;
+    const uint32_t y_smem = base + (uint32_t)p.kc * X_CHUNK_BYTES;
+
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        mbar_init(smem_u32(&bars.x_full), 1);
+        for (int s = 0; s < MAX_STAGES; ++s) {
+            mbar_init(smem_u32(&bars.y_full[s]), 1);
+            mbar_init(smem_u32(&bars.y_empty[s]), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(smem_u32(&bars.s_full[b]), 1);
+            mbar_init(smem_u32(&bars.w_full[b]), 4);      // one arrival per softmax warp
+        }
+        mbar_init(smem_u32(&bars.acc_full), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_s;
+
+    if (warp == 0) {
+        // ------------------------------ TMA producer ------------------------------------------
+        if (lane == 0) {
+            mbar_expect_tx(smem_u32(&bars.x_full), (uint32_t)p.kc * X_CHUNK_BYTES);
+            for (int c = 0; c < p.kc; ++c)
+                tma_load_2d(x_smem + c * X_CHUNK_BYTES, &mapX, c * 64, (int)x0,
+                            smem_u32(&bars.x_full));
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            auto load_chunk = [&](int chunk, int64_t row) {
+                if (!ok) return;
+                if (!mbar_wait(smem_u32(&bars.y_empty[stage]), phase ^ 1u, abort_flag)) {
+                    ok = false;
+                    return;
+                }
+                uint32_t full = smem_u32(&bars.y_full[stage]);
+                mbar_expect_tx(full, STAGE_BYTES);
+                tma_load_2d(y_smem + stage * STAGE_BYTES, &mapY, chunk * 64, (int)row, full);
+                if (++stage == p.nstage) { stage = 0; phase ^= 1u; }
+            };
+            for (int t = 0; t <= T && ok; ++t) {
+                if (t < T)
+                    for (int c = 0; c < p.kc; ++c) load_chunk(c, (lo + t) * SN);
+                if (MODE != MODE_FWD && t >= 1)
+                    for (int c = 0; c < c_count; ++c) load_chunk(c_begin + c, (lo + t - 1) * SN);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ----------------------------------------------
+        if (lane == 0) {
+            const uint32_t idesc_s = instr_desc(SN, false);
+            const uint32_t idesc_acc = instr_desc(64, true);
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = mbar_wait(smem_u32(&bars.x_full), 0, abort_flag);
+            tc_fence_after();
+            for (int t = 0; t <= T && ok; ++t) {
+                if (t < T) {
+                    const int b = t & 1;
+                    if (MODE == MODE_FWD && t >= 2) {
+                        ok = mbar_wait(smem_u32(&bars.w_full[b]), ((t - 2) >> 1) & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                    }
+                    const uint32_t d_tmem = tmem + S_COL0 + b * SN;
+                    for (int c = 0; c < p.kc && ok; ++c) {
+                        ok = mbar_wait(smem_u32(&bars.y_full[stage]), phase, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t xa = x_smem + c * X_CHUNK_BYTES;
+                        const uint32_t yb = y_smem + stage * STAGE_BYTES;
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            mma_ss(d_tmem, smem_desc(xa + k * 32), smem_desc(yb + k * 32), idesc_s,
+                                   (c | k) != 0);
+                        tc_commit(smem_u32(&bars.y_empty[stage]));
+                        if (++stage == p.nstage) { stage = 0; phase ^= 1u; }
+                    }
+                    if (!ok) break;
+                    tc_commit(smem_u32(&bars.s_full[b]));
+                }
+                if (MODE != MODE_FWD && t >= 1) {
+                    const int u = t - 1, b = u & 1;
+                    ok = mbar_wait(smem_u32(&bars.w_full[b]), (u >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t w_tmem = tmem + S_COL0 + b * SN;
+                    for (int c = 0; c < c_count && ok; ++c) {
+                        ok = mbar_wait(smem_u32(&bars.y_full[stage]), phase, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t yb = y_smem + stage * STAGE_BYTES;
+#pragma unroll
+                        for (int k = 0; k < SN / 16; ++k)
+                            mma_ts(tmem + c * 64, w_tmem + k * 8, smem_desc(yb + k * 2048),
+                                   idesc_acc, (u | k) != 0);
+                        tc_commit(smem_u32(&bars.y_empty[stage]));
+                        if (++stage == p.nstage) { stage = 0; phase ^= 1u; }
+                    }
+                }
+            }
+            if (ok && MODE != MODE_FWD) tc_commit(smem_u32(&bars.acc_full));
+        }
+    } else {
+        // ------------------------------ softmax / epilogue warps --------------------------------
+        const int q = warp & 3;                        // tensor-memory lane quarter of this warp
+        const int row = q * 32 + lane;
+        const int64_t x = x0 + row;
+        const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
+        const bool self_mask = (p.mask_mode == GC_MASK_SELF);
+        bool ok = true;
+
+        if (MODE == MODE_FWD) {
+            float m = -INFINITY, l = 0.f;
+            const int32_t pos_x = (x < p.nx) ? p.pos_idx[x] : -1;
+            for (int t = 0; t < T; ++t) {
+                const int b = t & 1;
+                ok = mbar_wait(smem_u32(&bars.s_full[b]), (t >> 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const int64_t y0 = (lo + t) * SN;
+#pragma unroll 1
+                for (int cb = 0; cb < SN / 32; ++cb) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem + lane_addr + S_COL0 + b * SN + cb * 32, v);
+                    tmem_ld_wait();
+                    const int64_t yb = y0 + cb * 32;
+                    if (yb >= p.ny) continue;
+                    if (pos_x >= yb && pos_x < yb + 32 && !(self_mask && x == pos_x)) {
+                        const int rel = (int)(pos_x - yb);
+                        float s = 0.f;
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (c == rel) s = __uint_as_float(v[c]);
+                        p.pos_logit[x] = s * p.inv_tau;
+                    }
+                    float s2[32];
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) s2[c] = __uint_as_float(v[c]) * p.c1;
+                    if (yb + 32 > p.ny) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (yb + c >= p.ny) s2[c] = -INFINITY;
+                    }
+                    if (self_mask && x >= yb && x < yb + 32) {
+                        const int rel = (int)(x - yb);
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (c == rel) s2[c] = -INFINITY;
+                    }
+                    float bm = s2[0];
+#pragma unroll
+                    for (int c = 1; c < 32; ++c) bm = fmaxf(bm, s2[c]);
+                    if (bm > -INFINITY) {
+                        const float mn = fmaxf(m, bm);
+                        float sum = 0.f;
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) sum += ex2(s2[c] - mn);
+                        l = l * ex2(m - mn) + sum;
+                        m = mn;
+                    }
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars.w_full[b]));
+            }
+            if (ok && x < p.nx) {
+                p.part_m[(int64_t)g * p.nq + x] = m * 0.69314718055994531f;   // back to natural log
+                p.part_l[(int64_t)g * p.nq + x] = l;
+            }
+        } else {
+            // per-row constants (DQ: the row is a query)
+            float lse2_x = 0.f;
+            int32_t pos_x = -1;
+            if (MODE == MODE_DQ && x < p.nx) {
+                lse2_x = p.row_lse[x] * 1.4426950408889634f;
+                pos_x = p.pos_idx[x];
+            }
+            for (int t = 0; t < T; ++t) {
+                const int b = t & 1;
+                const int64_t y0 = (lo + t) * SN;
+                // DP: the columns are queries; lane j holds lse / pos of column 32 cb + j
+                float lse2_y[SN / 32];
+                int32_t pos_y[SN / 32];
+                if (MODE == MODE_DP) {
+#pragma unroll
+                    for (int cb = 0; cb < SN / 32; ++cb) {
+                        const int64_t y = y0 + cb * 32 + lane;
+                        lse2_y[cb] = (y < p.ny) ? p.row_lse[y] * 1.4426950408889634f : INFINITY;
+                        pos_y[cb] = (y < p.ny) ? p.pos_idx[y] : -1;
+                    }
+                }
+                ok = mbar_wait(smem_u32(&bars.s_full[b]), (t >> 1) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t sbuf = tmem + lane_addr + S_COL0 + b * SN;
+#pragma unroll
+                for (int cb = 0; cb < SN / 32; ++cb) {
+                    uint32_t v[32];
+                    tmem_ld32(sbuf + cb * 32, v);
+                    tmem_ld_wait();
+                    const int64_t yb = y0 + cb * 32;
+                    float w[32];
+                    if (MODE == MODE_DQ) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            w[c] = ex2(fmaf(__uint_as_float(v[c]), p.c1, -lse2_x));
+                        if (pos_x >= yb && pos_x < yb + 32) {
+                            const int rel = (int)(pos_x - yb);
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (c == rel) w[c] -= 1.f;
+                        }
+                        if (yb + 32 > p.ny) {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (yb + c >= p.ny) w[c] = 0.f;
+                        }
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            const float ls = __shfl_sync(0xffffffffu, lse2_y[cb], c);
+                            w[c] = ex2(fmaf(__uint_as_float(v[c]), p.c1, -ls));   // OOB: ex2(-inf)
+                        }
+                        // one-hot: column c's query has its positive at row pos - x0 of this tile
+                        const int64_t rel_row = (int64_t)pos_y[cb] - x0;
+                        const bool mine = (pos_y[cb] >= 0) && rel_row >= q * 32 && rel_row < q * 32 + 32;
+                        unsigned hits = __ballot_sync(0xffffffffu, mine);
+                        while (hits) {
+                            const int col = __ffs(hits) - 1;
+                            hits &= hits - 1;
+                            const int target = (int)__shfl_sync(0xffffffffu, (int)rel_row, col) - q * 32;
+                            if (lane == target) {
+#pragma unroll
+                                for (int c = 0; c < 32; ++c)
+                                    if (c == col) w[c] -= 1.f;
+                            }
+                        }
+                    }
+                    if (self_mask && x >= yb && x < yb + 32) {
+                        const int rel = (int)(x - yb);
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (c == rel) w[c] = 0.f;
+                    }
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(w[2 * r], w[2 * r + 1]);
+                        packed[r] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                    tmem_st16(sbuf + cb * 16, packed);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars.w_full[b]));
+            }
+            // epilogue: accumulator columns of this part -> global memory
+            if (ok) ok = mbar_wait(smem_u32(&bars.acc_full), 0, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                const bool final_out = (p.groups == 1);
+                const int64_t d = (int64_t)p.kc * 64;
+                float* dst = final_out ? p.out + x * p.ldo + c_begin * 64
+                                       : p.partial + ((int64_t)g * p.nx + x) * d + c_begin * 64;
+                const float sc = final_out ? p.out_scale : 1.f;
+                for (int cb = 0; cb < c_count * 2; ++cb) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem + lane_addr + cb * 32, v);
+                    tmem_ld_wait();
+                    if (x < p.nx) {
+#pragma unroll
+                        for (int c = 0; c < 32; c += 4) {
+                            float4 o = make_float4(__uint_as_float(v[c]) * sc,
+                                                   __uint_as_float(v[c + 1]) * sc,
+                                                   __uint_as_float(v[c + 2]) * sc,
+                                                   __uint_as_float(v[c + 3]) * sc);
+                            *reinterpret_cast<float4*>(dst + cb * 32 + c) = o;
+                        }
+                    }
+                }
+            }
+        }
+    }
+
+    // ------------------------------ teardown ------------------------------------------------------
+    tc_fence_before();
+    __syncthreads();
+    if (*abort_flag) {
+        // let bulk copies still in flight land before the shared memory is released
+        uint64_t t0 = global_ns();
+        while (global_ns() - t0 < 200000ull) __nanosleep(1000);
+        if (threadIdx.x == 0 && p.dev_status) atomicOr(p.dev_status, GC_DEV_WAIT_LIMIT);
+        __syncthreads();
+    }
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                     ::"r"(tmem), "r"((uint32_t)TMEM_COLS) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Host side
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* sym = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) !=
+                cudaSuccess || qres != cudaDriverEntryPointSuccess)
+            return nullptr;
+        fn = reinterpret_cast<EncodeTiledFn>(sym);
+    }
+    return fn;
+}
+
+// Row-major bf16 matrix [rows x d], boxes of (box_rows x 64 columns), 128-byte swizzle,
+// out-of-range elements read as zero.
+bool make_map(CUtensorMap* map, const void* base, int64_t rows, int d, int64_t ld, int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+int parts_for(int kc) { return (kc + MAX_PART_CHUNKS - 1) / MAX_PART_CHUNKS; }
+int chunks_per_part(int kc) { int n = parts_for(kc); return (kc + n - 1) / n; }
+
+// S-tile width of the gradient sweeps: 128 when the accumulator part leaves room for two
+// 128-column S buffers, else 64.
+int sweep_sn(int kc) { return chunks_per_part(kc) * 64 + 256 <= TMEM_COLS ? 128 : 64; }
+
+struct SmemPlan { int nstage; size_t dynamic_bytes; };
+
+SmemPlan smem_plan(int kc, int sn) {
+    size_t xbytes = (size_t)kc * X_CHUNK_BYTES;
+    size_t stage = (size_t)sn * CHUNK_BYTES_PER_ROW;
+    size_t avail = SMEM_LIMIT - SMEM_STATIC_RESERVE - 1024 - xbytes;
+    int ns = (int)(avail / stage);
+    if (ns > MAX_STAGES) ns = MAX_STAGES;
+    SmemPlan sp;
+    sp.nstage = ns;
+    sp.dynamic_bytes = 1024 + xbytes + (size_t)ns * stage;
+    // keep one CTA per SM (each CTA allocates all 512 tensor-memory columns)
+    if (sp.dynamic_bytes < 120 * 1024) sp.dynamic_bytes = 120 * 1024;
+    return sp;
+}
+
+template <int MODE, int SN>
+cudaError_t launch(const CUtensorMap& mx, const CUtensorMap& my, const TcParams& p, int64_t units,
+                   cudaStream_t st) {
+    SmemPlan sp = smem_plan(p.kc, SN);
+    static bool configured = false;
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(tc_kernel<MODE, SN>,
+                                             cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)(SMEM_LIMIT - SMEM_STATIC_RESERVE));
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    tc_kernel<MODE, SN><<<(unsigned)units, NTHREADS, sp.dynamic_bytes, st>>>(mx, my, p);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+bool tc_supported(int64_t B, int64_t N, int d, int dtype) {
+    (void)B; (void)N;
+    return dtype == GC_BF16 && d % 64 == 0 && d >= 64 && d <= MAX_D;
+}
+
+int tc_fwd_groups(int64_t B, int64_t N, int d) {
+    (void)d;
+    int64_t tiles = (B + XROWS - 1) / XROWS, steps = (N + 127) / 128;
+    int64_t g = sm_count() / tiles;
+    if (g < 1) g = 1;
+    if (g > steps) g = steps;
+    if (g > 32) g = 32;
+    return (int)g;
+}
+
+int tc_sweep_groups(int64_t nx, int64_t ny, int d) {
+    int kc = d / 64;
+    int64_t units = ((nx + XROWS - 1) / XROWS) * parts_for(kc);
+    int64_t steps = (ny + sweep_sn(kc) - 1) / sweep_sn(kc);
+    int64_t g = sm_count() / units;
+    if (g < 1) g = 1;
+    if (g > steps) g = steps;
+    if (g > 8) g = 8;
+    return (int)g;
+}
+
+cudaError_t tc_launch_fwd(const FwdArgs& a, cudaStream_t st) {
+    const Problem& pr = a.p;
+    constexpr int SN = 128;
+    CUtensorMap mx, my;
+    if (!make_map(&mx, pr.Q, pr.B, pr.d, pr.ldq, XROWS) ||
+        !make_map(&my, pr.P, pr.N, pr.d, pr.ldp, SN))
+        return cudaErrorInvalidValue;
+    TcParams p{};
+    p.nx = pr.B; p.ny = pr.N; p.nq = pr.B;
+    p.kc = pr.d / 64; p.dparts = 1; p.dpc = 0; p.groups = a.groups;
+    p.nstage = smem_plan(p.kc, SN).nstage;
+    p.mask_mode = pr.mask_mode;
+    p.inv_tau = 1.f / pr.tau;
+    p.c1 = 1.4426950408889634f / pr.tau;
+    p.pos_idx = pr.pos_idx;
+    p.part_m = a.part_m; p.part_l = a.part_l; p.pos_logit = a.pos_logit;
+    p.dev_status = a.dev_status;
+    int64_t units = ((pr.B + XROWS - 1) / XROWS) * a.groups;
+    return launch<MODE_FWD, SN>(mx, my, p, units, st);
+}
+
+cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
+    const int kc = a.d / 64;
+    const int sn = sweep_sn(kc);
+    CUtensorMap mx, my;
+    if (!make_map(&mx, a.X, a.nx, a.d, a.ldx, XROWS) || !make_map(&my, a.Y, a.ny, a.d, a.ldy, sn))
+        return cudaErrorInvalidValue;
+    TcParams p{};
+    p.nx = a.nx; p.ny = a.ny; p.nq = 0;
+    p.kc = kc; p.dparts = parts_for(kc); p.dpc = chunks_per_part(kc); p.groups = a.groups;
+    p.nstage = smem_plan(kc, sn).nstage;
+    p.mask_mode = a.mask_mode;
+    p.inv_tau = a.inv_tau;
+    p.c1 = 1.4426950408889634f * a.inv_tau;
+    p.out_scale = a.out_scale;
+    p.row_lse = a.row_lse; p.pos_idx = a.pos_idx;
+    p.out = a.out; p.ldo = a.ldo; p.partial = a.partial;
+    p.dev_status = a.dev_status;
+    int64_t units = ((a.nx + XROWS - 1) / XROWS) * p.dparts * a.groups;
+    if (a.mode == SWEEP_DQ)
+        return sn == 128 ? launch<MODE_DQ, 128>(mx, my, p, units, st)
+                         : launch<MODE_DQ, 64>(mx, my, p, units, st);
+    return sn == 128 ? launch<MODE_DP, 128>(mx, my, p, units, st)
+                     : launch<MODE_DP, 64>(mx, my, p, units, st);
+}
+
+}  // namespace gc

@@ -17,11 +17,18 @@ def rel_err_scalar(got, ref):
     return abs(float(got) - float(ref)) / max(abs(float(ref)), 1e-30)
 
 
-def grad_err(got, ref):
-    """max_ij |got - ref| / max_ij |ref|."""
+def grad_err(got, ref, floor=1e-300):
+    """max_ij |got - ref| / max(max_ij |ref|, floor).  `floor` guards the degenerate cases whose
+    exact gradient is identically zero (e.g. a single passage)."""
     ref = np.asarray(ref, np.float64)
     got = np.asarray(got, np.float64)
-    return float(np.abs(got - ref).max() / max(np.abs(ref).max(), 1e-300))
+    return float(np.abs(got - ref).max() / max(np.abs(ref).max(), floor))
+
+
+def grad_floor(prob):
+    """1e-2 of the largest magnitude a gradient entry can have, max|row| / (B tau)."""
+    big = max(float(np.abs(prob.Q).max()), float(np.abs(prob.P).max()))
+    return 1e-2 * big / (prob.B * prob.tau)
 
 
 def run_build(prob, device="cuda"):
@@ -35,10 +42,13 @@ def run_build(prob, device="cuda"):
 def check_against_oracle(prob, out, ref, tol=None):
     tol = tol or TOL[prob.dtype]
     assert int(out.dev_status.item()) == 0
-    assert rel_err_scalar(out.loss.item(), ref["loss"]) <= tol["loss"]
+    # relative to the loss, or to the size of its terms when the loss itself is ~0 (N = 1)
+    loss_scale = max(abs(ref["loss"]), 1e-3 * float(np.abs(ref["row_lse"]).mean()), 1e-6)
+    assert abs(out.loss.item() - ref["loss"]) <= tol["loss"] * loss_scale
     lse = out.row_lse.cpu().numpy().astype(np.float64)
     assert np.abs(lse - ref["row_lse"]).max() <= tol["lse"] * max(1.0, np.abs(ref["row_lse"]).max())
     pl = out.pos_logit.cpu().numpy().astype(np.float64)
     assert np.abs(pl - ref["pos_logit"]).max() <= tol["lse"] * max(1.0, np.abs(ref["pos_logit"]).max())
-    assert grad_err(out.dQ.cpu().numpy(), ref["dQ"]) <= tol["grad"]
-    assert grad_err(out.dP.cpu().numpy(), ref["dP"]) <= tol["grad"]
+    floor = grad_floor(prob)
+    assert grad_err(out.dQ.cpu().numpy(), ref["dQ"], floor) <= tol["grad"]
+    assert grad_err(out.dP.cpu().numpy(), ref["dP"], floor) <= tol["grad"]

@@ -233,12 +233,13 @@ def test_self_mask_is_exact_zero(binding, dtype, d):
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 def test_mask_does_not_leak(binding, oracle, dtype):
-    """Huge diagonal logits (about +64): a single unmasked diagonal entry would move row_lse by
-    tens.  Sizes are not multiples of any tile."""
+    """Rows of norm 8 in random directions, shared between Q and P: every diagonal logit is 64
+    while the off-diagonal ones stay below about 30, so a single unmasked diagonal entry would
+    move that row's lse by tens.  Sizes are not multiples of any tile."""
     n, d = 333, 64
     rng = np.random.default_rng(5)
-    X = (rng.standard_normal((n, d)) * 0.1).astype(np.float32)
-    X[:, 0] = 8.0
+    X = rng.standard_normal((n, d))
+    X = (8.0 * X / np.linalg.norm(X, axis=1, keepdims=True)).astype(np.float32)
     prob = inputs._finish("leak", X, X, ((np.arange(n) + 1) % n).astype(np.int32), 1.0,
                           inputs.MASK_SELF, dtype, shared=True)
     out = run_build(prob)
