@@ -6,16 +6,21 @@
 //   DQ   (Eq. 5)    x = 128 queries,  y streams passages: W = exp(S - lse_x) - onehot, acc += W Y
 //   DP   (Eq. 6-7)  x = 128 passages, y streams queries:  W = exp(S - lse_y) - onehot, acc += W Y
 //
-// The stationary tile X (128 x d) stays resident in shared memory; Y arrives in (SN x 64)
-// chunks through an mbarrier ring.  S tiles (128 x SN, fp32) are double buffered in tensor
+// The stationary tile X (128 x d) stays resident in shared memory when d <= 512; for wider rows
+// only its first 6 column chunks stay and the others are re-streamed every step, which leaves
+// room for a ring of eight 16 KB stages: the load -> MMA -> release chain of a stage is about
+// 1500-2000 cycles long, so the bytes in flight, not the L2 bandwidth, bound the MMA rate.
+// Y arrives in (SN x 64) chunks through the same mbarrier ring.  S tiles (128 x SN, fp32) are double buffered in tensor
 // memory so the MMAs of step t+1 run while the softmax warps work on step t.  W is written
 // back over its S buffer as packed bf16 and used as the A operand (from tensor memory) of the
 // second MMA, whose B operand is the same Y chunk read MN-major.  An accumulator of 128 x 768
 // fp32 does not fit the 512 tensor-memory columns, so wide rows are split into column parts
 // (at most 384 columns each), one CTA per part.  S is never written to global memory.
 //
-// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = MMA issuer (and tensor-memory
-// allocator), warps 2..5 = softmax / epilogue, one thread per tile row.
+// Warp roles (288 threads): warps 0..3 = TMA producers (a single thread sustains only one bulk
+// tensor request per ~270 cycles, so the ring stages are dealt out to four issuing warps),
+// warp 4 = MMA issuer (and tensor-memory allocator), warps 5..8 = softmax / epilogue, one
+// thread per tile row.
 // Every wait is bounded: on a timeout the CTA raises GC_DEV_WAIT_LIMIT, drains and exits.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -30,8 +35,11 @@ namespace {
 constexpr int XROWS = 128;                 // rows of the stationary tile = MMA M
 constexpr int CHUNK_BYTES_PER_ROW = 128;   // 64 bf16 = one swizzle row
 constexpr uint32_t X_CHUNK_BYTES = XROWS * CHUNK_BYTES_PER_ROW;
-constexpr int NTHREADS = 192;
+constexpr int NPROD = 4;                   // TMA producer warps
+constexpr int MMA_WARP = NPROD;
+constexpr int NTHREADS = 32 * (NPROD + 5);
 constexpr int MAX_STAGES = 8;
+constexpr uint32_t STAGE_BYTES = 16384;    // one X chunk (128 rows) or 128 Y rows of one chunk
 constexpr int TMEM_COLS = 512;
 constexpr int MAX_D = 768;
 constexpr int MAX_PART_CHUNKS = 6;         // 384 accumulator columns
@@ -41,10 +49,27 @@ constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 
 enum { MODE_FWD = 0, MODE_DQ = 1, MODE_DP = 2 };
 
+// Optional diagnostics (-DGC_TC_TRACE): cycles each role spends waiting, summed over CTAs.
+#ifdef GC_TC_TRACE
+enum { TR_MMA_TOTAL, TR_MMA_WAIT_Y, TR_MMA_WAIT_W, TR_SM_TOTAL, TR_SM_WAIT_S, TR_SM_EPI,
+       TR_PROD_TOTAL, TR_PROD_WAIT, TR_CTAS, TR_MMA_ISSUE, TR_MMA_COMMIT, TR_ACC_ISSUE, TR_ACC_COMMIT, TR_SFULL_COMMIT, TR_COUNT };
+__device__ unsigned long long g_trace[3][TR_COUNT];
+#define TR_DECL(v) long long v = 0
+#define TR_BEGIN(v) long long v##_t0 = clock64()
+#define TR_END(v) v += clock64() - v##_t0
+#define TR_ADD(mode, slot, v) atomicAdd(&g_trace[mode][slot], (unsigned long long)(v))
+#else
+#define TR_DECL(v)
+#define TR_BEGIN(v)
+#define TR_END(v)
+#define TR_ADD(mode, slot, v)
+#endif
+
 struct TcParams {
     int64_t nx, ny;
     int64_t nq;               // number of queries B (pitch of the forward partial arrays)
     int kc;                   // d / 64
+    int xres;                 // X chunks [0, xres) stay resident, [xres, kc) are streamed
     int dparts, dpc;          // accumulator column parts and chunks per part
     int groups;
     int nstage;
@@ -119,6 +144,18 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
         : "memory");
 }
+// True on exactly one lane of a converged warp.  The surrounding loops run on all 32 lanes with
+// warp-uniform values, so that addresses and descriptors can stay in uniform registers, which
+// is where bulk-tensor and tcgen05 instructions read them from.
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "elect.sync _|P, 0xffffffff;\n\t"
+        "selp.u32 %0, 1, 0, P;\n\t}"
+        : "=r"(pred));
+    return pred != 0;
+}
 __device__ __forceinline__ void tc_fence_before() {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }
@@ -129,24 +166,40 @@ __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
                  ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
-                                       uint32_t idesc, uint32_t accumulate) {
+// Shared-memory matrix descriptors for 128-byte-swizzled tiles with 128-byte rows.  The high
+// word is constant: stride between 8-row groups = 1024 bytes (>> 4), descriptor version 1,
+// layout type 2 (SWIZZLE_128B).  The low word holds the start address (>> 4) and, in bits 16-29,
+// the leading byte offset (>> 4): the distance between 64-element atoms along M/N of an
+// MN-major operand (ignored for K-major operands).  A K-major operand advances 32 bytes
+// (low word + 2) per K = 16; an MN-major operand advances 16 rows = 2048 bytes (low word + 128).
+constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
+    return ((addr >> 4) & 0x3FFFu) | ((lbo_bytes >> 4) << 16);
+}
+// D[tmem] (+)= A[smem] * B[smem].  The issuing thread is alone on its scheduler, so every scalar
+// instruction spent per MMA shows up as idle tensor time: keep the operands precomputed.
+template <bool ACC>
+__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo,
+                                       uint32_t idesc) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 da, {%1, %4};\n\t"
+        "mov.b64 db, {%2, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(DESC_HI), "n"(ACC ? 1 : 0)
         : "memory");
 }
 // D[tmem] (+)= A[tmem] * B[smem]
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
-                                       uint32_t idesc, uint32_t accumulate) {
+template <bool ACC>
+__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo,
+                                       uint32_t idesc) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "mov.b64 db, {%2, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(DESC_HI), "n"(ACC ? 1 : 0)
         : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
@@ -183,19 +236,6 @@ __device__ __forceinline__ float ex2(float x) {
     return y;
 }
 
-// Shared-memory matrix descriptor for 128-byte-swizzled tiles whose rows are 128 bytes:
-// start address and stride-between-8-row-groups (1024 bytes) in 16-byte units, descriptor
-// version 1, layout type 2 (SWIZZLE_128B).  K-major operands step 32 bytes per K = 16 inside the
-// swizzle row; MN-major operands step 16 rows (2048 bytes) per K = 16.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFF);
-    d |= (uint64_t)(1024 >> 4) << 16;     // leading byte offset (next 64-element MN atom; unused)
-    d |= (uint64_t)(1024 >> 4) << 32;     // stride byte offset: 8 rows x 128 bytes
-    d |= (uint64_t)1 << 46;               // descriptor version
-    d |= (uint64_t)2 << 61;               // SWIZZLE_128B
-    return d;
-}
 // Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, M = 128.
 __device__ __forceinline__ uint32_t instr_desc(int n, bool b_mn_major) {
     uint32_t d = 0;
@@ -237,9 +277,11 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     __shared__ int abort_s;
     volatile int* abort_flag = &abort_s;
 
-    constexpr uint32_t STAGE_BYTES = SN * CHUNK_BYTES_PER_ROW;
+    constexpr uint32_t Y_CHUNK_BYTES = SN * CHUNK_BYTES_PER_ROW;
+    constexpr int YPER = 128 / SN;                      // Y chunks that share one ring stage
     constexpr uint32_t S_COL0 = TMEM_COLS - 2 * SN;     // S buffers sit at the top columns
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // warp-uniform
+    const int lane = threadIdx.x & 31;
 
     // work item: (x tile, column part, part of the streamed range)
     int unit = blockIdx.x;
@@ -257,7 +299,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t x_smem = base;
-    const uint32_t y_smem = base + (uint32_t)p.kc * X_CHUNK_BYTES;
+    const uint32_t y_smem = base + (uint32_t)p.xres * X_CHUNK_BYTES;   // the ring
 
     if (threadIdx.x == 0) {
         abort_s = 0;
@@ -273,7 +315,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
         mbar_init(smem_u32(&bars.acc_full), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {
+    if (warp == MMA_WARP) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -283,43 +325,115 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     tc_fence_after();
     const uint32_t tmem = tmem_base_s;
 
-    if (warp == 0) {
-        // ------------------------------ TMA producer ------------------------------------------
-        if (lane == 0) {
-            mbar_expect_tx(smem_u32(&bars.x_full), (uint32_t)p.kc * X_CHUNK_BYTES);
-            for (int c = 0; c < p.kc; ++c)
-                tma_load_2d(x_smem + c * X_CHUNK_BYTES, &mapX, c * 64, (int)x0,
-                            smem_u32(&bars.x_full));
-            int stage = 0;
-            uint32_t phase = 0;
+    if (warp < NPROD) {
+        // ------------------------------ TMA producers -----------------------------------------
+        // Chunk number n of the stream goes to ring stage n % nstage; a stage always belongs to
+        // the same producer warp (stage % NPROD), which therefore sees its phases in order.
+        {   // all 32 lanes run the loop; one elected lane issues
+            if (warp == 0 && elect_one())
+                mbar_expect_tx(smem_u32(&bars.x_full), (uint32_t)p.xres * X_CHUNK_BYTES);
+            for (int c = warp; c < p.xres; c += NPROD)
+                if (elect_one())
+                    tma_load_2d(x_smem + c * X_CHUNK_BYTES, &mapX, c * 64, (int)x0,
+                                smem_u32(&bars.x_full));
+            int next = 0;
+            uint32_t next_phase = 0;
             bool ok = true;
-            auto load_chunk = [&](int chunk, int64_t row) {
-                if (!ok) return;
-                if (!mbar_wait(smem_u32(&bars.y_empty[stage]), phase ^ 1u, abort_flag)) {
+            TR_DECL(tr_wait);
+            TR_BEGIN(tr_total);
+            // Claims the next ring stage if it belongs to this warp: waits until the MMAs that
+            // read its previous contents have completed.  Returns the stage or -1.
+            auto acquire = [&]() -> int {
+                const int stage = next;
+                const uint32_t phase = next_phase;
+                if (++next == p.nstage) { next = 0; next_phase ^= 1u; }
+                if (!ok || (stage & (NPROD - 1)) != warp) return -1;
+                TR_BEGIN(tr_wait);
+                const bool got = mbar_wait(smem_u32(&bars.y_empty[stage]), phase ^ 1u, abort_flag);
+                TR_END(tr_wait);
+                if (!got) {
                     ok = false;
-                    return;
+                    return -1;
                 }
-                uint32_t full = smem_u32(&bars.y_full[stage]);
-                mbar_expect_tx(full, STAGE_BYTES);
-                tma_load_2d(y_smem + stage * STAGE_BYTES, &mapY, chunk * 64, (int)row, full);
-                if (++stage == p.nstage) { stage = 0; phase ^= 1u; }
+                return stage;
+            };
+            auto load_y = [&](int chunk0, int count, int64_t row) {
+                const int stage = acquire();
+                if (stage < 0) return;
+                const uint32_t full = smem_u32(&bars.y_full[stage]);
+                if (elect_one()) {
+                    mbar_expect_tx(full, (uint32_t)count * Y_CHUNK_BYTES);
+                    for (int i = 0; i < count; ++i)
+                        tma_load_2d(y_smem + stage * STAGE_BYTES + i * Y_CHUNK_BYTES, &mapY,
+                                    (chunk0 + i) * 64, (int)row, full);
+                }
+            };
+            auto load_x = [&](int chunk) {
+                const int stage = acquire();
+                if (stage < 0) return;
+                const uint32_t full = smem_u32(&bars.y_full[stage]);
+                if (elect_one()) {
+                    mbar_expect_tx(full, X_CHUNK_BYTES);
+                    tma_load_2d(y_smem + stage * STAGE_BYTES, &mapX, chunk * 64, (int)x0, full);
+                }
             };
             for (int t = 0; t <= T && ok; ++t) {
-                if (t < T)
-                    for (int c = 0; c < p.kc; ++c) load_chunk(c, (lo + t) * SN);
-                if (MODE != MODE_FWD && t >= 1)
-                    for (int c = 0; c < c_count; ++c) load_chunk(c_begin + c, (lo + t - 1) * SN);
+                if (t < T) {
+                    for (int c = 0; c < p.kc; ++c) {
+                        if (c % YPER == 0) load_y(c, min(YPER, p.kc - c), (lo + t) * SN);
+                        if (c >= p.xres) load_x(c);
+                    }
+                }
+                if (MODE != MODE_FWD && t >= 1) {
+                    for (int c = 0; c < c_count; c += YPER)
+                        load_y(c_begin + c, min(YPER, c_count - c), (lo + t - 1) * SN);
+                }
             }
+#ifdef GC_TC_TRACE
+            if (warp == 0 && lane == 0) {
+                TR_ADD(MODE, TR_PROD_TOTAL, clock64() - tr_total_t0);
+                TR_ADD(MODE, TR_PROD_WAIT, tr_wait);
+                TR_ADD(MODE, TR_CTAS, 1);
+            }
+#endif
         }
-    } else if (warp == 1) {
+    } else if (warp == MMA_WARP) {
         // ------------------------------ MMA issuer ----------------------------------------------
-        if (lane == 0) {
+        {   // all 32 lanes run the loop; one elected lane issues the MMAs and commits
             const uint32_t idesc_s = instr_desc(SN, false);
-            const uint32_t idesc_acc = instr_desc(64, true);
-            int stage = 0;
-            uint32_t phase = 0;
+            const uint32_t idesc_acc64 = instr_desc(64, true);
+            const uint32_t idesc_acc128 = instr_desc(128, true);
+            const uint32_t x_lo = desc_lo(x_smem, 0);
+            const uint32_t ring_lo = desc_lo(y_smem, Y_CHUNK_BYTES);   // LBO: next chunk of a stage
+            constexpr uint32_t STAGE_LO = STAGE_BYTES >> 4, YCH_LO = Y_CHUNK_BYTES >> 4,
+                               XCH_LO = X_CHUNK_BYTES >> 4;
+            int next = 0;
+            uint32_t next_phase = 0;
+            TR_DECL(tr_wy);
+            TR_DECL(tr_ww);
+            TR_DECL(tr_is);
+            TR_DECL(tr_cm);
+            TR_DECL(tr_ai);
+            TR_DECL(tr_ac);
+            TR_DECL(tr_sf);
+            TR_BEGIN(tr_total);
             bool ok = mbar_wait(smem_u32(&bars.x_full), 0, abort_flag);
             tc_fence_after();
+            // Waits for the next ring stage to be filled; returns its index or -1.
+            auto next_stage = [&]() -> int {
+                const int stage = next;
+                const uint32_t phase = next_phase;
+                if (++next == p.nstage) { next = 0; next_phase ^= 1u; }
+                TR_BEGIN(tr_wy);
+                const bool got = mbar_wait(smem_u32(&bars.y_full[stage]), phase, abort_flag);
+                TR_END(tr_wy);
+                if (!got) {
+                    ok = false;
+                    return -1;
+                }
+                tc_fence_after();
+                return stage;
+            };
             for (int t = 0; t <= T && ok; ++t) {
                 if (t < T) {
                     const int b = t & 1;
@@ -329,43 +443,79 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         tc_fence_after();
                     }
                     const uint32_t d_tmem = tmem + S_COL0 + b * SN;
+                    int ys = 0;
                     for (int c = 0; c < p.kc && ok; ++c) {
-                        ok = mbar_wait(smem_u32(&bars.y_full[stage]), phase, abort_flag);
+                        const int sub = (YPER == 1) ? 0 : (c & (YPER - 1));
+                        if (sub == 0) ys = next_stage();
                         if (!ok) break;
-                        tc_fence_after();
-                        const uint32_t xa = x_smem + c * X_CHUNK_BYTES;
-                        const uint32_t yb = y_smem + stage * STAGE_BYTES;
-#pragma unroll
-                        for (int k = 0; k < 4; ++k)
-                            mma_ss(d_tmem, smem_desc(xa + k * 32), smem_desc(yb + k * 32), idesc_s,
-                                   (c | k) != 0);
-                        tc_commit(smem_u32(&bars.y_empty[stage]));
-                        if (++stage == p.nstage) { stage = 0; phase ^= 1u; }
+                        int xs = -1;
+                        uint32_t xa = x_lo + c * XCH_LO;
+                        if (c >= p.xres) {
+                            xs = next_stage();
+                            if (!ok) break;
+                            xa = ring_lo + xs * STAGE_LO;
+                        }
+                        const uint32_t yb = ring_lo + ys * STAGE_LO + sub * YCH_LO;
+                        TR_BEGIN(tr_is);
+                        if (elect_one()) {
+                            if (c == 0) mma_ss<false>(d_tmem, xa, yb, idesc_s);
+                            else        mma_ss<true>(d_tmem, xa, yb, idesc_s);
+                            mma_ss<true>(d_tmem, xa + 2, yb + 2, idesc_s);
+                            mma_ss<true>(d_tmem, xa + 4, yb + 4, idesc_s);
+                            mma_ss<true>(d_tmem, xa + 6, yb + 6, idesc_s);
+                            if (xs >= 0) tc_commit(smem_u32(&bars.y_empty[xs]));
+                            if (sub == YPER - 1 || c == p.kc - 1)
+                                tc_commit(smem_u32(&bars.y_empty[ys]));
+                        }
+                        TR_END(tr_is);
                     }
                     if (!ok) break;
-                    tc_commit(smem_u32(&bars.s_full[b]));
+                    TR_BEGIN(tr_sf);
+                    if (elect_one()) tc_commit(smem_u32(&bars.s_full[b]));
+                    TR_END(tr_sf);
                 }
                 if (MODE != MODE_FWD && t >= 1) {
                     const int u = t - 1, b = u & 1;
+                    TR_BEGIN(tr_ww);
                     ok = mbar_wait(smem_u32(&bars.w_full[b]), (u >> 1) & 1, abort_flag);
+                    TR_END(tr_ww);
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t w_tmem = tmem + S_COL0 + b * SN;
-                    for (int c = 0; c < c_count && ok; ++c) {
-                        ok = mbar_wait(smem_u32(&bars.y_full[stage]), phase, abort_flag);
+                    // one ring stage per iteration: YPER chunks = 64 * YPER accumulator columns
+                    for (int c = 0; c < c_count && ok; c += YPER) {
+                        const int ys = next_stage();
                         if (!ok) break;
-                        tc_fence_after();
-                        const uint32_t yb = y_smem + stage * STAGE_BYTES;
+                        const uint32_t yb = ring_lo + ys * STAGE_LO;
+                        const uint32_t d_tmem = tmem + c * 64;
+                        const bool wide = (YPER == 2) && (c + 1 < c_count);
+                        const uint32_t idesc = wide ? idesc_acc128 : idesc_acc64;
+                        TR_BEGIN(tr_ai);
+                        if (elect_one()) {
+                            if (u == 0) mma_ts<false>(d_tmem, w_tmem, yb, idesc);
+                            else        mma_ts<true>(d_tmem, w_tmem, yb, idesc);
 #pragma unroll
-                        for (int k = 0; k < SN / 16; ++k)
-                            mma_ts(tmem + c * 64, w_tmem + k * 8, smem_desc(yb + k * 2048),
-                                   idesc_acc, (u | k) != 0);
-                        tc_commit(smem_u32(&bars.y_empty[stage]));
-                        if (++stage == p.nstage) { stage = 0; phase ^= 1u; }
+                            for (int k = 1; k < SN / 16; ++k)
+                                mma_ts<true>(d_tmem, w_tmem + k * 8, yb + k * 128, idesc);
+                            tc_commit(smem_u32(&bars.y_empty[ys]));
+                        }
+                        TR_END(tr_ai);
                     }
                 }
             }
-            if (ok && MODE != MODE_FWD) tc_commit(smem_u32(&bars.acc_full));
+            if (ok && MODE != MODE_FWD && elect_one()) tc_commit(smem_u32(&bars.acc_full));
+#ifdef GC_TC_TRACE
+            if (lane == 0) {
+            TR_ADD(MODE, TR_MMA_TOTAL, clock64() - tr_total_t0);
+            TR_ADD(MODE, TR_MMA_WAIT_Y, tr_wy);
+            TR_ADD(MODE, TR_MMA_WAIT_W, tr_ww);
+            TR_ADD(MODE, TR_MMA_ISSUE, tr_is);
+            TR_ADD(MODE, TR_MMA_COMMIT, tr_cm);
+            TR_ADD(MODE, TR_ACC_ISSUE, tr_ai);
+            TR_ADD(MODE, TR_ACC_COMMIT, tr_ac);
+            TR_ADD(MODE, TR_SFULL_COMMIT, tr_sf);
+            }
+#endif
         }
     } else {
         // ------------------------------ softmax / epilogue warps --------------------------------
@@ -375,13 +525,18 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         const bool self_mask = (p.mask_mode == GC_MASK_SELF);
         bool ok = true;
+        TR_DECL(tr_ws);
+        TR_DECL(tr_epi);
+        TR_BEGIN(tr_total);
 
         if (MODE == MODE_FWD) {
             float m = -INFINITY, l = 0.f;
             const int32_t pos_x = (x < p.nx) ? p.pos_idx[x] : -1;
             for (int t = 0; t < T; ++t) {
                 const int b = t & 1;
+                TR_BEGIN(tr_ws);
                 ok = mbar_wait(smem_u32(&bars.s_full[b]), (t >> 1) & 1, abort_flag);
+                TR_END(tr_ws);
                 if (!ok) break;
                 tc_fence_after();
                 const int64_t y0 = (lo + t) * SN;
@@ -456,7 +611,9 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         pos_y[cb] = (y < p.ny) ? p.pos_idx[y] : -1;
                     }
                 }
+                TR_BEGIN(tr_ws);
                 ok = mbar_wait(smem_u32(&bars.s_full[b]), (t >> 1) & 1, abort_flag);
+                TR_END(tr_ws);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t sbuf = tmem + lane_addr + S_COL0 + b * SN;
@@ -523,6 +680,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 if (lane == 0) mbar_arrive(smem_u32(&bars.w_full[b]));
             }
             // epilogue: accumulator columns of this part -> global memory
+            TR_BEGIN(tr_epi);
             if (ok) ok = mbar_wait(smem_u32(&bars.acc_full), 0, abort_flag);
             if (ok) {
                 tc_fence_after();
@@ -547,7 +705,15 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     }
                 }
             }
+            TR_END(tr_epi);
         }
+#ifdef GC_TC_TRACE
+        if (q == 0 && lane == 0) {
+            TR_ADD(MODE, TR_SM_TOTAL, clock64() - tr_total_t0);
+            TR_ADD(MODE, TR_SM_WAIT_S, tr_ws);
+            TR_ADD(MODE, TR_SM_EPI, tr_epi);
+        }
+#endif
     }
 
     // ------------------------------ teardown ------------------------------------------------------
@@ -560,7 +726,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
         if (threadIdx.x == 0 && p.dev_status) atomicOr(p.dev_status, GC_DEV_WAIT_LIMIT);
         __syncthreads();
     }
-    if (warp == 1) {
+    if (warp == MMA_WARP) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
                      ::"r"(tmem), "r"((uint32_t)TMEM_COLS) : "memory");
@@ -611,17 +777,19 @@ int chunks_per_part(int kc) { int n = parts_for(kc); return (kc + n - 1) / n; }
 // 128-column S buffers, else 64.
 int sweep_sn(int kc) { return chunks_per_part(kc) * 64 + 256 <= TMEM_COLS ? 128 : 64; }
 
-struct SmemPlan { int nstage; size_t dynamic_bytes; };
+struct SmemPlan { int xres; int nstage; size_t dynamic_bytes; };
 
-SmemPlan smem_plan(int kc, int sn) {
-    size_t xbytes = (size_t)kc * X_CHUNK_BYTES;
-    size_t stage = (size_t)sn * CHUNK_BYTES_PER_ROW;
-    size_t avail = SMEM_LIMIT - SMEM_STATIC_RESERVE - 1024 - xbytes;
-    int ns = (int)(avail / stage);
-    if (ns > MAX_STAGES) ns = MAX_STAGES;
+// Rows up to 512 wide keep the whole X tile resident; wider rows keep 6 chunks so that the ring
+// still has eight stages.
+SmemPlan smem_plan(int kc) {
     SmemPlan sp;
+    sp.xres = kc <= 8 ? kc : 6;
+    size_t xbytes = (size_t)sp.xres * X_CHUNK_BYTES;
+    size_t avail = SMEM_LIMIT - SMEM_STATIC_RESERVE - 1024 - xbytes;
+    int ns = (int)(avail / STAGE_BYTES);
+    if (ns > MAX_STAGES) ns = MAX_STAGES;
     sp.nstage = ns;
-    sp.dynamic_bytes = 1024 + xbytes + (size_t)ns * stage;
+    sp.dynamic_bytes = 1024 + xbytes + (size_t)ns * STAGE_BYTES;
     // keep one CTA per SM (each CTA allocates all 512 tensor-memory columns)
     if (sp.dynamic_bytes < 120 * 1024) sp.dynamic_bytes = 120 * 1024;
     return sp;
@@ -630,7 +798,7 @@ SmemPlan smem_plan(int kc, int sn) {
 template <int MODE, int SN>
 cudaError_t launch(const CUtensorMap& mx, const CUtensorMap& my, const TcParams& p, int64_t units,
                    cudaStream_t st) {
-    SmemPlan sp = smem_plan(p.kc, SN);
+    SmemPlan sp = smem_plan(p.kc);
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(tc_kernel<MODE, SN>,
@@ -644,6 +812,17 @@ cudaError_t launch(const CUtensorMap& mx, const CUtensorMap& my, const TcParams&
 }
 
 }  // namespace
+
+#ifdef GC_TC_TRACE
+extern "C" int gc_debug_trace(unsigned long long* out, int clear) {
+    if (out && cudaMemcpyFromSymbol(out, g_trace, sizeof(g_trace)) != cudaSuccess) return 1;
+    if (clear) {
+        static unsigned long long zero[3][TR_COUNT] = {};
+        if (cudaMemcpyToSymbol(g_trace, zero, sizeof(zero)) != cudaSuccess) return 1;
+    }
+    return 0;
+}
+#endif
 
 bool tc_supported(int64_t B, int64_t N, int d, int dtype) {
     (void)B; (void)N;
@@ -681,7 +860,8 @@ cudaError_t tc_launch_fwd(const FwdArgs& a, cudaStream_t st) {
     TcParams p{};
     p.nx = pr.B; p.ny = pr.N; p.nq = pr.B;
     p.kc = pr.d / 64; p.dparts = 1; p.dpc = 0; p.groups = a.groups;
-    p.nstage = smem_plan(p.kc, SN).nstage;
+    p.nstage = smem_plan(p.kc).nstage;
+    p.xres = smem_plan(p.kc).xres;
     p.mask_mode = pr.mask_mode;
     p.inv_tau = 1.f / pr.tau;
     p.c1 = 1.4426950408889634f / pr.tau;
@@ -701,7 +881,8 @@ cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     TcParams p{};
     p.nx = a.nx; p.ny = a.ny; p.nq = 0;
     p.kc = kc; p.dparts = parts_for(kc); p.dpc = chunks_per_part(kc); p.groups = a.groups;
-    p.nstage = smem_plan(kc, sn).nstage;
+    p.nstage = smem_plan(kc).nstage;
+    p.xres = smem_plan(kc).xres;
     p.mask_mode = a.mask_mode;
     p.inv_tau = a.inv_tau;
     p.c1 = 1.4426950408889634f * a.inv_tau;
