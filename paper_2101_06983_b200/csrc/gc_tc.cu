@@ -17,10 +17,10 @@
 // fp32 does not fit the 512 tensor-memory columns, so wide rows are split into column parts
 // (at most 384 columns each), one CTA per part.  S is never written to global memory.
 //
-// Warp roles (288 threads): warps 0..3 = TMA producers (a single thread sustains only one bulk
-// tensor request per ~270 cycles, so the ring stages are dealt out to four issuing warps),
-// warp 4 = MMA issuer (and tensor-memory allocator), warps 5..8 = softmax / epilogue, one
-// thread per tile row.
+// Warp roles (416 threads): warps 0..3 = TMA producers (the ring stages are dealt out to four
+// issuing warps), warp 4 = MMA issuer (and tensor-memory allocator), warps 5..12 = softmax /
+// epilogue: two warps per tensor-memory lane quarter, each owning half of the tile's columns,
+// one thread per tile row.
 // Every wait is bounded: on a timeout the CTA raises GC_DEV_WAIT_LIMIT, drains and exits.
 #include <cuda.h>
 #include <cuda_bf16.h>
@@ -37,7 +37,8 @@ constexpr int CHUNK_BYTES_PER_ROW = 128;   // 64 bf16 = one swizzle row
 constexpr uint32_t X_CHUNK_BYTES = XROWS * CHUNK_BYTES_PER_ROW;
 constexpr int NPROD = 4;                   // TMA producer warps
 constexpr int MMA_WARP = NPROD;
-constexpr int NTHREADS = 32 * (NPROD + 5);
+constexpr int NSOFT = 8;                   // softmax / epilogue warps
+constexpr int NTHREADS = 32 * (NPROD + 1 + NSOFT);
 constexpr int MAX_STAGES = 8;
 constexpr uint32_t STAGE_BYTES = 16384;    // one X chunk (128 rows) or 128 Y rows of one chunk
 constexpr int TMEM_COLS = 512;
@@ -267,7 +268,7 @@ struct Bars {
 // ---------------------------------------------------------------------------------------------
 // The sweep kernel
 // ---------------------------------------------------------------------------------------------
-template <int MODE, int SN>
+template <int MODE, int SN, int NBUF>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
           const TcParams p) {
@@ -279,7 +280,9 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
 
     constexpr uint32_t Y_CHUNK_BYTES = SN * CHUNK_BYTES_PER_ROW;
     constexpr int YPER = 128 / SN;                      // Y chunks that share one ring stage
-    constexpr uint32_t S_COL0 = TMEM_COLS - 2 * SN;     // S buffers sit at the top columns
+    constexpr uint32_t S_COL0 = TMEM_COLS - NBUF * SN;  // S buffers sit at the top columns
+    constexpr int LAG = NBUF - 1;                       // steps between S(t) and acc(t) issue
+    constexpr int BSH = (NBUF == 2) ? 1 : 0;            // log2(NBUF)
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // warp-uniform
     const int lane = threadIdx.x & 31;
 
@@ -310,7 +313,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&bars.s_full[b]), 1);
-            mbar_init(smem_u32(&bars.w_full[b]), 4);      // one arrival per softmax warp
+            mbar_init(smem_u32(&bars.w_full[b]), NSOFT);  // one arrival per softmax warp
         }
         mbar_init(smem_u32(&bars.acc_full), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -377,16 +380,16 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     tma_load_2d(y_smem + stage * STAGE_BYTES, &mapX, chunk * 64, (int)x0, full);
                 }
             };
-            for (int t = 0; t <= T && ok; ++t) {
+            for (int t = 0; t < T + LAG && ok; ++t) {
                 if (t < T) {
                     for (int c = 0; c < p.kc; ++c) {
                         if (c % YPER == 0) load_y(c, min(YPER, p.kc - c), (lo + t) * SN);
                         if (c >= p.xres) load_x(c);
                     }
                 }
-                if (MODE != MODE_FWD && t >= 1) {
+                if (MODE != MODE_FWD && t >= LAG) {
                     for (int c = 0; c < c_count; c += YPER)
-                        load_y(c_begin + c, min(YPER, c_count - c), (lo + t - 1) * SN);
+                        load_y(c_begin + c, min(YPER, c_count - c), (lo + t - LAG) * SN);
                 }
             }
 #ifdef GC_TC_TRACE
@@ -431,14 +434,14 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     ok = false;
                     return -1;
                 }
-                tc_fence_after();
-                return stage;
+                return stage;   // filled by TMA (async proxy), read by the MMA: the mbarrier orders it
             };
-            for (int t = 0; t <= T && ok; ++t) {
+            for (int t = 0; t < T + LAG && ok; ++t) {
                 if (t < T) {
-                    const int b = t & 1;
-                    if (MODE == MODE_FWD && t >= 2) {
-                        ok = mbar_wait(smem_u32(&bars.w_full[b]), ((t - 2) >> 1) & 1, abort_flag);
+                    const int b = t & (NBUF - 1);
+                    if (MODE == MODE_FWD && t >= NBUF) {
+                        ok = mbar_wait(smem_u32(&bars.w_full[b]), ((t - NBUF) >> BSH) & 1,
+                                       abort_flag);
                         if (!ok) break;
                         tc_fence_after();
                     }
@@ -474,10 +477,10 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     if (elect_one()) tc_commit(smem_u32(&bars.s_full[b]));
                     TR_END(tr_sf);
                 }
-                if (MODE != MODE_FWD && t >= 1) {
-                    const int u = t - 1, b = u & 1;
+                if (MODE != MODE_FWD && t >= LAG) {
+                    const int u = t - LAG, b = u & (NBUF - 1);
                     TR_BEGIN(tr_ww);
-                    ok = mbar_wait(smem_u32(&bars.w_full[b]), (u >> 1) & 1, abort_flag);
+                    ok = mbar_wait(smem_u32(&bars.w_full[b]), (u >> BSH) & 1, abort_flag);
                     TR_END(tr_ww);
                     if (!ok) break;
                     tc_fence_after();
@@ -492,11 +495,15 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         const uint32_t idesc = wide ? idesc_acc128 : idesc_acc64;
                         TR_BEGIN(tr_ai);
                         if (elect_one()) {
+                            // k-steps of the first column half read W at columns 8 k, those of
+                            // the second half at SN/2 + 8 (k - KH)
+                            constexpr int KH = SN / 32;
                             if (u == 0) mma_ts<false>(d_tmem, w_tmem, yb, idesc);
                             else        mma_ts<true>(d_tmem, w_tmem, yb, idesc);
 #pragma unroll
                             for (int k = 1; k < SN / 16; ++k)
-                                mma_ts<true>(d_tmem, w_tmem + k * 8, yb + k * 128, idesc);
+                                mma_ts<true>(d_tmem, w_tmem + (k / KH) * (SN / 2) + (k % KH) * 8,
+                                             yb + k * 128, idesc);
                             tc_commit(smem_u32(&bars.y_empty[ys]));
                         }
                         TR_END(tr_ai);
@@ -520,6 +527,9 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     } else {
         // ------------------------------ softmax / epilogue warps --------------------------------
         const int q = warp & 3;                        // tensor-memory lane quarter of this warp
+        const int half = (warp - (NPROD + 1)) >> 2;    // which half of the tile's columns
+        constexpr int CB_PER = SN / 64;                // 32-column blocks per half
+        const int cb0 = half * CB_PER;
         const int row = q * 32 + lane;
         const int64_t x = x0 + row;
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
@@ -533,15 +543,15 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             float m = -INFINITY, l = 0.f;
             const int32_t pos_x = (x < p.nx) ? p.pos_idx[x] : -1;
             for (int t = 0; t < T; ++t) {
-                const int b = t & 1;
+                const int b = t & (NBUF - 1);
                 TR_BEGIN(tr_ws);
-                ok = mbar_wait(smem_u32(&bars.s_full[b]), (t >> 1) & 1, abort_flag);
+                ok = mbar_wait(smem_u32(&bars.s_full[b]), (t >> BSH) & 1, abort_flag);
                 TR_END(tr_ws);
                 if (!ok) break;
                 tc_fence_after();
                 const int64_t y0 = (lo + t) * SN;
 #pragma unroll 1
-                for (int cb = 0; cb < SN / 32; ++cb) {
+                for (int cb = cb0; cb < cb0 + CB_PER; ++cb) {
                     uint32_t v[32];
                     tmem_ld32(tmem + lane_addr + S_COL0 + b * SN + cb * 32, v);
                     tmem_ld_wait();
@@ -585,9 +595,11 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bars.w_full[b]));
             }
+            // one (max, sum) pair per row, part of the streamed range and column half
             if (ok && x < p.nx) {
-                p.part_m[(int64_t)g * p.nq + x] = m * 0.69314718055994531f;   // back to natural log
-                p.part_l[(int64_t)g * p.nq + x] = l;
+                const int64_t slot = (int64_t)(2 * g + half) * p.nq + x;
+                p.part_m[slot] = m * 0.69314718055994531f;   // back to natural log
+                p.part_l[slot] = l;
             }
         } else {
             // per-row constants (DQ: the row is a query)
@@ -598,27 +610,30 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 pos_x = p.pos_idx[x];
             }
             for (int t = 0; t < T; ++t) {
-                const int b = t & 1;
+                const int b = t & (NBUF - 1);
                 const int64_t y0 = (lo + t) * SN;
                 // DP: the columns are queries; lane j holds lse / pos of column 32 cb + j
-                float lse2_y[SN / 32];
-                int32_t pos_y[SN / 32];
+                float lse2_y[CB_PER];
+                int32_t pos_y[CB_PER];
                 if (MODE == MODE_DP) {
 #pragma unroll
-                    for (int cb = 0; cb < SN / 32; ++cb) {
-                        const int64_t y = y0 + cb * 32 + lane;
-                        lse2_y[cb] = (y < p.ny) ? p.row_lse[y] * 1.4426950408889634f : INFINITY;
-                        pos_y[cb] = (y < p.ny) ? p.pos_idx[y] : -1;
+                    for (int j = 0; j < CB_PER; ++j) {
+                        const int64_t y = y0 + (cb0 + j) * 32 + lane;
+                        lse2_y[j] = (y < p.ny) ? p.row_lse[y] * 1.4426950408889634f : INFINITY;
+                        pos_y[j] = (y < p.ny) ? p.pos_idx[y] : -1;
                     }
                 }
                 TR_BEGIN(tr_ws);
-                ok = mbar_wait(smem_u32(&bars.s_full[b]), (t >> 1) & 1, abort_flag);
+                ok = mbar_wait(smem_u32(&bars.s_full[b]), (t >> BSH) & 1, abort_flag);
                 TR_END(tr_ws);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t sbuf = tmem + lane_addr + S_COL0 + b * SN;
+                // W of this half goes to the first columns of the half's own S region (already
+                // read by this warp): columns half * SN/2 + 16 j for block j.
 #pragma unroll
-                for (int cb = 0; cb < SN / 32; ++cb) {
+                for (int j = 0; j < CB_PER; ++j) {
+                    const int cb = cb0 + j;
                     uint32_t v[32];
                     tmem_ld32(sbuf + cb * 32, v);
                     tmem_ld_wait();
@@ -642,12 +657,12 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     } else {
 #pragma unroll
                         for (int c = 0; c < 32; ++c) {
-                            const float ls = __shfl_sync(0xffffffffu, lse2_y[cb], c);
+                            const float ls = __shfl_sync(0xffffffffu, lse2_y[j], c);
                             w[c] = ex2(fmaf(__uint_as_float(v[c]), p.c1, -ls));   // OOB: ex2(-inf)
                         }
                         // one-hot: column c's query has its positive at row pos - x0 of this tile
-                        const int64_t rel_row = (int64_t)pos_y[cb] - x0;
-                        const bool mine = (pos_y[cb] >= 0) && rel_row >= q * 32 && rel_row < q * 32 + 32;
+                        const int64_t rel_row = (int64_t)pos_y[j] - x0;
+                        const bool mine = (pos_y[j] >= 0) && rel_row >= q * 32 && rel_row < q * 32 + 32;
                         unsigned hits = __ballot_sync(0xffffffffu, mine);
                         while (hits) {
                             const int col = __ffs(hits) - 1;
@@ -672,14 +687,15 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         __nv_bfloat162 h = __floats2bfloat162_rn(w[2 * r], w[2 * r + 1]);
                         packed[r] = *reinterpret_cast<uint32_t*>(&h);
                     }
-                    tmem_st16(sbuf + cb * 16, packed);
+                    tmem_st16(sbuf + half * (SN / 2) + j * 16, packed);
                 }
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bars.w_full[b]));
             }
-            // epilogue: accumulator columns of this part -> global memory
+            // epilogue: accumulator columns of this part -> global memory (32-column blocks are
+            // dealt alternately to the two warps of a lane quarter)
             TR_BEGIN(tr_epi);
             if (ok) ok = mbar_wait(smem_u32(&bars.acc_full), 0, abort_flag);
             if (ok) {
@@ -689,7 +705,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 float* dst = final_out ? p.out + x * p.ldo + c_begin * 64
                                        : p.partial + ((int64_t)g * p.nx + x) * d + c_begin * 64;
                 const float sc = final_out ? p.out_scale : 1.f;
-                for (int cb = 0; cb < c_count * 2; ++cb) {
+                for (int cb = half; cb < c_count * 2; cb += 2) {
                     uint32_t v[32];
                     tmem_ld32(tmem + lane_addr + cb * 32, v);
                     tmem_ld_wait();
@@ -708,7 +724,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             TR_END(tr_epi);
         }
 #ifdef GC_TC_TRACE
-        if (q == 0 && lane == 0) {
+        if (q == 0 && half == 0 && lane == 0) {
             TR_ADD(MODE, TR_SM_TOTAL, clock64() - tr_total_t0);
             TR_ADD(MODE, TR_SM_WAIT_S, tr_ws);
             TR_ADD(MODE, TR_SM_EPI, tr_epi);
@@ -773,9 +789,9 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int d, int64_t l
 int parts_for(int kc) { return (kc + MAX_PART_CHUNKS - 1) / MAX_PART_CHUNKS; }
 int chunks_per_part(int kc) { int n = parts_for(kc); return (kc + n - 1) / n; }
 
-// S-tile width of the gradient sweeps: 128 when the accumulator part leaves room for two
-// 128-column S buffers, else 64.
-int sweep_sn(int kc) { return chunks_per_part(kc) * 64 + 256 <= TMEM_COLS ? 128 : 64; }
+// The gradient sweeps use 128-wide S tiles: two buffers when the accumulator part leaves room
+// (up to 256 columns), one otherwise.
+int sweep_nbuf(int kc) { return chunks_per_part(kc) * 64 + 256 <= TMEM_COLS ? 2 : 1; }
 
 struct SmemPlan { int xres; int nstage; size_t dynamic_bytes; };
 
@@ -795,19 +811,19 @@ SmemPlan smem_plan(int kc) {
     return sp;
 }
 
-template <int MODE, int SN>
+template <int MODE, int SN, int NBUF>
 cudaError_t launch(const CUtensorMap& mx, const CUtensorMap& my, const TcParams& p, int64_t units,
                    cudaStream_t st) {
     SmemPlan sp = smem_plan(p.kc);
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(tc_kernel<MODE, SN>,
+        cudaError_t e = cudaFuncSetAttribute(tc_kernel<MODE, SN, NBUF>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)(SMEM_LIMIT - SMEM_STATIC_RESERVE));
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    tc_kernel<MODE, SN><<<(unsigned)units, NTHREADS, sp.dynamic_bytes, st>>>(mx, my, p);
+    tc_kernel<MODE, SN, NBUF><<<(unsigned)units, NTHREADS, sp.dynamic_bytes, st>>>(mx, my, p);
     return cudaGetLastError();
 }
 
@@ -829,20 +845,22 @@ bool tc_supported(int64_t B, int64_t N, int d, int dtype) {
     return dtype == GC_BF16 && d % 64 == 0 && d >= 64 && d <= MAX_D;
 }
 
+// Number of (max, sum) partial slots per query row written by the forward sweep: two column
+// halves for each part of the passage range.
 int tc_fwd_groups(int64_t B, int64_t N, int d) {
     (void)d;
     int64_t tiles = (B + XROWS - 1) / XROWS, steps = (N + 127) / 128;
     int64_t g = sm_count() / tiles;
     if (g < 1) g = 1;
     if (g > steps) g = steps;
-    if (g > 32) g = 32;
-    return (int)g;
+    if (g > 16) g = 16;
+    return (int)(2 * g);
 }
 
 int tc_sweep_groups(int64_t nx, int64_t ny, int d) {
     int kc = d / 64;
     int64_t units = ((nx + XROWS - 1) / XROWS) * parts_for(kc);
-    int64_t steps = (ny + sweep_sn(kc) - 1) / sweep_sn(kc);
+    int64_t steps = (ny + 127) / 128;
     int64_t g = sm_count() / units;
     if (g < 1) g = 1;
     if (g > steps) g = steps;
@@ -859,7 +877,7 @@ cudaError_t tc_launch_fwd(const FwdArgs& a, cudaStream_t st) {
         return cudaErrorInvalidValue;
     TcParams p{};
     p.nx = pr.B; p.ny = pr.N; p.nq = pr.B;
-    p.kc = pr.d / 64; p.dparts = 1; p.dpc = 0; p.groups = a.groups;
+    p.kc = pr.d / 64; p.dparts = 1; p.dpc = 0; p.groups = a.groups / 2;
     p.nstage = smem_plan(p.kc).nstage;
     p.xres = smem_plan(p.kc).xres;
     p.mask_mode = pr.mask_mode;
@@ -868,15 +886,15 @@ cudaError_t tc_launch_fwd(const FwdArgs& a, cudaStream_t st) {
     p.pos_idx = pr.pos_idx;
     p.part_m = a.part_m; p.part_l = a.part_l; p.pos_logit = a.pos_logit;
     p.dev_status = a.dev_status;
-    int64_t units = ((pr.B + XROWS - 1) / XROWS) * a.groups;
-    return launch<MODE_FWD, SN>(mx, my, p, units, st);
+    int64_t units = ((pr.B + XROWS - 1) / XROWS) * p.groups;
+    return launch<MODE_FWD, SN, 2>(mx, my, p, units, st);
 }
 
 cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     const int kc = a.d / 64;
-    const int sn = sweep_sn(kc);
+    constexpr int SN = 128;
     CUtensorMap mx, my;
-    if (!make_map(&mx, a.X, a.nx, a.d, a.ldx, XROWS) || !make_map(&my, a.Y, a.ny, a.d, a.ldy, sn))
+    if (!make_map(&mx, a.X, a.nx, a.d, a.ldx, XROWS) || !make_map(&my, a.Y, a.ny, a.d, a.ldy, SN))
         return cudaErrorInvalidValue;
     TcParams p{};
     p.nx = a.nx; p.ny = a.ny; p.nq = 0;
@@ -891,11 +909,12 @@ cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     p.out = a.out; p.ldo = a.ldo; p.partial = a.partial;
     p.dev_status = a.dev_status;
     int64_t units = ((a.nx + XROWS - 1) / XROWS) * p.dparts * a.groups;
+    const bool two = sweep_nbuf(kc) == 2;
     if (a.mode == SWEEP_DQ)
-        return sn == 128 ? launch<MODE_DQ, 128>(mx, my, p, units, st)
-                         : launch<MODE_DQ, 64>(mx, my, p, units, st);
-    return sn == 128 ? launch<MODE_DP, 128>(mx, my, p, units, st)
-                     : launch<MODE_DP, 64>(mx, my, p, units, st);
+        return two ? launch<MODE_DQ, SN, 2>(mx, my, p, units, st)
+                   : launch<MODE_DQ, SN, 1>(mx, my, p, units, st);
+    return two ? launch<MODE_DP, SN, 2>(mx, my, p, units, st)
+               : launch<MODE_DP, SN, 1>(mx, my, p, units, st);
 }
 
 }  // namespace gc
