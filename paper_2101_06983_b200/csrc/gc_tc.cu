@@ -40,7 +40,7 @@ constexpr int MMA_WARP = NPROD;
 constexpr int NSOFT = 8;                   // softmax / epilogue warps
 constexpr int NTHREADS = 32 * (NPROD + 1 + NSOFT);
 constexpr int MAX_STAGES = 8;
-constexpr uint32_t STAGE_BYTES = 16384;    // one X chunk (128 rows) or 128 Y rows of one chunk
+constexpr uint32_t CHUNK_BYTES = 16384;    // 128 rows x 64 columns: one X chunk or one Y chunk
 constexpr int TMEM_COLS = 512;
 constexpr int MAX_D = 768;
 constexpr int MAX_PART_CHUNKS = 6;         // 384 accumulator columns
@@ -71,6 +71,7 @@ struct TcParams {
     int64_t nq;               // number of queries B (pitch of the forward partial arrays)
     int kc;                   // d / 64
     int xres;                 // X chunks [0, xres) stay resident, [xres, kc) are streamed
+    int ipc;                  // chunks per ring item (1 or 2): a stage holds ipc * 16 KB
     int dparts, dpc;          // accumulator column parts and chunks per part
     int groups;
     int nstage;
@@ -278,8 +279,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     __shared__ int abort_s;
     volatile int* abort_flag = &abort_s;
 
-    constexpr uint32_t Y_CHUNK_BYTES = SN * CHUNK_BYTES_PER_ROW;
-    constexpr int YPER = 128 / SN;                      // Y chunks that share one ring stage
+    static_assert(SN == 128, "a Y chunk is 128 rows: the same 16 KB as an X chunk");
     constexpr uint32_t S_COL0 = TMEM_COLS - NBUF * SN;  // S buffers sit at the top columns
     constexpr int LAG = NBUF - 1;                       // steps between S(t) and acc(t) issue
     constexpr int BSH = (NBUF == 2) ? 1 : 0;            // log2(NBUF)
@@ -303,6 +303,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t x_smem = base;
     const uint32_t y_smem = base + (uint32_t)p.xres * X_CHUNK_BYTES;   // the ring
+    const uint32_t stage_bytes = (uint32_t)p.ipc * CHUNK_BYTES;
 
     if (threadIdx.x == 0) {
         abort_s = 0;
@@ -360,36 +361,28 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 }
                 return stage;
             };
-            auto load_y = [&](int chunk0, int count, int64_t row) {
+            // One ring item: p.ipc consecutive 64-column chunks of 128 rows of Y (or of X).
+            auto load_item = [&](const CUtensorMap* map, int chunk0, int64_t row) {
                 const int stage = acquire();
                 if (stage < 0) return;
                 const uint32_t full = smem_u32(&bars.y_full[stage]);
                 if (elect_one()) {
-                    mbar_expect_tx(full, (uint32_t)count * Y_CHUNK_BYTES);
-                    for (int i = 0; i < count; ++i)
-                        tma_load_2d(y_smem + stage * STAGE_BYTES + i * Y_CHUNK_BYTES, &mapY,
+                    mbar_expect_tx(full, stage_bytes);
+                    for (int i = 0; i < p.ipc; ++i)
+                        tma_load_2d(y_smem + stage * stage_bytes + i * CHUNK_BYTES, map,
                                     (chunk0 + i) * 64, (int)row, full);
-                }
-            };
-            auto load_x = [&](int chunk) {
-                const int stage = acquire();
-                if (stage < 0) return;
-                const uint32_t full = smem_u32(&bars.y_full[stage]);
-                if (elect_one()) {
-                    mbar_expect_tx(full, X_CHUNK_BYTES);
-                    tma_load_2d(y_smem + stage * STAGE_BYTES, &mapX, chunk * 64, (int)x0, full);
                 }
             };
             for (int t = 0; t < T + LAG && ok; ++t) {
                 if (t < T) {
-                    for (int c = 0; c < p.kc; ++c) {
-                        if (c % YPER == 0) load_y(c, min(YPER, p.kc - c), (lo + t) * SN);
-                        if (c >= p.xres) load_x(c);
+                    for (int c = 0; c < p.kc; c += p.ipc) {
+                        load_item(&mapY, c, (lo + t) * SN);
+                        if (c >= p.xres) load_item(&mapX, c, x0);
                     }
                 }
                 if (MODE != MODE_FWD && t >= LAG) {
-                    for (int c = 0; c < c_count; c += YPER)
-                        load_y(c_begin + c, min(YPER, c_count - c), (lo + t - LAG) * SN);
+                    for (int c = 0; c < c_count; c += p.ipc)
+                        load_item(&mapY, c_begin + c, (lo + t - LAG) * SN);
                 }
             }
 #ifdef GC_TC_TRACE
@@ -407,9 +400,10 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             const uint32_t idesc_acc64 = instr_desc(64, true);
             const uint32_t idesc_acc128 = instr_desc(128, true);
             const uint32_t x_lo = desc_lo(x_smem, 0);
-            const uint32_t ring_lo = desc_lo(y_smem, Y_CHUNK_BYTES);   // LBO: next chunk of a stage
-            constexpr uint32_t STAGE_LO = STAGE_BYTES >> 4, YCH_LO = Y_CHUNK_BYTES >> 4,
-                               XCH_LO = X_CHUNK_BYTES >> 4;
+            const uint32_t ring_lo = desc_lo(y_smem, CHUNK_BYTES);   // LBO: next chunk of a stage
+            constexpr uint32_t CH_LO = CHUNK_BYTES >> 4;
+            const uint32_t stage_lo = stage_bytes >> 4;
+            const uint32_t idesc_acc = (p.ipc == 2) ? idesc_acc128 : idesc_acc64;
             int next = 0;
             uint32_t next_phase = 0;
             TR_DECL(tr_wy);
@@ -446,19 +440,17 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         tc_fence_after();
                     }
                     const uint32_t d_tmem = tmem + S_COL0 + b * SN;
-                    int ys = 0;
-                    for (int c = 0; c < p.kc && ok; ++c) {
-                        const int sub = (YPER == 1) ? 0 : (c & (YPER - 1));
-                        if (sub == 0) ys = next_stage();
+                    for (int c = 0; c < p.kc && ok; c += p.ipc) {
+                        const int ys = next_stage();
                         if (!ok) break;
                         int xs = -1;
-                        uint32_t xa = x_lo + c * XCH_LO;
+                        uint32_t xa = x_lo + c * CH_LO;
                         if (c >= p.xres) {
                             xs = next_stage();
                             if (!ok) break;
-                            xa = ring_lo + xs * STAGE_LO;
+                            xa = ring_lo + xs * stage_lo;
                         }
-                        const uint32_t yb = ring_lo + ys * STAGE_LO + sub * YCH_LO;
+                        const uint32_t yb = ring_lo + ys * stage_lo;
                         TR_BEGIN(tr_is);
                         if (elect_one()) {
                             if (c == 0) mma_ss<false>(d_tmem, xa, yb, idesc_s);
@@ -466,9 +458,14 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                             mma_ss<true>(d_tmem, xa + 2, yb + 2, idesc_s);
                             mma_ss<true>(d_tmem, xa + 4, yb + 4, idesc_s);
                             mma_ss<true>(d_tmem, xa + 6, yb + 6, idesc_s);
+                            if (p.ipc == 2) {
+                                mma_ss<true>(d_tmem, xa + CH_LO, yb + CH_LO, idesc_s);
+                                mma_ss<true>(d_tmem, xa + CH_LO + 2, yb + CH_LO + 2, idesc_s);
+                                mma_ss<true>(d_tmem, xa + CH_LO + 4, yb + CH_LO + 4, idesc_s);
+                                mma_ss<true>(d_tmem, xa + CH_LO + 6, yb + CH_LO + 6, idesc_s);
+                            }
                             if (xs >= 0) tc_commit(smem_u32(&bars.y_empty[xs]));
-                            if (sub == YPER - 1 || c == p.kc - 1)
-                                tc_commit(smem_u32(&bars.y_empty[ys]));
+                            tc_commit(smem_u32(&bars.y_empty[ys]));
                         }
                         TR_END(tr_is);
                     }
@@ -485,25 +482,23 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     if (!ok) break;
                     tc_fence_after();
                     const uint32_t w_tmem = tmem + S_COL0 + b * SN;
-                    // one ring stage per iteration: YPER chunks = 64 * YPER accumulator columns
-                    for (int c = 0; c < c_count && ok; c += YPER) {
+                    // one ring item per iteration: ipc chunks = 64 * ipc accumulator columns
+                    for (int c = 0; c < c_count && ok; c += p.ipc) {
                         const int ys = next_stage();
                         if (!ok) break;
-                        const uint32_t yb = ring_lo + ys * STAGE_LO;
+                        const uint32_t yb = ring_lo + ys * stage_lo;
                         const uint32_t d_tmem = tmem + c * 64;
-                        const bool wide = (YPER == 2) && (c + 1 < c_count);
-                        const uint32_t idesc = wide ? idesc_acc128 : idesc_acc64;
                         TR_BEGIN(tr_ai);
                         if (elect_one()) {
                             // k-steps of the first column half read W at columns 8 k, those of
                             // the second half at SN/2 + 8 (k - KH)
                             constexpr int KH = SN / 32;
-                            if (u == 0) mma_ts<false>(d_tmem, w_tmem, yb, idesc);
-                            else        mma_ts<true>(d_tmem, w_tmem, yb, idesc);
+                            if (u == 0) mma_ts<false>(d_tmem, w_tmem, yb, idesc_acc);
+                            else        mma_ts<true>(d_tmem, w_tmem, yb, idesc_acc);
 #pragma unroll
                             for (int k = 1; k < SN / 16; ++k)
                                 mma_ts<true>(d_tmem, w_tmem + (k / KH) * (SN / 2) + (k % KH) * 8,
-                                             yb + k * 128, idesc);
+                                             yb + k * 128, idesc_acc);
                             tc_commit(smem_u32(&bars.y_empty[ys]));
                         }
                         TR_END(tr_ai);
@@ -793,19 +788,24 @@ int chunks_per_part(int kc) { int n = parts_for(kc); return (kc + n - 1) / n; }
 // (up to 256 columns), one otherwise.
 int sweep_nbuf(int kc) { return chunks_per_part(kc) * 64 + 256 <= TMEM_COLS ? 2 : 1; }
 
-struct SmemPlan { int xres; int nstage; size_t dynamic_bytes; };
+struct SmemPlan { int xres; int ipc; int nstage; size_t dynamic_bytes; };
 
 // Rows up to 512 wide keep the whole X tile resident; wider rows keep 6 chunks so that the ring
-// still has eight stages.
+// still has 128 KB.  Ring items hold two chunks when every chunk count involved is even.
 SmemPlan smem_plan(int kc) {
     SmemPlan sp;
     sp.xres = kc <= 8 ? kc : 6;
+    const int parts = parts_for(kc), dpc = chunks_per_part(kc);
+    const bool even = kc % 2 == 0 && sp.xres % 2 == 0 && dpc % 2 == 0 &&
+                      (kc - dpc * (parts - 1)) % 2 == 0;
+    sp.ipc = even ? 2 : 1;
     size_t xbytes = (size_t)sp.xres * X_CHUNK_BYTES;
+    size_t stage = (size_t)sp.ipc * CHUNK_BYTES;
     size_t avail = SMEM_LIMIT - SMEM_STATIC_RESERVE - 1024 - xbytes;
-    int ns = (int)(avail / STAGE_BYTES);
+    int ns = (int)(avail / stage);
     if (ns > MAX_STAGES) ns = MAX_STAGES;
     sp.nstage = ns;
-    sp.dynamic_bytes = 1024 + xbytes + (size_t)ns * STAGE_BYTES;
+    sp.dynamic_bytes = 1024 + xbytes + (size_t)ns * stage;
     // keep one CTA per SM (each CTA allocates all 512 tensor-memory columns)
     if (sp.dynamic_bytes < 120 * 1024) sp.dynamic_bytes = 120 * 1024;
     return sp;
@@ -880,6 +880,7 @@ cudaError_t tc_launch_fwd(const FwdArgs& a, cudaStream_t st) {
     p.kc = pr.d / 64; p.dparts = 1; p.dpc = 0; p.groups = a.groups / 2;
     p.nstage = smem_plan(p.kc).nstage;
     p.xres = smem_plan(p.kc).xres;
+    p.ipc = smem_plan(p.kc).ipc;
     p.mask_mode = pr.mask_mode;
     p.inv_tau = 1.f / pr.tau;
     p.c1 = 1.4426950408889634f / pr.tau;
@@ -901,6 +902,7 @@ cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     p.kc = kc; p.dparts = parts_for(kc); p.dpc = chunks_per_part(kc); p.groups = a.groups;
     p.nstage = smem_plan(kc).nstage;
     p.xres = smem_plan(kc).xres;
+    p.ipc = smem_plan(kc).ipc;
     p.mask_mode = a.mask_mode;
     p.inv_tau = a.inv_tau;
     p.c1 = 1.4426950408889634f * a.inv_tau;
