@@ -54,7 +54,8 @@ typedef enum {
     GC_ERR_ALIGN = 5,     /* a row does not start on a 16-byte boundary */
     GC_ERR_WORKSPACE = 6, /* workspace NULL, misaligned (256 bytes) or too small */
     GC_ERR_CUDA = 7,      /* a CUDA call or launch failed */
-    GC_ERR_ARCH = 8       /* the current device is not compute capability 10.x */
+    GC_ERR_ARCH = 8,      /* the current device is not compute capability 10.x */
+    GC_ERR_LIMIT = 9      /* problem too large for the library's built-in scratch area */
 } gc_status;
 
 typedef enum { GC_F32 = 0, GC_BF16 = 1 } gc_dtype;
@@ -102,6 +103,32 @@ int gc_build_cache(const void* Q, int64_t ldq, const void* P, int64_t ldp, const
                    float* loss, float* row_lse, float* pos_logit,
                    float* dQ, int64_t lddq, float* dP, int64_t lddp,
                    void* ws, size_t ws_bytes, int* dev_status, void* cuda_stream);
+
+/*
+ * Forward with library-owned scratch (no counterpart in the paper: it exists for the sake of
+ * callers, not of the method).  Same inputs, outputs and results as gc_loss_fwd, but the caller
+ * passes no workspace.  It is meant for callers that cannot obtain device memory at the point of
+ * the call: code running under a host framework that owns every byte of the device through its
+ * own pool and offers no allocation hook to a C library, and loops on a hot path where an
+ * allocator call is unwelcome because it may synchronise the whole device or fail late.  The
+ * call itself allocates nothing and frees nothing, on the device or through any library.
+ *
+ * The scratch (per-part row maxima, row sums and the gathered positive logits) lives in a
+ * fixed array of GC_STATIC_SCRATCH_BYTES inside the library image, so every GPU that loads the
+ * library carries that much extra memory until the process exits.  Problems whose forward
+ * scratch (gc_static_scratch_need) exceeds it are refused with GC_ERR_LIMIT and nothing is
+ * launched.  The first call on each device looks up the array's device address (once, with that
+ * device current); make that first call outside any stream capture.  All calls on a device
+ * share the one array, and it keeps whatever the previous call left: the kernels overwrite
+ * every entry they later read, so nothing has to be cleared, but two calls that overlap on the
+ * GPU (different streams, no ordering between them) would race on it.  Serialise them.
+ */
+#define GC_STATIC_SCRATCH_BYTES (2u << 20)
+size_t gc_static_scratch_need(int64_t B, int64_t N, int d, int dtype);
+int gc_loss_fwd_static(const void* Q, int64_t ldq, const void* P, int64_t ldp,
+                       const int32_t* pos_idx, int64_t B, int64_t N, int d, float tau,
+                       int mask_mode, int dtype, float* loss, float* row_lse, float* pos_logit,
+                       int* dev_status, void* cuda_stream);
 
 /*
  * Measurement aid (not part of the paper's method).  After gc_profile_enable(1) every call

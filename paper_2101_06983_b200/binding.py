@@ -20,7 +20,8 @@ GC_DEV_POS_RANGE, GC_DEV_POS_MASKED, GC_DEV_WAIT_LIMIT = 1, 2, 4
 
 EXPORTS = ("gc_workspace_bytes", "gc_plan_name", "gc_kernel_launches", "gc_loss_fwd",
            "gc_loss_bwd", "gc_build_cache", "gc_status_string", "gc_profile_enable",
-           "gc_profile_read")
+           "gc_profile_read", "gc_static_scratch_need", "gc_loss_fwd_static")
+GC_STATIC_SCRATCH_BYTES = 2 << 20
 
 
 class GradCacheError(RuntimeError):
@@ -53,6 +54,10 @@ def _load() -> ctypes.CDLL:
     lib.gc_build_cache.restype = i32
     lib.gc_build_cache.argtypes = common + [vp, vp, vp, vp, i64, vp, i64, vp, ctypes.c_size_t,
                                             vp, vp]
+    lib.gc_static_scratch_need.restype = ctypes.c_size_t
+    lib.gc_static_scratch_need.argtypes = [i64, i64, i32, i32]
+    lib.gc_loss_fwd_static.restype = i32
+    lib.gc_loss_fwd_static.argtypes = common + [vp, vp, vp, vp, vp]
     lib.gc_profile_enable.restype = i32
     lib.gc_profile_enable.argtypes = [i32]
     lib.gc_profile_read.restype = i32
@@ -127,6 +132,23 @@ def gc_loss_fwd(Q, P, pos_idx, tau, mask_mode, loss, row_lse, pos_logit=None, ws
                           ws.numel(), _ptr(dev_status), _stream())
     if rc != 0:
         raise GradCacheError(rc, "gc_loss_fwd")
+
+
+def gc_static_scratch_need(B: int, N: int, d: int, dtype: int) -> int:
+    return int(_lib.gc_static_scratch_need(B, N, d, dtype))
+
+
+def gc_loss_fwd_static(Q, P, pos_idx, tau, mask_mode, loss, row_lse, pos_logit=None,
+                       dev_status=None):
+    """gc_loss_fwd without a caller workspace: the scratch is a fixed array inside the library
+    (GC_STATIC_SCRATCH_BYTES).  Nothing is allocated by the call; all outputs are the caller's.
+    Raises GradCacheError with GC_ERR_LIMIT (9) when the problem needs more scratch than that.
+    Calls on one device share the array, so they must not overlap on the GPU."""
+    args, B, N, d, code = _common(Q, P, pos_idx, tau, mask_mode)
+    rc = _lib.gc_loss_fwd_static(*args, _ptr(loss), _ptr(row_lse), _ptr(pos_logit),
+                                 _ptr(dev_status), _stream())
+    if rc != 0:
+        raise GradCacheError(rc, "gc_loss_fwd_static")
 
 
 def gc_loss_bwd(Q, P, pos_idx, tau, mask_mode, row_lse, dQ, dP, ws=None, dev_status=None):

@@ -184,6 +184,33 @@ int run_sweep(const Problem& p, const Plan& pl, char* ws, int mode, const float*
 
 using namespace gc;
 
+// Scratch for gc_loss_fwd_static.  In host code this name is only a handle for the symbol: the
+// address a kernel can use comes from cudaGetSymbolAddress, looked up once per device.
+static __device__ __align__(256) unsigned char g_static_scratch[GC_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+// Device address of g_static_scratch on the current device, or nullptr on failure.
+void* static_scratch_ptr() {
+    static void* cached[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    if (!cached[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess) {
+            cudaGetLastError();
+            return nullptr;
+        }
+        cached[dev] = ptr;
+    }
+    return cached[dev];
+}
+
+}  // namespace
+
 extern "C" {
 
 size_t gc_workspace_bytes(int op, int64_t B, int64_t N, int d, int dtype) {
@@ -219,6 +246,28 @@ int gc_loss_fwd(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
     if ((rc = check_device())) return rc;
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
     return run_fwd(p, pl, static_cast<char*>(ws), loss, row_lse, pos_logit, dev_status,
+                   static_cast<cudaStream_t>(cuda_stream));
+}
+
+size_t gc_static_scratch_need(int64_t B, int64_t N, int d, int dtype) {
+    if (B <= 0 || N <= 0 || d <= 0 || (dtype != GC_F32 && dtype != GC_BF16)) return 0;
+    return make_plan(B, N, d, dtype).off_accq;   // the forward part of the workspace layout
+}
+
+int gc_loss_fwd_static(const void* Q, int64_t ldq, const void* P, int64_t ldp,
+                       const int32_t* pos_idx, int64_t B, int64_t N, int d, float tau,
+                       int mask_mode, int dtype, float* loss, float* row_lse, float* pos_logit,
+                       int* dev_status, void* cuda_stream) {
+    int rc = check_common(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
+    if (rc) return rc;
+    if (!loss || !row_lse) return GC_ERR_NULL;
+    Plan pl = make_plan(B, N, d, dtype);
+    if (pl.off_accq > (size_t)GC_STATIC_SCRATCH_BYTES) return GC_ERR_LIMIT;
+    if ((rc = check_device())) return rc;
+    void* scratch = static_scratch_ptr();
+    if (!scratch) return GC_ERR_CUDA;
+    Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
+    return run_fwd(p, pl, static_cast<char*>(scratch), loss, row_lse, pos_logit, dev_status,
                    static_cast<cudaStream_t>(cuda_stream));
 }
 
@@ -301,6 +350,7 @@ const char* gc_status_string(int status) {
         case GC_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case GC_ERR_CUDA: return "a CUDA call failed";
         case GC_ERR_ARCH: return "device is not compute capability 10.x";
+        case GC_ERR_LIMIT: return "problem needs more scratch than the library's built-in area holds";
         default: return "unknown status";
     }
 }

@@ -38,8 +38,8 @@ def test_every_declared_symbol_is_exported(binding):
 
 
 def test_status_strings(binding):
-    seen = {binding.status_string(i) for i in range(9)}
-    assert len(seen) == 9 and "ok" in seen
+    seen = {binding.status_string(i) for i in range(10)}
+    assert len(seen) == 10 and "ok" in seen
     assert binding.status_string(1234) == "unknown status"
 
 
