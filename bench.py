@@ -65,6 +65,23 @@ class ClockSampler(threading.Thread):
         except Exception:          # NVML missing: report nulls
             self.ok = False
 
+    def sample_once(self):
+        """One synchronous sample (called from the timed loop while a step is executing)."""
+        if not self.ok:
+            return
+        nv = self.nv
+        try:
+            self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+            mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+            for name in ("HwSlowdown", "HwThermalSlowdown", "SwThermalSlowdown", "SwPowerCap"):
+                if mask & getattr(nv, "nvmlClocksThrottleReason" + name):
+                    self.reasons.add({"HwSlowdown": "hw_slowdown",
+                                      "HwThermalSlowdown": "hw_thermal_slowdown",
+                                      "SwThermalSlowdown": "sw_thermal_slowdown",
+                                      "SwPowerCap": "sw_power_cap"}[name])
+        except Exception:
+            pass
+
     def run(self):
         if not self.ok:
             return
@@ -106,19 +123,6 @@ def physical_gpu_index(local_rank: int) -> int:
         except (ValueError, IndexError):
             return local_rank
     return local_rank
-
-
-def make_problem(index: int, rank: int):
-    from paper_2101_06983_b200 import inputs
-    if rank == 0:
-        return inputs.config(index)
-    # other replicas: same recipe, different seed
-    base = inputs.config  # noqa: F841
-    if index == 3:
-        return inputs.simclr_batch(4096, 128, "bf16", seed=inputs.BASE_SEED + 3 + 100 * rank)
-    B = {0: 64, 1: 128, 2: 4096, 4: 65536}[index]
-    return inputs.dpr_batch(B, 768, "f32" if index == 0 else "bf16",
-                            seed=inputs.BASE_SEED + index + 100 * rank)
 
 
 def run_reference(args, rank, world):
@@ -165,9 +169,9 @@ def run_ours(args, rank, local_rank, world):
     dev = torch.device("cuda", local_rank)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
-    from paper_2101_06983_b200 import binding
+    from paper_2101_06983_b200 import binding, replicas
 
-    prob = make_problem(args.config, rank)
+    prob = replicas.replica_problem(args.config, rank)
     B, N, d = prob.B, prob.N, prob.d
     code = binding.GC_BF16 if prob.dtype == "bf16" else binding.GC_F32
     Q, P, pos = binding.problem_tensors(prob, dev)
@@ -203,6 +207,7 @@ def run_ours(args, rank, local_rank, world):
         a.record()
         step()
         b.record()
+        sampler.sample_once()                   # the step is executing on the GPU right now
         ms = binding.gc_profile_read()          # waits for this step's kernels
         for k in range(3):
             kern[k] += ms[k]
@@ -260,10 +265,7 @@ def run_ours(args, rank, local_rank, world):
     status = int(out.dev_status.item())
 
     # ---- max over ranks ------------------------------------------------------------------------------
-    vals = torch.tensor([total_ms, warm_ms, e2e_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-    total_ms, warm_ms, e2e_ms = (float(x) for x in vals.tolist())
+    total_ms, warm_ms, e2e_ms = replicas.max_over_ranks([total_ms, warm_ms, e2e_ms], dev)
     ms_per_step = total_ms / args.steps
 
     if rank == 0:
@@ -272,7 +274,7 @@ def run_ours(args, rank, local_rank, world):
         # delivers one useful GEMM of 2 B N d
         sweep_ms = (kern[1] + kern[2]) / (2 * args.steps)
         achieved = (2.0 * B * N * d) / (sweep_ms * 1e-3) / 1e12 if sweep_ms > 0 else 0.0
-        value = world * flop / (ms_per_step * 1e-3) / 1e12
+        value = replicas.whole_job_rate(flop, world, ms_per_step) / 1e12
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,

@@ -2,7 +2,7 @@
 
 This module only *generates data*: representation matrices Q (B x d), P (N x d) and the
 relevance map pos_idx (the paper's r_i, Section 3.1).  It holds none of the method's
-arithmetic (no similarity, softmax, loss or gradient), so that the CPU oracle and the CUDA
+arithmetic (no similarity, softmax, loss or gradient), so that the CPU checker and the CUDA
 path can both be fed from it without sharing any computation.
 
 Random numbers come from numpy's Philox generator (a counter-based PRNG) keyed by the seed.

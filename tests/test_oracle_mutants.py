@@ -1,0 +1,105 @@
+"""Plants mistakes in copies of the oracle's C source (on the CPU) and checks that the pins of
+test_oracle_pins.py notice each one: a dropped term, a wrong sign, a wrong index, a misplaced
+temperature, a leaking mask, a transposed operand."""
+import ctypes
+import os
+import subprocess
+import types
+
+import numpy as np
+import pytest
+
+import test_oracle_pins as pins
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SRC = open(os.path.join(ROOT, "oracle", "gc_oracle.c")).read()
+
+MUTANTS = {
+    "one-hot term dropped": ("double onehot = (j == pos_idx[i]) ? 1.0 : 0.0;", "double onehot = 0.0;"),
+    "wrong sign of one-hot": ("row[j] = (p - onehot) / (double)B;", "row[j] = (p + onehot) / (double)B;"),
+    "1/B missing": ("row[j] = (p - onehot) / (double)B;", "row[j] = (p - onehot);"),
+    "dQ not divided by tau": ("for (int64_t k = 0; k < d; ++k) out[k] /= tau;\n            }\n        }\n        if (dP)",
+                              "}\n        }\n        if (dP)"),
+    "logits not divided by tau": ("S_row[j] = acc / tau;", "S_row[j] = acc;"),
+    "mask leaks into denominator": ("if (allowed(mask_mode, i, j)) sum += exp(S_row[j] - m);", "sum += exp(S_row[j] - m);"),
+    "dP uses wrong query row": ("const double* q = Q + i * d;\n                    for (int64_t k = 0; k < d; ++k) out[k] += g * q[k];",
+                                "const double* q = Q + ((i + 1) % B) * d;\n                    for (int64_t k = 0; k < d; ++k) out[k] += g * q[k];"),
+    "G read transposed in dP": ("double g = G[i * N + j];\n                    const double* q", "double g = G[(j % B) * N + (i % N)];\n                    const double* q"),
+    "positive index off by one": ("total += lse[i] - S[i * N + pos_idx[i]];", "total += lse[i] - S[i * N + (pos_idx[i] + 1) % N];"),
+    "max instead of logsumexp": ("return m + log(sum);", "return m;"),
+}
+
+
+def _build_mutant(tmp_path, name, old, new):
+    assert old in SRC, f"mutation site for '{name}' not found"
+    path = tmp_path / "mutant.c"
+    path.write_text(SRC.replace(old, new, 1))
+    lib = tmp_path / "libmutant.so"
+    subprocess.run(["gcc", "-O1", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", str(lib), str(path),
+                    "-lm"], check=True)
+    return str(lib)
+
+
+def _wrap(libpath):
+    """An object with the interface of the `oracle` package, backed by the mutant library."""
+    import oracle as real
+    lib = ctypes.CDLL(libpath)
+    dp = ctypes.POINTER(ctypes.c_double)
+    lib.gco_build_cache.restype = ctypes.c_int
+    lib.gco_build_cache.argtypes = [dp, dp, ctypes.POINTER(ctypes.c_int32), ctypes.c_int64,
+                                    ctypes.c_int64, ctypes.c_int64, ctypes.c_double, ctypes.c_int,
+                                    dp, dp, dp, dp, dp]
+
+    def build_cache(Q, P, pos_idx, tau=1.0, mask_mode=0, grads=True):
+        Q, P, pos = real._prep(Q, P, pos_idx)
+        B, d = Q.shape
+        N = P.shape[0]
+        loss = ctypes.c_double(0.0)
+        lse, pl = np.empty(B), np.empty(B)
+        dQ, dP = np.empty((B, d)), np.empty((N, d))
+        rc = lib.gco_build_cache(real._ptr(Q, ctypes.c_double), real._ptr(P, ctypes.c_double),
+                                 real._ptr(pos, ctypes.c_int32), B, N, d, float(tau), int(mask_mode),
+                                 ctypes.byref(loss), real._ptr(lse, ctypes.c_double),
+                                 real._ptr(pl, ctypes.c_double), real._ptr(dQ, ctypes.c_double),
+                                 real._ptr(dP, ctypes.c_double))
+        if rc != 0:
+            raise ValueError(f"rejected ({rc})")
+        return dict(loss=float(loss.value), row_lse=lse, pos_logit=pl, dQ=dQ, dP=dP)
+
+    return types.SimpleNamespace(
+        build_cache=build_cache,
+        loss_only=lambda Q, P, pos, tau=1.0, mask=0: build_cache(Q, P, pos, tau, mask)["loss"])
+
+
+def _pins(o):
+    yield lambda: pins.test_hand_worked_rational_example(o)
+    yield lambda: pins.test_gradients_match_finite_differences(o, 0.1, 1, (4, 8, 5))
+    yield lambda: pins.test_gradients_match_finite_differences(o, 1.0, 0, (3, 6, 4))
+    yield lambda: pins.test_rows_of_G_sum_to_zero(o, 1)
+    yield lambda: pins.test_identical_representations(o, 0.25)
+    yield lambda: pins.test_one_query_two_passages_is_logistic_loss(o)
+    yield lambda: pins.test_scale_and_permutation_symmetry(o)
+    yield lambda: pins.test_duplicate_positives_sum_in_epsilon(o)
+
+
+@pytest.mark.parametrize("name", sorted(MUTANTS))
+def test_pins_catch_planted_mistake(tmp_path, name):
+    old, new = MUTANTS[name]
+    mutant = _wrap(_build_mutant(tmp_path, name, old, new))
+    caught = 0
+    for pin in _pins(mutant):
+        try:
+            pin()
+        except (AssertionError, ValueError):
+            caught += 1
+    assert caught >= 1, f"no pin noticed: {name}"
+
+
+def test_unmutated_source_passes_the_same_pins(tmp_path):
+    path = tmp_path / "same.c"
+    path.write_text(SRC)
+    lib = tmp_path / "libsame.so"
+    subprocess.run(["gcc", "-O1", "-std=c11", "-fopenmp", "-fPIC", "-shared", "-o", str(lib), str(path),
+                    "-lm"], check=True)
+    for pin in _pins(_wrap(str(lib))):
+        pin()
