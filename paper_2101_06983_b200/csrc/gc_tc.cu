@@ -626,12 +626,15 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 const uint32_t sbuf = tmem + lane_addr + S_COL0 + b * SN;
                 // W of this half goes to the first columns of the half's own S region (already
                 // read by this warp): columns half * SN/2 + 16 j for block j.
+                // both 32-column blocks are requested before the single wait
+                uint32_t vv[CB_PER][32];
+#pragma unroll
+                for (int j = 0; j < CB_PER; ++j) tmem_ld32(sbuf + (cb0 + j) * 32, vv[j]);
+                tmem_ld_wait();
 #pragma unroll
                 for (int j = 0; j < CB_PER; ++j) {
                     const int cb = cb0 + j;
-                    uint32_t v[32];
-                    tmem_ld32(sbuf + cb * 32, v);
-                    tmem_ld_wait();
+                    uint32_t (&v)[32] = vv[j];
                     const int64_t yb = y0 + cb * 32;
                     float w[32];
                     if (MODE == MODE_DQ) {
