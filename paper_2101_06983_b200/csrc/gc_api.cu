@@ -39,18 +39,23 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype) {
         pl.g_dq = simt_sweep_groups(B, N, d);
         pl.g_dp = simt_sweep_groups(N, B, d);
     }
+    pl.fused = (pl.tc && tc_fused_applicable(d)) ? 1 : 0;
     size_t dpad = (size_t)((d + 3) & ~3);
+    // (max, sum) slots: the forward sweep writes g_fwd of them per row, the fused sweep 2 g_dq
+    size_t slots = (size_t)pl.g_fwd;
+    if (pl.fused && (size_t)(2 * pl.g_dq) > slots) slots = (size_t)(2 * pl.g_dq);
     size_t off = 0;
-    pl.off_m = off;    off += align256(sizeof(float) * (size_t)pl.g_fwd * (size_t)B);
-    pl.off_l = off;    off += align256(sizeof(float) * (size_t)pl.g_fwd * (size_t)B);
+    pl.off_m = off;    off += align256(sizeof(float) * slots * (size_t)B);
+    pl.off_l = off;    off += align256(sizeof(float) * slots * (size_t)B);
     pl.off_pos = off;  off += align256(sizeof(float) * (size_t)B);
     pl.off_accq = off;
-    if (pl.g_dq > 1) off += align256(sizeof(float) * (size_t)pl.g_dq * (size_t)B * dpad);
+    if (pl.g_dq > 1 || pl.fused) off += align256(sizeof(float) * (size_t)pl.g_dq * (size_t)B * dpad);
     pl.off_accp = off;
     if (pl.g_dp > 1) off += align256(sizeof(float) * (size_t)pl.g_dp * (size_t)N * dpad);
     pl.total = off;
     pl.launches_fwd = 2;  // sweep + combine
     pl.launches_bwd = 2 + (pl.g_dq > 1 ? 1 : 0) + (pl.g_dp > 1 ? 1 : 0);
+    pl.launches_build = pl.fused ? 4 + (pl.g_dp > 1 ? 1 : 0) : pl.launches_fwd + pl.launches_bwd;
     return pl;
 }
 
@@ -179,6 +184,33 @@ int run_sweep(const Problem& p, const Plan& pl, char* ws, int mode, const float*
     return GC_OK;
 }
 
+// gc_build_cache for wide bf16 rows: fused forward + dQ sweep, combine, dQ finalize.
+int run_fused_fwd_dq(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_lse,
+                     float* pos_logit, float* dQ, int64_t lddq, int* dev_status,
+                     cudaStream_t st) {
+    FwdArgs fa;
+    fa.p = p;
+    fa.part_m = reinterpret_cast<float*>(ws + pl.off_m);
+    fa.part_l = reinterpret_cast<float*>(ws + pl.off_l);
+    fa.pos_logit = reinterpret_cast<float*>(ws + pl.off_pos);
+    fa.groups = 2 * pl.g_dq;
+    fa.dev_status = dev_status;
+    float* partial = reinterpret_cast<float*>(ws + pl.off_accq);
+    cudaError_t e;
+    {
+        KernelTimer t(1, st);
+        e = tc_launch_fused_dq(fa, partial, pl.g_dq, st);
+    }
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
+                           p.mask_mode, row_lse, pos_logit, loss, dev_status, st);
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    e = launch_fused_dq_finalize(partial, pl.g_dq, fa.part_m, row_lse, fa.pos_logit, p.pos_idx, p.P,
+                                 p.ldp, p.B, p.N, p.d, p.mask_mode,
+                                 1.f / ((float)p.B * p.tau), dQ, lddq, st);
+    return e == cudaSuccess ? GC_OK : GC_ERR_CUDA;
+}
+
 }  // namespace
 }  // namespace gc
 
@@ -230,7 +262,7 @@ int gc_kernel_launches(int op, int64_t B, int64_t N, int d, int dtype) {
     Plan pl = make_plan(B, N, d, dtype);
     if (op == GC_OP_FWD) return pl.launches_fwd;
     if (op == GC_OP_BWD) return pl.launches_bwd + 1;   // + pos_idx validation
-    if (op == GC_OP_BUILD) return pl.launches_fwd + pl.launches_bwd;
+    if (op == GC_OP_BUILD) return pl.launches_build;
     return 0;
 }
 
@@ -308,8 +340,13 @@ int gc_build_cache(const void* Q, int64_t ldq, const void* P, int64_t ldp, const
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
     char* w = static_cast<char*>(ws);
-    if ((rc = run_fwd(p, pl, w, loss, row_lse, pos_logit, dev_status, st))) return rc;
-    if ((rc = run_sweep(p, pl, w, SWEEP_DQ, row_lse, dQ, lddq, dev_status, st))) return rc;
+    if (pl.fused) {
+        if ((rc = run_fused_fwd_dq(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dev_status, st)))
+            return rc;
+    } else {
+        if ((rc = run_fwd(p, pl, w, loss, row_lse, pos_logit, dev_status, st))) return rc;
+        if ((rc = run_sweep(p, pl, w, SWEEP_DQ, row_lse, dQ, lddq, dev_status, st))) return rc;
+    }
     if ((rc = run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, dev_status, st))) return rc;
     return GC_OK;
 }

@@ -1,6 +1,7 @@
 // Small fixed-order reductions that follow the tile sweeps: merging the per-part running
 // maximum / sum into row_lse and the loss (Eq. 1), validating pos_idx, and summing the
 // per-part gradient partials.  No atomics on floating-point data: results are reproducible.
+#include <cuda_bf16.h>
 #include <math.h>
 
 #include "gc_internal.h"
@@ -105,7 +106,61 @@ partial_reduce_kernel(const float4* __restrict__ partial, int groups, int64_t ro
     }
 }
 
+// Finishes the fused forward + dQ sweep (Eq. 5).  partial[g][i][:] = sum_j 2^(s2_ij - m2_g) P_j
+// over the part's allowed columns except the positive one; part_m holds m_g in natural-log
+// units (slot 2g of the row).  dQ_i = (sum_g partial_g exp(m_g - lse_i) + (p_pos - 1) P_pos)
+// / (B tau), with p_pos = exp(S_{i,r_i} - lse_i) and the positive row read exactly.  A row whose
+// pos_idx is unusable gets no positive term.
+__global__ void __launch_bounds__(256)
+fused_dq_finalize_kernel(const float4* __restrict__ partial, int groups,
+                         const float* __restrict__ part_m, const float* __restrict__ row_lse,
+                         const float* __restrict__ pos_ws, const int32_t* __restrict__ pos_idx,
+                         const __nv_bfloat16* __restrict__ P, int64_t ldp, int64_t B, int64_t N,
+                         int d4, int mask_mode, float scale, float* __restrict__ out,
+                         int64_t ldo) {
+    int64_t total = B * d4;
+    for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total;
+         e += (int64_t)gridDim.x * blockDim.x) {
+        int64_t i = e / d4;
+        int c = 4 * (int)(e - i * d4);
+        const float lse = row_lse[i];
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int g = 0; g < groups; ++g) {
+            const float w = expf(part_m[(int64_t)(2 * g) * B + i] - lse);
+            const float4 v = partial[(int64_t)g * total + e];
+            acc.x = fmaf(v.x, w, acc.x); acc.y = fmaf(v.y, w, acc.y);
+            acc.z = fmaf(v.z, w, acc.z); acc.w = fmaf(v.w, w, acc.w);
+        }
+        const int32_t r = pos_idx[i];
+        if (pos_flags(r, i, N, mask_mode) == 0) {
+            const float pm1 = expf(pos_ws[i] - lse) - 1.f;
+            const __nv_bfloat16* pr = P + (int64_t)r * ldp + c;
+            acc.x = fmaf(pm1, __bfloat162float(pr[0]), acc.x);
+            acc.y = fmaf(pm1, __bfloat162float(pr[1]), acc.y);
+            acc.z = fmaf(pm1, __bfloat162float(pr[2]), acc.z);
+            acc.w = fmaf(pm1, __bfloat162float(pr[3]), acc.w);
+        }
+        *reinterpret_cast<float4*>(out + i * ldo + c) =
+            make_float4(acc.x * scale, acc.y * scale, acc.z * scale, acc.w * scale);
+    }
+}
+
 }  // namespace
+
+cudaError_t launch_fused_dq_finalize(const float* partial, int groups, const float* part_m,
+                                     const float* row_lse, const float* pos_ws,
+                                     const int32_t* pos_idx, const void* P, int64_t ldp,
+                                     int64_t B, int64_t N, int d, int mask_mode, float scale,
+                                     float* out, int64_t ldo, cudaStream_t st) {
+    int64_t total = B * (d / 4);
+    int64_t blocks = (total + 255) / 256;
+    int cap = sm_count() * 8;
+    if (blocks > cap) blocks = cap;
+    fused_dq_finalize_kernel<<<(int)blocks, 256, 0, st>>>(
+        reinterpret_cast<const float4*>(partial), groups, part_m, row_lse, pos_ws, pos_idx,
+        static_cast<const __nv_bfloat16*>(P), ldp, B, N, d / 4, mask_mode, scale, out, ldo);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_lse_combine(const float* part_m, const float* part_l, const float* pos_ws,
                                const int32_t* pos_idx, int groups, int64_t B, int64_t N,

@@ -65,6 +65,8 @@ struct Plan {
     size_t off_m, off_l, off_pos, off_accq, off_accp;
     size_t total;           // workspace bytes (multiple of 256)
     int launches_fwd, launches_bwd;
+    int fused;              // 1: gc_build_cache runs the forward inside the dQ sweep
+    int launches_build;
 };
 
 int sm_count();
@@ -77,6 +79,11 @@ cudaError_t launch_lse_combine(const float* part_m, const float* part_l, const f
                                int* dev_status, cudaStream_t st);
 cudaError_t launch_pos_check(const int32_t* pos_idx, int64_t B, int64_t N, int mask_mode,
                              int* dev_status, cudaStream_t st);
+cudaError_t launch_fused_dq_finalize(const float* partial, int groups, const float* part_m,
+                                     const float* row_lse, const float* pos_ws,
+                                     const int32_t* pos_idx, const void* P, int64_t ldp,
+                                     int64_t B, int64_t N, int d, int mask_mode, float scale,
+                                     float* out, int64_t ldo, cudaStream_t st);
 cudaError_t launch_partial_reduce(const float* partial, int groups, int64_t rows, int d,
                                   float scale, float* out, int64_t ldo, cudaStream_t st);
 
@@ -91,6 +98,8 @@ bool tc_supported(int64_t B, int64_t N, int d, int dtype);
 cudaError_t tc_launch_fwd(const FwdArgs& a, cudaStream_t st);
 cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st);
 int tc_fwd_groups(int64_t B, int64_t N, int d);
+bool tc_fused_applicable(int d);
+cudaError_t tc_launch_fused_dq(const FwdArgs& a, float* partial, int groups, cudaStream_t st);
 int tc_sweep_groups(int64_t nx, int64_t ny, int d);
 
 }  // namespace gc

@@ -5,6 +5,11 @@
 //   FWD  (Eq. 1)    x = 128 queries,  y streams passages: S = X Y^T, online row max / sum.
 //   DQ   (Eq. 5)    x = 128 queries,  y streams passages: W = exp(S - lse_x) - onehot, acc += W Y
 //   DP   (Eq. 6-7)  x = 128 passages, y streams queries:  W = exp(S - lse_y) - onehot, acc += W Y
+//   FQ   (Eq. 1+5)  forward fused into the dQ sweep (used by gc_build_cache for wide rows): the
+//                   row maximum runs online, W = exp(S - m_ref) with the positive column left
+//                   out, acc += W Y; the accumulator is rescaled only when the maximum grows by
+//                   more than 2^8.  A finalize pass forms (sum_g acc_g exp(m_g - lse)
+//                   + (p_pos - 1) P_pos) / (B tau) with the positive term in fp32.
 //
 // The stationary tile X (128 x d) stays resident in shared memory when d <= 512; for wider rows
 // only its first 6 column chunks stay and the others are re-streamed every step, which leaves
@@ -48,13 +53,13 @@ constexpr size_t SMEM_LIMIT = 232448;      // 227 KB per block
 constexpr size_t SMEM_STATIC_RESERVE = 2048;
 constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
 
-enum { MODE_FWD = 0, MODE_DQ = 1, MODE_DP = 2 };
+enum { MODE_FWD = 0, MODE_DQ = 1, MODE_DP = 2, MODE_FQ = 3 };   // FQ: forward fused into dQ
 
 // Optional diagnostics (-DGC_TC_TRACE): cycles each role spends waiting, summed over CTAs.
 #ifdef GC_TC_TRACE
 enum { TR_MMA_TOTAL, TR_MMA_WAIT_Y, TR_MMA_WAIT_W, TR_SM_TOTAL, TR_SM_WAIT_S, TR_SM_EPI,
        TR_PROD_TOTAL, TR_PROD_WAIT, TR_CTAS, TR_MMA_ISSUE, TR_MMA_COMMIT, TR_ACC_ISSUE, TR_ACC_COMMIT, TR_SFULL_COMMIT, TR_COUNT };
-__device__ unsigned long long g_trace[3][TR_COUNT];
+__device__ unsigned long long g_trace[4][TR_COUNT];
 #define TR_DECL(v) long long v = 0
 #define TR_BEGIN(v) long long v##_t0 = clock64()
 #define TR_END(v) v += clock64() - v##_t0
@@ -264,6 +269,7 @@ struct Bars {
     uint64_t s_full[2];
     uint64_t w_full[2];
     uint64_t acc_full;
+    uint64_t pair[4];          // FQ: the two softmax warps of a lane quarter agree on the row max
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -277,6 +283,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     __shared__ __align__(8) Bars bars;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
+    __shared__ float row_max_xch[2][XROWS];      // FQ: [column half][row] block maxima
     volatile int* abort_flag = &abort_s;
 
     static_assert(SN == 128, "a Y chunk is 128 rows: the same 16 KB as an X chunk");
@@ -317,6 +324,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             mbar_init(smem_u32(&bars.w_full[b]), NSOFT);  // one arrival per softmax warp
         }
         mbar_init(smem_u32(&bars.acc_full), 1);
+        for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&bars.pair[i]), 2);   // one per warp
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == MMA_WARP) {
@@ -596,6 +604,164 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 p.part_m[slot] = m * 0.69314718055994531f;   // back to natural log
                 p.part_l[slot] = l;
             }
+        } else if (MODE == MODE_FQ) {
+            // ---------------- forward fused into the dQ sweep ----------------
+            // m_ref is the power-of-two scale all weights of a row share (both column halves);
+            // l is this half's sum of 2^(s2 - m_ref) over its allowed columns, positive included.
+            float m_ref = 0.f, l = 0.f;
+            const int32_t pos_x = (x < p.nx) ? p.pos_idx[x] : -1;
+            for (int t = 0; t < T; ++t) {
+                const int64_t y0 = (lo + t) * SN;
+                TR_BEGIN(tr_ws);
+                ok = mbar_wait(smem_u32(&bars.s_full[0]), t & 1, abort_flag);
+                TR_END(tr_ws);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t sbuf = tmem + lane_addr + S_COL0;
+                // ---- pass 1: maximum of this half's live logits (raw dot products; c1 > 0) ----
+                float bm = -INFINITY;
+                {
+                    uint32_t vv[CB_PER][32];
+#pragma unroll
+                    for (int j = 0; j < CB_PER; ++j) tmem_ld32(sbuf + (cb0 + j) * 32, vv[j]);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < CB_PER; ++j) {
+                        const int64_t yb = y0 + (cb0 + j) * 32;
+                        const bool has_pos = pos_x >= yb && pos_x < yb + 32 && pos_x < p.ny &&
+                                             !(self_mask && x == pos_x);
+                        if (has_pos) {
+                            const int rel = (int)(pos_x - yb);
+                            float sp = 0.f;
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (c == rel) sp = __uint_as_float(vv[j][c]);
+                            p.pos_logit[x] = sp * p.inv_tau;
+                        }
+                        if (yb + 32 > p.ny) {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (yb + c >= p.ny) vv[j][c] = __float_as_uint(-INFINITY);
+                        }
+                        if (self_mask && x >= yb && x < yb + 32) {
+                            const int rel = (int)(x - yb);
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (c == rel) vv[j][c] = __float_as_uint(-INFINITY);
+                        }
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) bm = fmaxf(bm, __uint_as_float(vv[j][c]));
+                    }
+                }
+                bm *= p.c1;                                            // log2 domain
+                // agree on the tile maximum with the warp that owns the other column half (the
+                // partner reads this before it arrives on w_full for this step, and the next
+                // write only happens after the S tile of the next step, which needs that arrival)
+                row_max_xch[half][row] = bm;
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars.pair[q]));
+                ok = mbar_wait(smem_u32(&bars.pair[q]), t & 1, abort_flag);
+                if (!ok) break;
+                const float tile_max = fmaxf(bm, row_max_xch[half ^ 1][row]);
+                if (t == 0) {
+                    m_ref = (tile_max > -INFINITY) ? tile_max : 0.f;
+                } else if (__any_sync(0xffffffffu, tile_max > m_ref + 8.f)) {
+                    // rare: some row's maximum outgrew its reference by more than 2^8.  The
+                    // tensor-memory accesses are warp-wide, so every lane moves its reference
+                    // to max(m_ref, tile_max) (factor 1 where nothing changes).  Both warps of
+                    // the quarter see the same rows and values, hence take the same branch, and
+                    // rescale alternate 32-column blocks of the accumulator.
+                    const float m_new = fmaxf(m_ref, tile_max);
+                    const float f = ex2(m_ref - m_new);
+                    l *= f;
+                    for (int cb = half; cb < c_count * 2; cb += 2) {
+                        uint32_t a[32];
+                        tmem_ld32(tmem + lane_addr + cb * 32, a);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            a[c] = __float_as_uint(__uint_as_float(a[c]) * f);
+                        tmem_st16(tmem + lane_addr + cb * 32,
+                                  *reinterpret_cast<const uint32_t(*)[16]>(&a[0]));
+                        tmem_st16(tmem + lane_addr + cb * 32 + 16,
+                                  *reinterpret_cast<const uint32_t(*)[16]>(&a[16]));
+                    }
+                    m_ref = m_new;
+                }
+                // ---- pass 2: weights 2^(s2 - m_ref), their sum, bf16 W without the positive ----
+#pragma unroll
+                for (int j = 0; j < CB_PER; ++j) {
+                    const int64_t yb = y0 + (cb0 + j) * 32;
+                    uint32_t v[32];
+                    tmem_ld32(sbuf + (cb0 + j) * 32, v);
+                    tmem_ld_wait();
+                    float w[32];
+#pragma unroll
+                    for (int c = 0; c < 32; ++c)
+                        w[c] = ex2(fmaf(__uint_as_float(v[c]), p.c1, -m_ref));
+                    if (yb + 32 > p.ny) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (yb + c >= p.ny) w[c] = 0.f;
+                    }
+                    if (self_mask && x >= yb && x < yb + 32) {
+                        const int rel = (int)(x - yb);
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (c == rel) w[c] = 0.f;
+                    }
+                    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 32; c += 4) {
+                        s0 += w[c]; s1 += w[c + 1]; s2 += w[c + 2]; s3 += w[c + 3];
+                    }
+                    l += (s0 + s1) + (s2 + s3);
+                    if (pos_x >= yb && pos_x < yb + 32) {                  // positive: fp32 later
+                        const int rel = (int)(pos_x - yb);
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (c == rel) w[c] = 0.f;
+                    }
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(w[2 * r], w[2 * r + 1]);
+                        packed[r] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                    tmem_st16(sbuf + half * (SN / 2) + j * 16, packed);
+                }
+                tmem_st_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars.w_full[0]));
+            }
+            // (scale, sum) of this half; only the first column part writes (both parts agree)
+            if (ok && x < p.nx && dp == 0) {
+                const int64_t slot = (int64_t)(2 * g + half) * p.nq + x;
+                p.part_m[slot] = m_ref * 0.69314718055994531f;
+                p.part_l[slot] = l;
+            }
+            // unscaled accumulator part -> partial buffer [g][nx][d]
+            TR_BEGIN(tr_epi);
+            if (ok) ok = mbar_wait(smem_u32(&bars.acc_full), 0, abort_flag);
+            if (ok) {
+                tc_fence_after();
+                const int64_t d = (int64_t)p.kc * 64;
+                float* dst = p.partial + ((int64_t)g * p.nx + x) * d + c_begin * 64;
+                for (int cb = half; cb < c_count * 2; cb += 2) {
+                    uint32_t v[32];
+                    tmem_ld32(tmem + lane_addr + cb * 32, v);
+                    tmem_ld_wait();
+                    if (x < p.nx) {
+#pragma unroll
+                        for (int c = 0; c < 32; c += 4)
+                            *reinterpret_cast<float4*>(dst + cb * 32 + c) =
+                                make_float4(__uint_as_float(v[c]), __uint_as_float(v[c + 1]),
+                                            __uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
+                    }
+                }
+            }
+            TR_END(tr_epi);
         } else {
             // per-row constants (DQ: the row is a query)
             float lse2_x = 0.f;
@@ -836,7 +1002,7 @@ cudaError_t launch(const CUtensorMap& mx, const CUtensorMap& my, const TcParams&
 extern "C" int gc_debug_trace(unsigned long long* out, int clear) {
     if (out && cudaMemcpyFromSymbol(out, g_trace, sizeof(g_trace)) != cudaSuccess) return 1;
     if (clear) {
-        static unsigned long long zero[3][TR_COUNT] = {};
+        static unsigned long long zero[4][TR_COUNT] = {};
         if (cudaMemcpyToSymbol(g_trace, zero, sizeof(zero)) != cudaSuccess) return 1;
     }
     return 0;
@@ -892,6 +1058,35 @@ cudaError_t tc_launch_fwd(const FwdArgs& a, cudaStream_t st) {
     p.dev_status = a.dev_status;
     int64_t units = ((pr.B + XROWS - 1) / XROWS) * p.groups;
     return launch<MODE_FWD, SN, 2>(mx, my, p, units, st);
+}
+
+bool tc_fused_applicable(int d) { return sweep_nbuf(d / 64) == 1; }
+
+// Forward fused into the dQ sweep: writes (scale, sum) slots [2 groups][B], pos_logit and the
+// unscaled accumulators partial[groups][B][d].
+cudaError_t tc_launch_fused_dq(const FwdArgs& a, float* partial, int groups, cudaStream_t st) {
+    const Problem& pr = a.p;
+    constexpr int SN = 128;
+    const int kc = pr.d / 64;
+    CUtensorMap mx, my;
+    if (!make_map(&mx, pr.Q, pr.B, pr.d, pr.ldq, XROWS) ||
+        !make_map(&my, pr.P, pr.N, pr.d, pr.ldp, SN))
+        return cudaErrorInvalidValue;
+    TcParams p{};
+    p.nx = pr.B; p.ny = pr.N; p.nq = pr.B;
+    p.kc = kc; p.dparts = parts_for(kc); p.dpc = chunks_per_part(kc); p.groups = groups;
+    p.nstage = smem_plan(kc).nstage;
+    p.xres = smem_plan(kc).xres;
+    p.ipc = smem_plan(kc).ipc;
+    p.mask_mode = pr.mask_mode;
+    p.inv_tau = 1.f / pr.tau;
+    p.c1 = 1.4426950408889634f / pr.tau;
+    p.pos_idx = pr.pos_idx;
+    p.part_m = a.part_m; p.part_l = a.part_l; p.pos_logit = a.pos_logit;
+    p.partial = partial;
+    p.dev_status = a.dev_status;
+    int64_t units = ((pr.B + XROWS - 1) / XROWS) * p.dparts * groups;
+    return launch<MODE_FQ, SN, 1>(mx, my, p, units, st);
 }
 
 cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {

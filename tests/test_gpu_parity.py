@@ -52,8 +52,10 @@ def test_self_mask_shared_rows(binding, oracle, n, d, tau, dtype):
 
 
 def test_fwd_then_bwd_equals_build(binding, oracle):
-    """The separate forward and backward calls reproduce the fused call bit for bit."""
-    for dtype, d in (("f32", 96), ("bf16", 768)):
+    """The separate forward and backward calls reproduce gc_build_cache: bit for bit where both
+    run the same kernels, within rounding where gc_build_cache fuses the forward into the dQ
+    sweep (wide bf16 rows)."""
+    for dtype, d in (("f32", 96), ("bf16", 128), ("bf16", 768)):
         prob = inputs.random_problem(150, 333, d, dtype, seed=9, tau=0.7, scale=d ** -0.5)
         Q, P, pos = to_device(prob)
         a = binding.build_cache(Q, P, pos, prob.tau, prob.mask_mode)
@@ -63,12 +65,19 @@ def test_fwd_then_bwd_equals_build(binding, oracle):
         binding.gc_loss_bwd(Q, P, pos, prob.tau, prob.mask_mode, b.row_lse, b.dQ, b.dP, b.ws,
                             b.dev_status)
         torch.cuda.synchronize()
-        for name in ("loss", "row_lse", "pos_logit", "dQ", "dP"):
-            assert torch.equal(getattr(a, name), getattr(b, name)), name
+        if d == 768:
+            assert torch.equal(a.pos_logit, b.pos_logit)
+            torch.testing.assert_close(a.loss, b.loss, rtol=1e-5, atol=0)
+            torch.testing.assert_close(a.row_lse, b.row_lse, rtol=1e-5, atol=1e-5)
+            assert grad_err(a.dQ.cpu().numpy(), b.dQ.cpu().numpy()) <= 1e-2
+            assert grad_err(a.dP.cpu().numpy(), b.dP.cpu().numpy()) <= 1e-2
+        else:
+            for name in ("loss", "row_lse", "pos_logit", "dQ", "dP"):
+                assert torch.equal(getattr(a, name), getattr(b, name)), name
         # either gradient may be skipped
         c = binding.Outputs(prob.B, prob.N, prob.d, binding._dtype_code(Q))
         c.dQ.fill_(7.0)
-        binding.gc_loss_bwd(Q, P, pos, prob.tau, prob.mask_mode, b.row_lse, None, c.dP, c.ws)
+        binding.gc_loss_bwd(Q, P, pos, prob.tau, prob.mask_mode, a.row_lse, None, c.dP, c.ws)
         torch.cuda.synchronize()
         assert torch.equal(c.dP, a.dP) and bool((c.dQ == 7.0).all())
 
