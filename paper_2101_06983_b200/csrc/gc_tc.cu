@@ -163,6 +163,44 @@ __device__ __forceinline__ bool elect_one() {
         : "=r"(pred));
     return pred != 0;
 }
+// ---- CTA-pair (cluster of 2) helpers -------------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\t"
+                 "barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];"
+                 ::"r"(cluster_addr) : "memory");
+}
+// Bulk tensor load of a CTA pair: the data lands in the executing CTA, the transaction bytes are
+// counted on an mbarrier that may live in the other CTA of the pair (no multicast).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0,
+                                                 int c1, uint32_t bar_cluster) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar_cluster)
+        : "memory");
+}
+// Arrives on the mbarrier at this offset in both CTAs of the pair once all MMAs issued so far
+// by this thread have completed.
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 "
+        "[%0], %1;"
+        ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
 __device__ __forceinline__ void tc_fence_before() {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }
@@ -185,29 +223,50 @@ __device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
 }
 // D[tmem] (+)= A[smem] * B[smem].  The issuing thread is alone on its scheduler, so every scalar
 // instruction spent per MMA shows up as idle tensor time: keep the operands precomputed.
-template <bool ACC>
+template <bool ACC, bool PAIR>
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo,
                                        uint32_t idesc) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-        "setp.ne.b32 p, %5, 0;\n\t"
-        "mov.b64 da, {%1, %4};\n\t"
-        "mov.b64 db, {%2, %4};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(DESC_HI), "n"(ACC ? 1 : 0)
-        : "memory");
+    if (PAIR) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+            "setp.ne.b32 p, %5, 0;\n\t"
+            "mov.b64 da, {%1, %4};\n\t"
+            "mov.b64 db, {%2, %4};\n\t"
+            "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(DESC_HI), "n"(ACC ? 1 : 0)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+            "setp.ne.b32 p, %5, 0;\n\t"
+            "mov.b64 da, {%1, %4};\n\t"
+            "mov.b64 db, {%2, %4};\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(DESC_HI), "n"(ACC ? 1 : 0)
+            : "memory");
+    }
 }
 // D[tmem] (+)= A[tmem] * B[smem]
-template <bool ACC>
+template <bool ACC, bool PAIR>
 __device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo,
                                        uint32_t idesc) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
-        "setp.ne.b32 p, %5, 0;\n\t"
-        "mov.b64 db, {%2, %4};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(DESC_HI), "n"(ACC ? 1 : 0)
-        : "memory");
+    if (PAIR) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+            "setp.ne.b32 p, %5, 0;\n\t"
+            "mov.b64 db, {%2, %4};\n\t"
+            "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], db, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(DESC_HI), "n"(ACC ? 1 : 0)
+            : "memory");
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
+            "setp.ne.b32 p, %5, 0;\n\t"
+            "mov.b64 db, {%2, %4};\n\t"
+            "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
+            ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(DESC_HI), "n"(ACC ? 1 : 0)
+            : "memory");
+    }
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile(
@@ -244,14 +303,14 @@ __device__ __forceinline__ float ex2(float x) {
 }
 
 // Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, M = 128.
-__device__ __forceinline__ uint32_t instr_desc(int n, bool b_mn_major) {
+__device__ __forceinline__ uint32_t instr_desc(int n, bool b_mn_major, int m = XROWS) {
     uint32_t d = 0;
     d |= 1u << 4;                          // D format f32
     d |= 1u << 7;                          // A format bf16
     d |= 1u << 10;                         // B format bf16
     d |= (b_mn_major ? 1u : 0u) << 16;     // B major
     d |= (uint32_t)(n >> 3) << 17;
-    d |= (uint32_t)(XROWS >> 4) << 24;
+    d |= (uint32_t)(m >> 4) << 24;          // 128, or 256 for an MMA across a CTA pair
     return d;
 }
 
@@ -275,10 +334,17 @@ struct Bars {
 // ---------------------------------------------------------------------------------------------
 // The sweep kernel
 // ---------------------------------------------------------------------------------------------
-template <int MODE, int SN, int NBUF>
+// PAIR: the kernel runs as clusters of two CTAs that own two neighbouring x tiles of the same
+// column part.  The leader (rank 0) issues every MMA with cta_group::2 (M = 256: 128 rows in each
+// CTA's tensor memory); each CTA loads its own X chunks but only its half of every Y chunk (the
+// 64 streamed rows of its rank for the S MMAs, the 64 columns of its rank for the accumulation
+// MMAs), which halves the Y traffic into shared memory.  "Full" barriers live in the leader and
+// count the bytes landing in both CTAs; "empty", s_full and acc_full are signalled in both CTAs by
+// multicast commits; the softmax warps of both CTAs arrive on the leader's w_full.
+template <int MODE, int SN, int NBUF, bool PAIR>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
-          const TcParams p) {
+          const __grid_constant__ CUtensorMap mapYh, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) Bars bars;
     __shared__ uint32_t tmem_base_s;
@@ -294,11 +360,14 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     const int lane = threadIdx.x & 31;
 
     // work item: (x tile, column part, part of the streamed range)
-    int unit = blockIdx.x;
+    const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
+    const bool leader = (rank == 0);
+    constexpr uint32_t NCTA = PAIR ? 2u : 1u;
+    int unit = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
     const int g = unit % p.groups;
     unit /= p.groups;
     const int dp = unit % p.dparts;
-    const int64_t xt = unit / p.dparts;
+    const int64_t xt = PAIR ? 2 * (int64_t)(unit / p.dparts) + rank : unit / p.dparts;
     const int64_t x0 = xt * XROWS;
     const int c_begin = dp * p.dpc;
     const int c_count = (MODE == MODE_FWD) ? 0 : min(p.dpc, p.kc - c_begin);
@@ -310,7 +379,10 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t x_smem = base;
     const uint32_t y_smem = base + (uint32_t)p.xres * X_CHUNK_BYTES;   // the ring
-    const uint32_t stage_bytes = (uint32_t)p.ipc * CHUNK_BYTES;
+    // a paired CTA holds half of every Y item, so its stages are one chunk (16 KB) and a streamed
+    // X item is a single chunk; otherwise a stage holds ipc chunks of Y or of X
+    const int xipc = PAIR ? 1 : p.ipc;
+    const uint32_t stage_bytes = (uint32_t)xipc * CHUNK_BYTES;
 
     if (threadIdx.x == 0) {
         abort_s = 0;
@@ -321,33 +393,46 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&bars.s_full[b]), 1);
-            mbar_init(smem_u32(&bars.w_full[b]), NSOFT);  // one arrival per softmax warp
+            mbar_init(smem_u32(&bars.w_full[b]), NCTA * NSOFT);   // one arrival per softmax warp
         }
         mbar_init(smem_u32(&bars.acc_full), 1);
         for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&bars.pair[i]), 2);   // one per warp
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == MMA_WARP) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                     ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)TMEM_COLS) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) {   // the same warp of both CTAs, same destination offset
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)TMEM_COLS) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                         ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)TMEM_COLS) : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();     // both CTAs' barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem = tmem_base_s;
+    // shared::cluster address, in the leader, of the barrier at the same offset as `local`
+    auto in_leader = [&](uint32_t local) -> uint32_t { return PAIR ? mapa_u32(local, 0) : local; };
 
     if (warp < NPROD) {
         // ------------------------------ TMA producers -----------------------------------------
         // Chunk number n of the stream goes to ring stage n % nstage; a stage always belongs to
         // the same producer warp (stage % NPROD), which therefore sees its phases in order.
         {   // all 32 lanes run the loop; one elected lane issues
-            if (warp == 0 && elect_one())
-                mbar_expect_tx(smem_u32(&bars.x_full), (uint32_t)p.xres * X_CHUNK_BYTES);
+            // one load, counted on the leader's barrier when the CTAs are paired
+            auto tma = [&](uint32_t dst, const CUtensorMap* map, int col, int64_t r, uint32_t bar) {
+                if (PAIR) tma_load_2d_pair(dst, map, col, (int)r, bar);
+                else      tma_load_2d(dst, map, col, (int)r, bar);
+            };
+            const uint32_t x_full_bar = in_leader(smem_u32(&bars.x_full));
+            if (warp == 0 && leader && elect_one())
+                mbar_expect_tx(smem_u32(&bars.x_full), NCTA * (uint32_t)p.xres * X_CHUNK_BYTES);
             for (int c = warp; c < p.xres; c += NPROD)
-                if (elect_one())
-                    tma_load_2d(x_smem + c * X_CHUNK_BYTES, &mapX, c * 64, (int)x0,
-                                smem_u32(&bars.x_full));
+                if (elect_one()) tma(x_smem + c * X_CHUNK_BYTES, &mapX, c * 64, x0, x_full_bar);
             int next = 0;
             uint32_t next_phase = 0;
             bool ok = true;
@@ -369,28 +454,46 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 }
                 return stage;
             };
-            // One ring item: p.ipc consecutive 64-column chunks of 128 rows of Y (or of X).
-            auto load_item = [&](const CUtensorMap* map, int chunk0, int64_t row) {
+            // Ring items.  kind 0: Y for the S MMAs (ipc chunks; a paired CTA loads the 64 rows of
+            // its rank); kind 1: streamed X chunks (ipc chunks of this CTA's 128 rows); kind 2: Y
+            // for the accumulation MMAs (ipc chunks; a paired CTA loads the one chunk of its rank).
+            auto load_item = [&](int kind, int chunk0, int64_t row) {
                 const int stage = acquire();
                 if (stage < 0) return;
                 const uint32_t full = smem_u32(&bars.y_full[stage]);
+                const uint32_t full_bar = in_leader(full);
+                const uint32_t dst = y_smem + stage * stage_bytes;
                 if (elect_one()) {
-                    mbar_expect_tx(full, stage_bytes);
-                    for (int i = 0; i < p.ipc; ++i)
-                        tma_load_2d(y_smem + stage * stage_bytes + i * CHUNK_BYTES, map,
-                                    (chunk0 + i) * 64, (int)row, full);
+                    if (kind == 1) {
+                        if (leader) mbar_expect_tx(full, NCTA * stage_bytes);
+                        for (int i = 0; i < xipc; ++i)
+                            tma(dst + i * CHUNK_BYTES, &mapX, (chunk0 + i) * 64, x0, full_bar);
+                    } else if (!PAIR) {
+                        mbar_expect_tx(full, stage_bytes);
+                        for (int i = 0; i < p.ipc; ++i)
+                            tma(dst + i * CHUNK_BYTES, &mapY, (chunk0 + i) * 64, row, full_bar);
+                    } else if (kind == 0) {
+                        if (leader) mbar_expect_tx(full, (uint32_t)p.ipc * CHUNK_BYTES);  // 2 halves
+                        for (int i = 0; i < p.ipc; ++i)
+                            tma(dst + i * (CHUNK_BYTES / 2), &mapYh, (chunk0 + i) * 64,
+                                row + 64 * rank, full_bar);
+                    } else {
+                        if (leader) mbar_expect_tx(full, 2 * CHUNK_BYTES);      // one chunk per CTA
+                        tma(dst, &mapY, (chunk0 + (int)rank) * 64, row, full_bar);
+                    }
                 }
             };
             for (int t = 0; t < T + LAG && ok; ++t) {
                 if (t < T) {
                     for (int c = 0; c < p.kc; c += p.ipc) {
-                        load_item(&mapY, c, (lo + t) * SN);
-                        if (c >= p.xres) load_item(&mapX, c, x0);
+                        load_item(0, c, (lo + t) * SN);
+                        if (c >= p.xres)
+                            for (int j = 0; j < p.ipc; j += xipc) load_item(1, c + j, x0);
                     }
                 }
                 if (MODE != MODE_FWD && t >= LAG) {
                     for (int c = 0; c < c_count; c += p.ipc)
-                        load_item(&mapY, c_begin + c, (lo + t - LAG) * SN);
+                        load_item(2, c_begin + c, (lo + t - LAG) * SN);
                 }
             }
 #ifdef GC_TC_TRACE
@@ -403,15 +506,23 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
         }
     } else if (warp == MMA_WARP) {
         // ------------------------------ MMA issuer ----------------------------------------------
-        {   // all 32 lanes run the loop; one elected lane issues the MMAs and commits
-            const uint32_t idesc_s = instr_desc(SN, false);
-            const uint32_t idesc_acc64 = instr_desc(64, true);
-            const uint32_t idesc_acc128 = instr_desc(128, true);
+        if (leader) {   // all 32 lanes run the loop; one elected lane issues the MMAs and commits
+            constexpr int MROWS = PAIR ? 2 * XROWS : XROWS;
+            const uint32_t idesc_s = instr_desc(SN, false, MROWS);
+            const uint32_t idesc_acc64 = instr_desc(64, true, MROWS);
+            const uint32_t idesc_acc128 = instr_desc(128, true, MROWS);
+            // arrives on the given barrier (of both CTAs when paired) when the MMAs so far are done
+            auto commit = [&](uint32_t bar) {
+                if (PAIR) tc_commit_pair(bar);
+                else      tc_commit(bar);
+            };
+            // S-phase Y chunks of one stage are 16 KB apart, or 8 KB when each CTA holds 64 rows
+            constexpr uint32_t YCH_LO = (PAIR ? CHUNK_BYTES / 2 : CHUNK_BYTES) >> 4;
             const uint32_t x_lo = desc_lo(x_smem, 0);
             const uint32_t ring_lo = desc_lo(y_smem, CHUNK_BYTES);   // LBO: next chunk of a stage
             constexpr uint32_t CH_LO = CHUNK_BYTES >> 4;
             const uint32_t stage_lo = stage_bytes >> 4;
-            const uint32_t idesc_acc = (p.ipc == 2) ? idesc_acc128 : idesc_acc64;
+            const uint32_t idesc_acc = (p.ipc == 2) ? idesc_acc128 : idesc_acc64;   // paired: ipc == 2
             int next = 0;
             uint32_t next_phase = 0;
             TR_DECL(tr_wy);
@@ -451,35 +562,64 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     for (int c = 0; c < p.kc && ok; c += p.ipc) {
                         const int ys = next_stage();
                         if (!ok) break;
-                        int xs = -1;
-                        uint32_t xa = x_lo + c * CH_LO;
-                        if (c >= p.xres) {
-                            xs = next_stage();
-                            if (!ok) break;
-                            xa = ring_lo + xs * stage_lo;
-                        }
                         const uint32_t yb = ring_lo + ys * stage_lo;
-                        TR_BEGIN(tr_is);
-                        if (elect_one()) {
-                            if (c == 0) mma_ss<false>(d_tmem, xa, yb, idesc_s);
-                            else        mma_ss<true>(d_tmem, xa, yb, idesc_s);
-                            mma_ss<true>(d_tmem, xa + 2, yb + 2, idesc_s);
-                            mma_ss<true>(d_tmem, xa + 4, yb + 4, idesc_s);
-                            mma_ss<true>(d_tmem, xa + 6, yb + 6, idesc_s);
-                            if (p.ipc == 2) {
-                                mma_ss<true>(d_tmem, xa + CH_LO, yb + CH_LO, idesc_s);
-                                mma_ss<true>(d_tmem, xa + CH_LO + 2, yb + CH_LO + 2, idesc_s);
-                                mma_ss<true>(d_tmem, xa + CH_LO + 4, yb + CH_LO + 4, idesc_s);
-                                mma_ss<true>(d_tmem, xa + CH_LO + 6, yb + CH_LO + 6, idesc_s);
+                        if (!PAIR) {
+                            // one ring item of Y and (for streamed chunks) one of X: ipc chunks,
+                            // issued from a single elected region (scalar work per item is what
+                            // limits the issuing warp)
+                            int xs = -1;
+                            uint32_t xa = x_lo + c * CH_LO;
+                            if (c >= p.xres) {
+                                xs = next_stage();
+                                if (!ok) break;
+                                xa = ring_lo + xs * stage_lo;
                             }
-                            if (xs >= 0) tc_commit(smem_u32(&bars.y_empty[xs]));
-                            tc_commit(smem_u32(&bars.y_empty[ys]));
+                            TR_BEGIN(tr_is);
+                            if (elect_one()) {
+                                if (c == 0) mma_ss<false, false>(d_tmem, xa, yb, idesc_s);
+                                else        mma_ss<true, false>(d_tmem, xa, yb, idesc_s);
+                                mma_ss<true, false>(d_tmem, xa + 2, yb + 2, idesc_s);
+                                mma_ss<true, false>(d_tmem, xa + 4, yb + 4, idesc_s);
+                                mma_ss<true, false>(d_tmem, xa + 6, yb + 6, idesc_s);
+                                if (p.ipc == 2) {
+                                    mma_ss<true, false>(d_tmem, xa + CH_LO, yb + CH_LO, idesc_s);
+                                    mma_ss<true, false>(d_tmem, xa + CH_LO + 2, yb + CH_LO + 2, idesc_s);
+                                    mma_ss<true, false>(d_tmem, xa + CH_LO + 4, yb + CH_LO + 4, idesc_s);
+                                    mma_ss<true, false>(d_tmem, xa + CH_LO + 6, yb + CH_LO + 6, idesc_s);
+                                }
+                                if (xs >= 0) tc_commit(smem_u32(&bars.y_empty[xs]));
+                                tc_commit(smem_u32(&bars.y_empty[ys]));
+                            }
+                            TR_END(tr_is);
+                        } else {
+                            // paired: the Y item holds this CTA's 64 rows of two chunks (8 KB
+                            // each), every streamed X chunk is an item of its own
+                            for (int j = 0; j < 2 && ok; ++j) {
+                                int xs = -1;
+                                uint32_t xa = x_lo + (c + j) * CH_LO;
+                                if (c + j >= p.xres) {
+                                    xs = next_stage();
+                                    if (!ok) break;
+                                    xa = ring_lo + xs * stage_lo;
+                                }
+                                const uint32_t yj = yb + j * YCH_LO;
+                                TR_BEGIN(tr_is);
+                                if (elect_one()) {
+                                    if (c + j == 0) mma_ss<false, true>(d_tmem, xa, yj, idesc_s);
+                                    else            mma_ss<true, true>(d_tmem, xa, yj, idesc_s);
+                                    mma_ss<true, true>(d_tmem, xa + 2, yj + 2, idesc_s);
+                                    mma_ss<true, true>(d_tmem, xa + 4, yj + 4, idesc_s);
+                                    mma_ss<true, true>(d_tmem, xa + 6, yj + 6, idesc_s);
+                                    if (xs >= 0) tc_commit_pair(smem_u32(&bars.y_empty[xs]));
+                                    if (j == 1) tc_commit_pair(smem_u32(&bars.y_empty[ys]));
+                                }
+                                TR_END(tr_is);
+                            }
                         }
-                        TR_END(tr_is);
                     }
                     if (!ok) break;
                     TR_BEGIN(tr_sf);
-                    if (elect_one()) tc_commit(smem_u32(&bars.s_full[b]));
+                    if (elect_one()) commit(smem_u32(&bars.s_full[b]));
                     TR_END(tr_sf);
                 }
                 if (MODE != MODE_FWD && t >= LAG) {
@@ -501,19 +641,20 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                             // k-steps of the first column half read W at columns 8 k, those of
                             // the second half at SN/2 + 8 (k - KH)
                             constexpr int KH = SN / 32;
-                            if (u == 0) mma_ts<false>(d_tmem, w_tmem, yb, idesc_acc);
-                            else        mma_ts<true>(d_tmem, w_tmem, yb, idesc_acc);
+                            if (u == 0) mma_ts<false, PAIR>(d_tmem, w_tmem, yb, idesc_acc);
+                            else        mma_ts<true, PAIR>(d_tmem, w_tmem, yb, idesc_acc);
 #pragma unroll
                             for (int k = 1; k < SN / 16; ++k)
-                                mma_ts<true>(d_tmem, w_tmem + (k / KH) * (SN / 2) + (k % KH) * 8,
-                                             yb + k * 128, idesc_acc);
-                            tc_commit(smem_u32(&bars.y_empty[ys]));
+                                mma_ts<true, PAIR>(d_tmem,
+                                                   w_tmem + (k / KH) * (SN / 2) + (k % KH) * 8,
+                                                   yb + k * 128, idesc_acc);
+                            commit(smem_u32(&bars.y_empty[ys]));
                         }
                         TR_END(tr_ai);
                     }
                 }
             }
-            if (ok && MODE != MODE_FWD && elect_one()) tc_commit(smem_u32(&bars.acc_full));
+            if (ok && MODE != MODE_FWD && elect_one()) commit(smem_u32(&bars.acc_full));
 #ifdef GC_TC_TRACE
             if (lane == 0) {
             TR_ADD(MODE, TR_MMA_TOTAL, clock64() - tr_total_t0);
@@ -538,6 +679,11 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         const bool self_mask = (p.mask_mode == GC_MASK_SELF);
         bool ok = true;
+        // w_full lives in the CTA that issues the MMAs
+        auto arrive_w = [&](uint32_t local) {
+            if (PAIR && !leader) mbar_arrive_cluster(mapa_u32(local, 0));
+            else                 mbar_arrive(local);
+        };
         TR_DECL(tr_ws);
         TR_DECL(tr_epi);
         TR_BEGIN(tr_total);
@@ -596,7 +742,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 }
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bars.w_full[b]));
+                if (lane == 0) arrive_w(smem_u32(&bars.w_full[b]));
             }
             // one (max, sum) pair per row, part of the streamed range and column half
             if (ok && x < p.nx) {
@@ -733,7 +879,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bars.w_full[0]));
+                if (lane == 0) arrive_w(smem_u32(&bars.w_full[0]));
             }
             // (scale, sum) of this half; only the first column part writes (both parts agree)
             if (ok && x < p.nx && dp == 0) {
@@ -856,7 +1002,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bars.w_full[b]));
+                if (lane == 0) arrive_w(smem_u32(&bars.w_full[b]));
             }
             // epilogue: accumulator columns of this part -> global memory (32-column blocks are
             // dealt alternately to the two warps of a lane quarter)
@@ -906,10 +1052,15 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
         if (threadIdx.x == 0 && p.dev_status) atomicOr(p.dev_status, GC_DEV_WAIT_LIMIT);
         __syncthreads();
     }
+    if (PAIR) cluster_sync_all();   // the peer's MMAs, loads and arrivals no longer touch this CTA
     if (warp == MMA_WARP) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
-                     ::"r"(tmem), "r"((uint32_t)TMEM_COLS) : "memory");
+        if (PAIR)
+            asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;"
+                         ::"r"(tmem), "r"((uint32_t)TMEM_COLS) : "memory");
+        else
+            asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;"
+                         ::"r"(tmem), "r"((uint32_t)TMEM_COLS) : "memory");
     }
 }
 
@@ -961,7 +1112,7 @@ struct SmemPlan { int xres; int ipc; int nstage; size_t dynamic_bytes; };
 
 // Rows up to 512 wide keep the whole X tile resident; wider rows keep 6 chunks so that the ring
 // still has 128 KB.  Ring items hold two chunks when every chunk count involved is even.
-SmemPlan smem_plan(int kc) {
+SmemPlan smem_plan(int kc, bool pair = false) {
     SmemPlan sp;
     sp.xres = kc <= 8 ? kc : 6;
     const int parts = parts_for(kc), dpc = chunks_per_part(kc);
@@ -969,7 +1120,7 @@ SmemPlan smem_plan(int kc) {
                       (kc - dpc * (parts - 1)) % 2 == 0;
     sp.ipc = even ? 2 : 1;
     size_t xbytes = (size_t)sp.xres * X_CHUNK_BYTES;
-    size_t stage = (size_t)sp.ipc * CHUNK_BYTES;
+    size_t stage = pair ? (size_t)CHUNK_BYTES : (size_t)sp.ipc * CHUNK_BYTES;
     size_t avail = SMEM_LIMIT - SMEM_STATIC_RESERVE - 1024 - xbytes;
     int ns = (int)(avail / stage);
     if (ns > MAX_STAGES) ns = MAX_STAGES;
@@ -980,20 +1131,64 @@ SmemPlan smem_plan(int kc) {
     return sp;
 }
 
-template <int MODE, int SN, int NBUF>
-cudaError_t launch(const CUtensorMap& mx, const CUtensorMap& my, const TcParams& p, int64_t units,
-                   cudaStream_t st) {
-    SmemPlan sp = smem_plan(p.kc);
+template <int MODE, int SN, int NBUF, bool PAIR>
+cudaError_t launch_one(const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& myh,
+                       const TcParams& p, int64_t ctas, cudaStream_t st) {
+    SmemPlan sp = smem_plan(p.kc, PAIR);
     static bool configured = false;
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(tc_kernel<MODE, SN, NBUF>,
+        cudaError_t e = cudaFuncSetAttribute(tc_kernel<MODE, SN, NBUF, PAIR>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)(SMEM_LIMIT - SMEM_STATIC_RESERVE));
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    tc_kernel<MODE, SN, NBUF><<<(unsigned)units, NTHREADS, sp.dynamic_bytes, st>>>(mx, my, p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)ctas);
+    cfg.blockDim = dim3(NTHREADS);
+    cfg.dynamicSmemBytes = sp.dynamic_bytes;
+    cfg.stream = st;
+    TcParams pp = p;
+    pp.nstage = sp.nstage;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = PAIR ? 2 : 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (!PAIR) {
+        tc_kernel<MODE, SN, NBUF, false><<<(unsigned)ctas, NTHREADS, sp.dynamic_bytes, st>>>(
+            mx, my, myh, pp);
+        return cudaGetLastError();
+    }
+    return cudaLaunchKernelEx(&cfg, tc_kernel<MODE, SN, NBUF, PAIR>, mx, my, myh, pp);
+}
+
+// CTA pairs need two-chunk ring items (the accumulation MMAs split them by rank) and at least
+// two x tiles.
+// Pairing halves the traffic of the streamed matrix but adds cross-SM hand-offs to every step:
+// it pays when that matrix does not stay in the L2 cache (measured: 2.4 % faster at
+// 65536 x 131072, 3 % slower at 4096 x 8192).
+bool use_pair(int kc, int64_t nx, int64_t ny) {
+    const int64_t streamed_bytes = ny * kc * 128;
+    return smem_plan(kc).ipc == 2 && nx > XROWS && sweep_nbuf(kc) == 1 &&
+           streamed_bytes > (int64_t)64 << 20;
+}
+
+// x tiles (rounded up to whole pairs when paired) * column parts * groups
+int64_t cta_count(int kc, int64_t nx, int64_t ny, int parts, int groups) {
+    int64_t tiles = (nx + XROWS - 1) / XROWS;
+    if (use_pair(kc, nx, ny)) tiles = (tiles + 1) / 2 * 2;
+    return tiles * parts * groups;
+}
+
+template <int MODE, int SN, int NBUF>
+cudaError_t launch(const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& myh,
+                   const TcParams& p, cudaStream_t st) {
+    const int64_t ctas = cta_count(p.kc, p.nx, p.ny, p.dparts, p.groups);
+    if (use_pair(p.kc, p.nx, p.ny)) return launch_one<MODE, SN, NBUF, true>(mx, my, myh, p, ctas, st);
+    return launch_one<MODE, SN, NBUF, false>(mx, my, myh, p, ctas, st);
 }
 
 }  // namespace
@@ -1040,9 +1235,10 @@ int tc_sweep_groups(int64_t nx, int64_t ny, int d) {
 cudaError_t tc_launch_fwd(const FwdArgs& a, cudaStream_t st) {
     const Problem& pr = a.p;
     constexpr int SN = 128;
-    CUtensorMap mx, my;
+    CUtensorMap mx, my, myh;
     if (!make_map(&mx, pr.Q, pr.B, pr.d, pr.ldq, XROWS) ||
-        !make_map(&my, pr.P, pr.N, pr.d, pr.ldp, SN))
+        !make_map(&my, pr.P, pr.N, pr.d, pr.ldp, SN) ||
+        !make_map(&myh, pr.P, pr.N, pr.d, pr.ldp, SN / 2))
         return cudaErrorInvalidValue;
     TcParams p{};
     p.nx = pr.B; p.ny = pr.N; p.nq = pr.B;
@@ -1056,8 +1252,7 @@ cudaError_t tc_launch_fwd(const FwdArgs& a, cudaStream_t st) {
     p.pos_idx = pr.pos_idx;
     p.part_m = a.part_m; p.part_l = a.part_l; p.pos_logit = a.pos_logit;
     p.dev_status = a.dev_status;
-    int64_t units = ((pr.B + XROWS - 1) / XROWS) * p.groups;
-    return launch<MODE_FWD, SN, 2>(mx, my, p, units, st);
+    return launch<MODE_FWD, SN, 2>(mx, my, myh, p, st);
 }
 
 bool tc_fused_applicable(int d) { return sweep_nbuf(d / 64) == 1; }
@@ -1068,9 +1263,10 @@ cudaError_t tc_launch_fused_dq(const FwdArgs& a, float* partial, int groups, cud
     const Problem& pr = a.p;
     constexpr int SN = 128;
     const int kc = pr.d / 64;
-    CUtensorMap mx, my;
+    CUtensorMap mx, my, myh;
     if (!make_map(&mx, pr.Q, pr.B, pr.d, pr.ldq, XROWS) ||
-        !make_map(&my, pr.P, pr.N, pr.d, pr.ldp, SN))
+        !make_map(&my, pr.P, pr.N, pr.d, pr.ldp, SN) ||
+        !make_map(&myh, pr.P, pr.N, pr.d, pr.ldp, SN / 2))
         return cudaErrorInvalidValue;
     TcParams p{};
     p.nx = pr.B; p.ny = pr.N; p.nq = pr.B;
@@ -1085,15 +1281,15 @@ cudaError_t tc_launch_fused_dq(const FwdArgs& a, float* partial, int groups, cud
     p.part_m = a.part_m; p.part_l = a.part_l; p.pos_logit = a.pos_logit;
     p.partial = partial;
     p.dev_status = a.dev_status;
-    int64_t units = ((pr.B + XROWS - 1) / XROWS) * p.dparts * groups;
-    return launch<MODE_FQ, SN, 1>(mx, my, p, units, st);
+    return launch<MODE_FQ, SN, 1>(mx, my, myh, p, st);
 }
 
 cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     const int kc = a.d / 64;
     constexpr int SN = 128;
-    CUtensorMap mx, my;
-    if (!make_map(&mx, a.X, a.nx, a.d, a.ldx, XROWS) || !make_map(&my, a.Y, a.ny, a.d, a.ldy, SN))
+    CUtensorMap mx, my, myh;
+    if (!make_map(&mx, a.X, a.nx, a.d, a.ldx, XROWS) ||
+        !make_map(&my, a.Y, a.ny, a.d, a.ldy, SN) || !make_map(&myh, a.Y, a.ny, a.d, a.ldy, SN / 2))
         return cudaErrorInvalidValue;
     TcParams p{};
     p.nx = a.nx; p.ny = a.ny; p.nq = 0;
@@ -1108,13 +1304,12 @@ cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     p.row_lse = a.row_lse; p.pos_idx = a.pos_idx;
     p.out = a.out; p.ldo = a.ldo; p.partial = a.partial;
     p.dev_status = a.dev_status;
-    int64_t units = ((a.nx + XROWS - 1) / XROWS) * p.dparts * a.groups;
     const bool two = sweep_nbuf(kc) == 2;
     if (a.mode == SWEEP_DQ)
-        return two ? launch<MODE_DQ, SN, 2>(mx, my, p, units, st)
-                   : launch<MODE_DQ, SN, 1>(mx, my, p, units, st);
-    return two ? launch<MODE_DP, SN, 2>(mx, my, p, units, st)
-               : launch<MODE_DP, SN, 1>(mx, my, p, units, st);
+        return two ? launch<MODE_DQ, SN, 2>(mx, my, myh, p, st)
+                   : launch<MODE_DQ, SN, 1>(mx, my, myh, p, st);
+    return two ? launch<MODE_DP, SN, 2>(mx, my, myh, p, st)
+               : launch<MODE_DP, SN, 1>(mx, my, myh, p, st);
 }
 
 }  // namespace gc

@@ -51,6 +51,26 @@ def test_self_mask_shared_rows(binding, oracle, n, d, tau, dtype):
     check_against_oracle(prob, out, _oracle_full(oracle, prob))
 
 
+@pytest.mark.parametrize("B,N", [(300, 45000), (45000, 300)])
+def test_streamed_matrix_larger_than_l2_uses_cta_pairs(binding, oracle, B, N):
+    """When the streamed matrix (P for the forward/dQ sweeps, Q for the dP sweep) exceeds 64 MB
+    the wide-row kernels run as CTA pairs that share every streamed chunk.  Both orientations,
+    with an odd number of 128-row tiles on the stationary side (3), against the full oracle."""
+    prob = inputs.random_problem(B, N, 768, "bf16", seed=B + N, tau=0.5, scale=768 ** -0.5)
+    Q, P, pos = to_device(prob)
+    out = binding.build_cache(Q, P, pos, prob.tau, prob.mask_mode)
+    ref = _oracle_full(oracle, prob)
+    check_against_oracle(prob, out, ref)
+    # the stand-alone forward and backward calls take the same paired kernels
+    b = binding.Outputs(prob.B, prob.N, prob.d, binding.GC_BF16)
+    binding.gc_loss_fwd(Q, P, pos, prob.tau, prob.mask_mode, b.loss, b.row_lse, b.pos_logit, b.ws,
+                        b.dev_status)
+    binding.gc_loss_bwd(Q, P, pos, prob.tau, prob.mask_mode, b.row_lse, b.dQ, b.dP, b.ws,
+                        b.dev_status)
+    torch.cuda.synchronize()
+    check_against_oracle(prob, b, ref)
+
+
 def test_fwd_then_bwd_equals_build(binding, oracle):
     """The separate forward and backward calls reproduce gc_build_cache: bit for bit where both
     run the same kernels, within rounding where gc_build_cache fuses the forward into the dQ
