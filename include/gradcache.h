@@ -69,7 +69,7 @@ enum { GC_DEV_POS_RANGE = 1, GC_DEV_POS_MASKED = 2, GC_DEV_WAIT_LIMIT = 4 };
 size_t gc_workspace_bytes(int op, int64_t B, int64_t N, int d, int dtype);
 
 /* Name of the kernel plan the library will use for these sizes: "tcgen05" (TMA + tcgen05 MMA
- * with TMEM accumulators; bf16, d a multiple of 64 up to 768) or "simt" (fp32 FMA tiles; every
+ * with TMEM accumulators; bf16, d a multiple of 64 up to 4096) or "simt" (fp32 FMA tiles; every
  * other case, including all fp32 inputs).  Static string. */
 const char* gc_plan_name(int op, int64_t B, int64_t N, int d, int dtype);
 

@@ -1,4 +1,4 @@
-// Tensor-core plan for bf16 inputs with d a multiple of 64 (up to 768): TMA-staged tiles in
+// Tensor-core plan for bf16 inputs with d a multiple of 64 (up to 4096): TMA-staged tiles in
 // 128-byte-swizzled shared memory, tcgen05 MMAs with fp32 accumulators in tensor memory, the
 // softmax arithmetic in registers.  One kernel template serves three sweeps:
 //
@@ -47,7 +47,7 @@ constexpr int NTHREADS = 32 * (NPROD + 1 + NSOFT);
 constexpr int MAX_STAGES = 8;
 constexpr uint32_t CHUNK_BYTES = 16384;    // 128 rows x 64 columns: one X chunk or one Y chunk
 constexpr int TMEM_COLS = 512;
-constexpr int MAX_D = 768;
+constexpr int MAX_D = 4096;                // wider rows just take more column parts
 constexpr int MAX_PART_CHUNKS = 6;         // 384 accumulator columns
 constexpr size_t SMEM_LIMIT = 232448;      // 227 KB per block
 constexpr size_t SMEM_STATIC_RESERVE = 2048;

@@ -28,7 +28,8 @@ def _oracle_full(oracle, prob):
 SHAPES = [
     # B, N, d
     (1, 2, 4), (1, 1, 8), (7, 2, 12), (64, 128, 64), (129, 257, 72), (130, 130, 128),
-    (200, 513, 192), (257, 1, 64), (65, 300, 768),
+    (200, 513, 192), (257, 1, 64), (65, 300, 768), (300, 200, 320), (140, 270, 448),
+    (150, 260, 576), (129, 300, 1024), (260, 131, 1536), (70, 140, 4096),
 ]
 
 
