@@ -296,6 +296,57 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16
 __device__ __forceinline__ void tmem_st_wait() {
     asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
+// ---- epilogue: accumulator blocks leave through shared memory and bulk tensor stores ---------------
+// One warp's block of 32 rows x 32 fp32 columns is written to a 4 KB buffer in the 128-byte
+// swizzle the tensor map expects (16-byte chunk j of row r at chunk j ^ (r & 7)), which also
+// makes the float4 stores conflict-free, and then leaves with one bulk tensor store; rows past
+// the end of the matrix are clipped by the tensor map.
+__device__ __forceinline__ void stage_block(uint32_t buf, const uint32_t (&v)[32], float sc,
+                                            int lane) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const uint32_t addr = buf + lane * 128 + ((j ^ (lane & 7)) << 4);
+        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};"
+                     ::"r"(addr), "f"(__uint_as_float(v[4 * j]) * sc),
+                       "f"(__uint_as_float(v[4 * j + 1]) * sc),
+                       "f"(__uint_as_float(v[4 * j + 2]) * sc),
+                       "f"(__uint_as_float(v[4 * j + 3]) * sc)
+                     : "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the bulk store
+}
+__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1,
+                                             int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+        ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+// Writes accumulator blocks cb = half, half + 2, ... (32 columns each) of this warp's 32 rows.
+// `slot` is the warp's 8 KB staging area (two buffers).
+__device__ __forceinline__ void store_acc_blocks(uint32_t tmem_rows, int nblocks, int half,
+                                                 uint32_t slot, float sc, int lane,
+                                                 const CUtensorMap* mapO, int col0, int row0,
+                                                 int plane) {
+    int n = 0;
+    for (int cb = half; cb < nblocks; cb += 2, ++n) {
+        uint32_t v[32];
+        tmem_ld32(tmem_rows + cb * 32, v);
+        if (n >= 2) {   // the store issued two blocks ago has finished reading this buffer
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+            __syncwarp();
+        }
+        tmem_ld_wait();
+        const uint32_t buf = slot + (n & 1) * 4096;
+        stage_block(buf, v, sc, lane);
+        __syncwarp();
+        if (lane == 0) tma_store_3d(mapO, buf, col0 + cb * 32, row0, plane);
+    }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+    __syncwarp();
+}
+
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -344,7 +395,8 @@ struct Bars {
 template <int MODE, int SN, int NBUF, bool PAIR>
 __global__ void __launch_bounds__(NTHREADS, 1)
 tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
-          const __grid_constant__ CUtensorMap mapYh, const TcParams p) {
+          const __grid_constant__ CUtensorMap mapYh, const __grid_constant__ CUtensorMap mapO,
+          const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) Bars bars;
     __shared__ uint32_t tmem_base_s;
@@ -892,20 +944,10 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             if (ok) ok = mbar_wait(smem_u32(&bars.acc_full), 0, abort_flag);
             if (ok) {
                 tc_fence_after();
-                const int64_t d = (int64_t)p.kc * 64;
-                float* dst = p.partial + ((int64_t)g * p.nx + x) * d + c_begin * 64;
-                for (int cb = half; cb < c_count * 2; cb += 2) {
-                    uint32_t v[32];
-                    tmem_ld32(tmem + lane_addr + cb * 32, v);
-                    tmem_ld_wait();
-                    if (x < p.nx) {
-#pragma unroll
-                        for (int c = 0; c < 32; c += 4)
-                            *reinterpret_cast<float4*>(dst + cb * 32 + c) =
-                                make_float4(__uint_as_float(v[c]), __uint_as_float(v[c + 1]),
-                                            __uint_as_float(v[c + 2]), __uint_as_float(v[c + 3]));
-                    }
-                }
+                // every MMA and every load has completed: the dynamic shared memory is free
+                const uint32_t slot = base + (uint32_t)(warp - (NPROD + 1)) * 8192u;
+                store_acc_blocks(tmem + lane_addr, c_count * 2, half, slot, 1.f, lane, &mapO,
+                                 c_begin * 64, (int)x0 + q * 32, g);
             }
             TR_END(tr_epi);
         } else {
@@ -1005,31 +1047,17 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 if (lane == 0) arrive_w(smem_u32(&bars.w_full[b]));
             }
             // epilogue: accumulator columns of this part -> global memory (32-column blocks are
-            // dealt alternately to the two warps of a lane quarter)
+            // dealt alternately to the two warps of a lane quarter); final values are scaled,
+            // partial sums of a split sweep are not
             TR_BEGIN(tr_epi);
             if (ok) ok = mbar_wait(smem_u32(&bars.acc_full), 0, abort_flag);
             if (ok) {
                 tc_fence_after();
                 const bool final_out = (p.groups == 1);
-                const int64_t d = (int64_t)p.kc * 64;
-                float* dst = final_out ? p.out + x * p.ldo + c_begin * 64
-                                       : p.partial + ((int64_t)g * p.nx + x) * d + c_begin * 64;
-                const float sc = final_out ? p.out_scale : 1.f;
-                for (int cb = half; cb < c_count * 2; cb += 2) {
-                    uint32_t v[32];
-                    tmem_ld32(tmem + lane_addr + cb * 32, v);
-                    tmem_ld_wait();
-                    if (x < p.nx) {
-#pragma unroll
-                        for (int c = 0; c < 32; c += 4) {
-                            float4 o = make_float4(__uint_as_float(v[c]) * sc,
-                                                   __uint_as_float(v[c + 1]) * sc,
-                                                   __uint_as_float(v[c + 2]) * sc,
-                                                   __uint_as_float(v[c + 3]) * sc);
-                            *reinterpret_cast<float4*>(dst + cb * 32 + c) = o;
-                        }
-                    }
-                }
+                const uint32_t slot = base + (uint32_t)(warp - (NPROD + 1)) * 8192u;
+                store_acc_blocks(tmem + lane_addr, c_count * 2, half, slot,
+                                 final_out ? p.out_scale : 1.f, lane, &mapO, c_begin * 64,
+                                 (int)x0 + q * 32, final_out ? 0 : g);
             }
             TR_END(tr_epi);
         }
@@ -1101,6 +1129,22 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int d, int64_t l
     return r == CUDA_SUCCESS;
 }
 
+// fp32 destination of the accumulators as [planes][rows][d]: the output matrix itself (one plane,
+// row pitch ld) or the per-part partial sums (planes = parts of the streamed range, pitch d).
+// Boxes of 32 rows x 32 columns, 128-byte swizzle.
+bool make_out_map(CUtensorMap* map, float* base, int64_t rows, int d, int64_t ld, int planes) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)rows, (cuuint64_t)planes};
+    cuuint64_t strides[2] = {(cuuint64_t)ld * 4, (cuuint64_t)rows * (cuuint64_t)ld * 4};
+    cuuint32_t box[3] = {32, 32, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 int parts_for(int kc) { return (kc + MAX_PART_CHUNKS - 1) / MAX_PART_CHUNKS; }
 int chunks_per_part(int kc) { int n = parts_for(kc); return (kc + n - 1) / n; }
 
@@ -1133,7 +1177,7 @@ SmemPlan smem_plan(int kc, bool pair = false) {
 
 template <int MODE, int SN, int NBUF, bool PAIR>
 cudaError_t launch_one(const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& myh,
-                       const TcParams& p, int64_t ctas, cudaStream_t st) {
+                       const CUtensorMap& mo, const TcParams& p, int64_t ctas, cudaStream_t st) {
     SmemPlan sp = smem_plan(p.kc, PAIR);
     static bool configured = false;
     if (!configured) {
@@ -1159,10 +1203,10 @@ cudaError_t launch_one(const CUtensorMap& mx, const CUtensorMap& my, const CUten
     cfg.numAttrs = 1;
     if (!PAIR) {
         tc_kernel<MODE, SN, NBUF, false><<<(unsigned)ctas, NTHREADS, sp.dynamic_bytes, st>>>(
-            mx, my, myh, pp);
+            mx, my, myh, mo, pp);
         return cudaGetLastError();
     }
-    return cudaLaunchKernelEx(&cfg, tc_kernel<MODE, SN, NBUF, PAIR>, mx, my, myh, pp);
+    return cudaLaunchKernelEx(&cfg, tc_kernel<MODE, SN, NBUF, PAIR>, mx, my, myh, mo, pp);
 }
 
 // CTA pairs need two-chunk ring items (the accumulation MMAs split them by rank) and at least
@@ -1185,10 +1229,11 @@ int64_t cta_count(int kc, int64_t nx, int64_t ny, int parts, int groups) {
 
 template <int MODE, int SN, int NBUF>
 cudaError_t launch(const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& myh,
-                   const TcParams& p, cudaStream_t st) {
+                   const CUtensorMap& mo, const TcParams& p, cudaStream_t st) {
     const int64_t ctas = cta_count(p.kc, p.nx, p.ny, p.dparts, p.groups);
-    if (use_pair(p.kc, p.nx, p.ny)) return launch_one<MODE, SN, NBUF, true>(mx, my, myh, p, ctas, st);
-    return launch_one<MODE, SN, NBUF, false>(mx, my, myh, p, ctas, st);
+    if (use_pair(p.kc, p.nx, p.ny))
+        return launch_one<MODE, SN, NBUF, true>(mx, my, myh, mo, p, ctas, st);
+    return launch_one<MODE, SN, NBUF, false>(mx, my, myh, mo, p, ctas, st);
 }
 
 }  // namespace
@@ -1252,7 +1297,7 @@ cudaError_t tc_launch_fwd(const FwdArgs& a, cudaStream_t st) {
     p.pos_idx = pr.pos_idx;
     p.part_m = a.part_m; p.part_l = a.part_l; p.pos_logit = a.pos_logit;
     p.dev_status = a.dev_status;
-    return launch<MODE_FWD, SN, 2>(mx, my, myh, p, st);
+    return launch<MODE_FWD, SN, 2>(mx, my, myh, mx, p, st);   // no accumulator output
 }
 
 bool tc_fused_applicable(int d) { return sweep_nbuf(d / 64) == 1; }
@@ -1281,7 +1326,9 @@ cudaError_t tc_launch_fused_dq(const FwdArgs& a, float* partial, int groups, cud
     p.part_m = a.part_m; p.part_l = a.part_l; p.pos_logit = a.pos_logit;
     p.partial = partial;
     p.dev_status = a.dev_status;
-    return launch<MODE_FQ, SN, 1>(mx, my, myh, p, st);
+    CUtensorMap mo;
+    if (!make_out_map(&mo, partial, pr.B, pr.d, pr.d, groups)) return cudaErrorInvalidValue;
+    return launch<MODE_FQ, SN, 1>(mx, my, myh, mo, p, st);
 }
 
 cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
@@ -1304,12 +1351,16 @@ cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     p.row_lse = a.row_lse; p.pos_idx = a.pos_idx;
     p.out = a.out; p.ldo = a.ldo; p.partial = a.partial;
     p.dev_status = a.dev_status;
+    CUtensorMap mo;
+    const bool ok_map = a.groups == 1 ? make_out_map(&mo, a.out, a.nx, a.d, a.ldo, 1)
+                                      : make_out_map(&mo, a.partial, a.nx, a.d, a.d, a.groups);
+    if (!ok_map) return cudaErrorInvalidValue;
     const bool two = sweep_nbuf(kc) == 2;
     if (a.mode == SWEEP_DQ)
-        return two ? launch<MODE_DQ, SN, 2>(mx, my, myh, p, st)
-                   : launch<MODE_DQ, SN, 1>(mx, my, myh, p, st);
-    return two ? launch<MODE_DP, SN, 2>(mx, my, myh, p, st)
-               : launch<MODE_DP, SN, 1>(mx, my, myh, p, st);
+        return two ? launch<MODE_DQ, SN, 2>(mx, my, myh, mo, p, st)
+                   : launch<MODE_DQ, SN, 1>(mx, my, myh, mo, p, st);
+    return two ? launch<MODE_DP, SN, 2>(mx, my, myh, mo, p, st)
+               : launch<MODE_DP, SN, 1>(mx, my, myh, mo, p, st);
 }
 
 }  // namespace gc
