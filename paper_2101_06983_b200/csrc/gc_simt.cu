@@ -14,7 +14,8 @@ namespace {
 
 constexpr int TX = 64;        // stationary rows per block
 constexpr int TY = 64;        // streamed rows per step
-constexpr int TK = 16;        // width of one staged k chunk
+constexpr int TK = 32;        // width of one staged k chunk of the logits product
+constexpr int TR = 16;        // streamed rows staged per pass of the accumulation product
 constexpr int TD = 128;       // accumulator columns per block in the sweep
 constexpr int PADX = TX + 4;  // row pitch of the k-major staging tiles (keeps float4 alignment)
 constexpr int THREADS = 256;
@@ -25,26 +26,47 @@ template <> __device__ __forceinline__ float to_float<__nv_bfloat16>(__nv_bfloat
     return __bfloat162float(v);
 }
 
-// Stage rows [row0, row0 + 64) x columns [k0, k0 + 16) of M into dst[k][row] as float,
-// zero-filled outside the matrix.  Thread t handles row t / 4, columns 4 (t % 4) .. + 3.
+// Thread t fetches 8 consecutive k values (columns k0 + 8 (t % 4) ..) of row row0 + t / 4 into
+// registers as float, zero outside the matrix: one or two 16-byte loads on the fast path.
 template <typename T>
-__device__ __forceinline__ void stage_chunk(const T* __restrict__ M, int64_t ld, int64_t rows,
-                                            int d, int64_t row0, int k0, float (*dst)[PADX]) {
-    int r = threadIdx.x >> 2;
-    int kq = (threadIdx.x & 3) * 4;
-    int64_t row = row0 + r;
-    float v[4] = {0.f, 0.f, 0.f, 0.f};
-    if (row < rows) {
-        const T* src = M + row * ld + k0 + kq;
+__device__ __forceinline__ void fetch8(const T* __restrict__ M, int64_t ld, int64_t rows, int d,
+                                       int64_t row0, int k0, float (&v)[8]) {
+    const int64_t row = row0 + (threadIdx.x >> 2);
+    const int k = k0 + (threadIdx.x & 3) * 8;
 #pragma unroll
-        for (int e = 0; e < 4; ++e)
-            if (k0 + kq + e < d) v[e] = to_float<T>(src[e]);
+    for (int e = 0; e < 8; ++e) v[e] = 0.f;
+    if (row >= rows || k >= d) return;
+    const T* src = M + row * ld + k;
+    if (k + 8 <= d) {
+        if (sizeof(T) == 4) {
+            const float4 a = *reinterpret_cast<const float4*>(src);
+            const float4 b = *reinterpret_cast<const float4*>(src + 4);
+            v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+            v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+        } else {
+            const uint4 u = *reinterpret_cast<const uint4*>(src);
+            const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                v[2 * e] = __uint_as_float(w[e] << 16);              // bf16 -> fp32 is a shift
+                v[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+            }
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            if (k + e < d) v[e] = to_float<T>(src[e]);
     }
-#pragma unroll
-    for (int e = 0; e < 4; ++e) dst[kq + e][r] = v[e];
 }
 
-// acc[a][b] = sum_k X[x0 + 4 ty + a][k] * Y[y0 + 4 tx + b][k] over the full width d.
+__device__ __forceinline__ void put8(const float (&v)[8], float (*dst)[PADX]) {
+    const int r = threadIdx.x >> 2, kq = (threadIdx.x & 3) * 8;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) dst[kq + e][r] = v[e];
+}
+
+// acc[a][b] = sum_k X[x0 + 4 ty + a][k] * Y[y0 + 4 tx + b][k] over the full width d.  The next
+// 32-wide k chunk is fetched into registers while the current one is multiplied.
 template <typename T>
 __device__ __forceinline__ void logits_tile(const T* __restrict__ X, int64_t ldx, int64_t nx,
                                             const T* __restrict__ Y, int64_t ldy, int64_t ny,
@@ -55,11 +77,18 @@ __device__ __forceinline__ void logits_tile(const T* __restrict__ X, int64_t ldx
     for (int a = 0; a < 4; ++a)
 #pragma unroll
         for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+    float xr[8], yr[8];
+    fetch8<T>(X, ldx, nx, d, x0, 0, xr);
+    fetch8<T>(Y, ldy, ny, d, y0, 0, yr);
     for (int k0 = 0; k0 < d; k0 += TK) {
+        __syncthreads();                      // the previous chunk has been consumed
+        put8(xr, Xs);
+        put8(yr, Ys);
         __syncthreads();
-        stage_chunk<T>(X, ldx, nx, d, x0, k0, Xs);
-        stage_chunk<T>(Y, ldy, ny, d, y0, k0, Ys);
-        __syncthreads();
+        if (k0 + TK < d) {
+            fetch8<T>(X, ldx, nx, d, x0, k0 + TK, xr);
+            fetch8<T>(Y, ldy, ny, d, y0, k0 + TK, yr);
+        }
 #pragma unroll
         for (int k = 0; k < TK; ++k) {
             float4 xv = *reinterpret_cast<const float4*>(&Xs[k][ty * 4]);
@@ -161,7 +190,7 @@ __global__ void __launch_bounds__(THREADS) simt_sweep_kernel(SweepArgs a) {
     __shared__ __align__(16) float Xs[TK][PADX];
     __shared__ __align__(16) float Ys[TK][PADX];
     __shared__ float Ws[TX][TY + 1];
-    __shared__ __align__(16) float Yd[TK][TD];
+    __shared__ __align__(16) float Yd[TR][TD];
     const T* X = static_cast<const T*>(a.X);
     const T* Y = static_cast<const T*>(a.Y);
     int ty = threadIdx.x >> 4, tx = threadIdx.x & 15;
@@ -216,7 +245,7 @@ __global__ void __launch_bounds__(THREADS) simt_sweep_kernel(SweepArgs a) {
             }
         }
         // out[x][c0 + 8 tx ..] += sum_y Ws[x][y] * Y[y0 + y][c0 + 8 tx ..]
-        for (int yb = 0; yb < TY; yb += TK) {
+        for (int yb = 0; yb < TY; yb += TR) {
             __syncthreads();   // Ws complete (first pass) / Yd free (later passes)
             {
                 int r = threadIdx.x >> 4;              // 16 rows x 16 threads of 8 columns
@@ -230,7 +259,7 @@ __global__ void __launch_bounds__(THREADS) simt_sweep_kernel(SweepArgs a) {
             }
             __syncthreads();
 #pragma unroll
-            for (int k = 0; k < TK; ++k) {
+            for (int k = 0; k < TR; ++k) {
                 float4 y0v = *reinterpret_cast<const float4*>(&Yd[k][tx * 8]);
                 float4 y1v = *reinterpret_cast<const float4*>(&Yd[k][tx * 8 + 4]);
                 float yv[8] = {y0v.x, y0v.y, y0v.z, y0v.w, y1v.x, y1v.y, y1v.z, y1v.w};
