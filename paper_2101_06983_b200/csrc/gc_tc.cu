@@ -380,6 +380,8 @@ struct Bars {
     uint64_t w_full[2];
     uint64_t acc_full;
     uint64_t pair[4];          // FQ: the two softmax warps of a lane quarter agree on the row max
+    uint64_t s_free;           // WS: every softmax warp has read the S tile (in the leader)
+    uint64_t w_empty[2];       // WS: the MMAs that read W buffer b have completed
 };
 
 // ---------------------------------------------------------------------------------------------
@@ -406,8 +408,15 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
 
     static_assert(SN == 128, "a Y chunk is 128 rows: the same 16 KB as an X chunk");
     constexpr uint32_t S_COL0 = TMEM_COLS - NBUF * SN;  // S buffers sit at the top columns
-    constexpr int LAG = NBUF - 1;                       // steps between S(t) and acc(t) issue
+    // WS ("W through shared memory"): paired wide-row sweeps write the bf16 weights to two
+    // shared-memory buffers instead of over the single S tile.  The S tile is then free as soon as
+    // the softmax warps have read it, S(t+1) is issued while softmax(t) computes, and acc(t)
+    // follows from W buffer t & 1: the tensor pipe no longer waits for the softmax.
+    constexpr bool WS = PAIR && NBUF == 1 && MODE != MODE_FWD;
+    constexpr int LAG = WS ? 1 : NBUF - 1;              // steps between S(t) and acc(t) issue
     constexpr int BSH = (NBUF == 2) ? 1 : 0;            // log2(NBUF)
+    constexpr int WBUF = WS ? 2 : NBUF;                 // W buffers (w_full barriers in use)
+    constexpr int WSH = (WBUF == 2) ? 1 : 0;
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // warp-uniform
     const int lane = threadIdx.x & 31;
 
@@ -430,7 +439,8 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t x_smem = base;
-    const uint32_t y_smem = base + (uint32_t)p.xres * X_CHUNK_BYTES;   // the ring
+    const uint32_t w_smem = base + (uint32_t)p.xres * X_CHUNK_BYTES;   // WS: two 32 KB W buffers
+    const uint32_t y_smem = w_smem + (WS ? 2u * 32768u : 0u);          // the ring
     // a paired CTA holds half of every Y item, so its stages are one chunk (16 KB) and a streamed
     // X item is a single chunk; otherwise a stage holds ipc chunks of Y or of X
     const int xipc = PAIR ? 1 : p.ipc;
@@ -449,6 +459,8 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
         }
         mbar_init(smem_u32(&bars.acc_full), 1);
         for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&bars.pair[i]), 2);   // one per warp
+        mbar_init(smem_u32(&bars.s_free), NCTA * NSOFT);
+        for (int b = 0; b < 2; ++b) mbar_init(smem_u32(&bars.w_empty[b]), 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == MMA_WARP) {
@@ -604,6 +616,11 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             for (int t = 0; t < T + LAG && ok; ++t) {
                 if (t < T) {
                     const int b = t & (NBUF - 1);
+                    if (WS && t >= 1) {     // the softmax warps have read S(t-1) out of the tile
+                        ok = mbar_wait(smem_u32(&bars.s_free), (t - 1) & 1, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                    }
                     if (MODE == MODE_FWD && t >= NBUF) {
                         ok = mbar_wait(smem_u32(&bars.w_full[b]), ((t - NBUF) >> BSH) & 1,
                                        abort_flag);
@@ -675,13 +692,14 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     TR_END(tr_sf);
                 }
                 if (MODE != MODE_FWD && t >= LAG) {
-                    const int u = t - LAG, b = u & (NBUF - 1);
+                    const int u = t - LAG, b = u & (WBUF - 1);
                     TR_BEGIN(tr_ww);
-                    ok = mbar_wait(smem_u32(&bars.w_full[b]), (u >> BSH) & 1, abort_flag);
+                    ok = mbar_wait(smem_u32(&bars.w_full[b]), (u >> WSH) & 1, abort_flag);
                     TR_END(tr_ww);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t w_tmem = tmem + S_COL0 + b * SN;
+                    const uint32_t w_tmem = tmem + S_COL0 + (WS ? 0 : b * SN);
+                    const uint32_t w_lo = desc_lo(w_smem + b * 32768u, 0);   // WS: K-major A operand
                     // one ring item per iteration: ipc chunks = 64 * ipc accumulator columns
                     for (int c = 0; c < c_count && ok; c += p.ipc) {
                         const int ys = next_stage();
@@ -693,17 +711,28 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                             // k-steps of the first column half read W at columns 8 k, those of
                             // the second half at SN/2 + 8 (k - KH)
                             constexpr int KH = SN / 32;
-                            if (u == 0) mma_ts<false, PAIR>(d_tmem, w_tmem, yb, idesc_acc);
-                            else        mma_ts<true, PAIR>(d_tmem, w_tmem, yb, idesc_acc);
+                            if (WS) {
+                                // W[128 x 128] sits in shared memory as two K-major chunks of 64
+                                if (u == 0) mma_ss<false, PAIR>(d_tmem, w_lo, yb, idesc_acc);
+                                else        mma_ss<true, PAIR>(d_tmem, w_lo, yb, idesc_acc);
 #pragma unroll
-                            for (int k = 1; k < SN / 16; ++k)
-                                mma_ts<true, PAIR>(d_tmem,
-                                                   w_tmem + (k / KH) * (SN / 2) + (k % KH) * 8,
-                                                   yb + k * 128, idesc_acc);
+                                for (int k = 1; k < SN / 16; ++k)
+                                    mma_ss<true, PAIR>(d_tmem, w_lo + (k / 4) * CH_LO + (k % 4) * 2,
+                                                       yb + k * 128, idesc_acc);
+                            } else {
+                                if (u == 0) mma_ts<false, PAIR>(d_tmem, w_tmem, yb, idesc_acc);
+                                else        mma_ts<true, PAIR>(d_tmem, w_tmem, yb, idesc_acc);
+#pragma unroll
+                                for (int k = 1; k < SN / 16; ++k)
+                                    mma_ts<true, PAIR>(d_tmem,
+                                                       w_tmem + (k / KH) * (SN / 2) + (k % KH) * 8,
+                                                       yb + k * 128, idesc_acc);
+                            }
                             commit(smem_u32(&bars.y_empty[ys]));
                         }
                         TR_END(tr_ai);
                     }
+                    if (WS && ok && elect_one()) commit(smem_u32(&bars.w_empty[b]));
                 }
             }
             if (ok && MODE != MODE_FWD && elect_one()) commit(smem_u32(&bars.acc_full));
@@ -731,10 +760,23 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         const bool self_mask = (p.mask_mode == GC_MASK_SELF);
         bool ok = true;
-        // w_full lives in the CTA that issues the MMAs
+        // w_full and s_free live in the CTA that issues the MMAs
         auto arrive_w = [&](uint32_t local) {
             if (PAIR && !leader) mbar_arrive_cluster(mapa_u32(local, 0));
             else                 mbar_arrive(local);
+        };
+        // WS: 32 packed bf16 weights (columns 32 j .. of this warp's column half) of this thread's
+        // row go to W buffer wb as four 16-byte pieces of the row's 128-byte line in K chunk
+        // `half`, at the swizzled piece index the K-major MMA descriptor expects.
+        auto put_w_block = [&](int wb, int j, const uint32_t (&pk)[16]) {
+            const uint32_t line = w_smem + wb * 32768u + half * CHUNK_BYTES + row * 128;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const uint32_t addr = line + (((4 * j + i) ^ (row & 7)) << 4);
+                asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                             ::"r"(addr), "r"(pk[4 * i]), "r"(pk[4 * i + 1]), "r"(pk[4 * i + 2]),
+                               "r"(pk[4 * i + 3]) : "memory");
+            }
         };
         TR_DECL(tr_ws);
         TR_DECL(tr_epi);
@@ -872,6 +914,12 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     const float m_new = fmaxf(m_ref, tile_max);
                     const float f = ex2(m_ref - m_new);
                     l *= f;
+                    if (WS) {   // acc(t-1) may still be running: wait for its completion
+                        ok = mbar_wait(smem_u32(&bars.w_empty[(t - 1) & 1]), ((t - 1) >> 1) & 1,
+                                       abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                    }
                     for (int cb = half; cb < c_count * 2; cb += 2) {
                         uint32_t a[32];
                         tmem_ld32(tmem + lane_addr + cb * 32, a);
@@ -887,12 +935,21 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     m_ref = m_new;
                 }
                 // ---- pass 2: weights 2^(s2 - m_ref), their sum, bf16 W without the positive ----
+                if (WS && t >= 2) {   // W buffer t & 1 has been consumed by acc(t-2)
+                    ok = mbar_wait(smem_u32(&bars.w_empty[t & 1]), ((t - 2) >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                }
 #pragma unroll
                 for (int j = 0; j < CB_PER; ++j) {
                     const int64_t yb = y0 + (cb0 + j) * 32;
                     uint32_t v[32];
                     tmem_ld32(sbuf + (cb0 + j) * 32, v);
                     tmem_ld_wait();
+                    if (WS && j == CB_PER - 1) {   // last read of the S tile: it may be overwritten
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) arrive_w(smem_u32(&bars.s_free));
+                    }
                     float w[32];
 #pragma unroll
                     for (int c = 0; c < 32; ++c)
@@ -926,12 +983,14 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         __nv_bfloat162 h = __floats2bfloat162_rn(w[2 * r], w[2 * r + 1]);
                         packed[r] = *reinterpret_cast<uint32_t*>(&h);
                     }
-                    tmem_st16(sbuf + half * (SN / 2) + j * 16, packed);
+                    if (WS) put_w_block(t & 1, j, packed);
+                    else    tmem_st16(sbuf + half * (SN / 2) + j * 16, packed);
                 }
-                tmem_st_wait();
+                if (WS) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                else    tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) arrive_w(smem_u32(&bars.w_full[0]));
+                if (lane == 0) arrive_w(smem_u32(&bars.w_full[WS ? (t & 1) : 0]));
             }
             // (scale, sum) of this half; only the first column part writes (both parts agree)
             if (ok && x < p.nx && dp == 0) {
@@ -985,6 +1044,16 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
 #pragma unroll
                 for (int j = 0; j < CB_PER; ++j) tmem_ld32(sbuf + (cb0 + j) * 32, vv[j]);
                 tmem_ld_wait();
+                if (WS) {
+                    // the S tile may be overwritten; W buffer t & 1 must have been consumed
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) arrive_w(smem_u32(&bars.s_free));
+                    if (t >= 2) {
+                        ok = mbar_wait(smem_u32(&bars.w_empty[t & 1]), ((t - 2) >> 1) & 1, abort_flag);
+                        if (!ok) break;
+                    }
+                }
 #pragma unroll
                 for (int j = 0; j < CB_PER; ++j) {
                     const int cb = cb0 + j;
@@ -1039,12 +1108,14 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         __nv_bfloat162 h = __floats2bfloat162_rn(w[2 * r], w[2 * r + 1]);
                         packed[r] = *reinterpret_cast<uint32_t*>(&h);
                     }
-                    tmem_st16(sbuf + half * (SN / 2) + j * 16, packed);
+                    if (WS) put_w_block(t & 1, j, packed);
+                    else    tmem_st16(sbuf + half * (SN / 2) + j * 16, packed);
                 }
-                tmem_st_wait();
+                if (WS) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                else    tmem_st_wait();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) arrive_w(smem_u32(&bars.w_full[b]));
+                if (lane == 0) arrive_w(smem_u32(&bars.w_full[WS ? (t & 1) : b]));
             }
             // epilogue: accumulator columns of this part -> global memory (32-column blocks are
             // dealt alternately to the two warps of a lane quarter); final values are scaled,
@@ -1156,20 +1227,23 @@ struct SmemPlan { int xres; int ipc; int nstage; size_t dynamic_bytes; };
 
 // Rows up to 512 wide keep the whole X tile resident; wider rows keep 6 chunks so that the ring
 // still has 128 KB.  Ring items hold two chunks when every chunk count involved is even.
-SmemPlan smem_plan(int kc, bool pair = false) {
+// `ws`: the paired wide-row sweeps also keep two 32 KB W buffers in shared memory and therefore
+// only 4 resident X chunks.
+SmemPlan smem_plan(int kc, bool pair = false, bool ws = false) {
     SmemPlan sp;
-    sp.xres = kc <= 8 ? kc : 6;
+    sp.xres = ws ? 4 : (kc <= 8 ? kc : 6);
     const int parts = parts_for(kc), dpc = chunks_per_part(kc);
     const bool even = kc % 2 == 0 && sp.xres % 2 == 0 && dpc % 2 == 0 &&
                       (kc - dpc * (parts - 1)) % 2 == 0;
     sp.ipc = even ? 2 : 1;
     size_t xbytes = (size_t)sp.xres * X_CHUNK_BYTES;
     size_t stage = pair ? (size_t)CHUNK_BYTES : (size_t)sp.ipc * CHUNK_BYTES;
-    size_t avail = SMEM_LIMIT - SMEM_STATIC_RESERVE - 1024 - xbytes;
+    size_t wbytes = ws ? 2 * 32768 : 0;
+    size_t avail = SMEM_LIMIT - SMEM_STATIC_RESERVE - 1024 - xbytes - wbytes;
     int ns = (int)(avail / stage);
     if (ns > MAX_STAGES) ns = MAX_STAGES;
     sp.nstage = ns;
-    sp.dynamic_bytes = 1024 + xbytes + (size_t)ns * stage;
+    sp.dynamic_bytes = 1024 + xbytes + wbytes + (size_t)ns * stage;
     // keep one CTA per SM (each CTA allocates all 512 tensor-memory columns)
     if (sp.dynamic_bytes < 120 * 1024) sp.dynamic_bytes = 120 * 1024;
     return sp;
@@ -1178,7 +1252,8 @@ SmemPlan smem_plan(int kc, bool pair = false) {
 template <int MODE, int SN, int NBUF, bool PAIR>
 cudaError_t launch_one(const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& myh,
                        const CUtensorMap& mo, const TcParams& p, int64_t ctas, cudaStream_t st) {
-    SmemPlan sp = smem_plan(p.kc, PAIR);
+    constexpr bool WS = PAIR && NBUF == 1 && MODE != MODE_FWD;
+    SmemPlan sp = smem_plan(p.kc, PAIR, WS);
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(tc_kernel<MODE, SN, NBUF, PAIR>,
@@ -1194,6 +1269,7 @@ cudaError_t launch_one(const CUtensorMap& mx, const CUtensorMap& my, const CUten
     cfg.stream = st;
     TcParams pp = p;
     pp.nstage = sp.nstage;
+    pp.xres = sp.xres;
     cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = PAIR ? 2 : 1;
@@ -1211,27 +1287,28 @@ cudaError_t launch_one(const CUtensorMap& mx, const CUtensorMap& my, const CUten
 
 // CTA pairs need two-chunk ring items (the accumulation MMAs split them by rank) and at least
 // two x tiles.
-// Pairing halves the traffic of the streamed matrix but adds cross-SM hand-offs to every step:
-// it pays when that matrix does not stay in the L2 cache (measured: 2.4 % faster at
-// 65536 x 131072, 3 % slower at 4096 x 8192).
-bool use_pair(int kc, int64_t nx, int64_t ny) {
-    const int64_t streamed_bytes = ny * kc * 128;
-    return smem_plan(kc).ipc == 2 && nx > XROWS && sweep_nbuf(kc) == 1 &&
-           streamed_bytes > (int64_t)64 << 20;
+// CTA pairs need two-chunk ring items and at least two x tiles.  The wide-row gradient sweeps
+// (one S buffer) always pair: together with W in shared memory this takes the softmax off the
+// tensor pipe's critical path.  The forward sweep pairs only when the streamed matrix does not
+// stay in the L2 cache, where halving its traffic outweighs the cross-SM hand-offs.
+bool use_pair(int mode, int kc, int64_t nx, int64_t ny) {
+    if (smem_plan(kc).ipc != 2 || nx <= XROWS || sweep_nbuf(kc) != 1) return false;
+    if (mode != MODE_FWD) return true;
+    return ny * kc * 128 > ((int64_t)64 << 20);
 }
 
 // x tiles (rounded up to whole pairs when paired) * column parts * groups
-int64_t cta_count(int kc, int64_t nx, int64_t ny, int parts, int groups) {
+int64_t cta_count(int mode, int kc, int64_t nx, int64_t ny, int parts, int groups) {
     int64_t tiles = (nx + XROWS - 1) / XROWS;
-    if (use_pair(kc, nx, ny)) tiles = (tiles + 1) / 2 * 2;
+    if (use_pair(mode, kc, nx, ny)) tiles = (tiles + 1) / 2 * 2;
     return tiles * parts * groups;
 }
 
 template <int MODE, int SN, int NBUF>
 cudaError_t launch(const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& myh,
                    const CUtensorMap& mo, const TcParams& p, cudaStream_t st) {
-    const int64_t ctas = cta_count(p.kc, p.nx, p.ny, p.dparts, p.groups);
-    if (use_pair(p.kc, p.nx, p.ny))
+    const int64_t ctas = cta_count(MODE, p.kc, p.nx, p.ny, p.dparts, p.groups);
+    if (use_pair(MODE, p.kc, p.nx, p.ny))
         return launch_one<MODE, SN, NBUF, true>(mx, my, myh, mo, p, ctas, st);
     return launch_one<MODE, SN, NBUF, false>(mx, my, myh, mo, p, ctas, st);
 }
