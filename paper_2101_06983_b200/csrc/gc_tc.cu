@@ -44,7 +44,7 @@ constexpr int NPROD = 4;                   // TMA producer warps
 constexpr int MMA_WARP = NPROD;
 constexpr int NSOFT = 8;                   // softmax / epilogue warps
 constexpr int NTHREADS = 32 * (NPROD + 1 + NSOFT);
-constexpr int MAX_STAGES = 8;
+constexpr int MAX_STAGES = 12;
 constexpr uint32_t CHUNK_BYTES = 16384;    // 128 rows x 64 columns: one X chunk or one Y chunk
 constexpr int TMEM_COLS = 512;
 constexpr int MAX_D = 4096;                // wider rows just take more column parts
@@ -58,7 +58,8 @@ enum { MODE_FWD = 0, MODE_DQ = 1, MODE_DP = 2, MODE_FQ = 3 };   // FQ: forward f
 // Optional diagnostics (-DGC_TC_TRACE): cycles each role spends waiting, summed over CTAs.
 #ifdef GC_TC_TRACE
 enum { TR_MMA_TOTAL, TR_MMA_WAIT_Y, TR_MMA_WAIT_W, TR_SM_TOTAL, TR_SM_WAIT_S, TR_SM_EPI,
-       TR_PROD_TOTAL, TR_PROD_WAIT, TR_CTAS, TR_MMA_ISSUE, TR_MMA_COMMIT, TR_ACC_ISSUE, TR_ACC_COMMIT, TR_SFULL_COMMIT, TR_COUNT };
+       TR_PROD_TOTAL, TR_PROD_WAIT, TR_CTAS, TR_MMA_ISSUE, TR_MMA_COMMIT, TR_ACC_ISSUE, TR_ACC_COMMIT, TR_SFULL_COMMIT,
+       TR_CTA_LIFE, TR_SETUP, TR_T0_MIN, TR_T0_MAX, TR_T1_MIN, TR_T1_MAX, TR_COUNT };
 __device__ unsigned long long g_trace[4][TR_COUNT];
 #define TR_DECL(v) long long v = 0
 #define TR_BEGIN(v) long long v##_t0 = clock64()
@@ -417,6 +418,10 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     constexpr int BSH = (NBUF == 2) ? 1 : 0;            // log2(NBUF)
     constexpr int WBUF = WS ? 2 : NBUF;                 // W buffers (w_full barriers in use)
     constexpr int WSH = (WBUF == 2) ? 1 : 0;
+#ifdef GC_TC_TRACE
+    const unsigned long long cta_t0 = global_ns();
+    const long long cta_c0 = clock64();
+#endif
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // warp-uniform
     const int lane = threadIdx.x & 31;
 
@@ -479,6 +484,9 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     if (PAIR) cluster_sync_all();     // both CTAs' barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem = tmem_base_s;
+#ifdef GC_TC_TRACE
+    if (threadIdx.x == 0) TR_ADD(MODE, TR_SETUP, clock64() - cta_c0);
+#endif
     // shared::cluster address, in the leader, of the barrier at the same offset as `local`
     auto in_leader = [&](uint32_t local) -> uint32_t { return PAIR ? mapa_u32(local, 0) : local; };
 
@@ -551,8 +559,8 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 if (t < T) {
                     for (int c = 0; c < p.kc; c += p.ipc) {
                         load_item(0, c, (lo + t) * SN);
-                        if (c >= p.xres)
-                            for (int j = 0; j < p.ipc; j += xipc) load_item(1, c + j, x0);
+                        for (int j = 0; j < p.ipc; j += xipc)
+                            if (c + j >= p.xres) load_item(1, c + j, x0);
                     }
                 }
                 if (MODE != MODE_FWD && t >= LAG) {
@@ -1152,6 +1160,16 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
         __syncthreads();
     }
     if (PAIR) cluster_sync_all();   // the peer's MMAs, loads and arrivals no longer touch this CTA
+#ifdef GC_TC_TRACE
+    if (threadIdx.x == 0) {
+        const unsigned long long t1 = global_ns();
+        TR_ADD(MODE, TR_CTA_LIFE, clock64() - cta_c0);
+        atomicMin(&g_trace[MODE][TR_T0_MIN], cta_t0);
+        atomicMax(&g_trace[MODE][TR_T0_MAX], cta_t0);
+        atomicMin(&g_trace[MODE][TR_T1_MIN], t1);
+        atomicMax(&g_trace[MODE][TR_T1_MAX], t1);
+    }
+#endif
     if (warp == MMA_WARP) {
         tc_fence_after();
         if (PAIR)
@@ -1227,11 +1245,12 @@ struct SmemPlan { int xres; int ipc; int nstage; size_t dynamic_bytes; };
 
 // Rows up to 512 wide keep the whole X tile resident; wider rows keep 6 chunks so that the ring
 // still has 128 KB.  Ring items hold two chunks when every chunk count involved is even.
-// `ws`: the paired wide-row sweeps also keep two 32 KB W buffers in shared memory and therefore
-// only 4 resident X chunks.
+// `ws`: the paired wide-row sweeps also keep two 32 KB W buffers in shared memory.  Their step
+// time follows the ring depth (measured at 4096 x 8192 x 768: 4 stages 0.388 ms, 6 stages 0.351,
+// 8 stages 0.341, 10 stages with no resident chunk 0.344), so only 2 X chunks stay resident.
 SmemPlan smem_plan(int kc, bool pair = false, bool ws = false) {
     SmemPlan sp;
-    sp.xres = ws ? 4 : (kc <= 8 ? kc : 6);
+    sp.xres = ws ? 2 : (kc <= 8 ? kc : 6);
     const int parts = parts_for(kc), dpc = chunks_per_part(kc);
     const bool even = kc % 2 == 0 && sp.xres % 2 == 0 && dpc % 2 == 0 &&
                       (kc - dpc * (parts - 1)) % 2 == 0;
@@ -1320,6 +1339,7 @@ extern "C" int gc_debug_trace(unsigned long long* out, int clear) {
     if (out && cudaMemcpyFromSymbol(out, g_trace, sizeof(g_trace)) != cudaSuccess) return 1;
     if (clear) {
         static unsigned long long zero[4][TR_COUNT] = {};
+        for (int m = 0; m < 4; ++m) zero[m][TR_T0_MIN] = zero[m][TR_T1_MIN] = ~0ull;
         if (cudaMemcpyToSymbol(g_trace, zero, sizeof(zero)) != cudaSuccess) return 1;
     }
     return 0;
