@@ -40,7 +40,7 @@ namespace {
 constexpr int XROWS = 128;                 // rows of the stationary tile = MMA M
 constexpr int CHUNK_BYTES_PER_ROW = 128;   // 64 bf16 = one swizzle row
 constexpr uint32_t X_CHUNK_BYTES = XROWS * CHUNK_BYTES_PER_ROW;
-constexpr int NPROD = 4;                   // TMA producer warps
+constexpr int NPROD = 2;                   // TMA producer warps
 constexpr int MMA_WARP = NPROD;
 constexpr int NSOFT = 8;                   // softmax / epilogue warps
 constexpr int NTHREADS = 32 * (NPROD + 1 + NSOFT);
@@ -866,42 +866,45 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t sbuf = tmem + lane_addr + S_COL0;
-                // ---- pass 1: maximum of this half's live logits (raw dot products; c1 > 0) ----
-                float bm = -INFINITY;
-                {
-                    uint32_t vv[CB_PER][32];
+                // ---- read the tile once: raw dot products of this half, dead columns at -inf ----
+                uint32_t vv[CB_PER][32];
 #pragma unroll
-                    for (int j = 0; j < CB_PER; ++j) tmem_ld32(sbuf + (cb0 + j) * 32, vv[j]);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int j = 0; j < CB_PER; ++j) {
-                        const int64_t yb = y0 + (cb0 + j) * 32;
-                        const bool has_pos = pos_x >= yb && pos_x < yb + 32 && pos_x < p.ny &&
-                                             !(self_mask && x == pos_x);
-                        if (has_pos) {
-                            const int rel = (int)(pos_x - yb);
-                            float sp = 0.f;
-#pragma unroll
-                            for (int c = 0; c < 32; ++c)
-                                if (c == rel) sp = __uint_as_float(vv[j][c]);
-                            p.pos_logit[x] = sp * p.inv_tau;
-                        }
-                        if (yb + 32 > p.ny) {
-#pragma unroll
-                            for (int c = 0; c < 32; ++c)
-                                if (yb + c >= p.ny) vv[j][c] = __float_as_uint(-INFINITY);
-                        }
-                        if (self_mask && x >= yb && x < yb + 32) {
-                            const int rel = (int)(x - yb);
-#pragma unroll
-                            for (int c = 0; c < 32; ++c)
-                                if (c == rel) vv[j][c] = __float_as_uint(-INFINITY);
-                        }
-#pragma unroll
-                        for (int c = 0; c < 32; ++c) bm = fmaxf(bm, __uint_as_float(vv[j][c]));
-                    }
+                for (int j = 0; j < CB_PER; ++j) tmem_ld32(sbuf + (cb0 + j) * 32, vv[j]);
+                tmem_ld_wait();
+                if (WS) {   // the S tile may be overwritten now
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) arrive_w(smem_u32(&bars.s_free));
                 }
-                bm *= p.c1;                                            // log2 domain
+                float bm = -INFINITY;
+#pragma unroll
+                for (int j = 0; j < CB_PER; ++j) {
+                    const int64_t yb = y0 + (cb0 + j) * 32;
+                    const bool has_pos = pos_x >= yb && pos_x < yb + 32 && pos_x < p.ny &&
+                                         !(self_mask && x == pos_x);
+                    if (has_pos) {
+                        const int rel = (int)(pos_x - yb);
+                        float sp = 0.f;
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (c == rel) sp = __uint_as_float(vv[j][c]);
+                        p.pos_logit[x] = sp * p.inv_tau;
+                    }
+                    if (yb + 32 > p.ny) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (yb + c >= p.ny) vv[j][c] = __float_as_uint(-INFINITY);
+                    }
+                    if (self_mask && x >= yb && x < yb + 32) {
+                        const int rel = (int)(x - yb);
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (c == rel) vv[j][c] = __float_as_uint(-INFINITY);
+                    }
+#pragma unroll
+                    for (int c = 0; c < 32; ++c) bm = fmaxf(bm, __uint_as_float(vv[j][c]));
+                }
+                bm *= p.c1;                                            // log2 domain (c1 > 0)
                 // agree on the tile maximum with the warp that owns the other column half (the
                 // partner reads this before it arrives on w_full for this step, and the next
                 // write only happens after the S tile of the next step, which needs that arrival)
@@ -942,7 +945,8 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     }
                     m_ref = m_new;
                 }
-                // ---- pass 2: weights 2^(s2 - m_ref), their sum, bf16 W without the positive ----
+                // ---- weights 2^(s2 - m_ref) (0 for dead columns), their sum, bf16 W without the
+                // positive ----
                 if (WS && t >= 2) {   // W buffer t & 1 has been consumed by acc(t-2)
                     ok = mbar_wait(smem_u32(&bars.w_empty[t & 1]), ((t - 2) >> 1) & 1, abort_flag);
                     if (!ok) break;
@@ -950,45 +954,31 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
 #pragma unroll
                 for (int j = 0; j < CB_PER; ++j) {
                     const int64_t yb = y0 + (cb0 + j) * 32;
-                    uint32_t v[32];
-                    tmem_ld32(sbuf + (cb0 + j) * 32, v);
-                    tmem_ld_wait();
-                    if (WS && j == CB_PER - 1) {   // last read of the S tile: it may be overwritten
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) arrive_w(smem_u32(&bars.s_free));
-                    }
-                    float w[32];
-#pragma unroll
-                    for (int c = 0; c < 32; ++c)
-                        w[c] = ex2(fmaf(__uint_as_float(v[c]), p.c1, -m_ref));
-                    if (yb + 32 > p.ny) {
-#pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            if (yb + c >= p.ny) w[c] = 0.f;
-                    }
-                    if (self_mask && x >= yb && x < yb + 32) {
-                        const int rel = (int)(x - yb);
-#pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            if (c == rel) w[c] = 0.f;
-                    }
                     float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
                     for (int c = 0; c < 32; c += 4) {
-                        s0 += w[c]; s1 += w[c + 1]; s2 += w[c + 2]; s3 += w[c + 3];
+                        float w0 = ex2(fmaf(__uint_as_float(vv[j][c]), p.c1, -m_ref));
+                        float w1 = ex2(fmaf(__uint_as_float(vv[j][c + 1]), p.c1, -m_ref));
+                        float w2 = ex2(fmaf(__uint_as_float(vv[j][c + 2]), p.c1, -m_ref));
+                        float w3 = ex2(fmaf(__uint_as_float(vv[j][c + 3]), p.c1, -m_ref));
+                        s0 += w0; s1 += w1; s2 += w2; s3 += w3;
+                        vv[j][c] = __float_as_uint(w0);
+                        vv[j][c + 1] = __float_as_uint(w1);
+                        vv[j][c + 2] = __float_as_uint(w2);
+                        vv[j][c + 3] = __float_as_uint(w3);
                     }
                     l += (s0 + s1) + (s2 + s3);
                     if (pos_x >= yb && pos_x < yb + 32) {                  // positive: fp32 later
                         const int rel = (int)(pos_x - yb);
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
-                            if (c == rel) w[c] = 0.f;
+                            if (c == rel) vv[j][c] = 0u;
                     }
                     uint32_t packed[16];
 #pragma unroll
                     for (int r = 0; r < 16; ++r) {
-                        __nv_bfloat162 h = __floats2bfloat162_rn(w[2 * r], w[2 * r + 1]);
+                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(vv[j][2 * r]),
+                                                                 __uint_as_float(vv[j][2 * r + 1]));
                         packed[r] = *reinterpret_cast<uint32_t*>(&h);
                     }
                     if (WS) put_w_block(t & 1, j, packed);
