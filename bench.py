@@ -191,16 +191,19 @@ def run_ours(args, rank, local_rank, world):
     B, N, d = prob.B, prob.N, prob.d
     code = binding.GC_BF16 if prob.dtype == "bf16" else binding.GC_F32
     Q, P, pos = binding.problem_tensors(prob, dev)
-    out = binding.Outputs(B, N, d, code, dev)
+    stored = args.plan == "stored"
+    op = binding.GC_OP_BUILD_STORED if stored else binding.GC_OP_BUILD
+    build = binding.gc_build_cache_stored if stored else binding.gc_build_cache
+    out = binding.Outputs(B, N, d, code, dev, op)
     flop = useful_flop(B, N, d)
-    plan = binding.gc_plan_name(binding.GC_OP_BUILD, B, N, d, code)
-    launches = binding.gc_kernel_launches(binding.GC_OP_BUILD, B, N, d, code)
+    plan = binding.gc_plan_name(binding.GC_OP_BUILD, B, N, d, code) + ("+stored" if stored else "")
+    launches = binding.gc_kernel_launches(op, B, N, d, code)
 
     flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)   # larger than the 126 MB L2
 
     def step():
-        binding.gc_build_cache(Q, P, pos, prob.tau, prob.mask_mode, out.loss, out.row_lse,
-                               out.dQ, out.dP, out.pos_logit, out.ws, out.dev_status)
+        build(Q, P, pos, prob.tau, prob.mask_mode, out.loss, out.row_lse, out.dQ, out.dP,
+              out.pos_logit, out.ws, out.dev_status)
 
     def barrier():
         if world > 1:
@@ -259,7 +262,7 @@ def run_ours(args, rank, local_rank, world):
     for _ in range(NB):
         q_ = torch.empty_like(Q)
         d_in.append((q_, q_ if prob.shared else torch.empty_like(P), torch.empty_like(pos)))
-    d_out = [out] + [binding.Outputs(B, N, d, code, dev) for _ in range(NB - 1)]
+    d_out = [out] + [binding.Outputs(B, N, d, code, dev, op) for _ in range(NB - 1)]
     s_up, s_run, s_down = (torch.cuda.Stream(dev) for _ in range(3))
     ev_up = [torch.cuda.Event() for _ in range(NB)]
     ev_run = [torch.cuda.Event() for _ in range(NB)]
@@ -278,8 +281,8 @@ def run_ours(args, rank, local_rank, world):
             s_run.wait_event(ev_up[k])
             s_run.wait_event(ev_down[k])          # the previous results of this set are out
             o = d_out[k]
-            binding.gc_build_cache(d_in[k][0], d_in[k][1], d_in[k][2], prob.tau, prob.mask_mode,
-                                   o.loss, o.row_lse, o.dQ, o.dP, o.pos_logit, o.ws, o.dev_status)
+            build(d_in[k][0], d_in[k][1], d_in[k][2], prob.tau, prob.mask_mode, o.loss, o.row_lse,
+                  o.dQ, o.dP, o.pos_logit, o.ws, o.dev_status)
             ev_run[k].record(s_run)
         with torch.cuda.stream(s_down):
             s_down.wait_event(ev_run[k])
@@ -315,9 +318,14 @@ def run_ours(args, rank, local_rank, world):
         # dominant kernel: the tile sweep kernel, launched twice per step for the gradients.  The
         # dP launch delivers one useful GEMM (2 B N d); the dQ launch delivers one, or two when the
         # forward is fused into it (no separate forward launch was timed).
+        # The stored-weights plan has three tensor kernels of one useful GEMM each.
         fused = kern[0] == 0.0
-        sweep_ms = (kern[1] + kern[2]) / (2 * args.steps)
-        sweep_flop = (6.0 if fused else 4.0) * B * N * d / 2.0          # per launch, averaged
+        if stored:
+            sweep_ms = (kern[0] + kern[1] + kern[2]) / (3 * args.steps)
+            sweep_flop = 2.0 * B * N * d
+        else:
+            sweep_ms = (kern[1] + kern[2]) / (2 * args.steps)
+            sweep_flop = (6.0 if fused else 4.0) * B * N * d / 2.0      # per launch, averaged
         achieved = sweep_flop / (sweep_ms * 1e-3) / 1e12 if sweep_ms > 0 else 0.0
         value = replicas.whole_job_rate(flop, world, ms_per_step) / 1e12
         line = {
@@ -341,7 +349,7 @@ def run_ours(args, rank, local_rank, world):
             "roofline": {"bound": "tensor", "kernel": f"{plan} tile sweep (the two gradient launches per step)",
                          "achieved": achieved, "peak": pk["tf_burst"], "unit": "TFLOP/s",
                          "frac": achieved / pk["tf_burst"], "peak_source": pk["source"],
-                         "traffic": ncu_traffic(prob.name)},
+                         "traffic": None if stored else ncu_traffic(prob.name)},
             "e2e": {"value": world * flop / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
                     "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "loss_read_back": e2e_loss,
@@ -379,6 +387,10 @@ def main():
                     help="query rows in the CPU sample (default: whole batch for ours' "
                          "cpu_baseline, 512 for --impl reference)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--plan", default="recompute", choices=["recompute", "stored"],
+                    help="recompute: gc_build_cache (nothing of size B x N leaves the chip); "
+                         "stored: gc_build_cache_stored, the comparison plan that keeps the "
+                         "B x N bf16 weights in the workspace")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

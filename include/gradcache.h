@@ -55,17 +55,18 @@ typedef enum {
     GC_ERR_WORKSPACE = 6, /* workspace NULL, misaligned (256 bytes) or too small */
     GC_ERR_CUDA = 7,      /* a CUDA call or launch failed */
     GC_ERR_ARCH = 8,      /* the current device is not compute capability 10.x */
-    GC_ERR_LIMIT = 9      /* problem too large for the library's built-in scratch area */
+    GC_ERR_LIMIT = 9      /* problem exceeds a built-in limit of the entry point that was called */
 } gc_status;
 
 typedef enum { GC_F32 = 0, GC_BF16 = 1 } gc_dtype;
 typedef enum { GC_MASK_NONE = 0, GC_MASK_SELF = 1 } gc_mask; /* SELF: drop the pair (i, i) */
-typedef enum { GC_OP_FWD = 0, GC_OP_BWD = 1, GC_OP_BUILD = 2 } gc_op;
+typedef enum { GC_OP_FWD = 0, GC_OP_BWD = 1, GC_OP_BUILD = 2, GC_OP_BUILD_STORED = 3 } gc_op;
 
 enum { GC_DEV_POS_RANGE = 1, GC_DEV_POS_MASKED = 2, GC_DEV_WAIT_LIMIT = 4 };
 
 /* Bytes of workspace the given call needs for these sizes on the current device (a multiple
- * of 256; O((B + N) d), never O(B N)).  Returns 0 for invalid arguments. */
+ * of 256).  O((B + N) d), never O(B N), for the three calls of the paper's path;
+ * GC_OP_BUILD_STORED adds 2 B N bytes for its weight matrix.  Returns 0 for invalid arguments. */
 size_t gc_workspace_bytes(int op, int64_t B, int64_t N, int d, int dtype);
 
 /* Name of the kernel plan the library will use for these sizes: "tcgen05" (TMA + tcgen05 MMA
@@ -103,6 +104,25 @@ int gc_build_cache(const void* Q, int64_t ldq, const void* P, int64_t ldp, const
                    float* loss, float* row_lse, float* pos_logit,
                    float* dQ, int64_t lddq, float* dP, int64_t lddp,
                    void* ws, size_t ws_bytes, int* dev_status, void* cuda_stream);
+
+/*
+ * The same results as gc_build_cache by a different route, kept as a measured comparison point:
+ * Eq. 1 and Eq. 5-7 need every logit three times (loss, dQ, dP), and gc_build_cache recomputes
+ * them so that nothing of size B x N ever leaves the chip.  This call trades memory for work: one
+ * forward sweep writes the un-normalised bf16 softmax weights 2^((S_ij - S_{i,r_i}) log2 e) of
+ * all pairs to the workspace (2 B N bytes; 0 at masked pairs and at the positive column, whose
+ * terms are added in fp32), and two plain GEMMs over that matrix form dQ and dP.  Rows whose
+ * logits lie more than 100 powers of two above their positive logit cannot be stored this way; a
+ * device flag then hands the whole call to the recomputing kernels, which are always launched
+ * after the GEMMs and return at once when the flag is down.  bf16 inputs with d a multiple of 64
+ * only, and a weight matrix of at most 40 GiB: other problems are refused with GC_ERR_LIMIT.
+ * Workspace size: gc_workspace_bytes(GC_OP_BUILD_STORED, ...).
+ */
+int gc_build_cache_stored(const void* Q, int64_t ldq, const void* P, int64_t ldp,
+                          const int32_t* pos_idx, int64_t B, int64_t N, int d, float tau,
+                          int mask_mode, int dtype, float* loss, float* row_lse, float* pos_logit,
+                          float* dQ, int64_t lddq, float* dP, int64_t lddp,
+                          void* ws, size_t ws_bytes, int* dev_status, void* cuda_stream);
 
 /*
  * Forward with library-owned scratch (no counterpart in the paper: it exists for the sake of

@@ -15,11 +15,12 @@ from . import _build
 
 GC_F32, GC_BF16 = 0, 1
 GC_MASK_NONE, GC_MASK_SELF = 0, 1
-GC_OP_FWD, GC_OP_BWD, GC_OP_BUILD = 0, 1, 2
+GC_OP_FWD, GC_OP_BWD, GC_OP_BUILD, GC_OP_BUILD_STORED = 0, 1, 2, 3
 GC_DEV_POS_RANGE, GC_DEV_POS_MASKED, GC_DEV_WAIT_LIMIT = 1, 2, 4
 
 EXPORTS = ("gc_workspace_bytes", "gc_plan_name", "gc_kernel_launches", "gc_loss_fwd",
-           "gc_loss_bwd", "gc_build_cache", "gc_status_string", "gc_profile_enable",
+           "gc_loss_bwd", "gc_build_cache", "gc_build_cache_stored", "gc_status_string",
+           "gc_profile_enable",
            "gc_profile_read", "gc_static_scratch_need", "gc_loss_fwd_static")
 GC_STATIC_SCRATCH_BYTES = 2 << 20
 
@@ -54,6 +55,8 @@ def _load() -> ctypes.CDLL:
     lib.gc_build_cache.restype = i32
     lib.gc_build_cache.argtypes = common + [vp, vp, vp, vp, i64, vp, i64, vp, ctypes.c_size_t,
                                             vp, vp]
+    lib.gc_build_cache_stored.restype = i32
+    lib.gc_build_cache_stored.argtypes = lib.gc_build_cache.argtypes
     lib.gc_static_scratch_need.restype = ctypes.c_size_t
     lib.gc_static_scratch_need.argtypes = [i64, i64, i32, i32]
     lib.gc_loss_fwd_static.restype = i32
@@ -176,6 +179,19 @@ def gc_build_cache(Q, P, pos_idx, tau, mask_mode, loss, row_lse, dQ, dP, pos_log
         raise GradCacheError(rc, "gc_build_cache")
 
 
+def gc_build_cache_stored(Q, P, pos_idx, tau, mask_mode, loss, row_lse, dQ, dP, pos_logit=None,
+                          ws=None, dev_status=None):
+    """gc_build_cache by way of a stored B x N bf16 weight matrix and two GEMMs (comparison plan)."""
+    args, B, N, d, code = _common(Q, P, pos_idx, tau, mask_mode)
+    if ws is None:
+        ws = alloc_workspace(GC_OP_BUILD_STORED, B, N, d, code, Q.device)
+    rc = _lib.gc_build_cache_stored(*args, _ptr(loss), _ptr(row_lse), _ptr(pos_logit), _ptr(dQ),
+                                    dQ.stride(0), _ptr(dP), dP.stride(0), _ptr(ws), ws.numel(),
+                                    _ptr(dev_status), _stream())
+    if rc != 0:
+        raise GradCacheError(rc, "gc_build_cache_stored")
+
+
 def gc_profile_enable(on: bool) -> None:
     rc = _lib.gc_profile_enable(1 if on else 0)
     if rc != 0:
@@ -208,7 +224,7 @@ def problem_tensors(prob, device="cuda"):
 class Outputs:
     """Device buffers for one problem size, allocated once and reused across calls."""
 
-    def __init__(self, B: int, N: int, d: int, dtype: int, device="cuda"):
+    def __init__(self, B: int, N: int, d: int, dtype: int, device="cuda", op: int = GC_OP_BUILD):
         f = dict(dtype=torch.float32, device=device)
         self.loss = torch.zeros(1, **f)
         self.row_lse = torch.empty(B, **f)
@@ -216,7 +232,7 @@ class Outputs:
         self.dQ = torch.empty(B, d, **f)
         self.dP = torch.empty(N, d, **f)
         self.dev_status = torch.zeros(1, dtype=torch.int32, device=device)
-        self.ws = alloc_workspace(GC_OP_BUILD, B, N, d, dtype, device)
+        self.ws = alloc_workspace(op, B, N, d, dtype, device)
 
 
 def build_cache(Q, P, pos_idx, tau=1.0, mask_mode=GC_MASK_NONE, out: Outputs | None = None):

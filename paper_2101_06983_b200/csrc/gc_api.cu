@@ -27,7 +27,10 @@ int sm_count() {
 
 static size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
-Plan make_plan(int64_t B, int64_t N, int d, int dtype) {
+// Largest weight matrix gc_build_cache will ask the workspace to hold.
+constexpr size_t kMaxStoredWeightBytes = (size_t)40 << 30;
+
+Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored) {
     Plan pl{};
     pl.tc = tc_supported(B, N, d, dtype) ? 1 : 0;
     if (pl.tc) {
@@ -48,14 +51,39 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype) {
     pl.off_m = off;    off += align256(sizeof(float) * slots * (size_t)B);
     pl.off_l = off;    off += align256(sizeof(float) * slots * (size_t)B);
     pl.off_pos = off;  off += align256(sizeof(float) * (size_t)B);
+    pl.off_red = off;  off += 2048;      // loss reduction: block ticket + up to 256 block sums
     pl.off_accq = off;
     if (pl.g_dq > 1 || pl.fused) off += align256(sizeof(float) * (size_t)pl.g_dq * (size_t)B * dpad);
     pl.off_accp = off;
     if (pl.g_dp > 1) off += align256(sizeof(float) * (size_t)pl.g_dp * (size_t)N * dpad);
-    pl.total = off;
     pl.launches_fwd = 2;  // sweep + combine
     pl.launches_bwd = 2 + (pl.g_dq > 1 ? 1 : 0) + (pl.g_dp > 1 ? 1 : 0);
     pl.launches_build = pl.fused ? 4 + (pl.g_dp > 1 ? 1 : 0) : pl.launches_fwd + pl.launches_bwd;
+    // Stored weights: B x N bf16 (pitch rounded up to 64 elements), kept when they fit the limit
+    // below; the gradient partials share the regions of the sweeps they replace.
+    pl.ldw = (N + 63) / 64 * 64;
+    const size_t w_bytes = (size_t)B * (size_t)pl.ldw * 2;
+    pl.mat = (stored && pl.tc && w_bytes <= kMaxStoredWeightBytes) ? 1 : 0;
+    if (pl.mat) {
+        pl.g_mq = gemm_groups(B, N, d);
+        pl.g_mp = gemm_groups(N, B, d);
+        size_t accq = align256(sizeof(float) * (size_t)pl.g_mq * (size_t)B * dpad);
+        size_t accp = pl.g_mp > 1 ? align256(sizeof(float) * (size_t)pl.g_mp * (size_t)N * dpad) : 0;
+        if (pl.off_accp - pl.off_accq < accq) {       // grow the dQ partial region
+            size_t old_accp = off - pl.off_accp;
+            pl.off_accp = pl.off_accq + accq;
+            off = pl.off_accp + old_accp;
+        }
+        if (off - pl.off_accp < accp) off = pl.off_accp + accp;
+        pl.off_ref = off;   off += align256(sizeof(float) * (size_t)B);
+        pl.off_flag = off;  off += 256;
+        pl.off_qs = off;    off += align256((size_t)B * (size_t)d * 2);
+        pl.off_w = off;     off += align256(w_bytes);
+        // anchor, sweep, combine, row scaling, dQ GEMM, dQ finalize, dP GEMM (+ reduce),
+        // positive terms, then the gated fallback sequence
+        pl.launches_build = 8 + (pl.g_mp > 1 ? 1 : 0) + pl.launches_build;
+    }
+    pl.total = off;
     return pl;
 }
 
@@ -73,11 +101,11 @@ Profile g_prof;
 struct KernelTimer {
     int k;
     cudaStream_t st;
-    KernelTimer(int kernel, cudaStream_t s) : k(kernel), st(s) {
-        if (g_prof.on) { cudaEventRecord(g_prof.ev[2 * k], st); g_prof.used[k] = true; }
+    KernelTimer(int kernel, cudaStream_t s) : k(kernel), st(s) {   // kernel < 0: not timed
+        if (g_prof.on && k >= 0) { cudaEventRecord(g_prof.ev[2 * k], st); g_prof.used[k] = true; }
     }
     ~KernelTimer() {
-        if (g_prof.on) cudaEventRecord(g_prof.ev[2 * k + 1], st);
+        if (g_prof.on && k >= 0) cudaEventRecord(g_prof.ev[2 * k + 1], st);
     }
 };
 
@@ -133,28 +161,32 @@ Problem make_problem(const void* Q, int64_t ldq, const void* P, int64_t ldp,
 }
 
 int run_fwd(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_lse,
-            float* pos_logit, int* dev_status, cudaStream_t st) {
-    FwdArgs fa;
+            float* pos_logit, int* dev_status, cudaStream_t st, const int* run_if = nullptr) {
+    FwdArgs fa{};
     fa.p = p;
+    fa.run_if = run_if;
     fa.part_m = reinterpret_cast<float*>(ws + pl.off_m);
     fa.part_l = reinterpret_cast<float*>(ws + pl.off_l);
     fa.pos_logit = reinterpret_cast<float*>(ws + pl.off_pos);
+    fa.red = reinterpret_cast<float*>(ws + pl.off_red);
     fa.groups = pl.g_fwd;
     fa.dev_status = dev_status;
     cudaError_t e;
     {
-        KernelTimer t(0, st);
+        KernelTimer t(run_if ? -1 : 0, st);
         e = pl.tc ? tc_launch_fwd(fa, st) : simt_launch_fwd(fa, st);
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, dev_status, st);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, run_if, st);
     return e == cudaSuccess ? GC_OK : GC_ERR_CUDA;
 }
 
 int run_sweep(const Problem& p, const Plan& pl, char* ws, int mode, const float* row_lse,
-              float* out, int64_t ldo, int* dev_status, cudaStream_t st) {
-    SweepArgs sa;
+              float* out, int64_t ldo, int* dev_status, cudaStream_t st,
+              const int* run_if = nullptr) {
+    SweepArgs sa{};
+    sa.run_if = run_if;
     const bool dq = (mode == SWEEP_DQ);
     sa.X = dq ? p.Q : p.P;   sa.ldx = dq ? p.ldq : p.ldp;   sa.nx = dq ? p.B : p.N;
     sa.Y = dq ? p.P : p.Q;   sa.ldy = dq ? p.ldp : p.ldq;   sa.ny = dq ? p.N : p.B;
@@ -173,12 +205,13 @@ int run_sweep(const Problem& p, const Plan& pl, char* ws, int mode, const float*
     sa.dev_status = dev_status;
     cudaError_t e;
     {
-        KernelTimer t(dq ? 1 : 2, st);
+        KernelTimer t(run_if ? -1 : (dq ? 1 : 2), st);
         e = pl.tc ? tc_launch_sweep(sa, st) : simt_launch_sweep(sa, st);
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     if (sa.groups > 1) {
-        e = launch_partial_reduce(sa.partial, sa.groups, sa.nx, sa.d, sa.out_scale, out, ldo, st);
+        e = launch_partial_reduce(sa.partial, sa.groups, sa.nx, sa.d, sa.out_scale, out, ldo, run_if,
+                                  st);
         if (e != cudaSuccess) return GC_ERR_CUDA;
     }
     return GC_OK;
@@ -187,28 +220,115 @@ int run_sweep(const Problem& p, const Plan& pl, char* ws, int mode, const float*
 // gc_build_cache for wide bf16 rows: fused forward + dQ sweep, combine, dQ finalize.
 int run_fused_fwd_dq(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_lse,
                      float* pos_logit, float* dQ, int64_t lddq, int* dev_status,
-                     cudaStream_t st) {
-    FwdArgs fa;
+                     cudaStream_t st, const int* run_if = nullptr) {
+    FwdArgs fa{};
     fa.p = p;
+    fa.run_if = run_if;
     fa.part_m = reinterpret_cast<float*>(ws + pl.off_m);
     fa.part_l = reinterpret_cast<float*>(ws + pl.off_l);
     fa.pos_logit = reinterpret_cast<float*>(ws + pl.off_pos);
+    fa.red = reinterpret_cast<float*>(ws + pl.off_red);
     fa.groups = 2 * pl.g_dq;
     fa.dev_status = dev_status;
     float* partial = reinterpret_cast<float*>(ws + pl.off_accq);
     cudaError_t e;
     {
-        KernelTimer t(1, st);
+        KernelTimer t(run_if ? -1 : 1, st);
         e = tc_launch_fused_dq(fa, partial, pl.g_dq, st);
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, dev_status, st);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, run_if, st);
     if (e != cudaSuccess) return GC_ERR_CUDA;
-    e = launch_fused_dq_finalize(partial, pl.g_dq, fa.part_m, row_lse, fa.pos_logit, p.pos_idx, p.P,
-                                 p.ldp, p.B, p.N, p.d, p.mask_mode,
-                                 1.f / ((float)p.B * p.tau), dQ, lddq, st);
+    e = launch_fused_dq_finalize(partial, pl.g_dq, fa.part_m, nullptr, row_lse, fa.pos_logit,
+                                 p.pos_idx, p.P, p.ldp, p.B, p.N, p.d, p.mask_mode,
+                                 1.f / ((float)p.B * p.tau), dQ, lddq, run_if, st);
     return e == cudaSuccess ? GC_OK : GC_ERR_CUDA;
+}
+
+// The recomputing sequence of gc_build_cache; with run_if every kernel of it is gated.
+int run_build_sweeps(const Problem& p, const Plan& pl, char* w, float* loss, float* row_lse,
+                     float* pos_logit, float* dQ, int64_t lddq, float* dP, int64_t lddp,
+                     int* dev_status, cudaStream_t st, const int* run_if = nullptr) {
+    int rc;
+    if (pl.fused) {
+        if ((rc = run_fused_fwd_dq(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dev_status, st,
+                                   run_if)))
+            return rc;
+    } else {
+        if ((rc = run_fwd(p, pl, w, loss, row_lse, pos_logit, dev_status, st, run_if))) return rc;
+        if ((rc = run_sweep(p, pl, w, SWEEP_DQ, row_lse, dQ, lddq, dev_status, st, run_if)))
+            return rc;
+    }
+    return run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, dev_status, st, run_if);
+}
+
+// gc_build_cache with stored weights (Eq. 1, 5, 6-7 without recomputing a logit):
+//   anchor      ref2_i = log2(e) S_{i,r_i}, the scale all weights of row i are measured against
+//   sweep       W~_ij = 2^(s2_ij - ref2_i) as bf16 (0 at masked pairs and at the positive), the
+//               row sums in fp32, pos_logit; a weight beyond 2^100 raises the range flag
+//   combine     row_lse, loss
+//   dQ          (2^(ref2_i - lse2_i) sum_j W~_ij P_j + (p_pos - 1) P_pos) / (B tau)
+//   dP          (sum_i W~_ij Q'_i) / (B tau) with Q'_i = 2^(ref2_i - lse2_i) Q_i, then the
+//               positive terms (p_pos - 1) Q_i / (B tau) added in fp32 in query order
+// When the range flag is up (logits more than 100 powers of two above the positive's) these
+// results are not usable; the gated recomputing sequence that follows then overwrites them all.
+int run_build_stored(const Problem& p, const Plan& pl, char* w, float* loss, float* row_lse,
+                     float* pos_logit, float* dQ, int64_t lddq, float* dP, int64_t lddp,
+                     int* dev_status, cudaStream_t st) {
+    float* ref2 = reinterpret_cast<float*>(w + pl.off_ref);
+    int* flag = reinterpret_cast<int*>(w + pl.off_flag);
+    void* qs = w + pl.off_qs;
+    void* weights = w + pl.off_w;
+    float* partq = reinterpret_cast<float*>(w + pl.off_accq);
+    float* partp = reinterpret_cast<float*>(w + pl.off_accp);
+    const float scale = 1.f / ((float)p.B * p.tau);
+    cudaError_t e = launch_pos_anchor(p.Q, p.ldq, p.P, p.ldp, p.pos_idx, p.B, p.N, p.d, p.mask_mode,
+                                      1.4426950408889634f / p.tau, ref2, flag, st);
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    FwdArgs fa{};
+    fa.p = p;
+    fa.part_m = reinterpret_cast<float*>(w + pl.off_m);
+    fa.part_l = reinterpret_cast<float*>(w + pl.off_l);
+    fa.pos_logit = reinterpret_cast<float*>(w + pl.off_pos);
+    fa.red = reinterpret_cast<float*>(w + pl.off_red);
+    fa.groups = pl.g_fwd;
+    fa.dev_status = dev_status;
+    {
+        KernelTimer t(0, st);
+        e = tc_launch_fwd_store(fa, weights, pl.ldw, ref2, flag, st);
+    }
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, nullptr, st);
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    e = launch_scale_rows(p.Q, p.ldq, p.B, p.d, ref2, row_lse, qs, st);
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    {
+        KernelTimer t(1, st);
+        e = launch_weight_gemm(weights, pl.ldw, p.B, p.N, 0, p.P, p.ldp, p.d, pl.g_mq, 1.f,
+                               nullptr, 0, partq, dev_status, st);
+    }
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    e = launch_fused_dq_finalize(partq, pl.g_mq, nullptr, ref2, row_lse, fa.pos_logit, p.pos_idx,
+                                 p.P, p.ldp, p.B, p.N, p.d, p.mask_mode, scale, dQ, lddq, nullptr,
+                                 st);
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    {
+        KernelTimer t(2, st);
+        e = launch_weight_gemm(weights, pl.ldw, p.B, p.N, 1, qs, p.d, p.d, pl.g_mp, scale, dP, lddp,
+                               partp, dev_status, st);
+    }
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    if (pl.g_mp > 1) {
+        e = launch_partial_reduce(partp, pl.g_mp, p.N, p.d, scale, dP, lddp, nullptr, st);
+        if (e != cudaSuccess) return GC_ERR_CUDA;
+    }
+    e = launch_dp_positive(p.pos_idx, p.B, p.N, p.mask_mode, fa.pos_logit, row_lse, p.Q, p.ldq, p.d,
+                           scale, dP, lddp, st);
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    return run_build_sweeps(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status, st,
+                            flag);
 }
 
 }  // namespace
@@ -246,9 +366,11 @@ void* static_scratch_ptr() {
 extern "C" {
 
 size_t gc_workspace_bytes(int op, int64_t B, int64_t N, int d, int dtype) {
-    if (op < GC_OP_FWD || op > GC_OP_BUILD || B <= 0 || N <= 0 || d <= 0) return 0;
+    if (op < GC_OP_FWD || op > GC_OP_BUILD_STORED || B <= 0 || N <= 0 || d <= 0) return 0;
     if (dtype != GC_F32 && dtype != GC_BF16) return 0;
-    return make_plan(B, N, d, dtype).total;   // one layout serves all three calls
+    // one layout serves the three calls of the paper's path; the stored-weights build appends its
+    // own regions to it
+    return make_plan(B, N, d, dtype, op == GC_OP_BUILD_STORED).total;
 }
 
 const char* gc_plan_name(int op, int64_t B, int64_t N, int d, int dtype) {
@@ -263,6 +385,7 @@ int gc_kernel_launches(int op, int64_t B, int64_t N, int d, int dtype) {
     if (op == GC_OP_FWD) return pl.launches_fwd;
     if (op == GC_OP_BWD) return pl.launches_bwd + 1;   // + pos_idx validation
     if (op == GC_OP_BUILD) return pl.launches_build;
+    if (op == GC_OP_BUILD_STORED) return make_plan(B, N, d, dtype, true).launches_build;
     return 0;
 }
 
@@ -340,15 +463,27 @@ int gc_build_cache(const void* Q, int64_t ldq, const void* P, int64_t ldp, const
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
     char* w = static_cast<char*>(ws);
-    if (pl.fused) {
-        if ((rc = run_fused_fwd_dq(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dev_status, st)))
-            return rc;
-    } else {
-        if ((rc = run_fwd(p, pl, w, loss, row_lse, pos_logit, dev_status, st))) return rc;
-        if ((rc = run_sweep(p, pl, w, SWEEP_DQ, row_lse, dQ, lddq, dev_status, st))) return rc;
-    }
-    if ((rc = run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, dev_status, st))) return rc;
-    return GC_OK;
+    return run_build_sweeps(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status, st);
+}
+
+int gc_build_cache_stored(const void* Q, int64_t ldq, const void* P, int64_t ldp,
+                          const int32_t* pos_idx, int64_t B, int64_t N, int d, float tau,
+                          int mask_mode, int dtype, float* loss, float* row_lse, float* pos_logit,
+                          float* dQ, int64_t lddq, float* dP, int64_t lddp, void* ws,
+                          size_t ws_bytes, int* dev_status, void* cuda_stream) {
+    int rc = check_common(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
+    if (rc) return rc;
+    if (!loss || !row_lse || !dQ || !dP) return GC_ERR_NULL;
+    if ((rc = check_grad_out(dQ, lddq, d))) return rc;
+    if ((rc = check_grad_out(dP, lddp, d))) return rc;
+    Plan pl = make_plan(B, N, d, dtype, true);
+    if (!pl.mat) return GC_ERR_LIMIT;       // not a tcgen05 shape, or the weights exceed the limit
+    if ((rc = check_ws(ws, ws_bytes, pl.total))) return rc;
+    if ((rc = check_device())) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
+    return run_build_stored(p, pl, static_cast<char*>(ws), loss, row_lse, pos_logit, dQ, lddq, dP,
+                            lddp, dev_status, st);
 }
 
 int gc_profile_enable(int on) {
@@ -387,7 +522,9 @@ const char* gc_status_string(int status) {
         case GC_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case GC_ERR_CUDA: return "a CUDA call failed";
         case GC_ERR_ARCH: return "device is not compute capability 10.x";
-        case GC_ERR_LIMIT: return "problem needs more scratch than the library's built-in area holds";
+        case GC_ERR_LIMIT:
+            return "problem exceeds a built-in limit of this entry point (static scratch size, or "
+                   "dtype / shape / size of the stored weights)";
         default: return "unknown status";
     }
 }

@@ -47,6 +47,7 @@ struct SweepArgs {
     float* partial;         // [groups x nx x d] unscaled partial sums (used when groups > 1)
     int groups;             // the y range is split into this many contiguous parts
     int* dev_status;        // may be NULL
+    const int* run_if;      // when not NULL the kernels return at once unless *run_if != 0
 };
 
 struct FwdArgs {
@@ -54,38 +55,58 @@ struct FwdArgs {
     float* part_m;          // [groups x B] running maximum of each part
     float* part_l;          // [groups x B] sum of exp(S - m) of each part
     float* pos_logit;       // [B] written only by the owner of column pos_idx[i]
+    float* red;             // scratch of the loss reduction that follows; the sweep clears its
+                            // first word (the block ticket)
     int groups;
     int* dev_status;        // may be NULL
+    const int* run_if;      // when not NULL the kernels return at once unless *run_if != 0
 };
 
 // How one call is carried out for given sizes on the current device.
 struct Plan {
     int tc;                 // 1: tcgen05 kernels, 0: SIMT kernels
     int g_fwd, g_dq, g_dp;  // split factors of the streamed range
-    size_t off_m, off_l, off_pos, off_accq, off_accp;
+    size_t off_m, off_l, off_pos, off_red, off_accq, off_accp;
     size_t total;           // workspace bytes (multiple of 256)
     int launches_fwd, launches_bwd;
     int fused;              // 1: gc_build_cache runs the forward inside the dQ sweep
     int launches_build;
+    // Stored-weights plan of gc_build_cache (tcgen05 only): one forward sweep keeps the bf16
+    // weights, two GEMMs form the gradients; the sweeps above stay as its fallback.
+    int mat;
+    int g_mq, g_mp;         // split factors of the two GEMMs' contraction ranges
+    int64_t ldw;            // row pitch of the stored weights, elements
+    size_t off_ref, off_flag, off_qs, off_w;
 };
 
 int sm_count();
-Plan make_plan(int64_t B, int64_t N, int d, int dtype);
+Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored = false);
 
 // gc_combine.cu
 cudaError_t launch_lse_combine(const float* part_m, const float* part_l, const float* pos_ws,
                                const int32_t* pos_idx, int groups, int64_t B, int64_t N,
                                int mask_mode, float* row_lse, float* pos_logit, float* loss,
-                               int* dev_status, cudaStream_t st);
+                               float* red, int* dev_status, const int* run_if, cudaStream_t st);
 cudaError_t launch_pos_check(const int32_t* pos_idx, int64_t B, int64_t N, int mask_mode,
                              int* dev_status, cudaStream_t st);
 cudaError_t launch_fused_dq_finalize(const float* partial, int groups, const float* part_m,
-                                     const float* row_lse, const float* pos_ws,
-                                     const int32_t* pos_idx, const void* P, int64_t ldp,
-                                     int64_t B, int64_t N, int d, int mask_mode, float scale,
-                                     float* out, int64_t ldo, cudaStream_t st);
+                                     const float* row_ref2, const float* row_lse,
+                                     const float* pos_ws, const int32_t* pos_idx, const void* P,
+                                     int64_t ldp, int64_t B, int64_t N, int d, int mask_mode,
+                                     float scale, float* out, int64_t ldo, const int* run_if,
+                                     cudaStream_t st);
 cudaError_t launch_partial_reduce(const float* partial, int groups, int64_t rows, int d,
-                                  float scale, float* out, int64_t ldo, cudaStream_t st);
+                                  float scale, float* out, int64_t ldo, const int* run_if,
+                                  cudaStream_t st);
+cudaError_t launch_pos_anchor(const void* Q, int64_t ldq, const void* P, int64_t ldp,
+                              const int32_t* pos_idx, int64_t B, int64_t N, int d, int mask_mode,
+                              float c1, float* ref2, int* range_flag, cudaStream_t st);
+cudaError_t launch_scale_rows(const void* Q, int64_t ldq, int64_t B, int d, const float* ref2,
+                              const float* row_lse, void* Qs, cudaStream_t st);
+cudaError_t launch_dp_positive(const int32_t* pos_idx, int64_t B, int64_t N, int mask_mode,
+                               const float* pos_ws, const float* row_lse, const void* Q,
+                               int64_t ldq, int d, float scale, float* out, int64_t ldo,
+                               cudaStream_t st);
 
 // gc_simt.cu
 cudaError_t simt_launch_fwd(const FwdArgs& a, cudaStream_t st);
@@ -101,5 +122,14 @@ int tc_fwd_groups(int64_t B, int64_t N, int d);
 bool tc_fused_applicable(int d);
 cudaError_t tc_launch_fused_dq(const FwdArgs& a, float* partial, int groups, cudaStream_t st);
 int tc_sweep_groups(int64_t nx, int64_t ny, int d);
+cudaError_t tc_launch_fwd_store(const FwdArgs& a, void* weights, int64_t ldw, const float* row_ref,
+                                int* range_flag, cudaStream_t st);
+
+// gc_gemm.cu
+int gemm_groups(int64_t m_rows, int64_t k_len, int d);
+cudaError_t launch_weight_gemm(const void* weights, int64_t ldw, int64_t B, int64_t N, int transpose,
+                               const void* V, int64_t ldv, int d, int groups, float out_scale,
+                               float* out, int64_t ldo, float* partial, int* dev_status,
+                               cudaStream_t st);
 
 }  // namespace gc

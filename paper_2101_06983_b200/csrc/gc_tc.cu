@@ -27,40 +27,21 @@
 // epilogue: two warps per tensor-memory lane quarter, each owning half of the tile's columns,
 // one thread per tile row.
 // Every wait is bounded: on a timeout the CTA raises GC_DEV_WAIT_LIMIT, drains and exits.
-#include <cuda.h>
-#include <cuda_bf16.h>
-#include <math.h>
-
-#include "gc_internal.h"
+#include "tc_common.cuh"
 
 namespace gc {
 
 namespace {
 
-constexpr int XROWS = 128;                 // rows of the stationary tile = MMA M
-constexpr int CHUNK_BYTES_PER_ROW = 128;   // 64 bf16 = one swizzle row
-constexpr uint32_t X_CHUNK_BYTES = XROWS * CHUNK_BYTES_PER_ROW;
-constexpr int NPROD = 2;                   // TMA producer warps
-constexpr int MMA_WARP = NPROD;
-constexpr int NSOFT = 8;                   // softmax / epilogue warps
-constexpr int NTHREADS = 32 * (NPROD + 1 + NSOFT);
-constexpr int MAX_STAGES = 12;
-constexpr uint32_t CHUNK_BYTES = 16384;    // 128 rows x 64 columns: one X chunk or one Y chunk
-constexpr int TMEM_COLS = 512;
-constexpr int MAX_D = 4096;                // wider rows just take more column parts
-constexpr int MAX_PART_CHUNKS = 6;         // 384 accumulator columns
-constexpr size_t SMEM_LIMIT = 232448;      // 227 KB per block
-constexpr size_t SMEM_STATIC_RESERVE = 2048;
-constexpr uint64_t WAIT_LIMIT_NS = 2000000000ull;
-
-enum { MODE_FWD = 0, MODE_DQ = 1, MODE_DP = 2, MODE_FQ = 3 };   // FQ: forward fused into dQ
+// FQ: forward fused into dQ; FS: forward that also stores the bf16 weights
+enum { MODE_FWD = 0, MODE_DQ = 1, MODE_DP = 2, MODE_FQ = 3, MODE_FS = 4 };
 
 // Optional diagnostics (-DGC_TC_TRACE): cycles each role spends waiting, summed over CTAs.
 #ifdef GC_TC_TRACE
 enum { TR_MMA_TOTAL, TR_MMA_WAIT_Y, TR_MMA_WAIT_W, TR_SM_TOTAL, TR_SM_WAIT_S, TR_SM_EPI,
        TR_PROD_TOTAL, TR_PROD_WAIT, TR_CTAS, TR_MMA_ISSUE, TR_MMA_COMMIT, TR_ACC_ISSUE, TR_ACC_COMMIT, TR_SFULL_COMMIT,
        TR_CTA_LIFE, TR_SETUP, TR_T0_MIN, TR_T0_MAX, TR_T1_MIN, TR_T1_MAX, TR_COUNT };
-__device__ unsigned long long g_trace[4][TR_COUNT];
+__device__ unsigned long long g_trace[5][TR_COUNT];
 #define TR_DECL(v) long long v = 0
 #define TR_BEGIN(v) long long v##_t0 = clock64()
 #define TR_END(v) v += clock64() - v##_t0
@@ -94,284 +75,11 @@ struct TcParams {
     float* part_l;
     float* pos_logit;
     int* dev_status;
+    const float* row_ref;     // FS: per-query anchor of the stored weights, log2 domain
+    int* range_flag;          // FS: set to 1 when a weight leaves the range the anchor allows
+    const int* run_if;        // when not NULL and *run_if == 0 the kernel returns at once
+    int* zero_me;             // forward sweeps: the ticket word of the reduction that follows
 };
-
-// ---------------------------------------------------------------------------------------------
-// PTX wrappers
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-    return (uint32_t)__cvta_generic_to_shared(p);
-}
-__device__ __forceinline__ uint64_t global_ns() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bounded wait: false when the CTA is aborting or the time limit passed.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try(bar, parity)) return true;
-    uint64_t t0 = global_ns();
-    uint32_t spins = 0;
-    while (true) {
-        if (mbar_try(bar, parity)) return true;
-        if ((++spins & 127u) == 0u) {
-            if (*abort_flag) return false;
-            if (global_ns() - t0 > WAIT_LIMIT_NS) {
-                *abort_flag = 1;
-                return false;
-            }
-        }
-    }
-}
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1,
-                                            uint32_t bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes "
-        "[%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
-        : "memory");
-}
-// True on exactly one lane of a converged warp.  The surrounding loops run on all 32 lanes with
-// warp-uniform values, so that addresses and descriptors can stay in uniform registers, which
-// is where bulk-tensor and tcgen05 instructions read them from.
-__device__ __forceinline__ bool elect_one() {
-    uint32_t pred;
-    asm volatile(
-        "{\n\t.reg .pred P;\n\t"
-        "elect.sync _|P, 0xffffffff;\n\t"
-        "selp.u32 %0, 1, 0, P;\n\t}"
-        : "=r"(pred));
-    return pred != 0;
-}
-// ---- CTA-pair (cluster of 2) helpers -------------------------------------------------------------
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster
-__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
-    uint32_t r;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\t"
-                 "barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];"
-                 ::"r"(cluster_addr) : "memory");
-}
-// Bulk tensor load of a CTA pair: the data lands in the executing CTA, the transaction bytes are
-// counted on an mbarrier that may live in the other CTA of the pair (no multicast).
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int c0,
-                                                 int c1, uint32_t bar_cluster) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
-        "[%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar_cluster)
-        : "memory");
-}
-// Arrives on the mbarrier at this offset in both CTAs of the pair once all MMAs issued so far
-// by this thread have completed.
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
-    asm volatile(
-        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 "
-        "[%0], %1;"
-        ::"r"(bar), "h"((uint16_t)3) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() {
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-}
-__device__ __forceinline__ void tc_fence_after() {
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-}
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
-                 ::"r"(bar) : "memory");
-}
-// Shared-memory matrix descriptors for 128-byte-swizzled tiles with 128-byte rows.  The high
-// word is constant: stride between 8-row groups = 1024 bytes (>> 4), descriptor version 1,
-// layout type 2 (SWIZZLE_128B).  The low word holds the start address (>> 4) and, in bits 16-29,
-// the leading byte offset (>> 4): the distance between 64-element atoms along M/N of an
-// MN-major operand (ignored for K-major operands).  A K-major operand advances 32 bytes
-// (low word + 2) per K = 16; an MN-major operand advances 16 rows = 2048 bytes (low word + 128).
-constexpr uint32_t DESC_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
-__device__ __forceinline__ uint32_t desc_lo(uint32_t addr, uint32_t lbo_bytes) {
-    return ((addr >> 4) & 0x3FFFu) | ((lbo_bytes >> 4) << 16);
-}
-// D[tmem] (+)= A[smem] * B[smem].  The issuing thread is alone on its scheduler, so every scalar
-// instruction spent per MMA shows up as idle tensor time: keep the operands precomputed.
-template <bool ACC, bool PAIR>
-__device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo,
-                                       uint32_t idesc) {
-    if (PAIR) {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-            "setp.ne.b32 p, %5, 0;\n\t"
-            "mov.b64 da, {%1, %4};\n\t"
-            "mov.b64 db, {%2, %4};\n\t"
-            "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %3, p;\n\t}"
-            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(DESC_HI), "n"(ACC ? 1 : 0)
-            : "memory");
-    } else {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-            "setp.ne.b32 p, %5, 0;\n\t"
-            "mov.b64 da, {%1, %4};\n\t"
-            "mov.b64 db, {%2, %4};\n\t"
-            "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p;\n\t}"
-            ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(DESC_HI), "n"(ACC ? 1 : 0)
-            : "memory");
-    }
-}
-// D[tmem] (+)= A[tmem] * B[smem]
-template <bool ACC, bool PAIR>
-__device__ __forceinline__ void mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo,
-                                       uint32_t idesc) {
-    if (PAIR) {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
-            "setp.ne.b32 p, %5, 0;\n\t"
-            "mov.b64 db, {%2, %4};\n\t"
-            "tcgen05.mma.cta_group::2.kind::f16 [%0], [%1], db, %3, p;\n\t}"
-            ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(DESC_HI), "n"(ACC ? 1 : 0)
-            : "memory");
-    } else {
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t.reg .b64 db;\n\t"
-            "setp.ne.b32 p, %5, 0;\n\t"
-            "mov.b64 db, {%2, %4};\n\t"
-            "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p;\n\t}"
-            ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(DESC_HI), "n"(ACC ? 1 : 0)
-            : "memory");
-    }
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
-          "=r"(v[7]), "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]),
-          "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]),
-          "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]),
-          "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() {
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
-        ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]),
-          "r"(v[7]), "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]),
-          "r"(v[14]), "r"(v[15])
-        : "memory");
-}
-__device__ __forceinline__ void tmem_st_wait() {
-    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-}
-// ---- epilogue: accumulator blocks leave through shared memory and bulk tensor stores ---------------
-// One warp's block of 32 rows x 32 fp32 columns is written to a 4 KB buffer in the 128-byte
-// swizzle the tensor map expects (16-byte chunk j of row r at chunk j ^ (r & 7)), which also
-// makes the float4 stores conflict-free, and then leaves with one bulk tensor store; rows past
-// the end of the matrix are clipped by the tensor map.
-__device__ __forceinline__ void stage_block(uint32_t buf, const uint32_t (&v)[32], float sc,
-                                            int lane) {
-#pragma unroll
-    for (int j = 0; j < 8; ++j) {
-        const uint32_t addr = buf + lane * 128 + ((j ^ (lane & 7)) << 4);
-        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};"
-                     ::"r"(addr), "f"(__uint_as_float(v[4 * j]) * sc),
-                       "f"(__uint_as_float(v[4 * j + 1]) * sc),
-                       "f"(__uint_as_float(v[4 * j + 2]) * sc),
-                       "f"(__uint_as_float(v[4 * j + 3]) * sc)
-                     : "memory");
-    }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // visible to the bulk store
-}
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap* map, uint32_t src, int c0, int c1,
-                                             int c2) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
-        ::"l"(reinterpret_cast<uint64_t>(map)), "r"(src), "r"(c0), "r"(c1), "r"(c2)
-        : "memory");
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-// Writes accumulator blocks cb = half, half + 2, ... (32 columns each) of this warp's 32 rows.
-// `slot` is the warp's 8 KB staging area (two buffers).
-__device__ __forceinline__ void store_acc_blocks(uint32_t tmem_rows, int nblocks, int half,
-                                                 uint32_t slot, float sc, int lane,
-                                                 const CUtensorMap* mapO, int col0, int row0,
-                                                 int plane) {
-    int n = 0;
-    for (int cb = half; cb < nblocks; cb += 2, ++n) {
-        uint32_t v[32];
-        tmem_ld32(tmem_rows + cb * 32, v);
-        if (n >= 2) {   // the store issued two blocks ago has finished reading this buffer
-            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
-            __syncwarp();
-        }
-        tmem_ld_wait();
-        const uint32_t buf = slot + (n & 1) * 4096;
-        stage_block(buf, v, sc, lane);
-        __syncwarp();
-        if (lane == 0) tma_store_3d(mapO, buf, col0 + cb * 32, row0, plane);
-    }
-    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-    __syncwarp();
-}
-
-__device__ __forceinline__ float ex2(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
-// Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, M = 128.
-__device__ __forceinline__ uint32_t instr_desc(int n, bool b_mn_major, int m = XROWS) {
-    uint32_t d = 0;
-    d |= 1u << 4;                          // D format f32
-    d |= 1u << 7;                          // A format bf16
-    d |= 1u << 10;                         // B format bf16
-    d |= (b_mn_major ? 1u : 0u) << 16;     // B major
-    d |= (uint32_t)(n >> 3) << 17;
-    d |= (uint32_t)(m >> 4) << 24;          // 128, or 256 for an MMA across a CTA pair
-    return d;
-}
-
-__device__ __forceinline__ void part_range(int64_t steps, int groups, int g, int64_t* lo,
-                                           int64_t* hi) {
-    int64_t base = steps / groups, rem = steps % groups;
-    *lo = g * base + (g < rem ? g : rem);
-    *hi = *lo + base + (g < rem ? 1 : 0);
-}
 
 struct Bars {
     uint64_t x_full;
@@ -406,6 +114,8 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     __shared__ int abort_s;
     __shared__ float row_max_xch[2][XROWS];      // FQ: [column half][row] block maxima
     volatile int* abort_flag = &abort_s;
+    if (p.run_if && *p.run_if == 0) return;     // same answer in every CTA
+    if ((MODE == MODE_FWD || MODE == MODE_FS || MODE == MODE_FQ) && blockIdx.x == 0 && threadIdx.x == 0 && p.zero_me) *p.zero_me = 0;
 
     static_assert(SN == 128, "a Y chunk is 128 rows: the same 16 KB as an X chunk");
     constexpr uint32_t S_COL0 = TMEM_COLS - NBUF * SN;  // S buffers sit at the top columns
@@ -413,7 +123,10 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     // shared-memory buffers instead of over the single S tile.  The S tile is then free as soon as
     // the softmax warps have read it, S(t+1) is issued while softmax(t) computes, and acc(t)
     // follows from W buffer t & 1: the tensor pipe no longer waits for the softmax.
-    constexpr bool WS = PAIR && NBUF == 1 && MODE != MODE_FWD;
+    constexpr bool NOACC = MODE == MODE_FWD || MODE == MODE_FS;   // no accumulation MMAs
+    constexpr bool WS = PAIR && NBUF == 1 && !NOACC;
+    // FS: the softmax warps stage their bf16 weights in two 32 KB buffers (where WS keeps W)
+    constexpr bool WBUFS = WS || MODE == MODE_FS;
     constexpr int LAG = WS ? 1 : NBUF - 1;              // steps between S(t) and acc(t) issue
     constexpr int BSH = (NBUF == 2) ? 1 : 0;            // log2(NBUF)
     constexpr int WBUF = WS ? 2 : NBUF;                 // W buffers (w_full barriers in use)
@@ -436,7 +149,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     const int64_t xt = PAIR ? 2 * (int64_t)(unit / p.dparts) + rank : unit / p.dparts;
     const int64_t x0 = xt * XROWS;
     const int c_begin = dp * p.dpc;
-    const int c_count = (MODE == MODE_FWD) ? 0 : min(p.dpc, p.kc - c_begin);
+    const int c_count = NOACC ? 0 : min(p.dpc, p.kc - c_begin);
 
     int64_t lo, hi;
     part_range((p.ny + SN - 1) / SN, p.groups, g, &lo, &hi);
@@ -445,7 +158,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t x_smem = base;
     const uint32_t w_smem = base + (uint32_t)p.xres * X_CHUNK_BYTES;   // WS: two 32 KB W buffers
-    const uint32_t y_smem = w_smem + (WS ? 2u * 32768u : 0u);          // the ring
+    const uint32_t y_smem = w_smem + (WBUFS ? 2u * 32768u : 0u);       // the ring
     // a paired CTA holds half of every Y item, so its stages are one chunk (16 KB) and a streamed
     // X item is a single chunk; otherwise a stage holds ipc chunks of Y or of X
     const int xipc = PAIR ? 1 : p.ipc;
@@ -563,7 +276,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                             if (c + j >= p.xres) load_item(1, c + j, x0);
                     }
                 }
-                if (MODE != MODE_FWD && t >= LAG) {
+                if (!NOACC && t >= LAG) {
                     for (int c = 0; c < c_count; c += p.ipc)
                         load_item(2, c_begin + c, (lo + t - LAG) * SN);
                 }
@@ -629,7 +342,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         if (!ok) break;
                         tc_fence_after();
                     }
-                    if (MODE == MODE_FWD && t >= NBUF) {
+                    if (NOACC && t >= NBUF) {
                         ok = mbar_wait(smem_u32(&bars.w_full[b]), ((t - NBUF) >> BSH) & 1,
                                        abort_flag);
                         if (!ok) break;
@@ -699,7 +412,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     if (elect_one()) commit(smem_u32(&bars.s_full[b]));
                     TR_END(tr_sf);
                 }
-                if (MODE != MODE_FWD && t >= LAG) {
+                if (!NOACC && t >= LAG) {
                     const int u = t - LAG, b = u & (WBUF - 1);
                     TR_BEGIN(tr_ww);
                     ok = mbar_wait(smem_u32(&bars.w_full[b]), (u >> WSH) & 1, abort_flag);
@@ -743,7 +456,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     if (WS && ok && elect_one()) commit(smem_u32(&bars.w_empty[b]));
                 }
             }
-            if (ok && MODE != MODE_FWD && elect_one()) commit(smem_u32(&bars.acc_full));
+            if (ok && !NOACC && elect_one()) commit(smem_u32(&bars.acc_full));
 #ifdef GC_TC_TRACE
             if (lane == 0) {
             TR_ADD(MODE, TR_MMA_TOTAL, clock64() - tr_total_t0);
@@ -851,6 +564,112 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 const int64_t slot = (int64_t)(2 * g + half) * p.nq + x;
                 p.part_m[slot] = m * 0.69314718055994531f;   // back to natural log
                 p.part_l[slot] = l;
+            }
+        } else if (MODE == MODE_FS) {
+            // ---------------- forward sweep that also stores the weights ----------------
+            // Every weight of query x is 2^(s2 - ref2[x]) with an anchor chosen before the sweep,
+            // so all parts of the streamed range, and every later kernel, share one scale per
+            // row.  l is this half's sum over its allowed columns, positive included; the stored
+            // bf16 weight of the positive column is 0 (its term is added in fp32 later).
+            const float ref2 = (x < p.nx) ? p.row_ref[x] : 0.f;
+            const int32_t pos_x = (x < p.nx) ? p.pos_idx[x] : -1;
+            float l = 0.f, wmax = 0.f;
+            // this warp's 32 rows x 64 columns of a staging buffer: 4 KB, stored on their own
+            const uint32_t my_stage = w_smem + half * CHUNK_BYTES + q * 4096;
+            const bool rows_live = x0 + q * 32 < p.nx;
+            for (int t = 0; t < T; ++t) {
+                const int b = t & (NBUF - 1);
+                const int64_t y0 = (lo + t) * SN;
+                TR_BEGIN(tr_ws);
+                ok = mbar_wait(smem_u32(&bars.s_full[b]), (t >> BSH) & 1, abort_flag);
+                TR_END(tr_ws);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t sbuf = tmem + lane_addr + S_COL0 + b * SN;
+                uint32_t vv[CB_PER][32];
+#pragma unroll
+                for (int j = 0; j < CB_PER; ++j) tmem_ld32(sbuf + (cb0 + j) * 32, vv[j]);
+                tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) arrive_w(smem_u32(&bars.w_full[b]));   // S buffer b may be reused
+                // the store issued two steps ago has finished reading staging buffer t & 1
+                if (t >= 2) {
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                    __syncwarp();
+                }
+#pragma unroll
+                for (int j = 0; j < CB_PER; ++j) {
+                    const int64_t yb = y0 + (cb0 + j) * 32;
+                    const bool has_pos = pos_x >= yb && pos_x < yb + 32 && pos_x < p.ny &&
+                                         !(self_mask && x == pos_x);
+                    if (has_pos) {
+                        const int rel = (int)(pos_x - yb);
+                        float sp = 0.f;
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (c == rel) sp = __uint_as_float(vv[j][c]);
+                        p.pos_logit[x] = sp * p.inv_tau;
+                    }
+                    if (yb + 32 > p.ny) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (yb + c >= p.ny) vv[j][c] = __float_as_uint(-INFINITY);
+                    }
+                    if (self_mask && x >= yb && x < yb + 32) {
+                        const int rel = (int)(x - yb);
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (c == rel) vv[j][c] = __float_as_uint(-INFINITY);
+                    }
+                    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+                    float m0 = 0.f, m1 = 0.f;
+#pragma unroll
+                    for (int c = 0; c < 32; c += 4) {
+                        float w0 = ex2(fmaf(__uint_as_float(vv[j][c]), p.c1, -ref2));
+                        float w1 = ex2(fmaf(__uint_as_float(vv[j][c + 1]), p.c1, -ref2));
+                        float w2 = ex2(fmaf(__uint_as_float(vv[j][c + 2]), p.c1, -ref2));
+                        float w3 = ex2(fmaf(__uint_as_float(vv[j][c + 3]), p.c1, -ref2));
+                        s0 += w0; s1 += w1; s2 += w2; s3 += w3;
+                        m0 = fmaxf(m0, fmaxf(w0, w1));
+                        m1 = fmaxf(m1, fmaxf(w2, w3));
+                        vv[j][c] = __float_as_uint(w0);
+                        vv[j][c + 1] = __float_as_uint(w1);
+                        vv[j][c + 2] = __float_as_uint(w2);
+                        vv[j][c + 3] = __float_as_uint(w3);
+                    }
+                    l += (s0 + s1) + (s2 + s3);
+                    wmax = fmaxf(wmax, fmaxf(m0, m1));
+                    if (pos_x >= yb && pos_x < yb + 32) {                  // positive: fp32 later
+                        const int rel = (int)(pos_x - yb);
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            if (c == rel) vv[j][c] = 0u;
+                    }
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(vv[j][2 * r]),
+                                                                 __uint_as_float(vv[j][2 * r + 1]));
+                        packed[r] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+                    put_w_block(t & 1, j, packed);
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                // rows past nx and columns past ny are clipped by the tensor map
+                if (lane == 0 && rows_live && y0 + half * 64 < p.ny)
+                    tma_store_2d(&mapO, my_stage + (t & 1) * 32768u, (int)(y0 + half * 64),
+                                 (int)x0 + q * 32);
+            }
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+            __syncwarp();
+            if (ok && x < p.nx) {
+                const int64_t slot = (int64_t)(2 * g + half) * p.nq + x;
+                p.part_m[slot] = ref2 * 0.69314718055994531f;   // natural log units
+                p.part_l[slot] = l;
+                // weights beyond 2^100 (or not finite) cannot be accumulated safely
+                if (!(wmax <= 1.2676506e30f)) *p.range_flag = 1;
             }
         } else if (MODE == MODE_FQ) {
             // ---------------- forward fused into the dQ sweep ----------------
@@ -1171,62 +990,6 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     }
 }
 
-// ---------------------------------------------------------------------------------------------
-// Host side
-// ---------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
-                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
-                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
-                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (!fn) {
-        void* sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) !=
-                cudaSuccess || qres != cudaDriverEntryPointSuccess)
-            return nullptr;
-        fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    return fn;
-}
-
-// Row-major bf16 matrix [rows x d], boxes of (box_rows x 64 columns), 128-byte swizzle,
-// out-of-range elements read as zero.
-bool make_map(CUtensorMap* map, const void* base, int64_t rows, int d, int64_t ld, int box_rows) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-    cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
-                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
-}
-
-// fp32 destination of the accumulators as [planes][rows][d]: the output matrix itself (one plane,
-// row pitch ld) or the per-part partial sums (planes = parts of the streamed range, pitch d).
-// Boxes of 32 rows x 32 columns, 128-byte swizzle.
-bool make_out_map(CUtensorMap* map, float* base, int64_t rows, int d, int64_t ld, int planes) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)rows, (cuuint64_t)planes};
-    cuuint64_t strides[2] = {(cuuint64_t)ld * 4, (cuuint64_t)rows * (cuuint64_t)ld * 4};
-    cuuint32_t box[3] = {32, 32, 1};
-    cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, base, dims, strides, box, estr,
-                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-                    CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
-}
-
-int parts_for(int kc) { return (kc + MAX_PART_CHUNKS - 1) / MAX_PART_CHUNKS; }
-int chunks_per_part(int kc) { int n = parts_for(kc); return (kc + n - 1) / n; }
-
 // The gradient sweeps use 128-wide S tiles: two buffers when the accumulator part leaves room
 // (up to 256 columns), one otherwise.
 int sweep_nbuf(int kc) { return chunks_per_part(kc) * 64 + 256 <= TMEM_COLS ? 2 : 1; }
@@ -1240,7 +1003,7 @@ struct SmemPlan { int xres; int ipc; int nstage; size_t dynamic_bytes; };
 // 8 stages 0.341, 10 stages with no resident chunk 0.344), so only 2 X chunks stay resident.
 SmemPlan smem_plan(int kc, bool pair = false, bool ws = false) {
     SmemPlan sp;
-    sp.xres = ws ? 2 : (kc <= 8 ? kc : 6);
+    sp.xres = ws ? (kc < 2 ? kc : 2) : (kc <= 8 ? kc : 6);
     const int parts = parts_for(kc), dpc = chunks_per_part(kc);
     const bool even = kc % 2 == 0 && sp.xres % 2 == 0 && dpc % 2 == 0 &&
                       (kc - dpc * (parts - 1)) % 2 == 0;
@@ -1261,8 +1024,8 @@ SmemPlan smem_plan(int kc, bool pair = false, bool ws = false) {
 template <int MODE, int SN, int NBUF, bool PAIR>
 cudaError_t launch_one(const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& myh,
                        const CUtensorMap& mo, const TcParams& p, int64_t ctas, cudaStream_t st) {
-    constexpr bool WS = PAIR && NBUF == 1 && MODE != MODE_FWD;
-    SmemPlan sp = smem_plan(p.kc, PAIR, WS);
+    constexpr bool WBUFS = (PAIR && NBUF == 1 && MODE != MODE_FWD) || MODE == MODE_FS;
+    SmemPlan sp = smem_plan(p.kc, PAIR, WBUFS);
     static bool configured = false;
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(tc_kernel<MODE, SN, NBUF, PAIR>,
@@ -1301,6 +1064,7 @@ cudaError_t launch_one(const CUtensorMap& mx, const CUtensorMap& my, const CUten
 // tensor pipe's critical path.  The forward sweep pairs only when the streamed matrix does not
 // stay in the L2 cache, where halving its traffic outweighs the cross-SM hand-offs.
 bool use_pair(int mode, int kc, int64_t nx, int64_t ny) {
+    if (mode == MODE_FS) return smem_plan(kc, false, true).ipc == 2 && nx > XROWS;
     if (smem_plan(kc).ipc != 2 || nx <= XROWS || sweep_nbuf(kc) != 1) return false;
     if (mode != MODE_FWD) return true;
     return ny * kc * 128 > ((int64_t)64 << 20);
@@ -1383,8 +1147,43 @@ cudaError_t tc_launch_fwd(const FwdArgs& a, cudaStream_t st) {
     p.c1 = 1.4426950408889634f / pr.tau;
     p.pos_idx = pr.pos_idx;
     p.part_m = a.part_m; p.part_l = a.part_l; p.pos_logit = a.pos_logit;
+    p.zero_me = reinterpret_cast<int*>(a.red);
     p.dev_status = a.dev_status;
+    p.run_if = a.run_if;
     return launch<MODE_FWD, SN, 2>(mx, my, myh, mx, p, st);   // no accumulator output
+}
+
+// Forward sweep that also stores the weights 2^(s2_ij - row_ref[i]) as bf16 [B x N] (row pitch
+// ldw elements; 0 at masked pairs and at the positive column).  Writes the same (scale, sum) slots
+// and pos_logit as the plain forward sweep, with row_ref as the scale of every slot.
+cudaError_t tc_launch_fwd_store(const FwdArgs& a, void* weights, int64_t ldw, const float* row_ref,
+                                int* range_flag, cudaStream_t st) {
+    const Problem& pr = a.p;
+    constexpr int SN = 128;
+    const int kc = pr.d / 64;
+    CUtensorMap mx, my, myh, mw;
+    if (!make_map(&mx, pr.Q, pr.B, pr.d, pr.ldq, XROWS) ||
+        !make_map(&my, pr.P, pr.N, pr.d, pr.ldp, SN) ||
+        !make_map(&myh, pr.P, pr.N, pr.d, pr.ldp, SN / 2) ||
+        !make_map(&mw, weights, pr.B, (int)pr.N, ldw, 32))
+        return cudaErrorInvalidValue;
+    TcParams p{};
+    p.nx = pr.B; p.ny = pr.N; p.nq = pr.B;
+    p.kc = kc; p.dparts = 1; p.dpc = 0; p.groups = a.groups / 2;
+    const SmemPlan sp = smem_plan(kc, false, true);
+    p.nstage = sp.nstage;
+    p.xres = sp.xres;
+    p.ipc = sp.ipc;
+    p.mask_mode = pr.mask_mode;
+    p.inv_tau = 1.f / pr.tau;
+    p.c1 = 1.4426950408889634f / pr.tau;
+    p.pos_idx = pr.pos_idx;
+    p.part_m = a.part_m; p.part_l = a.part_l; p.pos_logit = a.pos_logit;
+    p.zero_me = reinterpret_cast<int*>(a.red);
+    p.dev_status = a.dev_status;
+    p.row_ref = row_ref;
+    p.range_flag = range_flag;
+    return launch<MODE_FS, SN, 2>(mx, my, myh, mw, p, st);
 }
 
 bool tc_fused_applicable(int d) { return sweep_nbuf(d / 64) == 1; }
@@ -1411,8 +1210,10 @@ cudaError_t tc_launch_fused_dq(const FwdArgs& a, float* partial, int groups, cud
     p.c1 = 1.4426950408889634f / pr.tau;
     p.pos_idx = pr.pos_idx;
     p.part_m = a.part_m; p.part_l = a.part_l; p.pos_logit = a.pos_logit;
+    p.zero_me = reinterpret_cast<int*>(a.red);
     p.partial = partial;
     p.dev_status = a.dev_status;
+    p.run_if = a.run_if;
     CUtensorMap mo;
     if (!make_out_map(&mo, partial, pr.B, pr.d, pr.d, groups)) return cudaErrorInvalidValue;
     return launch<MODE_FQ, SN, 1>(mx, my, myh, mo, p, st);
@@ -1438,6 +1239,7 @@ cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     p.row_lse = a.row_lse; p.pos_idx = a.pos_idx;
     p.out = a.out; p.ldo = a.ldo; p.partial = a.partial;
     p.dev_status = a.dev_status;
+    p.run_if = a.run_if;
     CUtensorMap mo;
     const bool ok_map = a.groups == 1 ? make_out_map(&mo, a.out, a.nx, a.d, a.ldo, 1)
                                       : make_out_map(&mo, a.partial, a.nx, a.d, a.d, a.groups);

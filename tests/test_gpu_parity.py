@@ -160,12 +160,12 @@ def _check_sampled(oracle, prob, out, n_q, n_p, full_lse=None, seed=0):
         assert grad_err(dp, dp_ref) <= tol["grad"]
 
 
-def _check_properties(prob, out, Q, P):
+def _check_properties(prob, out, Q, P, units=4):
     """Identities that hold at any size: sum_j dP_j = 0 and sum <Q, dQ> = sum <P, dP>."""
     dP64 = out.dP.double()
     scale = float(dP64.abs().max())
     col = dP64.sum(dim=0).abs().max().item()
-    assert col <= 2e-2 * scale * 4                       # bf16 weights: a few rounding units
+    assert col <= 2e-2 * scale * units                   # bf16 weights: a few rounding units
     a = (Q.double() * out.dQ.double()).sum().item()
     b = (P.double() * dP64).sum().item()
     norm = (Q.double().abs() * out.dQ.double().abs()).sum().item()
