@@ -125,6 +125,11 @@ int tc_sweep_groups(int64_t nx, int64_t ny, int d);
 cudaError_t tc_launch_fwd_store(const FwdArgs& a, void* weights, int64_t ldw, const float* row_ref,
                                 int* range_flag, cudaStream_t st);
 
+// gc_quad.cu
+bool quad_applicable(int64_t nx, int d);
+int quad_groups(int64_t nx, int64_t ny);
+cudaError_t quad_launch_sweep(const SweepArgs& a, cudaStream_t st);
+
 // gc_gemm.cu
 int gemm_groups(int64_t m_rows, int64_t k_len, int d);
 cudaError_t launch_weight_gemm(const void* weights, int64_t ldw, int64_t B, int64_t N, int transpose,

@@ -46,7 +46,23 @@ __device__ unsigned long long g_trace[5][TR_COUNT];
 #define TR_BEGIN(v) long long v##_t0 = clock64()
 #define TR_END(v) v += clock64() - v##_t0
 #define TR_ADD(mode, slot, v) atomicAdd(&g_trace[mode][slot], (unsigned long long)(v))
+// Event timeline of CTA 0 in the mode g_ev_mode selects: per role, (tag, low clock bits) pairs.
+__device__ unsigned int g_evlog[3][16384];
+__device__ int g_ev_mode = -1;
+#define EV_DECL(cnt) int cnt = 0
+#define EV(role, cnt, kind, idx)                                                       \
+    do {                                                                               \
+        if (ev_on && (cnt) < 8190) {                                                   \
+            g_evlog[role][2 * (cnt)] = ((unsigned)(kind) << 16) | ((unsigned)(idx) & 0xffffu); \
+            g_evlog[role][2 * (cnt) + 1] = (unsigned)clock64();                        \
+            ++(cnt);                                                                   \
+        }                                                                              \
+    } while (0)
+#define EV_END(role, cnt) do { if (ev_on) g_evlog[role][2 * 8191] = (unsigned)(cnt); } while (0)
 #else
+#define EV_DECL(cnt)
+#define EV(role, cnt, kind, idx)
+#define EV_END(role, cnt)
 #define TR_DECL(v)
 #define TR_BEGIN(v)
 #define TR_END(v)
@@ -137,6 +153,9 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
 #endif
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // warp-uniform
     const int lane = threadIdx.x & 31;
+#ifdef GC_TC_TRACE
+    const bool ev_on = blockIdx.x == 0 && lane == 0 && g_ev_mode == MODE;
+#endif
 
     // work item: (x tile, column part, part of the streamed range)
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
@@ -221,6 +240,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             int next = 0;
             uint32_t next_phase = 0;
             bool ok = true;
+            EV_DECL(ev_p);
             TR_DECL(tr_wait);
             TR_BEGIN(tr_total);
             // Claims the next ring stage if it belongs to this warp: waits until the MMAs that
@@ -237,6 +257,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     ok = false;
                     return -1;
                 }
+                if (warp == 0) EV(0, ev_p, 20, stage);
                 return stage;
             };
             // Ring items.  kind 0: Y for the S MMAs (ipc chunks; a paired CTA loads the 64 rows of
@@ -281,6 +302,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         load_item(2, c_begin + c, (lo + t - LAG) * SN);
                 }
             }
+            if (warp == 0) EV_END(0, ev_p);
 #ifdef GC_TC_TRACE
             if (warp == 0 && lane == 0) {
                 TR_ADD(MODE, TR_PROD_TOTAL, clock64() - tr_total_t0);
@@ -317,8 +339,10 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             TR_DECL(tr_ai);
             TR_DECL(tr_ac);
             TR_DECL(tr_sf);
+            EV_DECL(ev_m);
             TR_BEGIN(tr_total);
             bool ok = mbar_wait(smem_u32(&bars.x_full), 0, abort_flag);
+            EV(1, ev_m, 0, 0);
             tc_fence_after();
             // Waits for the next ring stage to be filled; returns its index or -1.
             auto next_stage = [&]() -> int {
@@ -332,15 +356,18 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     ok = false;
                     return -1;
                 }
+                EV(1, ev_m, 1, stage);
                 return stage;   // filled by TMA (async proxy), read by the MMA: the mbarrier orders it
             };
             for (int t = 0; t < T + LAG && ok; ++t) {
                 if (t < T) {
                     const int b = t & (NBUF - 1);
                     if (WS && t >= 1) {     // the softmax warps have read S(t-1) out of the tile
+                        EV(1, ev_m, 2, t);
                         ok = mbar_wait(smem_u32(&bars.s_free), (t - 1) & 1, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
+                        EV(1, ev_m, 3, t);
                     }
                     if (NOACC && t >= NBUF) {
                         ok = mbar_wait(smem_u32(&bars.w_full[b]), ((t - NBUF) >> BSH) & 1,
@@ -411,6 +438,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     TR_BEGIN(tr_sf);
                     if (elect_one()) commit(smem_u32(&bars.s_full[b]));
                     TR_END(tr_sf);
+                    EV(1, ev_m, 4, t);
                 }
                 if (!NOACC && t >= LAG) {
                     const int u = t - LAG, b = u & (WBUF - 1);
@@ -419,6 +447,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     TR_END(tr_ww);
                     if (!ok) break;
                     tc_fence_after();
+                    EV(1, ev_m, 5, u);
                     const uint32_t w_tmem = tmem + S_COL0 + (WS ? 0 : b * SN);
                     const uint32_t w_lo = desc_lo(w_smem + b * 32768u, 0);   // WS: K-major A operand
                     // one ring item per iteration: ipc chunks = 64 * ipc accumulator columns
@@ -454,9 +483,11 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         TR_END(tr_ai);
                     }
                     if (WS && ok && elect_one()) commit(smem_u32(&bars.w_empty[b]));
+                    EV(1, ev_m, 6, u);
                 }
             }
             if (ok && !NOACC && elect_one()) commit(smem_u32(&bars.acc_full));
+            EV_END(1, ev_m);
 #ifdef GC_TC_TRACE
             if (lane == 0) {
             TR_ADD(MODE, TR_MMA_TOTAL, clock64() - tr_total_t0);
@@ -501,6 +532,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
         };
         TR_DECL(tr_ws);
         TR_DECL(tr_epi);
+        EV_DECL(ev_s);
         TR_BEGIN(tr_total);
 
         if (MODE == MODE_FWD) {
@@ -853,6 +885,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 TR_END(tr_ws);
                 if (!ok) break;
                 tc_fence_after();
+                if (q == 0 && half == 0) EV(2, ev_s, 10, t);
                 const uint32_t sbuf = tmem + lane_addr + S_COL0 + b * SN;
                 // W of this half goes to the first columns of the half's own S region (already
                 // read by this warp): columns half * SN/2 + 16 j for block j.
@@ -866,10 +899,12 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) arrive_w(smem_u32(&bars.s_free));
+                    if (q == 0 && half == 0) EV(2, ev_s, 11, t);
                     if (t >= 2) {
                         ok = mbar_wait(smem_u32(&bars.w_empty[t & 1]), ((t - 2) >> 1) & 1, abort_flag);
                         if (!ok) break;
                     }
+                    if (q == 0 && half == 0) EV(2, ev_s, 12, t);
                 }
 #pragma unroll
                 for (int j = 0; j < CB_PER; ++j) {
@@ -933,7 +968,9 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) arrive_w(smem_u32(&bars.w_full[WS ? (t & 1) : b]));
+                if (q == 0 && half == 0) EV(2, ev_s, 13, t);
             }
+            if (q == 0 && half == 0) EV_END(2, ev_s);
             // epilogue: accumulator columns of this part -> global memory (32-column blocks are
             // dealt alternately to the two warps of a lane quarter); final values are scaled,
             // partial sums of a split sweep are not
@@ -1089,11 +1126,16 @@ cudaError_t launch(const CUtensorMap& mx, const CUtensorMap& my, const CUtensorM
 }  // namespace
 
 #ifdef GC_TC_TRACE
+extern "C" int gc_debug_evlog(unsigned int* out, int mode) {
+    if (out && cudaMemcpyFromSymbol(out, g_evlog, sizeof(g_evlog)) != cudaSuccess) return 1;
+    if (cudaMemcpyToSymbol(g_ev_mode, &mode, sizeof(int)) != cudaSuccess) return 1;
+    return 0;
+}
 extern "C" int gc_debug_trace(unsigned long long* out, int clear) {
     if (out && cudaMemcpyFromSymbol(out, g_trace, sizeof(g_trace)) != cudaSuccess) return 1;
     if (clear) {
-        static unsigned long long zero[4][TR_COUNT] = {};
-        for (int m = 0; m < 4; ++m) zero[m][TR_T0_MIN] = zero[m][TR_T1_MIN] = ~0ull;
+        static unsigned long long zero[5][TR_COUNT] = {};
+        for (int m = 0; m < 5; ++m) zero[m][TR_T0_MIN] = zero[m][TR_T1_MIN] = ~0ull;
         if (cudaMemcpyToSymbol(g_trace, zero, sizeof(zero)) != cudaSuccess) return 1;
     }
     return 0;
@@ -1118,6 +1160,7 @@ int tc_fwd_groups(int64_t B, int64_t N, int d) {
 }
 
 int tc_sweep_groups(int64_t nx, int64_t ny, int d) {
+    if (quad_applicable(nx, d)) return quad_groups(nx, ny);
     int kc = d / 64;
     int64_t units = ((nx + XROWS - 1) / XROWS) * parts_for(kc);
     int64_t steps = (ny + 127) / 128;
@@ -1220,6 +1263,7 @@ cudaError_t tc_launch_fused_dq(const FwdArgs& a, float* partial, int groups, cud
 }
 
 cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
+    if (quad_applicable(a.nx, a.d)) return quad_launch_sweep(a, st);
     const int kc = a.d / 64;
     constexpr int SN = 128;
     CUtensorMap mx, my, myh;
