@@ -43,10 +43,13 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored) {
         pl.g_dp = simt_sweep_groups(N, B, d);
     }
     pl.fused = (pl.tc && tc_fused_applicable(d)) ? 1 : 0;
+    pl.anchored = (pl.fused && quad_applicable(B, d)) ? 1 : 0;
     size_t dpad = (size_t)((d + 3) & ~3);
-    // (max, sum) slots: the forward sweep writes g_fwd of them per row, the fused sweep 2 g_dq
+    // (max, sum) slots: the forward sweep writes g_fwd of them per row, the fused sweep 2 g_dq,
+    // the anchored fused sweep 4 g_dq
     size_t slots = (size_t)pl.g_fwd;
     if (pl.fused && (size_t)(2 * pl.g_dq) > slots) slots = (size_t)(2 * pl.g_dq);
+    if (pl.anchored && (size_t)(4 * pl.g_dq) > slots) slots = (size_t)(4 * pl.g_dq);
     size_t off = 0;
     pl.off_m = off;    off += align256(sizeof(float) * slots * (size_t)B);
     pl.off_l = off;    off += align256(sizeof(float) * slots * (size_t)B);
@@ -59,8 +62,13 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored) {
     pl.launches_fwd = 2;  // sweep + combine
     pl.launches_bwd = 2 + (pl.g_dq > 1 ? 1 : 0) + (pl.g_dp > 1 ? 1 : 0);
     pl.launches_build = pl.fused ? 4 + (pl.g_dp > 1 ? 1 : 0) : pl.launches_fwd + pl.launches_bwd;
+    if (pl.anchored) pl.launches_build = 1 + 2 * pl.launches_build;   // anchor, sequence, fallback
     // Stored weights: B x N bf16 (pitch rounded up to 64 elements), kept when they fit the limit
     // below; the gradient partials share the regions of the sweeps they replace.
+    if (pl.anchored) {
+        pl.off_ref = off;   off += align256(sizeof(float) * (size_t)B);
+        pl.off_flag = off;  off += 256;
+    }
     pl.ldw = (N + 63) / 64 * 64;
     const size_t w_bytes = (size_t)B * (size_t)pl.ldw * 2;
     pl.mat = (stored && pl.tc && w_bytes <= kMaxStoredWeightBytes) ? 1 : 0;
@@ -75,8 +83,10 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored) {
             off = pl.off_accp + old_accp;
         }
         if (off - pl.off_accp < accp) off = pl.off_accp + accp;
-        pl.off_ref = off;   off += align256(sizeof(float) * (size_t)B);
-        pl.off_flag = off;  off += 256;
+        if (!pl.anchored) {
+            pl.off_ref = off;   off += align256(sizeof(float) * (size_t)B);
+            pl.off_flag = off;  off += 256;
+        }
         pl.off_qs = off;    off += align256((size_t)B * (size_t)d * 2);
         pl.off_w = off;     off += align256(w_bytes);
         // anchor, sweep, combine, row scaling, dQ GEMM, dQ finalize, dP GEMM (+ reduce),
@@ -247,10 +257,50 @@ int run_fused_fwd_dq(const Problem& p, const Plan& pl, char* ws, float* loss, fl
 }
 
 // The recomputing sequence of gc_build_cache; with run_if every kernel of it is gated.
+// Forward fused into the four-CTA dQ sweep with the positive logit as each row's scale, then the
+// combine and the dQ finalize.  A weight beyond 2^100 raises the range flag at pl.off_flag.
+int run_anchored_fwd_dq(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_lse,
+                        float* pos_logit, float* dQ, int64_t lddq, int* dev_status,
+                        cudaStream_t st) {
+    float* ref2 = reinterpret_cast<float*>(ws + pl.off_ref);
+    int* flag = reinterpret_cast<int*>(ws + pl.off_flag);
+    cudaError_t e = launch_pos_anchor(p.Q, p.ldq, p.P, p.ldp, p.pos_idx, p.B, p.N, p.d, p.mask_mode,
+                                      1.4426950408889634f / p.tau, ref2, flag, st);
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    FwdArgs fa{};
+    fa.p = p;
+    fa.part_m = reinterpret_cast<float*>(ws + pl.off_m);
+    fa.part_l = reinterpret_cast<float*>(ws + pl.off_l);
+    fa.pos_logit = reinterpret_cast<float*>(ws + pl.off_pos);
+    fa.red = reinterpret_cast<float*>(ws + pl.off_red);
+    fa.groups = 4 * pl.g_dq;
+    fa.dev_status = dev_status;
+    float* partial = reinterpret_cast<float*>(ws + pl.off_accq);
+    {
+        KernelTimer t(1, st);
+        e = quad_launch_fused_dq(fa, partial, pl.g_dq, ref2, flag, st);
+    }
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, nullptr, st);
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    e = launch_fused_dq_finalize(partial, pl.g_dq, nullptr, ref2, row_lse, fa.pos_logit, p.pos_idx,
+                                 p.P, p.ldp, p.B, p.N, p.d, p.mask_mode,
+                                 1.f / ((float)p.B * p.tau), dQ, lddq, nullptr, st);
+    return e == cudaSuccess ? GC_OK : GC_ERR_CUDA;
+}
+
 int run_build_sweeps(const Problem& p, const Plan& pl, char* w, float* loss, float* row_lse,
                      float* pos_logit, float* dQ, int64_t lddq, float* dP, int64_t lddp,
                      int* dev_status, cudaStream_t st, const int* run_if = nullptr) {
     int rc;
+    if (pl.anchored && !run_if) {
+        // anchored sequence first; the online-maximum sequence below then runs gated by its flag
+        if ((rc = run_anchored_fwd_dq(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dev_status, st)))
+            return rc;
+        if ((rc = run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, dev_status, st))) return rc;
+        run_if = reinterpret_cast<const int*>(w + pl.off_flag);
+    }
     if (pl.fused) {
         if ((rc = run_fused_fwd_dq(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dev_status, st,
                                    run_if)))

@@ -70,6 +70,8 @@ struct Plan {
     size_t total;           // workspace bytes (multiple of 256)
     int launches_fwd, launches_bwd;
     int fused;              // 1: gc_build_cache runs the forward inside the dQ sweep
+    int anchored;           // 1: ... with the positive logit as the fixed scale of each row (four-
+                            // CTA sweep); the online-maximum sweep then is its gated fallback
     int launches_build;
     // Stored-weights plan of gc_build_cache (tcgen05 only): one forward sweep keeps the bf16
     // weights, two GEMMs form the gradients; the sweeps above stay as its fallback.
@@ -129,6 +131,8 @@ cudaError_t tc_launch_fwd_store(const FwdArgs& a, void* weights, int64_t ldw, co
 bool quad_applicable(int64_t nx, int d);
 int quad_groups(int64_t nx, int64_t ny);
 cudaError_t quad_launch_sweep(const SweepArgs& a, cudaStream_t st);
+cudaError_t quad_launch_fused_dq(const FwdArgs& a, float* partial, int groups, const float* row_ref,
+                                 int* range_flag, cudaStream_t st);
 
 // gc_gemm.cu
 int gemm_groups(int64_t m_rows, int64_t k_len, int d);

@@ -501,10 +501,9 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
         if (MODE == QMODE_FA && ok && x < p.nx) {
             // one (scale, sum) slot per row, part of the streamed range, duty pair and column half
             const int64_t slot = (int64_t)((2 * g + pr) * 2 + half) * p.nq + x;
-            if (c_begin == 0 || true) {
-                p.part_m[slot] = lse2_x * 0.69314718055994531f;
-                p.part_l[slot] = l;
-            }
+            p.part_m[slot] = lse2_x * 0.69314718055994531f;
+            p.part_l[slot] = l;
+            // weights beyond 2^100 (or not finite) cannot be accumulated safely
             if (!(wmax <= 1.2676506e30f)) *p.range_flag = 1;
         }
         // epilogue: accumulator columns of this CTA's half -> global memory
@@ -609,6 +608,37 @@ cudaError_t quad_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     const int64_t clusters = (((a.nx + XROWS - 1) / XROWS + 1) / 2) * a.groups;
     if (a.mode == SWEEP_DQ) return launch_quad<QMODE_DQ>(mx, my, myh, mo, p, clusters, st);
     return launch_quad<QMODE_DP>(mx, my, myh, mo, p, clusters, st);
+}
+
+// Forward fused into the dQ sweep with the positive logit as each row's fixed scale (row_ref,
+// log2 domain): writes (scale, sum) slots [4 groups][B] (scale = row_ref in natural-log units),
+// pos_logit and the unscaled accumulators partial[groups][B][d] of sum_j 2^(s2_ij - ref_i) P_j
+// over all allowed columns but the positive one; raises *range_flag when a weight exceeds 2^100.
+cudaError_t quad_launch_fused_dq(const FwdArgs& a, float* partial, int groups, const float* row_ref,
+                                 int* range_flag, cudaStream_t st) {
+    const Problem& pr = a.p;
+    const int kc = pr.d / 64;
+    CUtensorMap mx, my, myh, mo;
+    if (!make_map(&mx, pr.Q, pr.B, pr.d, pr.ldq, XROWS) ||
+        !make_map(&my, pr.P, pr.N, pr.d, pr.ldp, 128) ||
+        !make_map(&myh, pr.P, pr.N, pr.d, pr.ldp, 64) ||
+        !make_out_map(&mo, partial, pr.B, pr.d, pr.d, groups))
+        return cudaErrorInvalidValue;
+    QuadParams p{};
+    p.nx = pr.B; p.ny = pr.N; p.nq = pr.B;
+    p.kc = kc; p.dpc = chunks_per_part(kc); p.groups = groups;
+    p.mask_mode = pr.mask_mode;
+    p.inv_tau = 1.f / pr.tau;
+    p.c1 = 1.4426950408889634f / pr.tau;
+    p.pos_idx = pr.pos_idx;
+    p.row_ref = row_ref;
+    p.part_m = a.part_m; p.part_l = a.part_l; p.pos_logit = a.pos_logit;
+    p.range_flag = range_flag;
+    p.dev_status = a.dev_status;
+    p.run_if = a.run_if;
+    p.zero_me = reinterpret_cast<int*>(a.red);
+    const int64_t clusters = (((pr.B + XROWS - 1) / XROWS + 1) / 2) * groups;
+    return launch_quad<QMODE_FA>(mx, my, myh, mo, p, clusters, st);
 }
 
 }  // namespace gc

@@ -276,6 +276,18 @@ def test_mask_does_not_leak(binding, oracle, dtype):
     check_against_oracle(prob, out, _oracle_full(oracle, prob))
 
 
+@pytest.mark.parametrize("B,N,d,tau", [(200, 300, 128, 0.01), (300, 520, 768, 0.004)])
+def test_logits_far_above_the_positive(binding, oracle, B, N, d, tau):
+    """Rows whose largest logit lies hundreds of powers of two above their positive logit: the
+    wide-row build scales its weights by the positive logit and must hand such inputs to the
+    kernels that track the running row maximum."""
+    prob = inputs.random_problem(B, N, d, "bf16", seed=21, tau=tau, scale=1.0)
+    ref = _oracle_full(oracle, prob)
+    assert np.max(ref["row_lse"] - ref["pos_logit"]) > 500.0       # natural-log units
+    out = run_build(prob)
+    check_against_oracle(prob, out, ref)
+
+
 def test_bad_positives_are_flagged_not_fatal(binding, oracle):
     prob = inputs.random_problem(40, 50, 64, "f32", seed=1, tau=1.0, scale=0.3,
                                  mask_mode=inputs.MASK_SELF)
