@@ -53,15 +53,41 @@ struct QuadParams {
 
 constexpr int Q_XRES = 2;     // X chunks that stay resident
 
+// Optional diagnostics (-DGC_TC_TRACE): event timeline of the two pair leaders of cluster 0 in
+// the mode g_qev_mode selects; per role (tag, low clock bits) pairs.
+#ifdef GC_TC_TRACE
+__device__ unsigned int g_qevlog[4][8192];
+__device__ int g_qev_mode = -1;
+#define QEV_DECL(cnt) int cnt = 0
+#define QEV(role, cnt, kind, idx)                                                          \
+    do {                                                                                   \
+        if (qev_on && (cnt) < 4094) {                                                      \
+            g_qevlog[role][2 * (cnt)] = ((unsigned)(kind) << 16) | ((unsigned)(idx) & 0xffffu); \
+            g_qevlog[role][2 * (cnt) + 1] = (unsigned)clock64();                           \
+            ++(cnt);                                                                       \
+        }                                                                                  \
+    } while (0)
+#define QEV_END(role, cnt) do { if (qev_on) g_qevlog[role][2 * 4095] = (unsigned)(cnt); } while (0)
+#else
+#define QEV_DECL(cnt)
+#define QEV(role, cnt, kind, idx)
+#define QEV_END(role, cnt)
+#endif
+
 struct QBars {
     uint64_t x_full;
     uint64_t y_full[MAX_STAGES];
     uint64_t y_empty[MAX_STAGES];
+    // A remote arrive with cluster-scope release costs the arriving warp well over a thousand
+    // cycles, so the softmax warps only ever arrive on barriers of their own CTA; the MMA warp of
+    // the pair's second CTA, otherwise idle, forwards each completed phase to the leader.
     uint64_t s_full;           // S tile of the duty pair complete (both CTAs of the pair)
-    uint64_t s_free;           // leader: all 16 softmax warps of the pair have read the S tile
-    uint64_t w_self;           // leader: the pair's own W is in both CTAs (16 arrivals)
-    uint64_t w_recv;           // every CTA: the other pair's W has landed (8 arrivals + 32 KB)
-    uint64_t w_peer;           // leader: the other CTA of the pair saw its w_recv complete
+    uint64_t s_read;           // this CTA's 8 softmax warps have read the S tile
+    uint64_t s_read_peer;      // leader: forwarded s_read of the second CTA
+    uint64_t w_done;           // this CTA's 8 softmax warps have written their part of W
+    uint64_t w_done_peer;      // leader: forwarded w_done of the second CTA
+    uint64_t w_recv;           // the other pair's W has landed here (1 arrival + 32 KB)
+    uint64_t w_peer;           // leader: forwarded w_recv of the second CTA
     uint64_t w_empty[2][2];    // [W buffer][consuming pair], committed to all four CTAs
     uint64_t acc_full;
 };
@@ -106,6 +132,9 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
 
     const uint32_t rank = cluster_ctarank();        // 0..3
     const int pr = (int)(rank >> 1);                // pair = column half = duty parity
+#ifdef GC_TC_TRACE
+    const bool qev_on = (blockIdx.x == 0 || blockIdx.x == 2) && lane == 0 && g_qev_mode == MODE;
+#endif
     const int side = (int)(rank & 1);               // which of the two x tiles
     const bool leader = (side == 0);
     const uint32_t leader_rank = rank & ~1u;
@@ -140,9 +169,11 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
             mbar_init(smem_u32(&bars.y_empty[s]), 1);
         }
         mbar_init(smem_u32(&bars.s_full), 1);
-        mbar_init(smem_u32(&bars.s_free), 2 * NSOFT);
-        mbar_init(smem_u32(&bars.w_self), 2 * NSOFT);
-        mbar_init(smem_u32(&bars.w_recv), NSOFT);
+        mbar_init(smem_u32(&bars.s_read), NSOFT);
+        mbar_init(smem_u32(&bars.s_read_peer), 1);
+        mbar_init(smem_u32(&bars.w_done), NSOFT);
+        mbar_init(smem_u32(&bars.w_done_peer), 1);
+        mbar_init(smem_u32(&bars.w_recv), 1);
         mbar_init(smem_u32(&bars.w_peer), 1);
         for (int b = 0; b < 2; ++b)
             for (int q = 0; q < 2; ++q) mbar_init(smem_u32(&bars.w_empty[b][q]), 1);
@@ -239,8 +270,10 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
             const uint32_t ring_lo = desc_lo(y_smem, CHUNK_BYTES);
             int next = 0;
             uint32_t next_phase = 0;
+            QEV_DECL(ev_m);
             bool ok = mbar_wait(smem_u32(&bars.x_full), 0, abort_flag);
             tc_fence_after();
+            QEV(pr, ev_m, 0, 0);
             auto next_stage = [&]() -> int {
                 const int stage = next;
                 const uint32_t phase = next_phase;
@@ -254,11 +287,14 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
             for_each_op([&](int kind, int idx) {
                 if (!ok) return;
                 if (kind == 0) {
+                    QEV(pr, ev_m, 1, idx);
                     if (idx >= 1) {     // the softmax warps have read the previous duty tile
-                        ok = mbar_wait(smem_u32(&bars.s_free), (idx - 1) & 1, abort_flag);
+                        ok = mbar_wait(smem_u32(&bars.s_read), (idx - 1) & 1, abort_flag) &&
+                             mbar_wait(smem_u32(&bars.s_read_peer), (idx - 1) & 1, abort_flag);
                         if (!ok) return;
                         tc_fence_after();
                     }
+                    QEV(pr, ev_m, 2, idx);
                     const uint32_t d_tmem = tmem + S_COL0;
                     for (int c = 0; c < p.kc && ok; c += 2) {
                         const int ys = next_stage();
@@ -285,16 +321,20 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                         }
                     }
                     if (ok && elect_one()) tc_commit_mask(smem_u32(&bars.s_full), pair_mask);
+                    QEV(pr, ev_m, 3, idx);
                 } else {
                     const int u = idx, b = u & 1, round = u >> 1;
+                    QEV(pr, ev_m, 4, idx);
                     if (b == pr) {
-                        ok = mbar_wait(smem_u32(&bars.w_self), round & 1, abort_flag);
+                        ok = mbar_wait(smem_u32(&bars.w_done), round & 1, abort_flag) &&
+                             mbar_wait(smem_u32(&bars.w_done_peer), round & 1, abort_flag);
                     } else {
                         ok = mbar_wait(smem_u32(&bars.w_recv), round & 1, abort_flag) &&
                              mbar_wait(smem_u32(&bars.w_peer), round & 1, abort_flag);
                     }
                     if (!ok) return;
                     tc_fence_after();
+                    QEV(pr, ev_m, 5, idx);
                     const uint32_t w_lo = desc_lo(w_smem + b * 32768u, 0);   // K-major A operand
                     for (int a = 0; a < na && ok; ++a) {
                         const int ys = next_stage();
@@ -314,17 +354,48 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                                 tc_commit_mask(smem_u32(&bars.w_empty[b][pr]), (uint16_t)0xF);
                         }
                     }
+                    QEV(pr, ev_m, 6, idx);
                 }
             });
+            QEV_END(pr, ev_m);
             if (ok && elect_one()) tc_commit_mask(smem_u32(&bars.acc_full), pair_mask);
         } else {
-            // the other CTA of the pair tells the leader when its copy of a received W has landed
-            const uint32_t peer_bar = in_leader(smem_u32(&bars.w_peer));
-            for (int round = 0; round < rounds; ++round) {
-                if (2 * round + (1 - pr) >= T) break;
-                if (!mbar_wait(smem_u32(&bars.w_recv), round & 1, abort_flag)) break;
-                if (lane == 0) mbar_arrive_cluster(peer_bar);
+            // Forwarder: the second CTA's completed phases (S tile read, W written, received W
+            // landed) become single arrivals on the leader's barriers.  The three sequences are
+            // polled together so that none waits behind another.
+            const uint32_t fs = in_leader(smem_u32(&bars.s_read_peer));
+            const uint32_t fw = in_leader(smem_u32(&bars.w_done_peer));
+            const uint32_t fr = in_leader(smem_u32(&bars.w_peer));
+            const int nrecv = (T - (1 - pr) + 1) / 2;       // tiles 1 - pr, 3 - pr, ... < T
+            int js = 0, jw = 0, jr = 0;
+            uint64_t t_last = global_ns();
+            while (js < nd || jw < nd || jr < nrecv) {
+                bool progress = false;
+                if (js < nd && mbar_test(smem_u32(&bars.s_read), js & 1)) {
+                    if (lane == 0) mbar_arrive_cluster(fs);
+                    ++js;
+                    progress = true;
+                }
+                if (jw < nd && mbar_test(smem_u32(&bars.w_done), jw & 1)) {
+                    if (lane == 0) mbar_arrive_cluster(fw);
+                    ++jw;
+                    progress = true;
+                }
+                if (jr < nrecv && mbar_test(smem_u32(&bars.w_recv), jr & 1)) {
+                    if (lane == 0) mbar_arrive_cluster(fr);
+                    ++jr;
+                    progress = true;
+                }
                 __syncwarp();
+                if (progress) {
+                    t_last = global_ns();
+                } else {
+                    if (*abort_flag) break;
+                    if (global_ns() - t_last > WAIT_LIMIT_NS) {
+                        *abort_flag = 1;
+                        break;
+                    }
+                }
             }
         }
     } else {
@@ -338,13 +409,12 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         const bool self_mask = (p.mask_mode == GC_MASK_SELF);
         bool ok = true;
-        const uint32_t s_free_bar = in_leader(smem_u32(&bars.s_free));
-        const uint32_t w_self_bar = in_leader(smem_u32(&bars.w_self));
-        // this warp's 32 rows x 64 columns of W buffer pr: 4 KB, copied on their own to the same
-        // place in the CTA that holds this x tile in the other pair
-        const uint32_t my_w = w_smem + pr * 32768u + half * CHUNK_BYTES + q * 4096;
+        // W buffer pr (32 KB) goes as one copy to the same place in the CTA that holds this x tile
+        // in the other pair; the last softmax warp sends it once all eight have written
+        const uint32_t my_w = w_smem + pr * 32768u;
         const uint32_t remote_w = mapa_u32(my_w, rank ^ 2u);
         const uint32_t remote_bar = mapa_u32(smem_u32(&bars.w_recv), rank ^ 2u);
+        const bool sender = (q == 3 && half == 1);
         auto put_w_block = [&](int j, const uint32_t (&pk)[16]) {
             const uint32_t line = w_smem + pr * 32768u + half * CHUNK_BYTES + row * 128;
 #pragma unroll
@@ -357,6 +427,10 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
         };
         float lse2_x = 0.f, l = 0.f, wmax = 0.f;
         int32_t pos_x = -1;
+#ifdef GC_TC_TRACE
+        const bool sev = (q == 0 && half == 0);
+        long long ph[7] = {0, 0, 0, 0, 0, 0, 0};
+#endif
         if (MODE != QMODE_DP && x < p.nx) {
             lse2_x = (MODE == QMODE_FA) ? p.row_ref[x] : p.row_lse[x] * 1.4426950408889634f;
             pos_x = p.pos_idx[x];
@@ -374,23 +448,33 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                     pos_y[jj] = (y < p.ny) ? p.pos_idx[y] : -1;
                 }
             }
+#ifdef GC_TC_TRACE
+            const long long c0_ = clock64();
+#endif
             ok = mbar_wait(smem_u32(&bars.s_full), j & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
+#ifdef GC_TC_TRACE
+            const long long c1_ = clock64(); ph[0] += c1_ - c0_;
+#endif
             const uint32_t sbuf = tmem + lane_addr + S_COL0;
             uint32_t vv[CB_PER][32];
 #pragma unroll
             for (int jj = 0; jj < CB_PER; ++jj) tmem_ld32(sbuf + (cb0 + jj) * 32, vv[jj]);
             tmem_ld_wait();
+#ifdef GC_TC_TRACE
+            const long long c2_ = clock64(); ph[1] += c2_ - c1_;
+#endif
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_cluster(s_free_bar);     // the S tile may be overwritten
-            // W buffer pr of both pairs must have been consumed (accumulation of tile t - 2)
-            if (j >= 1) {
-                ok = mbar_wait(smem_u32(&bars.w_empty[pr][0]), (j - 1) & 1, abort_flag) &&
-                     mbar_wait(smem_u32(&bars.w_empty[pr][1]), (j - 1) & 1, abort_flag);
-                if (!ok) break;
-            }
+            if (lane == 0) mbar_arrive(smem_u32(&bars.s_read));  // the S tile may be overwritten
+#ifdef GC_TC_TRACE
+            const long long c3_ = clock64(); ph[2] += c3_ - c2_;
+#endif
+#ifdef GC_TC_TRACE
+            const long long c4_ = c3_;
+#endif
+            uint32_t packed[CB_PER][16];
 #pragma unroll
             for (int jj = 0; jj < CB_PER; ++jj) {
                 const int cb = cb0 + jj;
@@ -481,23 +565,49 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                     for (int c = 0; c < 32; ++c)
                         if (c == rel) w[c] = 0.f;
                 }
-                uint32_t packed[16];
 #pragma unroll
                 for (int r = 0; r < 16; ++r) {
                     __nv_bfloat162 h = __floats2bfloat162_rn(w[2 * r], w[2 * r + 1]);
-                    packed[r] = *reinterpret_cast<uint32_t*>(&h);
+                    packed[jj][r] = *reinterpret_cast<uint32_t*>(&h);
                 }
-                put_w_block(jj, packed);
             }
+            // W buffer pr of both pairs must have been consumed (accumulation of tile t - 2)
+            if (j >= 1) {
+                ok = mbar_wait(smem_u32(&bars.w_empty[pr][0]), (j - 1) & 1, abort_flag) &&
+                     mbar_wait(smem_u32(&bars.w_empty[pr][1]), (j - 1) & 1, abort_flag);
+                if (!ok) break;
+            }
+#pragma unroll
+            for (int jj = 0; jj < CB_PER; ++jj) put_w_block(jj, packed[jj]);
+#ifdef GC_TC_TRACE
+            const long long c5_ = clock64(); ph[4] += c5_ - c4_;
+#endif
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive_expect_cluster(remote_bar, 4096u);
-                dsmem_copy(remote_w, my_w, 4096u, remote_bar);
-                mbar_arrive_cluster(w_self_bar);
+#ifdef GC_TC_TRACE
+            const long long c6_ = clock64(); ph[5] += c6_ - c5_;
+#endif
+            if (lane == 0) mbar_arrive(smem_u32(&bars.w_done));
+            if (sender) {
+                ok = mbar_wait(smem_u32(&bars.w_done), j & 1, abort_flag);
+                if (!ok) break;
+                if (lane == 0) {
+                    mbar_arrive_expect_cluster(remote_bar, 32768u);
+                    dsmem_copy(remote_w, my_w, 32768u, remote_bar);
+                }
+                __syncwarp();
             }
+#ifdef GC_TC_TRACE
+            ph[6] += clock64() - c6_;
+#endif
         }
+#ifdef GC_TC_TRACE
+        if (sev && qev_on) {
+            for (int k = 0; k < 7; ++k) g_qevlog[2 + pr][2 * k + 1] = (unsigned)(ph[k] / max(nd, 1));
+            g_qevlog[2 + pr][2 * 4095] = 7;
+        }
+#endif
         if (MODE == QMODE_FA && ok && x < p.nx) {
             // one (scale, sum) slot per row, part of the streamed range, duty pair and column half
             const int64_t slot = (int64_t)((2 * g + pr) * 2 + half) * p.nq + x;
@@ -567,6 +677,14 @@ cudaError_t launch_quad(const CUtensorMap& mx, const CUtensorMap& my, const CUte
 }
 
 }  // namespace
+
+#ifdef GC_TC_TRACE
+extern "C" int gc_debug_qevlog(unsigned int* out, int mode) {
+    if (out && cudaMemcpyFromSymbol(out, g_qevlog, sizeof(g_qevlog)) != cudaSuccess) return 1;
+    if (cudaMemcpyToSymbol(g_qev_mode, &mode, sizeof(int)) != cudaSuccess) return 1;
+    return 0;
+}
+#endif
 
 // Two column halves of an even number of chunks each, at most 384 columns per half, more than
 // one x tile.
