@@ -170,11 +170,13 @@ Problem make_problem(const void* Q, int64_t ldq, const void* P, int64_t ldp,
     return p;
 }
 
+constexpr Gate kOpen = {nullptr, 0};
+
 int run_fwd(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_lse,
-            float* pos_logit, int* dev_status, cudaStream_t st, const int* run_if = nullptr) {
+            float* pos_logit, int* dev_status, cudaStream_t st, Gate gate = kOpen) {
     FwdArgs fa{};
     fa.p = p;
-    fa.run_if = run_if;
+    fa.gate = gate;
     fa.part_m = reinterpret_cast<float*>(ws + pl.off_m);
     fa.part_l = reinterpret_cast<float*>(ws + pl.off_l);
     fa.pos_logit = reinterpret_cast<float*>(ws + pl.off_pos);
@@ -183,20 +185,21 @@ int run_fwd(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_
     fa.dev_status = dev_status;
     cudaError_t e;
     {
-        KernelTimer t(run_if ? -1 : 0, st);
+        KernelTimer t(gate.flag ? -1 : 0, st);
         e = pl.tc ? tc_launch_fwd(fa, st) : simt_launch_fwd(fa, st);
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, run_if, st);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, gate, st);
     return e == cudaSuccess ? GC_OK : GC_ERR_CUDA;
 }
 
+// `timed`: bracket the sweep with the profiling events (only the sweeps that normally run are).
 int run_sweep(const Problem& p, const Plan& pl, char* ws, int mode, const float* row_lse,
-              float* out, int64_t ldo, int* dev_status, cudaStream_t st,
-              const int* run_if = nullptr) {
+              float* out, int64_t ldo, int* dev_status, cudaStream_t st, Gate gate = kOpen,
+              bool timed = true) {
     SweepArgs sa{};
-    sa.run_if = run_if;
+    sa.gate = gate;
     const bool dq = (mode == SWEEP_DQ);
     sa.X = dq ? p.Q : p.P;   sa.ldx = dq ? p.ldq : p.ldp;   sa.nx = dq ? p.B : p.N;
     sa.Y = dq ? p.P : p.Q;   sa.ldy = dq ? p.ldp : p.ldq;   sa.ny = dq ? p.N : p.B;
@@ -215,12 +218,12 @@ int run_sweep(const Problem& p, const Plan& pl, char* ws, int mode, const float*
     sa.dev_status = dev_status;
     cudaError_t e;
     {
-        KernelTimer t(run_if ? -1 : (dq ? 1 : 2), st);
+        KernelTimer t(timed ? (dq ? 1 : 2) : -1, st);
         e = pl.tc ? tc_launch_sweep(sa, st) : simt_launch_sweep(sa, st);
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     if (sa.groups > 1) {
-        e = launch_partial_reduce(sa.partial, sa.groups, sa.nx, sa.d, sa.out_scale, out, ldo, run_if,
+        e = launch_partial_reduce(sa.partial, sa.groups, sa.nx, sa.d, sa.out_scale, out, ldo, gate,
                                   st);
         if (e != cudaSuccess) return GC_ERR_CUDA;
     }
@@ -230,10 +233,10 @@ int run_sweep(const Problem& p, const Plan& pl, char* ws, int mode, const float*
 // gc_build_cache for wide bf16 rows: fused forward + dQ sweep, combine, dQ finalize.
 int run_fused_fwd_dq(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_lse,
                      float* pos_logit, float* dQ, int64_t lddq, int* dev_status,
-                     cudaStream_t st, const int* run_if = nullptr) {
+                     cudaStream_t st, Gate gate = kOpen) {
     FwdArgs fa{};
     fa.p = p;
-    fa.run_if = run_if;
+    fa.gate = gate;
     fa.part_m = reinterpret_cast<float*>(ws + pl.off_m);
     fa.part_l = reinterpret_cast<float*>(ws + pl.off_l);
     fa.pos_logit = reinterpret_cast<float*>(ws + pl.off_pos);
@@ -243,27 +246,85 @@ int run_fused_fwd_dq(const Problem& p, const Plan& pl, char* ws, float* loss, fl
     float* partial = reinterpret_cast<float*>(ws + pl.off_accq);
     cudaError_t e;
     {
-        KernelTimer t(run_if ? -1 : 1, st);
+        KernelTimer t(gate.flag ? -1 : 1, st);
         e = tc_launch_fused_dq(fa, partial, pl.g_dq, st);
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, run_if, st);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, gate, st);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_fused_dq_finalize(partial, pl.g_dq, fa.part_m, nullptr, row_lse, fa.pos_logit,
                                  p.pos_idx, p.P, p.ldp, p.B, p.N, p.d, p.mask_mode,
-                                 1.f / ((float)p.B * p.tau), dQ, lddq, run_if, st);
+                                 1.f / ((float)p.B * p.tau), dQ, lddq, gate, st);
     return e == cudaSuccess ? GC_OK : GC_ERR_CUDA;
 }
 
-// The recomputing sequence of gc_build_cache; with run_if every kernel of it is gated.
-// Forward fused into the four-CTA dQ sweep with the positive logit as each row's scale, then the
-// combine and the dQ finalize.  A weight beyond 2^100 raises the range flag at pl.off_flag.
-int run_anchored_fwd_dq(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_lse,
-                        float* pos_logit, float* dQ, int64_t lddq, int* dev_status,
-                        cudaStream_t st) {
+// The sequence that tracks the running row maximum: forward (fused into the dQ sweep for wide
+// rows), dQ, dP.  With a gate every kernel of it is gated.
+int run_online_sweeps(const Problem& p, const Plan& pl, char* w, float* loss, float* row_lse,
+                      float* pos_logit, float* dQ, int64_t lddq, float* dP, int64_t lddp,
+                      int* dev_status, cudaStream_t st, Gate gate = kOpen) {
+    int rc;
+    if (pl.fused) {
+        if ((rc = run_fused_fwd_dq(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dev_status, st,
+                                   gate)))
+            return rc;
+    } else {
+        if ((rc = run_fwd(p, pl, w, loss, row_lse, pos_logit, dev_status, st, gate))) return rc;
+        if ((rc = run_sweep(p, pl, w, SWEEP_DQ, row_lse, dQ, lddq, dev_status, st, gate,
+                            gate.flag == nullptr)))
+            return rc;
+    }
+    return run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, dev_status, st, gate,
+                     gate.flag == nullptr);
+}
+
+// A side stream and three events per device, created on first use: work that is off a call's
+// critical path (the dQ finalize, the gated fallback) runs there between a fork from and a join
+// back into the caller's stream, so the call stays asynchronous on that stream alone.
+struct SideStream {
+    bool tried = false, ok = false;
+    cudaStream_t st = nullptr;
+    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+};
+SideStream* side_stream() {
+    static SideStream per_dev[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    SideStream& s = per_dev[dev];
+    if (!s.tried) {
+        s.tried = true;
+        bool good = cudaStreamCreateWithFlags(&s.st, cudaStreamNonBlocking) == cudaSuccess;
+        for (int i = 0; i < 3 && good; ++i)
+            good = cudaEventCreateWithFlags(&s.ev[i], cudaEventDisableTiming) == cudaSuccess;
+        if (!good) cudaGetLastError();
+        s.ok = good;
+    }
+    return s.ok ? &s : nullptr;
+}
+
+// gc_build_cache for rows of two column halves (four-CTA sweeps).  The forward is fused into the
+// dQ sweep with the positive logit as each row's fixed scale (anchor kernel), so no running
+// maximum has to be agreed across the cluster.  A weight beyond 2^100 raises the range flag; the
+// kernels after the fused sweep run only while it is down, and the online-maximum sequence, which
+// is always launched, runs only when it is up and then produces every output.
+//
+//   caller's stream:  anchor, fused sweep, combine, dP sweep (+ reduce)
+//   side stream:      after the fused sweep: the gated online-maximum sequence;
+//                     after the combine: the dQ finalize
+// Both are joined back before the call returns.  Without a side stream everything is queued on
+// the caller's stream in dependency order.
+int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_lse,
+                       float* pos_logit, float* dQ, int64_t lddq, float* dP, int64_t lddp,
+                       int* dev_status, cudaStream_t st) {
     float* ref2 = reinterpret_cast<float*>(ws + pl.off_ref);
     int* flag = reinterpret_cast<int*>(ws + pl.off_flag);
+    const Gate in_range = {flag, 0}, out_of_range = {flag, 1};
+    SideStream* side = side_stream();
+    cudaStream_t aux = side ? side->st : st;
     cudaError_t e = launch_pos_anchor(p.Q, p.ldq, p.P, p.ldp, p.pos_idx, p.B, p.N, p.d, p.mask_mode,
                                       1.4426950408889634f / p.tau, ref2, flag, st);
     if (e != cudaSuccess) return GC_ERR_CUDA;
@@ -281,36 +342,44 @@ int run_anchored_fwd_dq(const Problem& p, const Plan& pl, char* ws, float* loss,
         e = quad_launch_fused_dq(fa, partial, pl.g_dq, ref2, flag, st);
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
+    if (side && (cudaEventRecord(side->ev[0], st) != cudaSuccess ||
+                 cudaStreamWaitEvent(aux, side->ev[0], 0) != cudaSuccess))
+        return GC_ERR_CUDA;
+    int rc;
+    if (side) {
+        // fallback first on the side stream: it only needs the flag
+        if ((rc = run_online_sweeps(p, pl, ws, loss, row_lse, pos_logit, dQ, lddq, dP, lddp,
+                                    dev_status, aux, out_of_range)))
+            return rc;
+    }
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, nullptr, st);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, in_range, st);
     if (e != cudaSuccess) return GC_ERR_CUDA;
+    if (side && (cudaEventRecord(side->ev[1], st) != cudaSuccess ||
+                 cudaStreamWaitEvent(aux, side->ev[1], 0) != cudaSuccess))
+        return GC_ERR_CUDA;
     e = launch_fused_dq_finalize(partial, pl.g_dq, nullptr, ref2, row_lse, fa.pos_logit, p.pos_idx,
                                  p.P, p.ldp, p.B, p.N, p.d, p.mask_mode,
-                                 1.f / ((float)p.B * p.tau), dQ, lddq, nullptr, st);
-    return e == cudaSuccess ? GC_OK : GC_ERR_CUDA;
+                                 1.f / ((float)p.B * p.tau), dQ, lddq, in_range, aux);
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    if ((rc = run_sweep(p, pl, ws, SWEEP_DP, row_lse, dP, lddp, dev_status, st, in_range))) return rc;
+    if (side) {
+        if (cudaEventRecord(side->ev[2], aux) != cudaSuccess ||
+            cudaStreamWaitEvent(st, side->ev[2], 0) != cudaSuccess)
+            return GC_ERR_CUDA;
+        return GC_OK;
+    }
+    return run_online_sweeps(p, pl, ws, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status, st,
+                             out_of_range);
 }
 
 int run_build_sweeps(const Problem& p, const Plan& pl, char* w, float* loss, float* row_lse,
                      float* pos_logit, float* dQ, int64_t lddq, float* dP, int64_t lddp,
-                     int* dev_status, cudaStream_t st, const int* run_if = nullptr) {
-    int rc;
-    if (pl.anchored && !run_if) {
-        // anchored sequence first; the online-maximum sequence below then runs gated by its flag
-        if ((rc = run_anchored_fwd_dq(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dev_status, st)))
-            return rc;
-        if ((rc = run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, dev_status, st))) return rc;
-        run_if = reinterpret_cast<const int*>(w + pl.off_flag);
-    }
-    if (pl.fused) {
-        if ((rc = run_fused_fwd_dq(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dev_status, st,
-                                   run_if)))
-            return rc;
-    } else {
-        if ((rc = run_fwd(p, pl, w, loss, row_lse, pos_logit, dev_status, st, run_if))) return rc;
-        if ((rc = run_sweep(p, pl, w, SWEEP_DQ, row_lse, dQ, lddq, dev_status, st, run_if)))
-            return rc;
-    }
-    return run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, dev_status, st, run_if);
+                     int* dev_status, cudaStream_t st) {
+    if (pl.anchored)
+        return run_anchored_build(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status,
+                                  st);
+    return run_online_sweeps(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status, st);
 }
 
 // gc_build_cache with stored weights (Eq. 1, 5, 6-7 without recomputing a logit):
@@ -350,7 +419,7 @@ int run_build_stored(const Problem& p, const Plan& pl, char* w, float* loss, flo
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, nullptr, st);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, kOpen, st);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_scale_rows(p.Q, p.ldq, p.B, p.d, ref2, row_lse, qs, st);
     if (e != cudaSuccess) return GC_ERR_CUDA;
@@ -361,7 +430,7 @@ int run_build_stored(const Problem& p, const Plan& pl, char* w, float* loss, flo
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_fused_dq_finalize(partq, pl.g_mq, nullptr, ref2, row_lse, fa.pos_logit, p.pos_idx,
-                                 p.P, p.ldp, p.B, p.N, p.d, p.mask_mode, scale, dQ, lddq, nullptr,
+                                 p.P, p.ldp, p.B, p.N, p.d, p.mask_mode, scale, dQ, lddq, kOpen,
                                  st);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     {
@@ -371,14 +440,15 @@ int run_build_stored(const Problem& p, const Plan& pl, char* w, float* loss, flo
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     if (pl.g_mp > 1) {
-        e = launch_partial_reduce(partp, pl.g_mp, p.N, p.d, scale, dP, lddp, nullptr, st);
+        e = launch_partial_reduce(partp, pl.g_mp, p.N, p.d, scale, dP, lddp, kOpen, st);
         if (e != cudaSuccess) return GC_ERR_CUDA;
     }
     e = launch_dp_positive(p.pos_idx, p.B, p.N, p.mask_mode, fa.pos_logit, row_lse, p.Q, p.ldq, p.d,
                            scale, dP, lddp, st);
     if (e != cudaSuccess) return GC_ERR_CUDA;
-    return run_build_sweeps(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status, st,
-                            flag);
+    const Gate out_of_range = {flag, 1};
+    return run_online_sweeps(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status, st,
+                             out_of_range);
 }
 
 }  // namespace

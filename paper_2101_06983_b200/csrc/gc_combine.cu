@@ -29,8 +29,8 @@ lse_combine_kernel(const float* __restrict__ part_m, const float* __restrict__ p
                    const float* __restrict__ pos_ws, const int32_t* __restrict__ pos_idx,
                    int groups, int64_t B, int64_t N, int mask_mode, float* __restrict__ row_lse,
                    float* __restrict__ pos_logit, float* __restrict__ loss, float* red,
-                   int* __restrict__ dev_status, const int* __restrict__ run_if) {
-    if (run_if && *run_if == 0) return;
+                   int* __restrict__ dev_status, const Gate gate) {
+    if (gate_closed(gate)) return;
     __shared__ float warp_sum[kCombineThreads / 32];
     __shared__ int warp_flag[kCombineThreads / 32];
     __shared__ int is_last;
@@ -103,8 +103,8 @@ pos_check_kernel(const int32_t* __restrict__ pos_idx, int64_t B, int64_t N, int 
 __global__ void __launch_bounds__(256)
 partial_reduce_kernel(const float4* __restrict__ partial, int groups, int64_t rows, int d, int d4,
                       float scale, float* __restrict__ out, int64_t ldo,
-                      const int* __restrict__ run_if) {
-    if (run_if && *run_if == 0) return;
+                      const Gate gate) {
+    if (gate_closed(gate)) return;
     int64_t total = rows * d4;
     for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total;
          e += (int64_t)gridDim.x * blockDim.x) {
@@ -140,8 +140,8 @@ fused_dq_finalize_kernel(const float4* __restrict__ partial, int groups,
                          const float* __restrict__ pos_ws, const int32_t* __restrict__ pos_idx,
                          const __nv_bfloat16* __restrict__ P, int64_t ldp, int64_t B, int64_t N,
                          int d4, int mask_mode, float scale, float* __restrict__ out,
-                         int64_t ldo, const int* __restrict__ run_if) {
-    if (run_if && *run_if == 0) return;
+                         int64_t ldo, const Gate gate) {
+    if (gate_closed(gate)) return;
     int64_t total = B * d4;
     for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total;
          e += (int64_t)gridDim.x * blockDim.x) {
@@ -328,7 +328,7 @@ cudaError_t launch_fused_dq_finalize(const float* partial, int groups, const flo
                                      const float* row_ref2, const float* row_lse,
                                      const float* pos_ws, const int32_t* pos_idx, const void* P,
                                      int64_t ldp, int64_t B, int64_t N, int d, int mask_mode,
-                                     float scale, float* out, int64_t ldo, const int* run_if,
+                                     float scale, float* out, int64_t ldo, Gate gate,
                                      cudaStream_t st) {
     int64_t total = B * (d / 4);
     int64_t blocks = (total + 255) / 256;
@@ -337,21 +337,21 @@ cudaError_t launch_fused_dq_finalize(const float* partial, int groups, const flo
     fused_dq_finalize_kernel<<<(int)blocks, 256, 0, st>>>(
         reinterpret_cast<const float4*>(partial), groups, part_m, row_ref2, row_lse, pos_ws,
         pos_idx, static_cast<const __nv_bfloat16*>(P), ldp, B, N, d / 4, mask_mode, scale, out, ldo,
-        run_if);
+        gate);
     return cudaGetLastError();
 }
 
 cudaError_t launch_lse_combine(const float* part_m, const float* part_l, const float* pos_ws,
                                const int32_t* pos_idx, int groups, int64_t B, int64_t N,
                                int mask_mode, float* row_lse, float* pos_logit, float* loss,
-                               float* red, int* dev_status, const int* run_if, cudaStream_t st) {
+                               float* red, int* dev_status, Gate gate, cudaStream_t st) {
     int64_t blocks = (B + kCombineThreads - 1) / kCombineThreads;
     if (blocks > sm_count()) blocks = sm_count();
     if (blocks > 256) blocks = 256;          // the scratch holds this many block sums
     lse_combine_kernel<<<(int)blocks, kCombineThreads, 0, st>>>(part_m, part_l, pos_ws, pos_idx,
                                                                groups, B, N, mask_mode, row_lse,
                                                                pos_logit, loss, red, dev_status,
-                                                               run_if);
+                                                               gate);
     return cudaGetLastError();
 }
 
@@ -364,7 +364,7 @@ cudaError_t launch_pos_check(const int32_t* pos_idx, int64_t B, int64_t N, int m
 }
 
 cudaError_t launch_partial_reduce(const float* partial, int groups, int64_t rows, int d,
-                                  float scale, float* out, int64_t ldo, const int* run_if,
+                                  float scale, float* out, int64_t ldo, Gate gate,
                                   cudaStream_t st) {
     int d4 = (d + 3) / 4;
     int64_t total = rows * d4;
@@ -373,7 +373,7 @@ cudaError_t launch_partial_reduce(const float* partial, int groups, int64_t rows
     if (blocks > cap) blocks = cap;
     partial_reduce_kernel<<<(int)blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(partial),
                                                       groups, rows, d, d4, scale, out, ldo,
-                                                      run_if);
+                                                      gate);
     return cudaGetLastError();
 }
 

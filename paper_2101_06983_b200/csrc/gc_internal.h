@@ -9,6 +9,18 @@
 
 namespace gc {
 
+// A kernel launched with a gate returns at once unless (*flag != 0) == (want != 0); with
+// flag == NULL it always runs.  The flag is written by an earlier kernel of the same call.
+struct Gate {
+    const int* flag;
+    int want;
+};
+#ifdef __CUDACC__
+__device__ __forceinline__ bool gate_closed(const Gate& g) {
+    return g.flag && ((*g.flag != 0) != (g.want != 0));
+}
+#endif
+
 // One problem instance as the entry points receive it.
 struct Problem {
     const void* Q;
@@ -47,7 +59,7 @@ struct SweepArgs {
     float* partial;         // [groups x nx x d] unscaled partial sums (used when groups > 1)
     int groups;             // the y range is split into this many contiguous parts
     int* dev_status;        // may be NULL
-    const int* run_if;      // when not NULL the kernels return at once unless *run_if != 0
+    Gate gate;
 };
 
 struct FwdArgs {
@@ -59,7 +71,7 @@ struct FwdArgs {
                             // first word (the block ticket)
     int groups;
     int* dev_status;        // may be NULL
-    const int* run_if;      // when not NULL the kernels return at once unless *run_if != 0
+    Gate gate;
 };
 
 // How one call is carried out for given sizes on the current device.
@@ -88,17 +100,17 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored = false);
 cudaError_t launch_lse_combine(const float* part_m, const float* part_l, const float* pos_ws,
                                const int32_t* pos_idx, int groups, int64_t B, int64_t N,
                                int mask_mode, float* row_lse, float* pos_logit, float* loss,
-                               float* red, int* dev_status, const int* run_if, cudaStream_t st);
+                               float* red, int* dev_status, Gate gate, cudaStream_t st);
 cudaError_t launch_pos_check(const int32_t* pos_idx, int64_t B, int64_t N, int mask_mode,
                              int* dev_status, cudaStream_t st);
 cudaError_t launch_fused_dq_finalize(const float* partial, int groups, const float* part_m,
                                      const float* row_ref2, const float* row_lse,
                                      const float* pos_ws, const int32_t* pos_idx, const void* P,
                                      int64_t ldp, int64_t B, int64_t N, int d, int mask_mode,
-                                     float scale, float* out, int64_t ldo, const int* run_if,
+                                     float scale, float* out, int64_t ldo, Gate gate,
                                      cudaStream_t st);
 cudaError_t launch_partial_reduce(const float* partial, int groups, int64_t rows, int d,
-                                  float scale, float* out, int64_t ldo, const int* run_if,
+                                  float scale, float* out, int64_t ldo, Gate gate,
                                   cudaStream_t st);
 cudaError_t launch_pos_anchor(const void* Q, int64_t ldq, const void* P, int64_t ldp,
                               const int32_t* pos_idx, int64_t B, int64_t N, int d, int mask_mode,

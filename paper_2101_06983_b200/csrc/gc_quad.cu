@@ -47,11 +47,11 @@ struct QuadParams {
     float* pos_logit;         // FA
     int* range_flag;          // FA
     int* dev_status;
-    const int* run_if;
+    Gate gate;
     int* zero_me;
 };
 
-constexpr int Q_XRES = 2;     // X chunks that stay resident
+constexpr int Q_XRES = 0;     // X chunks that stay resident (a deeper ring serves better)
 
 // Optional diagnostics (-DGC_TC_TRACE): event timeline of the two pair leaders of cluster 0 in
 // the mode g_qev_mode selects; per role (tag, low clock bits) pairs.
@@ -122,7 +122,7 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
     volatile int* abort_flag = &abort_s;
-    if (p.run_if && *p.run_if == 0) return;     // same answer in every CTA
+    if (gate_closed(p.gate)) return;            // same answer in every CTA
     if (MODE == QMODE_FA && blockIdx.x == 0 && threadIdx.x == 0 && p.zero_me) *p.zero_me = 0;
 
     constexpr int SN = 128;
@@ -719,7 +719,7 @@ cudaError_t quad_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     p.out_scale = a.out_scale;
     p.row_lse = a.row_lse; p.pos_idx = a.pos_idx;
     p.dev_status = a.dev_status;
-    p.run_if = a.run_if;
+    p.gate = a.gate;
     const bool ok_map = a.groups == 1 ? make_out_map(&mo, a.out, a.nx, a.d, a.ldo, 1)
                                       : make_out_map(&mo, a.partial, a.nx, a.d, a.d, a.groups);
     if (!ok_map) return cudaErrorInvalidValue;
@@ -753,7 +753,7 @@ cudaError_t quad_launch_fused_dq(const FwdArgs& a, float* partial, int groups, c
     p.part_m = a.part_m; p.part_l = a.part_l; p.pos_logit = a.pos_logit;
     p.range_flag = range_flag;
     p.dev_status = a.dev_status;
-    p.run_if = a.run_if;
+    p.gate = a.gate;
     p.zero_me = reinterpret_cast<int*>(a.red);
     const int64_t clusters = (((pr.B + XROWS - 1) / XROWS + 1) / 2) * groups;
     return launch_quad<QMODE_FA>(mx, my, myh, mo, p, clusters, st);

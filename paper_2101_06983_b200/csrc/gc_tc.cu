@@ -93,7 +93,7 @@ struct TcParams {
     int* dev_status;
     const float* row_ref;     // FS: per-query anchor of the stored weights, log2 domain
     int* range_flag;          // FS: set to 1 when a weight leaves the range the anchor allows
-    const int* run_if;        // when not NULL and *run_if == 0 the kernel returns at once
+    Gate gate;                // closed: the kernel returns at once
     int* zero_me;             // forward sweeps: the ticket word of the reduction that follows
 };
 
@@ -130,7 +130,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     __shared__ int abort_s;
     __shared__ float row_max_xch[2][XROWS];      // FQ: [column half][row] block maxima
     volatile int* abort_flag = &abort_s;
-    if (p.run_if && *p.run_if == 0) return;     // same answer in every CTA
+    if (gate_closed(p.gate)) return;            // same answer in every CTA
     if ((MODE == MODE_FWD || MODE == MODE_FS || MODE == MODE_FQ) && blockIdx.x == 0 && threadIdx.x == 0 && p.zero_me) *p.zero_me = 0;
 
     static_assert(SN == 128, "a Y chunk is 128 rows: the same 16 KB as an X chunk");
@@ -1192,7 +1192,7 @@ cudaError_t tc_launch_fwd(const FwdArgs& a, cudaStream_t st) {
     p.part_m = a.part_m; p.part_l = a.part_l; p.pos_logit = a.pos_logit;
     p.zero_me = reinterpret_cast<int*>(a.red);
     p.dev_status = a.dev_status;
-    p.run_if = a.run_if;
+    p.gate = a.gate;
     return launch<MODE_FWD, SN, 2>(mx, my, myh, mx, p, st);   // no accumulator output
 }
 
@@ -1256,7 +1256,7 @@ cudaError_t tc_launch_fused_dq(const FwdArgs& a, float* partial, int groups, cud
     p.zero_me = reinterpret_cast<int*>(a.red);
     p.partial = partial;
     p.dev_status = a.dev_status;
-    p.run_if = a.run_if;
+    p.gate = a.gate;
     CUtensorMap mo;
     if (!make_out_map(&mo, partial, pr.B, pr.d, pr.d, groups)) return cudaErrorInvalidValue;
     return launch<MODE_FQ, SN, 1>(mx, my, myh, mo, p, st);
@@ -1283,7 +1283,7 @@ cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     p.row_lse = a.row_lse; p.pos_idx = a.pos_idx;
     p.out = a.out; p.ldo = a.ldo; p.partial = a.partial;
     p.dev_status = a.dev_status;
-    p.run_if = a.run_if;
+    p.gate = a.gate;
     CUtensorMap mo;
     const bool ok_map = a.groups == 1 ? make_out_map(&mo, a.out, a.nx, a.d, a.ldo, 1)
                                       : make_out_map(&mo, a.partial, a.nx, a.d, a.d, a.groups);
