@@ -214,6 +214,9 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
         int next = 0;
         uint32_t next_phase = 0;
         bool ok = true;
+#ifdef GC_TC_TRACE
+        int ev_p = 0;
+#endif
         auto acquire = [&]() -> int {
             const int stage = next;
             const uint32_t phase = next_phase;
@@ -223,6 +226,16 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                 ok = false;
                 return -1;
             }
+#ifdef GC_TC_TRACE
+            if (blockIdx.x == 0 && lane == 0 && g_qev_mode == MODE + 16) {
+                if (ev_p < 4094) {
+                    g_qevlog[2 + warp][2 * ev_p] = (20u << 16) | (unsigned)stage;
+                    g_qevlog[2 + warp][2 * ev_p + 1] = (unsigned)clock64();
+                    ++ev_p;
+                    g_qevlog[2 + warp][2 * 4095] = (unsigned)ev_p;
+                }
+            }
+#endif
             return stage;
         };
         // kind 0: this CTA's 64 rows of two Y chunks (S phase); kind 1: one X chunk of its 128
@@ -282,6 +295,16 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                     ok = false;
                     return -1;
                 }
+#ifdef GC_TC_TRACE
+                if (blockIdx.x == 0 && lane == 0 && g_qev_mode == MODE + 16) {
+                    if (ev_m < 4094) {
+                        g_qevlog[0][2 * ev_m] = (1u << 16) | (unsigned)stage;
+                        g_qevlog[0][2 * ev_m + 1] = (unsigned)clock64();
+                        ++ev_m;
+                        g_qevlog[0][2 * 4095] = (unsigned)ev_m;
+                    }
+                }
+#endif
                 return stage;
             };
             for_each_op([&](int kind, int idx) {

@@ -52,6 +52,39 @@ def test_self_mask_shared_rows(binding, oracle, n, d, tau, dtype):
     check_against_oracle(prob, out, _oracle_full(oracle, prob))
 
 
+# Rows of two column halves (d = 512, 640, 768) with more than one x tile run as clusters of four
+# CTAs whose two pairs alternate over the streamed tiles: 1, 2, 3 and more tiles per cluster, odd
+# and even counts, an odd number of x tiles, split streamed ranges, both mask modes.
+QUAD_SHAPES = [
+    (130, 100, 768), (200, 200, 768), (257, 330, 512), (300, 520, 640), (385, 900, 768),
+    (520, 260, 512), (1030, 1300, 768), (2100, 3000, 640),
+]
+
+
+@pytest.mark.parametrize("B,N,d", QUAD_SHAPES)
+def test_four_cta_cluster_sweeps(binding, oracle, B, N, d):
+    prob = inputs.random_problem(B, N, d, "bf16", seed=B + N + d, tau=0.3, scale=d ** -0.5)
+    out = run_build(prob)
+    ref = _oracle_full(oracle, prob)
+    check_against_oracle(prob, out, ref)
+    # the same kernels with a given row_lse (gc_loss_bwd), from the forward call's lse
+    Q, P, pos = to_device(prob)
+    b = binding.Outputs(prob.B, prob.N, prob.d, binding.GC_BF16)
+    binding.gc_loss_fwd(Q, P, pos, prob.tau, prob.mask_mode, b.loss, b.row_lse, b.pos_logit, b.ws,
+                        b.dev_status)
+    binding.gc_loss_bwd(Q, P, pos, prob.tau, prob.mask_mode, b.row_lse, b.dQ, b.dP, b.ws,
+                        b.dev_status)
+    torch.cuda.synchronize()
+    check_against_oracle(prob, b, ref)
+
+
+def test_four_cta_cluster_sweeps_self_mask(binding, oracle):
+    prob = inputs.random_problem(700, 700, 768, "bf16", seed=77, tau=0.2,
+                                 mask_mode=inputs.MASK_SELF, scale=768 ** -0.5, shared=True)
+    out = run_build(prob)
+    check_against_oracle(prob, out, _oracle_full(oracle, prob))
+
+
 @pytest.mark.parametrize("B,N", [(300, 45000), (45000, 300)])
 def test_streamed_matrix_larger_than_l2_uses_cta_pairs(binding, oracle, B, N):
     """When the streamed matrix (P for the forward/dQ sweeps, Q for the dP sweep) exceeds 64 MB
