@@ -27,16 +27,16 @@ if ROOT not in sys.path:
 METRIC = "gc_build_cache TFLOP/s (3 GEMMs of 2*B*N*d) at B=4096,N=8192,d=768"
 UNIT = "TFLOP/s"
 NOMINAL_BF16_TFLOPS = 2250.0      # public dense bf16 figure for B200, context only
-# dram__bytes_read.sum + dram__bytes_write.sum per gradient-sweep launch at the headline shape,
-# from the ncu capture summarised in profiles/tc_kernel_cfg2_B4096_N8192_d768.txt.  Reported only
-# while the kernel source still has the hash it had when the counters were taken.
-NCU_TRAFFIC_BYTES = 18.97e6
-NCU_TRAFFIC_SOURCE_SHA1 = "da73b84221bcbb2d0d62375070a74b30519f05cd"
+# dram__bytes_read.sum + dram__bytes_write.sum per sweep launch at the headline shape, from the
+# ncu capture summarised in profiles/quad_kernel_cfg2_B4096_N8192_d768.txt.  Reported only while
+# the kernel source still has the hash it had when the counters were taken.
+NCU_TRAFFIC_BYTES = 19.0e6
+NCU_TRAFFIC_SOURCE_SHA1 = "dd3e923aa3355f8e776780c11a5c32246f66a5e4"
 
 
 def ncu_traffic(workload: str):
     import hashlib
-    src = os.path.join(ROOT, "paper_2101_06983_b200", "csrc", "gc_tc.cu")
+    src = os.path.join(ROOT, "paper_2101_06983_b200", "csrc", "gc_quad.cu")
     try:
         with open(src, "rb") as fh:
             same = hashlib.sha1(fh.read()).hexdigest() == NCU_TRAFFIC_SOURCE_SHA1
@@ -346,7 +346,8 @@ def run_ours(args, rank, local_rank, world):
                         "value": world * flop / (warm_ms * 1e-3) / 1e12, "unit": UNIT},
             "kernel_ms": {"fwd_sweep": kern[0] / args.steps, "dq_sweep": kern[1] / args.steps,
                           "dp_sweep": kern[2] / args.steps},
-            "roofline": {"bound": "tensor", "kernel": f"{plan} tile sweep (the two gradient launches per step)",
+            "roofline": {"bound": "tensor",
+                         "kernel": f"{plan} sweeps (the tensor-core launches of a step)",
                          "achieved": achieved, "peak": pk["tf_burst"], "unit": "TFLOP/s",
                          "frac": achieved / pk["tf_burst"], "peak_source": pk["source"],
                          "traffic": None if stored else ncu_traffic(prob.name)},

@@ -70,8 +70,9 @@ enum { GC_DEV_POS_RANGE = 1, GC_DEV_POS_MASKED = 2, GC_DEV_WAIT_LIMIT = 4 };
 size_t gc_workspace_bytes(int op, int64_t B, int64_t N, int d, int dtype);
 
 /* Name of the kernel plan the library will use for these sizes: "tcgen05" (TMA + tcgen05 MMA
- * with TMEM accumulators; bf16, d a multiple of 64 up to 4096) or "simt" (fp32 FMA tiles; every
- * other case, including all fp32 inputs).  Static string. */
+ * with TMEM accumulators; bf16, d a multiple of 64 up to 4096; one CTA, a CTA pair or a cluster
+ * of four per tile, by shape) or "simt" (fp32 FMA tiles; every other case, including all fp32
+ * inputs).  Static string. */
 const char* gc_plan_name(int op, int64_t B, int64_t N, int d, int dtype);
 
 /* Number of kernels one call launches for these sizes (for launch accounting). */
@@ -97,7 +98,11 @@ int gc_loss_bwd(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
                 void* ws, size_t ws_bytes, int* dev_status, void* cuda_stream);
 
 /*
- * Step 2 of Section 3.3 in one call: loss, row_lse, (pos_logit) and the cache dQ, dP.
+ * Step 2 of Section 3.3 in one call: loss, row_lse, (pos_logit) and the cache dQ, dP.  Nothing of
+ * size B x N is written to global memory.  For bf16 rows wider than 256 the forward runs inside
+ * the dQ sweep.  Part of the work may be queued on a stream the library owns, between a fork from
+ * and a join back into `cuda_stream`: the call is asynchronous on `cuda_stream` alone, but the
+ * first such call on a device creates that stream and belongs outside any stream capture.
  */
 int gc_build_cache(const void* Q, int64_t ldq, const void* P, int64_t ldp, const int32_t* pos_idx,
                    int64_t B, int64_t N, int d, float tau, int mask_mode, int dtype,

@@ -1,31 +1,34 @@
-// Tensor-core plan for bf16 inputs with d a multiple of 64 (up to 4096): TMA-staged tiles in
-// 128-byte-swizzled shared memory, tcgen05 MMAs with fp32 accumulators in tensor memory, the
-// softmax arithmetic in registers.  One kernel template serves three sweeps:
+// Tensor-core sweeps with one CTA, or one CTA pair, per (x tile, accumulator part): bf16 inputs
+// with d a multiple of 64 (up to 4096).  TMA-staged tiles in 128-byte-swizzled shared memory,
+// tcgen05 MMAs with fp32 accumulators in tensor memory, the softmax arithmetic in registers.  One
+// kernel template serves five sweeps:
 //
 //   FWD  (Eq. 1)    x = 128 queries,  y streams passages: S = X Y^T, online row max / sum.
 //   DQ   (Eq. 5)    x = 128 queries,  y streams passages: W = exp(S - lse_x) - onehot, acc += W Y
 //   DP   (Eq. 6-7)  x = 128 passages, y streams queries:  W = exp(S - lse_y) - onehot, acc += W Y
-//   FQ   (Eq. 1+5)  forward fused into the dQ sweep (used by gc_build_cache for wide rows): the
-//                   row maximum runs online, W = exp(S - m_ref) with the positive column left
-//                   out, acc += W Y; the accumulator is rescaled only when the maximum grows by
-//                   more than 2^8.  A finalize pass forms (sum_g acc_g exp(m_g - lse)
-//                   + (p_pos - 1) P_pos) / (B tau) with the positive term in fp32.
+//   FQ   (Eq. 1+5)  forward fused into the dQ sweep: the row maximum runs online, W = exp(S -
+//                   m_ref) with the positive column left out, acc += W Y; the accumulator is
+//                   rescaled only when the maximum grows by more than 2^8.  A finalize pass forms
+//                   (sum_g acc_g exp(m_g - lse) + (p_pos - 1) P_pos) / (B tau), positive term in fp32.
+//   FS   (Eq. 1)    forward that also stores the bf16 weights 2^(s2 - ref2_x) of all pairs (the
+//                   stored-weights comparison plan).
+//
+// Rows of two column halves with more than one x tile are served by the four-CTA sweeps of
+// gc_quad.cu instead; there FQ and DP remain as the gated fallback.
 //
 // The stationary tile X (128 x d) stays resident in shared memory when d <= 512; for wider rows
-// only its first 6 column chunks stay and the others are re-streamed every step, which leaves
-// room for a ring of eight 16 KB stages: the load -> MMA -> release chain of a stage is about
-// 1500-2000 cycles long, so the bytes in flight, not the L2 bandwidth, bound the MMA rate.
-// Y arrives in (SN x 64) chunks through the same mbarrier ring.  S tiles (128 x SN, fp32) are double buffered in tensor
-// memory so the MMAs of step t+1 run while the softmax warps work on step t.  W is written
-// back over its S buffer as packed bf16 and used as the A operand (from tensor memory) of the
-// second MMA, whose B operand is the same Y chunk read MN-major.  An accumulator of 128 x 768
-// fp32 does not fit the 512 tensor-memory columns, so wide rows are split into column parts
-// (at most 384 columns each), one CTA per part.  S is never written to global memory.
+// only its first chunks stay (6, or 2 beside shared-memory W buffers) and the others are
+// re-streamed every step through the ring that also carries Y in (128 x 64) chunks.  Narrow rows
+// double-buffer the S tile (128 x 128, fp32) in tensor memory and write W back over it as packed
+// bf16 (A operand from tensor memory); wide rows have one S tile and, when paired, keep W in two
+// shared-memory buffers so that S(t+1) is issued while softmax(t) runs.  The B operand of the
+// accumulation MMA is the Y chunk read MN-major.  An accumulator of 128 x 768 fp32 does not fit
+// the 512 tensor-memory columns, so wide rows are split into column parts (at most 384 columns),
+// one CTA per part.  S is never written to global memory.
 //
-// Warp roles (416 threads): warps 0..3 = TMA producers (the ring stages are dealt out to four
-// issuing warps), warp 4 = MMA issuer (and tensor-memory allocator), warps 5..12 = softmax /
-// epilogue: two warps per tensor-memory lane quarter, each owning half of the tile's columns,
-// one thread per tile row.
+// Warp roles (352 threads): warps 0..1 = TMA producers (ring stages dealt out alternately), warp
+// 2 = MMA issuer (and tensor-memory allocator), warps 3..10 = softmax / epilogue: two warps per
+// tensor-memory lane quarter, each owning half of the tile's columns, one thread per tile row.
 // Every wait is bounded: on a timeout the CTA raises GC_DEV_WAIT_LIMIT, drains and exits.
 #include "tc_common.cuh"
 
