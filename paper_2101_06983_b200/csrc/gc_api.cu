@@ -197,9 +197,11 @@ int run_fwd(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_
 // `timed`: bracket the sweep with the profiling events (only the sweeps that normally run are).
 int run_sweep(const Problem& p, const Plan& pl, char* ws, int mode, const float* row_lse,
               float* out, int64_t ldo, int* dev_status, cudaStream_t st, Gate gate = kOpen,
-              bool timed = true) {
+              bool timed = true, const float* slot_m = nullptr, const float* slot_l = nullptr,
+              int slots = 0) {
     SweepArgs sa{};
     sa.gate = gate;
+    sa.slot_m = slot_m; sa.slot_l = slot_l; sa.slots = slots;
     const bool dq = (mode == SWEEP_DQ);
     sa.X = dq ? p.Q : p.P;   sa.ldx = dq ? p.ldq : p.ldp;   sa.nx = dq ? p.B : p.N;
     sa.Y = dq ? p.P : p.Q;   sa.ldy = dq ? p.ldp : p.ldq;   sa.ny = dq ? p.N : p.B;
@@ -312,18 +314,20 @@ SideStream* side_stream() {
 // kernels after the fused sweep run only while it is down, and the online-maximum sequence, which
 // is always launched, runs only when it is up and then produces every output.
 //
-//   caller's stream:  anchor, fused sweep, combine, dP sweep (+ reduce)
-//   side stream:      after the fused sweep: the gated online-maximum sequence;
-//                     after the combine: the dQ finalize
-// Both are joined back before the call returns.  Without a side stream everything is queued on
-// the caller's stream in dependency order.
+//   caller's stream:  anchor, fused sweep, dP sweep (+ reduce), which merges the forward slots
+//                     of its streamed queries itself
+//   side stream:      after the fused sweep: combine (row_lse, loss), dQ finalize, then the
+//                     gated online-maximum sequence
+// Both are joined back before the call returns.  Without a side stream, or when the dP sweep is
+// not a four-CTA sweep (N <= 128), everything is queued on the caller's stream in dependency
+// order with the combine before the dP sweep.
 int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_lse,
                        float* pos_logit, float* dQ, int64_t lddq, float* dP, int64_t lddp,
                        int* dev_status, cudaStream_t st) {
     float* ref2 = reinterpret_cast<float*>(ws + pl.off_ref);
     int* flag = reinterpret_cast<int*>(ws + pl.off_flag);
     const Gate in_range = {flag, 0}, out_of_range = {flag, 1};
-    SideStream* side = side_stream();
+    SideStream* side = quad_applicable(p.N, p.d) ? side_stream() : nullptr;
     cudaStream_t aux = side ? side->st : st;
     cudaError_t e = launch_pos_anchor(p.Q, p.ldq, p.P, p.ldp, p.pos_idx, p.B, p.N, p.d, p.mask_mode,
                                       1.4426950408889634f / p.tau, ref2, flag, st);
@@ -345,30 +349,28 @@ int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, 
     if (side && (cudaEventRecord(side->ev[0], st) != cudaSuccess ||
                  cudaStreamWaitEvent(aux, side->ev[0], 0) != cudaSuccess))
         return GC_ERR_CUDA;
-    int rc;
-    if (side) {
-        // fallback first on the side stream: it only needs the flag
-        if ((rc = run_online_sweeps(p, pl, ws, loss, row_lse, pos_logit, dQ, lddq, dP, lddp,
-                                    dev_status, aux, out_of_range)))
-            return rc;
-    }
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, in_range, st);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, in_range, aux);
     if (e != cudaSuccess) return GC_ERR_CUDA;
-    if (side && (cudaEventRecord(side->ev[1], st) != cudaSuccess ||
-                 cudaStreamWaitEvent(aux, side->ev[1], 0) != cudaSuccess))
-        return GC_ERR_CUDA;
     e = launch_fused_dq_finalize(partial, pl.g_dq, nullptr, ref2, row_lse, fa.pos_logit, p.pos_idx,
                                  p.P, p.ldp, p.B, p.N, p.d, p.mask_mode,
                                  1.f / ((float)p.B * p.tau), dQ, lddq, in_range, aux);
     if (e != cudaSuccess) return GC_ERR_CUDA;
-    if ((rc = run_sweep(p, pl, ws, SWEEP_DP, row_lse, dP, lddp, dev_status, st, in_range))) return rc;
+    int rc;
     if (side) {
+        if ((rc = run_online_sweeps(p, pl, ws, loss, row_lse, pos_logit, dQ, lddq, dP, lddp,
+                                    dev_status, aux, out_of_range)))
+            return rc;
+        // the dP sweep does not wait for the combine: it merges the slots it needs itself
+        if ((rc = run_sweep(p, pl, ws, SWEEP_DP, row_lse, dP, lddp, dev_status, st, in_range, true,
+                            fa.part_m, fa.part_l, fa.groups)))
+            return rc;
         if (cudaEventRecord(side->ev[2], aux) != cudaSuccess ||
             cudaStreamWaitEvent(st, side->ev[2], 0) != cudaSuccess)
             return GC_ERR_CUDA;
         return GC_OK;
     }
+    if ((rc = run_sweep(p, pl, ws, SWEEP_DP, row_lse, dP, lddp, dev_status, st, in_range))) return rc;
     return run_online_sweeps(p, pl, ws, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status, st,
                              out_of_range);
 }

@@ -38,14 +38,7 @@ lse_combine_kernel(const float* __restrict__ part_m, const float* __restrict__ p
     int flags = 0;
     for (int64_t i = blockIdx.x * (int64_t)kCombineThreads + threadIdx.x; i < B;
          i += (int64_t)gridDim.x * kCombineThreads) {
-        float m = -INFINITY;
-        for (int g = 0; g < groups; ++g) m = fmaxf(m, part_m[(int64_t)g * B + i]);
-        float l = 0.f;
-        for (int g = 0; g < groups; ++g) {
-            float mg = part_m[(int64_t)g * B + i];
-            if (mg > -INFINITY) l += part_l[(int64_t)g * B + i] * expf(mg - m);
-        }
-        float lse = m + logf(l);
+        const float lse = combined_lse(part_m, part_l, groups, B, i);
         row_lse[i] = lse;
         int f = pos_flags(pos_idx[i], i, N, mask_mode);
         float pl = f ? 0.f : pos_ws[i];

@@ -19,6 +19,21 @@ struct Gate {
 __device__ __forceinline__ bool gate_closed(const Gate& g) {
     return g.flag && ((*g.flag != 0) != (g.want != 0));
 }
+// Logsumexp of row i from its per-part (scale, sum) slots, slot g at [g * pitch + i]: the one
+// definition every kernel that merges slots uses, with explicit roundings so that all of them
+// get the same bits.
+__device__ __forceinline__ float combined_lse(const float* __restrict__ part_m,
+                                              const float* __restrict__ part_l, int slots,
+                                              int64_t pitch, int64_t i) {
+    float m = -INFINITY;
+    for (int g = 0; g < slots; ++g) m = fmaxf(m, part_m[(int64_t)g * pitch + i]);
+    float l = 0.f;
+    for (int g = 0; g < slots; ++g) {
+        const float mg = part_m[(int64_t)g * pitch + i];
+        if (mg > -INFINITY) l = __fmaf_rn(part_l[(int64_t)g * pitch + i], expf(mg - m), l);
+    }
+    return __fadd_rn(m, logf(l));
+}
 #endif
 
 // One problem instance as the entry points receive it.
@@ -60,6 +75,11 @@ struct SweepArgs {
     int groups;             // the y range is split into this many contiguous parts
     int* dev_status;        // may be NULL
     Gate gate;
+    // SWEEP_DP of the four-CTA kernels only: when slot_l is set, row_lse is not read; the
+    // logsumexp of each streamed query is merged from these forward slots ([slots][ny]) instead.
+    const float* slot_m;
+    const float* slot_l;
+    int slots;
 };
 
 struct FwdArgs {

@@ -31,6 +31,7 @@ enum { QMODE_DQ = 1, QMODE_DP = 2, QMODE_FA = 3 };
 struct QuadParams {
     int64_t nx, ny;
     int64_t nq;               // number of queries B (pitch of the forward slot arrays)
+    int nslots;               // DP: forward slots per query to merge (0: read row_lse)
     int kc;                   // d / 64
     int dpc;                  // chunks per column half
     int groups;
@@ -42,8 +43,10 @@ struct QuadParams {
     const float* row_lse;
     const int32_t* pos_idx;
     const float* row_ref;     // FA: anchor of each query's weights, log2 domain
-    float* part_m;            // FA: [4 groups][B] slots (scale, natural log)
-    float* part_l;            // FA: [4 groups][B] slots (sum)
+    float* part_m;            // FA: [4 groups][B] slots (scale, natural log), written
+    float* part_l;            // FA: [4 groups][B] slots (sum), written
+    const float* slot_m;      // DP with nslots > 0: the slots a forward sweep wrote
+    const float* slot_l;
     float* pos_logit;         // FA
     int* range_flag;          // FA
     int* dev_status;
@@ -467,7 +470,11 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
 #pragma unroll
                 for (int jj = 0; jj < CB_PER; ++jj) {
                     const int64_t y = y0 + (cb0 + jj) * 32 + lane;
-                    lse2_y[jj] = (y < p.ny) ? p.row_lse[y] * 1.4426950408889634f : INFINITY;
+                    float lse_y = INFINITY;
+                    if (y < p.ny)
+                        lse_y = p.nslots > 0 ? combined_lse(p.slot_m, p.slot_l, p.nslots, p.nq, y)
+                                             : p.row_lse[y];
+                    lse2_y[jj] = lse_y * 1.4426950408889634f;
                     pos_y[jj] = (y < p.ny) ? p.pos_idx[y] : -1;
                 }
             }
@@ -743,6 +750,9 @@ cudaError_t quad_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     p.row_lse = a.row_lse; p.pos_idx = a.pos_idx;
     p.dev_status = a.dev_status;
     p.gate = a.gate;
+    if (a.mode == SWEEP_DP && a.slot_l) {
+        p.slot_m = a.slot_m; p.slot_l = a.slot_l; p.nslots = a.slots; p.nq = a.ny;
+    }
     const bool ok_map = a.groups == 1 ? make_out_map(&mo, a.out, a.nx, a.d, a.ldo, 1)
                                       : make_out_map(&mo, a.partial, a.nx, a.d, a.d, a.groups);
     if (!ok_map) return cudaErrorInvalidValue;
