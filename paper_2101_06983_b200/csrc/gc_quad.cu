@@ -429,6 +429,7 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
         const int q = warp & 3;                        // tensor-memory lane quarter of this warp
         const int half = (warp - (NPROD + 1)) >> 2;    // which half of the tile's columns
         constexpr int CB_PER = SN / 64;
+        static_assert(CB_PER == 2, "the softmax loop reads two 32-column blocks per thread");
         const int cb0 = half * CB_PER;
         const int row = q * 32 + lane;
         const int64_t x = x0 + row;
@@ -464,8 +465,8 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
         for (int j = 0; j < nd; ++j) {
             const int t = 2 * j + pr;
             const int64_t y0 = (lo + t) * SN;
-            float lse2_y[CB_PER];
-            int32_t pos_y[CB_PER];
+            float lse2_y[CB_PER] = {};
+            int32_t pos_y[CB_PER] = {};
             if (MODE == QMODE_DP) {
 #pragma unroll
                 for (int jj = 0; jj < CB_PER; ++jj) {
@@ -486,29 +487,34 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
             tc_fence_after();
 #ifdef GC_TC_TRACE
             const long long c1_ = clock64(); ph[0] += c1_ - c0_;
+            long long c2_ = c1_, c3_ = c1_;
 #endif
             const uint32_t sbuf = tmem + lane_addr + S_COL0;
-            uint32_t vv[CB_PER][32];
-#pragma unroll
-            for (int jj = 0; jj < CB_PER; ++jj) tmem_ld32(sbuf + (cb0 + jj) * 32, vv[jj]);
+            // Both 32-column blocks are read at once, so that the S tile is free again; the
+            // arithmetic then takes one block at a time in a loop that is not unrolled: the body is
+            // long, and the first pass through it runs at instruction-fetch speed.
+            uint32_t va[32], vb[32];
+            tmem_ld32(sbuf + cb0 * 32, va);
+            tmem_ld32(sbuf + (cb0 + 1) * 32, vb);
             tmem_ld_wait();
 #ifdef GC_TC_TRACE
-            const long long c2_ = clock64(); ph[1] += c2_ - c1_;
+            c2_ = clock64(); ph[1] += c2_ - c1_;
 #endif
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bars.s_read));  // the S tile may be overwritten
 #ifdef GC_TC_TRACE
-            const long long c3_ = clock64(); ph[2] += c3_ - c2_;
+            c3_ = clock64(); ph[2] += c3_ - c2_;
 #endif
-#ifdef GC_TC_TRACE
-            const long long c4_ = c3_;
-#endif
-            uint32_t packed[CB_PER][16];
-#pragma unroll
+            uint32_t keep_a[16], keep_b[16];
+#pragma unroll 1
             for (int jj = 0; jj < CB_PER; ++jj) {
                 const int cb = cb0 + jj;
-                uint32_t (&v)[32] = vv[jj];
+                uint32_t v[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c) v[c] = jj == 0 ? va[c] : vb[c];
+                const float lse2_yj = jj == 0 ? lse2_y[0] : lse2_y[CB_PER - 1];
+                const int32_t pos_yj = jj == 0 ? pos_y[0] : pos_y[CB_PER - 1];
                 const int64_t yb = y0 + cb * 32;
                 float w[32];
                 if (MODE == QMODE_FA) {
@@ -571,12 +577,12 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                 } else {
 #pragma unroll
                     for (int c = 0; c < 32; ++c) {
-                        const float ls = __shfl_sync(0xffffffffu, lse2_y[jj], c);
+                        const float ls = __shfl_sync(0xffffffffu, lse2_yj, c);
                         w[c] = ex2(fmaf(__uint_as_float(v[c]), p.c1, -ls));   // OOB: ex2(-inf)
                     }
                     // one-hot: column c's query has its positive at row pos - x0 of this tile
-                    const int64_t rel_row = (int64_t)pos_y[jj] - x0;
-                    const bool mine = (pos_y[jj] >= 0) && rel_row >= q * 32 && rel_row < q * 32 + 32;
+                    const int64_t rel_row = (int64_t)pos_yj - x0;
+                    const bool mine = (pos_yj >= 0) && rel_row >= q * 32 && rel_row < q * 32 + 32;
                     unsigned hits = __ballot_sync(0xffffffffu, mine);
                     while (hits) {
                         const int col = __ffs(hits) - 1;
@@ -595,10 +601,18 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                     for (int c = 0; c < 32; ++c)
                         if (c == rel) w[c] = 0.f;
                 }
+                uint32_t packed[16];
 #pragma unroll
                 for (int r = 0; r < 16; ++r) {
                     __nv_bfloat162 h = __floats2bfloat162_rn(w[2 * r], w[2 * r + 1]);
-                    packed[jj][r] = *reinterpret_cast<uint32_t*>(&h);
+                    packed[r] = *reinterpret_cast<uint32_t*>(&h);
+                }
+                if (jj == 0) {
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) keep_a[r] = packed[r];
+                } else {
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) keep_b[r] = packed[r];
                 }
             }
             // W buffer pr of both pairs must have been consumed (accumulation of tile t - 2)
@@ -607,10 +621,10 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                      mbar_wait(smem_u32(&bars.w_empty[pr][1]), (j - 1) & 1, abort_flag);
                 if (!ok) break;
             }
-#pragma unroll
-            for (int jj = 0; jj < CB_PER; ++jj) put_w_block(jj, packed[jj]);
+            put_w_block(0, keep_a);
+            put_w_block(1, keep_b);
 #ifdef GC_TC_TRACE
-            const long long c5_ = clock64(); ph[4] += c5_ - c4_;
+            const long long c5_ = clock64(); ph[4] += c5_ - c3_;
 #endif
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             tc_fence_before();
@@ -630,6 +644,12 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
             }
 #ifdef GC_TC_TRACE
             ph[6] += clock64() - c6_;
+            if (sev && qev_on && j < 6) {       // first tiles one by one: clocks at the phase ends
+                unsigned int* e = &g_qevlog[2 + pr][64 + 16 * j];
+                e[0] = (unsigned)c0_; e[1] = (unsigned)c1_; e[2] = (unsigned)c2_;
+                e[3] = (unsigned)c3_; e[4] = (unsigned)c5_; e[5] = (unsigned)c6_;
+                e[6] = (unsigned)clock64();
+            }
 #endif
         }
 #ifdef GC_TC_TRACE
