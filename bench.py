@@ -30,8 +30,8 @@ NOMINAL_BF16_TFLOPS = 2250.0      # public dense bf16 figure for B200, context o
 # dram__bytes_read.sum + dram__bytes_write.sum per sweep launch at the headline shape, from the
 # ncu capture summarised in profiles/quad_kernel_cfg2_B4096_N8192_d768.txt.  Reported only while
 # the kernel source still has the hash it had when the counters were taken.
-NCU_TRAFFIC_BYTES = 19.0e6
-NCU_TRAFFIC_SOURCE_SHA1 = "dd3e923aa3355f8e776780c11a5c32246f66a5e4"
+NCU_TRAFFIC_BYTES = 19.1e6
+NCU_TRAFFIC_SOURCE_SHA1 = "502a9f7cd1fe23b2413012fd5dc559175f624525"
 
 
 def ncu_traffic(workload: str):
