@@ -51,6 +51,8 @@ def _load():
         lib.gco_passage_rows.restype = ctypes.c_int
         lib.gco_passage_rows.argtypes = [dp, dp, ip, i64, i64, i64, ctypes.c_double, ctypes.c_int,
                                          dp, lp, i64, dp]
+        lib.gco_cache_apply.restype = ctypes.c_int
+        lib.gco_cache_apply.argtypes = [dp, dp, i64, i64, i64, ctypes.c_int, dp]
         _lib = lib
     return _lib
 
@@ -138,3 +140,26 @@ def passage_rows(Q, P, pos_idx, row_lse, rows, tau=1.0, mask_mode=0):
     if rc != 0:
         raise ValueError(f"oracle rejected the problem (code {rc})")
     return dP
+
+
+def cache_apply(U, X, dW=None):
+    """Eq. 8 / Eq. 9 for a linear encoder: returns dW (+)= U^T X in float64, where U [rows x d]
+    is a slice of the cache and X [rows x d_in] the encoder inputs of the same sub-batch.  With
+    dW given (d x d_in, float64, contiguous) the sum is added to it in place."""
+    U = _f64(U)
+    X = _f64(X)
+    if U.ndim != 2 or X.ndim != 2 or U.shape[0] != X.shape[0]:
+        raise ValueError("shape mismatch")
+    rows, d = U.shape
+    d_in = X.shape[1]
+    acc = dW is not None
+    if acc:
+        if dW.dtype != np.float64 or dW.shape != (d, d_in) or not dW.flags.c_contiguous:
+            raise ValueError("dW must be a contiguous float64 array of shape (d, d_in)")
+    else:
+        dW = np.empty((d, d_in), np.float64)
+    rc = _load().gco_cache_apply(_ptr(U, ctypes.c_double), _ptr(X, ctypes.c_double), rows, d, d_in,
+                                 int(acc), _ptr(dW, ctypes.c_double))
+    if rc != 0:
+        raise ValueError(f"oracle rejected the problem (code {rc})")
+    return dW

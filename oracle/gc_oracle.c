@@ -11,7 +11,9 @@
  * Parity pins (see tests/test_oracle_pins.py): central finite differences of the loss, row
  * sums of softmax-minus-onehot, closed forms for identical representations and for the 1x2
  * logistic case, scale and permutation symmetries, and the paper's exactness claim on a linear
- * encoder.  No function here is "parity unpinned".
+ * encoder; gco_cache_apply (Step 3 for a linear encoder) by the finite-difference gradient with
+ * respect to the encoder matrix and a hand-worked example.  No function here is "parity
+ * unpinned".
  *
  * Notation (paper, Section 3.1-3.2): Q row i is f(s_i), P row j is g(t_j), pos_idx[i] is r_i,
  * tau the temperature, S_ij = <f(s_i), g(t_j)> / tau.
@@ -229,6 +231,33 @@ int gco_passage_rows(const double* Q, const double* P, const int32_t* pos_idx, i
             for (int64_t k = 0; k < d; ++k) out[k] += g * q[k];
         }
         for (int64_t k = 0; k < d; ++k) out[k] /= tau;
+    }
+    return 0;
+}
+
+/*
+ * Step 3 for a linear encoder f(s) = W s (Section 3.3, Eq. 8; Eq. 9 for g): the representation
+ * gradients u_i of one sub-batch, taken from the cache, are pushed through the encoder's
+ * parameters.  For the linear map, d f(s_i) / d W applied to u_i is the outer product u_i s_i^T,
+ * so the sub-batch's term of Eq. 8 is
+ *
+ *     dW[a][b] (+)= sum_i U[i][a] * X[i][b]        U: rows x d (cache slice), X: rows x d_in
+ *
+ * With accumulate == 0 dW is overwritten (first sub-batch), otherwise the sum is added to it
+ * (the outer summation of Eq. 8 over sub-batches).  Pinned by the finite-difference gradient of
+ * the full-batch loss with respect to W and by a hand-worked integer example.
+ */
+int gco_cache_apply(const double* U, const double* X, int64_t rows, int64_t d, int64_t d_in,
+                    int accumulate, double* dW) {
+    if (!U || !X || !dW || rows <= 0 || d <= 0 || d_in <= 0) return 1;
+#pragma omp parallel for schedule(static)
+    for (int64_t a = 0; a < d; ++a) {
+        for (int64_t b = 0; b < d_in; ++b) {
+            double s = 0.0;
+            for (int64_t i = 0; i < rows; ++i) s += U[i * d + a] * X[i * d_in + b];
+            if (accumulate) dW[a * d_in + b] += s;
+            else dW[a * d_in + b] = s;
+        }
     }
     return 0;
 }

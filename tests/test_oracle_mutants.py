@@ -27,6 +27,10 @@ MUTANTS = {
     "G read transposed in dP": ("double g = G[i * N + j];\n                    const double* q", "double g = G[(j % B) * N + (i % N)];\n                    const double* q"),
     "positive index off by one": ("total += lse[i] - S[i * N + pos_idx[i]];", "total += lse[i] - S[i * N + (pos_idx[i] + 1) % N];"),
     "max instead of logsumexp": ("return m + log(sum);", "return m;"),
+    "cache_apply reads U transposed": ("s += U[i * d + a] * X[i * d_in + b];",
+                                       "s += U[(a % rows) * d + (i % d)] * X[i * d_in + b];"),
+    "cache_apply overwrites instead of accumulating": ("if (accumulate) dW[a * d_in + b] += s;",
+                                                       "if (accumulate) dW[a * d_in + b] = s;"),
 }
 
 
@@ -66,8 +70,25 @@ def _wrap(libpath):
             raise ValueError(f"rejected ({rc})")
         return dict(loss=float(loss.value), row_lse=lse, pos_logit=pl, dQ=dQ, dP=dP)
 
+    lib.gco_cache_apply.restype = ctypes.c_int
+    lib.gco_cache_apply.argtypes = [dp, dp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
+                                    ctypes.c_int, dp]
+
+    def cache_apply(U, X, dW=None):
+        U, X = real._f64(U), real._f64(X)
+        rows, d = U.shape
+        d_in = X.shape[1]
+        acc = dW is not None
+        if not acc:
+            dW = np.empty((d, d_in))
+        rc = lib.gco_cache_apply(real._ptr(U, ctypes.c_double), real._ptr(X, ctypes.c_double), rows,
+                                 d, d_in, int(acc), real._ptr(dW, ctypes.c_double))
+        if rc != 0:
+            raise ValueError(f"rejected ({rc})")
+        return dW
+
     return types.SimpleNamespace(
-        build_cache=build_cache,
+        build_cache=build_cache, cache_apply=cache_apply,
         loss_only=lambda Q, P, pos, tau=1.0, mask=0: build_cache(Q, P, pos, tau, mask)["loss"])
 
 
@@ -80,6 +101,8 @@ def _pins(o):
     yield lambda: pins.test_one_query_two_passages_is_logistic_loss(o)
     yield lambda: pins.test_scale_and_permutation_symmetry(o)
     yield lambda: pins.test_duplicate_positives_sum_in_epsilon(o)
+    yield lambda: pins.test_cache_apply_hand_worked_example(o)
+    yield lambda: pins.test_cache_apply_chunks_reproduce_full_batch_parameter_gradient(o)
 
 
 @pytest.mark.parametrize("name", sorted(MUTANTS))

@@ -285,3 +285,49 @@ def test_rejects_bad_positives(oracle):
     bad[1] = 1                                   # equals the masked column of row 1
     with pytest.raises(ValueError):
         oracle.build_cache(Q, P, bad, 1.0, 1)
+
+
+# ---- Step 3 for a linear encoder (Eq. 8-9): oracle.cache_apply ----------------------------------
+def test_cache_apply_hand_worked_example(oracle):
+    """rows = 2, d = 2, d_in = 3 with small integers: dW[a][b] = sum_i U[i][a] X[i][b], written
+    out by hand (u_1 x_1^T + u_2 x_2^T); a transposed operand or swapped index changes it."""
+    U = np.array([[1.0, -2.0], [3.0, 4.0]])
+    X = np.array([[5.0, 0.0, -1.0], [2.0, 7.0, 1.0]])
+    # u_1 x_1^T = [[5, 0, -1], [-10, 0, 2]];  u_2 x_2^T = [[6, 21, 3], [8, 28, 4]]
+    want = np.array([[11.0, 21.0, 2.0], [-2.0, 28.0, 6.0]])
+    got = oracle.cache_apply(U, X)
+    assert got.shape == (2, 3) and np.array_equal(got, want)
+    # accumulation adds in place; a second call with the rows swapped gives the same sum
+    acc = want.copy()
+    oracle.cache_apply(U[::-1], X[::-1], acc)
+    assert np.array_equal(acc, 2 * want)
+
+
+def test_cache_apply_chunks_reproduce_full_batch_parameter_gradient(oracle):
+    """Eq. 8-9 through the oracle's own Step-3 routine: accumulating cache_apply over ragged
+    sub-batches gives dL/dW_f and dL/dW_g of the FULL batch, checked against central finite
+    differences of the full-batch loss with respect to the encoder matrices (tau != 1, so a
+    dropped 1/tau or 1/B anywhere between Step 2 and Step 3 shows)."""
+    rng = np.random.default_rng(68983)
+    B, N, din, d, tau = 7, 14, 6, 3, 0.7
+    Xs = rng.standard_normal((B, din))
+    Xt = rng.standard_normal((N, din))
+    Wf = rng.standard_normal((d, din)) * 0.4
+    Wg = rng.standard_normal((d, din)) * 0.4
+    pos = (2 * np.arange(B)).astype(np.int32)
+
+    def full_loss():
+        return oracle.loss_only(Xs @ Wf.T, Xt @ Wg.T, pos, tau, 0)
+
+    gWf = _fd_grad(full_loss, Wf)
+    gWg = _fd_grad(full_loss, Wg)
+    cache = oracle.build_cache(Xs @ Wf.T, Xt @ Wg.T, pos, tau, 0)
+    accWf = oracle.cache_apply(cache["dQ"][0:3], Xs[0:3])
+    for lo in (3, 5):
+        oracle.cache_apply(cache["dQ"][lo:lo + 2], Xs[lo:lo + 2], accWf)
+    accWg = oracle.cache_apply(cache["dP"][0:9], Xt[0:9])
+    oracle.cache_apply(cache["dP"][9:], Xt[9:], accWg)
+    assert np.abs(accWf - gWf).max() <= 1e-7 * max(1.0, np.abs(gWf).max())
+    assert np.abs(accWg - gWg).max() <= 1e-7 * max(1.0, np.abs(gWg).max())
+    # one call over the whole batch is the same sum
+    np.testing.assert_allclose(oracle.cache_apply(cache["dQ"], Xs), accWf, rtol=1e-12, atol=1e-15)
