@@ -377,6 +377,62 @@ def run_ours(args, rank, local_rank, world):
         dist.destroy_process_group()
 
 
+def run_apply(args):
+    """Side measurement (not the headline metric): gc_cache_apply, Step 3 for a linear encoder,
+    dW (+)= U^T X over one sub-batch of --apply-rows rows with d = d_in = 768.  HBM-bound by its
+    algorithmic bytes (U fp32 and X bf16 read once, dW fp32 written once)."""
+    import numpy as np
+    import torch
+    from paper_2101_06983_b200 import binding, inputs
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    rows, d, d_in = args.apply_rows, 768, 768
+    U = inputs.cache_rows(rows, d, seed=1)
+    xbits, X = inputs.encoder_inputs(rows, d_in, seed=2)
+    dU = torch.from_numpy(U).cuda()
+    dX = torch.from_numpy(xbits.view(np.int16)).view(torch.bfloat16).cuda()
+    dW = torch.empty(d, d_in, device="cuda")
+    ws = torch.empty(binding.gc_cache_apply_workspace_bytes(rows, d, d_in), dtype=torch.uint8,
+                     device="cuda")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    for _ in range(max(args.warmup, 3)):
+        flush.fill_(1)
+        binding.gc_cache_apply(dU, dX, dW, False, ws)
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+          for _ in range(args.steps)]
+    for a, b in ev:
+        flush.fill_(1)
+        a.record()
+        binding.gc_cache_apply(dU, dX, dW, False, ws)
+        b.record()
+    torch.cuda.synchronize()
+    ms = sum(a.elapsed_time(b) for a, b in ev) / args.steps
+    pk = load_peaks()
+    nbytes = 4.0 * rows * d + 2.0 * rows * d_in + 4.0 * d * d_in
+    import oracle
+    t0 = time.perf_counter()
+    ref = oracle.cache_apply(U, X)
+    dt = time.perf_counter() - t0
+    err = float(np.abs(dW.cpu().numpy() - ref).max() / np.abs(ref).max())
+    line = {
+        "metric": f"gc_cache_apply rows/s at rows={rows},d={d},d_in={d_in}", "value": rows / (ms * 1e-3),
+        "unit": "rows/s", "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms, "higher_is_better": True, "dtype": "bf16 x (bf16 + bf16), fp32 accumulate",
+        "data": "synthetic",
+        "config": {"workload": f"apply_rows{rows}_d{d}_din{d_in}",
+                   "l2": "flushed before every timed step (256 MiB write)"},
+        "tflops": 2.0 * rows * d * d_in / (ms * 1e-3) / 1e12,
+        "roofline": {"bound": "hbm", "achieved": nbytes / (ms * 1e-3) / 1e9, "peak": pk["hbm"],
+                     "unit": "GB/s", "frac": nbytes / (ms * 1e-3) / 1e9 / pk["hbm"],
+                     "peak_source": pk["source"], "traffic": None},
+        "cpu_baseline": {"value": rows / dt, "unit": "rows/s", "cores": oracle.num_threads(),
+                         "kind": "oracle", "sample": "the same sub-batch, one pass, double precision"},
+        "max_err_vs_oracle": err, "gpu_launches": 3 * args.steps,
+    }
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -392,7 +448,15 @@ def main():
                     help="recompute: gc_build_cache (nothing of size B x N leaves the chip); "
                          "stored: gc_build_cache_stored, the comparison plan that keeps the "
                          "B x N bf16 weights in the workspace")
+    ap.add_argument("--op", default="build", choices=["build", "apply"],
+                    help="build: gc_build_cache, the headline; apply: the side measurement of "
+                         "gc_cache_apply (one GPU)")
+    ap.add_argument("--apply-rows", type=int, default=4096)
     args = ap.parse_args()
+    if args.op == "apply":
+        if int(os.environ.get("RANK", "0")) == 0:
+            run_apply(args)
+        return
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))

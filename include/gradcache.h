@@ -130,6 +130,32 @@ int gc_build_cache_stored(const void* Q, int64_t ldq, const void* P, int64_t ldp
                           void* ws, size_t ws_bytes, int* dev_status, void* cuda_stream);
 
 /*
+ * Step 3 of Section 3.3 (Eq. 8 for f, Eq. 9 for g) for a linear encoder f(s) = W s: the cached
+ * representation gradients u_i of one sub-batch are propagated to the encoder matrix,
+ *
+ *     dW[a][b] (+)= sum_i U[i][a] * X[i][b],     a < d, b < d_in,
+ *
+ * the term d f(s_i)/dW applied to u_i being the outer product u_i s_i^T.  Summed over the
+ * sub-batches this is the full-batch gradient dL/dW (the equality the paper states after Eq. 9).
+ *   U      [rows x d] float, leading dimension ldu: a row range of dQ (or dP) as gc_build_cache
+ *          wrote it; pass the pointer to its first row.
+ *   X      [rows x d_in] bf16 (x_dtype = GC_BF16; anything else is GC_ERR_DTYPE), leading
+ *          dimension ldx: the encoder inputs s_i of the same rows.
+ *   dW     [d x d_in] float, leading dimension lddw.  accumulate == 0 overwrites it (first
+ *          sub-batch), otherwise the sub-batch's sum is added to it (outer sum of Eq. 8).
+ * Each u is used as the sum of two bf16 terms (its rounding and the rounding of the remainder,
+ * together exact to 2^-17 |u|), products are exact and accumulation is fp32 on the tensor cores.
+ * Limits: d a multiple of 8, d_in a multiple of 64 and at most 4096 (else GC_ERR_LIMIT); rows of
+ * U, X and dW start on 16-byte boundaries.  Workspace: gc_cache_apply_workspace_bytes (0 for
+ * sizes outside the limits), 256-byte aligned, caller-owned.  Asynchronous on cuda_stream;
+ * deterministic; GC_DEV_WAIT_LIMIT in *dev_status (may be NULL) as for the other calls.
+ */
+size_t gc_cache_apply_workspace_bytes(int64_t rows, int d, int d_in);
+int gc_cache_apply(const float* U, int64_t ldu, const void* X, int64_t ldx, int64_t rows, int d,
+                   int d_in, int x_dtype, float* dW, int64_t lddw, int accumulate,
+                   void* ws, size_t ws_bytes, int* dev_status, void* cuda_stream);
+
+/*
  * Forward with library-owned scratch (no counterpart in the paper: it exists for the sake of
  * callers, not of the method).  Same inputs, outputs and results as gc_loss_fwd, but the caller
  * passes no workspace.  It is meant for callers that cannot obtain device memory at the point of

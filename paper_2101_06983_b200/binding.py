@@ -21,7 +21,8 @@ GC_DEV_POS_RANGE, GC_DEV_POS_MASKED, GC_DEV_WAIT_LIMIT = 1, 2, 4
 EXPORTS = ("gc_workspace_bytes", "gc_plan_name", "gc_kernel_launches", "gc_loss_fwd",
            "gc_loss_bwd", "gc_build_cache", "gc_build_cache_stored", "gc_status_string",
            "gc_profile_enable",
-           "gc_profile_read", "gc_static_scratch_need", "gc_loss_fwd_static")
+           "gc_profile_read", "gc_static_scratch_need", "gc_loss_fwd_static",
+           "gc_cache_apply_workspace_bytes", "gc_cache_apply")
 GC_STATIC_SCRATCH_BYTES = 2 << 20
 
 
@@ -61,6 +62,11 @@ def _load() -> ctypes.CDLL:
     lib.gc_static_scratch_need.argtypes = [i64, i64, i32, i32]
     lib.gc_loss_fwd_static.restype = i32
     lib.gc_loss_fwd_static.argtypes = common + [vp, vp, vp, vp, vp]
+    lib.gc_cache_apply_workspace_bytes.restype = ctypes.c_size_t
+    lib.gc_cache_apply_workspace_bytes.argtypes = [i64, i32, i32]
+    lib.gc_cache_apply.restype = i32
+    lib.gc_cache_apply.argtypes = [vp, i64, vp, i64, i64, i32, i32, i32, vp, i64, i32, vp,
+                                   ctypes.c_size_t, vp, vp]
     lib.gc_profile_enable.restype = i32
     lib.gc_profile_enable.argtypes = [i32]
     lib.gc_profile_read.restype = i32
@@ -190,6 +196,32 @@ def gc_build_cache_stored(Q, P, pos_idx, tau, mask_mode, loss, row_lse, dQ, dP, 
                                     _ptr(dev_status), _stream())
     if rc != 0:
         raise GradCacheError(rc, "gc_build_cache_stored")
+
+
+def gc_cache_apply_workspace_bytes(rows: int, d: int, d_in: int) -> int:
+    return int(_lib.gc_cache_apply_workspace_bytes(rows, d, d_in))
+
+
+def gc_cache_apply(U, X, dW, accumulate: bool, ws=None, dev_status=None):
+    """Step 3 for a linear encoder (Eq. 8-9): dW[d x d_in] (+)= U^T X with U [rows x d] float32
+    (rows of the cache) and X [rows x d_in] bfloat16 (the same rows' encoder inputs)."""
+    if U.dim() != 2 or X.dim() != 2 or dW.dim() != 2 or U.stride(1) != 1 or X.stride(1) != 1 \
+            or dW.stride(1) != 1:
+        raise ValueError("U, X and dW must be 2-D with unit stride along their rows")
+    if U.dtype != torch.float32 or dW.dtype != torch.float32:
+        raise TypeError("U and dW must be float32")
+    rows, d = U.shape
+    d_in = X.shape[1]
+    if X.shape[0] != rows or tuple(dW.shape) != (d, d_in):
+        raise ValueError("shape mismatch")
+    if ws is None:
+        ws = torch.empty(max(gc_cache_apply_workspace_bytes(rows, d, d_in), 256),
+                         dtype=torch.uint8, device=U.device)
+    rc = _lib.gc_cache_apply(_ptr(U), U.stride(0), _ptr(X), X.stride(0), rows, d, d_in,
+                             _dtype_code(X), _ptr(dW), dW.stride(0), 1 if accumulate else 0,
+                             _ptr(ws), ws.numel(), _ptr(dev_status), _stream())
+    if rc != 0:
+        raise GradCacheError(rc, "gc_cache_apply")
 
 
 def gc_profile_enable(on: bool) -> None:

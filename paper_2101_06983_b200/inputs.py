@@ -173,3 +173,19 @@ def config(index: int) -> Problem:
     if index == 4:
         return dpr_batch(65536, 768, "bf16", s, name="cfg4_B65536_N131072_d768_bf16")
     raise ValueError("config index must be 0..4")
+
+
+def encoder_inputs(rows: int, d_in: int, seed: int = 0, sigma: float = 1.0):
+    """Stand-in for the inputs s_i of a linear encoder (Step 3, Eq. 8-9): a [rows x d_in] matrix
+    of N(0, sigma^2) values rounded to bf16.  Returns (uint16 bit patterns, float32 values)."""
+    return bf16_round(_normal(_rng(BASE_SEED + 1000 + seed), (rows, d_in), sigma))
+
+
+def cache_rows(rows: int, d: int, seed: int = 0, spread: float = 4.0) -> np.ndarray:
+    """Stand-in for rows of a representation gradient cache: float32 values of mixed sign whose
+    magnitudes span about 2^(+-spread) around 1/rows (a few rows carry most of the gradient, as
+    after a softmax), so that a sloppy low-precision product would show."""
+    rng = _rng(BASE_SEED + 2000 + seed)
+    mag = np.exp2(rng.uniform(-spread, spread, size=(rows, 1)).astype(np.float32))
+    u = rng.standard_normal(size=(rows, d), dtype=np.float32) * mag / np.float32(rows)
+    return np.ascontiguousarray(u, dtype=np.float32)
