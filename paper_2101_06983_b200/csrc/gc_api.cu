@@ -43,26 +43,32 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored) {
         pl.g_dp = simt_sweep_groups(N, B, d);
     }
     pl.fused = (pl.tc && tc_fused_applicable(d)) ? 1 : 0;
-    pl.anchored = (pl.fused && quad_applicable(B, d)) ? 1 : 0;
+    // 1: four-CTA sweeps (rows of two column halves); 2: narrow rows (two S buffers)
+    pl.anchored = (pl.fused && quad_applicable(B, d)) ? 1
+                  : (pl.tc && !pl.fused && tc_anchor_applicable(d)) ? 2 : 0;
     size_t dpad = (size_t)((d + 3) & ~3);
     // (max, sum) slots: the forward sweep writes g_fwd of them per row, the fused sweep 2 g_dq,
     // the anchored fused sweep 4 g_dq
     size_t slots = (size_t)pl.g_fwd;
     if (pl.fused && (size_t)(2 * pl.g_dq) > slots) slots = (size_t)(2 * pl.g_dq);
-    if (pl.anchored && (size_t)(4 * pl.g_dq) > slots) slots = (size_t)(4 * pl.g_dq);
+    if (pl.anchored == 1 && (size_t)(4 * pl.g_dq) > slots) slots = (size_t)(4 * pl.g_dq);
+    if (pl.anchored == 2 && (size_t)(2 * pl.g_dq) > slots) slots = (size_t)(2 * pl.g_dq);
     size_t off = 0;
     pl.off_m = off;    off += align256(sizeof(float) * slots * (size_t)B);
     pl.off_l = off;    off += align256(sizeof(float) * slots * (size_t)B);
     pl.off_pos = off;  off += align256(sizeof(float) * (size_t)B);
     pl.off_red = off;  off += 2048;      // loss reduction: block ticket + up to 256 block sums
     pl.off_accq = off;
-    if (pl.g_dq > 1 || pl.fused) off += align256(sizeof(float) * (size_t)pl.g_dq * (size_t)B * dpad);
+    if (pl.g_dq > 1 || pl.fused || pl.anchored) off += align256(sizeof(float) * (size_t)pl.g_dq * (size_t)B * dpad);
     pl.off_accp = off;
     if (pl.g_dp > 1) off += align256(sizeof(float) * (size_t)pl.g_dp * (size_t)N * dpad);
     pl.launches_fwd = 2;  // sweep + combine
     pl.launches_bwd = 2 + (pl.g_dq > 1 ? 1 : 0) + (pl.g_dp > 1 ? 1 : 0);
     pl.launches_build = pl.fused ? 4 + (pl.g_dp > 1 ? 1 : 0) : pl.launches_fwd + pl.launches_bwd;
-    if (pl.anchored) pl.launches_build = 1 + 2 * pl.launches_build;   // anchor, sequence, fallback
+    if (pl.anchored == 1) pl.launches_build = 1 + 2 * pl.launches_build;   // anchor, sequence, fallback
+    // anchor, fused sweep, combine, finalize, dP sweep (+ reduce), then the gated forward + sweeps
+    if (pl.anchored == 2)
+        pl.launches_build = 5 + (pl.g_dp > 1 ? 1 : 0) + pl.launches_fwd + pl.launches_bwd;
     // Stored weights: B x N bf16 (pitch rounded up to 64 elements), kept when they fit the limit
     // below; the gradient partials share the regions of the sweeps they replace.
     if (pl.anchored) {
@@ -318,16 +324,17 @@ SideStream* side_stream() {
 //                     of its streamed queries itself
 //   side stream:      after the fused sweep: combine (row_lse, loss), dQ finalize, then the
 //                     gated online-maximum sequence
-// Both are joined back before the call returns.  Without a side stream, or when the dP sweep is
-// not a four-CTA sweep (N <= 128), everything is queued on the caller's stream in dependency
-// order with the combine before the dP sweep.
+// Both are joined back before the call returns.  Without a side stream everything is queued on
+// the caller's stream in dependency order with the combine before the dP sweep.  Narrow rows
+// (two S buffers in tensor memory) take the same sequence with the one-CTA sweeps, and forward,
+// dQ and dP sweeps as the gated fallback.
 int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_lse,
                        float* pos_logit, float* dQ, int64_t lddq, float* dP, int64_t lddp,
                        int* dev_status, cudaStream_t st) {
     float* ref2 = reinterpret_cast<float*>(ws + pl.off_ref);
     int* flag = reinterpret_cast<int*>(ws + pl.off_flag);
     const Gate in_range = {flag, 0}, out_of_range = {flag, 1};
-    SideStream* side = quad_applicable(p.N, p.d) ? side_stream() : nullptr;
+    SideStream* side = side_stream();
     cudaStream_t aux = side ? side->st : st;
     cudaError_t e = launch_pos_anchor(p.Q, p.ldq, p.P, p.ldp, p.pos_idx, p.B, p.N, p.d, p.mask_mode,
                                       1.4426950408889634f / p.tau, ref2, flag, st);
@@ -338,20 +345,30 @@ int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, 
     fa.part_l = reinterpret_cast<float*>(ws + pl.off_l);
     fa.pos_logit = reinterpret_cast<float*>(ws + pl.off_pos);
     fa.red = reinterpret_cast<float*>(ws + pl.off_red);
-    fa.groups = 4 * pl.g_dq;
+    fa.groups = (pl.anchored == 1 ? 4 : 2) * pl.g_dq;
     fa.dev_status = dev_status;
     float* partial = reinterpret_cast<float*>(ws + pl.off_accq);
     {
         KernelTimer t(1, st);
-        e = quad_launch_fused_dq(fa, partial, pl.g_dq, ref2, flag, st);
+        e = pl.anchored == 1 ? quad_launch_fused_dq(fa, partial, pl.g_dq, ref2, flag, st)
+                             : tc_launch_anchored_dq(fa, partial, pl.g_dq, ref2, flag, st);
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
-    if (side && (cudaEventRecord(side->ev[0], st) != cudaSuccess ||
-                 cudaStreamWaitEvent(aux, side->ev[0], 0) != cudaSuccess))
+    // Wide rows: a sweep step is long enough to hide the slot merge of the streamed queries,
+    // so the dP sweep does not wait for the combine.  Narrow rows have short steps: there the
+    // combine stays on the caller's stream and the dP sweep reads row_lse.
+    const bool dp_merges = side && pl.anchored == 1;
+    cudaStream_t comb = dp_merges ? aux : st;
+    if (dp_merges && (cudaEventRecord(side->ev[0], st) != cudaSuccess ||
+                      cudaStreamWaitEvent(aux, side->ev[0], 0) != cudaSuccess))
         return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, in_range, aux);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, in_range,
+                           comb);
     if (e != cudaSuccess) return GC_ERR_CUDA;
+    if (side && !dp_merges && (cudaEventRecord(side->ev[0], st) != cudaSuccess ||
+                               cudaStreamWaitEvent(aux, side->ev[0], 0) != cudaSuccess))
+        return GC_ERR_CUDA;
     e = launch_fused_dq_finalize(partial, pl.g_dq, nullptr, ref2, row_lse, fa.pos_logit, p.pos_idx,
                                  p.P, p.ldp, p.B, p.N, p.d, p.mask_mode,
                                  1.f / ((float)p.B * p.tau), dQ, lddq, in_range, aux);
@@ -361,10 +378,12 @@ int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, 
         if ((rc = run_online_sweeps(p, pl, ws, loss, row_lse, pos_logit, dQ, lddq, dP, lddp,
                                     dev_status, aux, out_of_range)))
             return rc;
-        // the dP sweep does not wait for the combine: it merges the slots it needs itself
-        if ((rc = run_sweep(p, pl, ws, SWEEP_DP, row_lse, dP, lddp, dev_status, st, in_range, true,
-                            fa.part_m, fa.part_l, fa.groups)))
-            return rc;
+        if (dp_merges)
+            rc = run_sweep(p, pl, ws, SWEEP_DP, row_lse, dP, lddp, dev_status, st, in_range, true,
+                           fa.part_m, fa.part_l, fa.groups);
+        else
+            rc = run_sweep(p, pl, ws, SWEEP_DP, row_lse, dP, lddp, dev_status, st, in_range);
+        if (rc) return rc;
         if (cudaEventRecord(side->ev[2], aux) != cudaSuccess ||
             cudaStreamWaitEvent(st, side->ev[2], 0) != cudaSuccess)
             return GC_ERR_CUDA;

@@ -75,7 +75,7 @@ struct SweepArgs {
     int groups;             // the y range is split into this many contiguous parts
     int* dev_status;        // may be NULL
     Gate gate;
-    // SWEEP_DP of the four-CTA kernels only: when slot_l is set, row_lse is not read; the
+    // SWEEP_DP of the tensor-core kernels only: when slot_l is set, row_lse is not read; the
     // logsumexp of each streamed query is merged from these forward slots ([slots][ny]) instead.
     const float* slot_m;
     const float* slot_l;
@@ -154,6 +154,9 @@ cudaError_t tc_launch_fwd(const FwdArgs& a, cudaStream_t st);
 cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st);
 int tc_fwd_groups(int64_t B, int64_t N, int d);
 bool tc_fused_applicable(int d);
+bool tc_anchor_applicable(int d);
+cudaError_t tc_launch_anchored_dq(const FwdArgs& a, float* partial, int groups,
+                                  const float* row_ref, int* range_flag, cudaStream_t st);
 cudaError_t tc_launch_fused_dq(const FwdArgs& a, float* partial, int groups, cudaStream_t st);
 int tc_sweep_groups(int64_t nx, int64_t ny, int d);
 cudaError_t tc_launch_fwd_store(const FwdArgs& a, void* weights, int64_t ldw, const float* row_ref,

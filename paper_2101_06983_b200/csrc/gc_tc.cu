@@ -10,6 +10,11 @@
 //                   m_ref) with the positive column left out, acc += W Y; the accumulator is
 //                   rescaled only when the maximum grows by more than 2^8.  A finalize pass forms
 //                   (sum_g acc_g exp(m_g - lse) + (p_pos - 1) P_pos) / (B tau), positive term in fp32.
+//   DA   (Eq. 1+5)  forward fused into the dQ sweep with a scale fixed before the sweep: W =
+//                   2^(s2 - ref2_x), ref2_x = the row's positive logit (anchor kernel), positive
+//                   column left out, row sums kept per part; used for rows narrow enough for two S
+//                   buffers, where no running maximum has to be tracked.  Weights beyond 2^100
+//                   raise a flag that hands the call to FWD + DQ + DP.
 //   FS   (Eq. 1)    forward that also stores the bf16 weights 2^(s2 - ref2_x) of all pairs (the
 //                   stored-weights comparison plan).
 //
@@ -37,14 +42,14 @@ namespace gc {
 namespace {
 
 // FQ: forward fused into dQ; FS: forward that also stores the bf16 weights
-enum { MODE_FWD = 0, MODE_DQ = 1, MODE_DP = 2, MODE_FQ = 3, MODE_FS = 4 };
+enum { MODE_FWD = 0, MODE_DQ = 1, MODE_DP = 2, MODE_FQ = 3, MODE_FS = 4, MODE_DA = 5 };
 
 // Optional diagnostics (-DGC_TC_TRACE): cycles each role spends waiting, summed over CTAs.
 #ifdef GC_TC_TRACE
 enum { TR_MMA_TOTAL, TR_MMA_WAIT_Y, TR_MMA_WAIT_W, TR_SM_TOTAL, TR_SM_WAIT_S, TR_SM_EPI,
        TR_PROD_TOTAL, TR_PROD_WAIT, TR_CTAS, TR_MMA_ISSUE, TR_MMA_COMMIT, TR_ACC_ISSUE, TR_ACC_COMMIT, TR_SFULL_COMMIT,
        TR_CTA_LIFE, TR_SETUP, TR_T0_MIN, TR_T0_MAX, TR_T1_MIN, TR_T1_MAX, TR_COUNT };
-__device__ unsigned long long g_trace[5][TR_COUNT];
+__device__ unsigned long long g_trace[6][TR_COUNT];
 #define TR_DECL(v) long long v = 0
 #define TR_BEGIN(v) long long v##_t0 = clock64()
 #define TR_END(v) v += clock64() - v##_t0
@@ -94,8 +99,11 @@ struct TcParams {
     float* part_l;
     float* pos_logit;
     int* dev_status;
-    const float* row_ref;     // FS: per-query anchor of the stored weights, log2 domain
-    int* range_flag;          // FS: set to 1 when a weight leaves the range the anchor allows
+    const float* row_ref;     // FS, DA: per-query anchor of the weights, log2 domain
+    int* range_flag;          // FS, DA: set to 1 when a weight leaves the range the anchor allows
+    const float* slot_m;      // DP with nslots > 0: forward slots [nslots][ny] to merge instead of
+    const float* slot_l;      //   reading row_lse
+    int nslots;
     Gate gate;                // closed: the kernel returns at once
     int* zero_me;             // forward sweeps: the ticket word of the reduction that follows
 };
@@ -134,7 +142,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     __shared__ float row_max_xch[2][XROWS];      // FQ: [column half][row] block maxima
     volatile int* abort_flag = &abort_s;
     if (gate_closed(p.gate)) return;            // same answer in every CTA
-    if ((MODE == MODE_FWD || MODE == MODE_FS || MODE == MODE_FQ) && blockIdx.x == 0 && threadIdx.x == 0 && p.zero_me) *p.zero_me = 0;
+    if ((MODE == MODE_FWD || MODE == MODE_FS || MODE == MODE_FQ || MODE == MODE_DA) && blockIdx.x == 0 && threadIdx.x == 0 && p.zero_me) *p.zero_me = 0;
 
     static_assert(SN == 128, "a Y chunk is 128 rows: the same 16 KB as an X chunk");
     constexpr uint32_t S_COL0 = TMEM_COLS - NBUF * SN;  // S buffers sit at the top columns
@@ -863,10 +871,10 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             TR_END(tr_epi);
         } else {
             // per-row constants (DQ: the row is a query)
-            float lse2_x = 0.f;
+            float lse2_x = 0.f, l_sum = 0.f, wmax = 0.f;
             int32_t pos_x = -1;
-            if (MODE == MODE_DQ && x < p.nx) {
-                lse2_x = p.row_lse[x] * 1.4426950408889634f;
+            if ((MODE == MODE_DQ || MODE == MODE_DA) && x < p.nx) {
+                lse2_x = (MODE == MODE_DA) ? p.row_ref[x] : p.row_lse[x] * 1.4426950408889634f;
                 pos_x = p.pos_idx[x];
             }
             for (int t = 0; t < T; ++t) {
@@ -879,7 +887,12 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
 #pragma unroll
                     for (int j = 0; j < CB_PER; ++j) {
                         const int64_t y = y0 + (cb0 + j) * 32 + lane;
-                        lse2_y[j] = (y < p.ny) ? p.row_lse[y] * 1.4426950408889634f : INFINITY;
+                        float lse_y = INFINITY;
+                        if (y < p.ny)
+                            lse_y = p.nslots > 0
+                                        ? combined_lse(p.slot_m, p.slot_l, p.nslots, p.ny, y)
+                                        : p.row_lse[y];
+                        lse2_y[j] = lse_y * 1.4426950408889634f;
                         pos_y[j] = (y < p.ny) ? p.pos_idx[y] : -1;
                     }
                 }
@@ -930,6 +943,46 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                             for (int c = 0; c < 32; ++c)
                                 if (yb + c >= p.ny) w[c] = 0.f;
                         }
+                    } else if (MODE == MODE_DA) {
+                        const bool has_pos = pos_x >= yb && pos_x < yb + 32 && pos_x < p.ny &&
+                                             !(self_mask && x == pos_x);
+                        if (has_pos) {
+                            const int rel = (int)(pos_x - yb);
+                            float sp = 0.f;
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (c == rel) sp = __uint_as_float(v[c]);
+                            p.pos_logit[x] = sp * p.inv_tau;
+                        }
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            w[c] = ex2(fmaf(__uint_as_float(v[c]), p.c1, -lse2_x));
+                        if (yb + 32 > p.ny) {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (yb + c >= p.ny) w[c] = 0.f;
+                        }
+                        if (self_mask && x >= yb && x < yb + 32) {
+                            const int rel = (int)(x - yb);
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (c == rel) w[c] = 0.f;
+                        }
+                        float s0 = 0.f, s1 = 0.f, m0 = 0.f;
+#pragma unroll
+                        for (int c = 0; c < 32; c += 2) {
+                            s0 += w[c];
+                            s1 += w[c + 1];
+                            m0 = fmaxf(m0, fmaxf(w[c], w[c + 1]));
+                        }
+                        l_sum += s0 + s1;
+                        wmax = fmaxf(wmax, m0);
+                        if (pos_x >= yb && pos_x < yb + 32) {      // positive: fp32, in the finalize
+                            const int rel = (int)(pos_x - yb);
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (c == rel) w[c] = 0.f;
+                        }
                     } else {
 #pragma unroll
                         for (int c = 0; c < 32; ++c) {
@@ -974,6 +1027,14 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 if (q == 0 && half == 0) EV(2, ev_s, 13, t);
             }
             if (q == 0 && half == 0) EV_END(2, ev_s);
+            if (MODE == MODE_DA && ok && x < p.nx) {
+                // one (scale, sum) slot per row, part of the streamed range and column half
+                const int64_t slot = (int64_t)(2 * g + half) * p.nq + x;
+                p.part_m[slot] = lse2_x * 0.69314718055994531f;
+                p.part_l[slot] = l_sum;
+                // weights beyond 2^100 (or not finite) cannot be accumulated safely
+                if (!(wmax <= 1.2676506e30f)) *p.range_flag = 1;
+            }
             // epilogue: accumulator columns of this part -> global memory (32-column blocks are
             // dealt alternately to the two warps of a lane quarter); final values are scaled,
             // partial sums of a split sweep are not
@@ -981,7 +1042,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             if (ok) ok = mbar_wait(smem_u32(&bars.acc_full), 0, abort_flag);
             if (ok) {
                 tc_fence_after();
-                const bool final_out = (p.groups == 1);
+                const bool final_out = (p.groups == 1) && MODE != MODE_DA;
                 const uint32_t slot = base + (uint32_t)(warp - (NPROD + 1)) * 8192u;
                 store_acc_blocks(tmem + lane_addr, c_count * 2, half, slot,
                                  final_out ? p.out_scale : 1.f, lane, &mapO, c_begin * 64,
@@ -1137,8 +1198,8 @@ extern "C" int gc_debug_evlog(unsigned int* out, int mode) {
 extern "C" int gc_debug_trace(unsigned long long* out, int clear) {
     if (out && cudaMemcpyFromSymbol(out, g_trace, sizeof(g_trace)) != cudaSuccess) return 1;
     if (clear) {
-        static unsigned long long zero[5][TR_COUNT] = {};
-        for (int m = 0; m < 5; ++m) zero[m][TR_T0_MIN] = zero[m][TR_T1_MIN] = ~0ull;
+        static unsigned long long zero[6][TR_COUNT] = {};
+        for (int m = 0; m < 6; ++m) zero[m][TR_T0_MIN] = zero[m][TR_T1_MIN] = ~0ull;
         if (cudaMemcpyToSymbol(g_trace, zero, sizeof(zero)) != cudaSuccess) return 1;
     }
     return 0;
@@ -1265,6 +1326,43 @@ cudaError_t tc_launch_fused_dq(const FwdArgs& a, float* partial, int groups, cud
     return launch<MODE_FQ, SN, 1>(mx, my, myh, mo, p, st);
 }
 
+bool tc_anchor_applicable(int d) { return sweep_nbuf(d / 64) == 2; }
+
+// Forward fused into the dQ sweep of narrow rows with row_ref (log2 domain) as each row's fixed
+// scale: writes (scale, sum) slots [2 groups][B] (scale = row_ref in natural-log units),
+// pos_logit and the unscaled accumulators partial[groups][B][d] of sum_j 2^(s2_ij - ref_i) P_j
+// over all allowed columns but the positive one; raises *range_flag when a weight exceeds 2^100.
+cudaError_t tc_launch_anchored_dq(const FwdArgs& a, float* partial, int groups,
+                                  const float* row_ref, int* range_flag, cudaStream_t st) {
+    const Problem& pr = a.p;
+    constexpr int SN = 128;
+    const int kc = pr.d / 64;
+    CUtensorMap mx, my, myh, mo;
+    if (!make_map(&mx, pr.Q, pr.B, pr.d, pr.ldq, XROWS) ||
+        !make_map(&my, pr.P, pr.N, pr.d, pr.ldp, SN) ||
+        !make_map(&myh, pr.P, pr.N, pr.d, pr.ldp, SN / 2) ||
+        !make_out_map(&mo, partial, pr.B, pr.d, pr.d, groups))
+        return cudaErrorInvalidValue;
+    TcParams p{};
+    p.nx = pr.B; p.ny = pr.N; p.nq = pr.B;
+    p.kc = kc; p.dparts = parts_for(kc); p.dpc = chunks_per_part(kc); p.groups = groups;
+    p.nstage = smem_plan(kc).nstage;
+    p.xres = smem_plan(kc).xres;
+    p.ipc = smem_plan(kc).ipc;
+    p.mask_mode = pr.mask_mode;
+    p.inv_tau = 1.f / pr.tau;
+    p.c1 = 1.4426950408889634f / pr.tau;
+    p.pos_idx = pr.pos_idx;
+    p.partial = partial;
+    p.part_m = a.part_m; p.part_l = a.part_l; p.pos_logit = a.pos_logit;
+    p.row_ref = row_ref;
+    p.range_flag = range_flag;
+    p.zero_me = reinterpret_cast<int*>(a.red);
+    p.dev_status = a.dev_status;
+    p.gate = a.gate;
+    return launch<MODE_DA, SN, 2>(mx, my, myh, mo, p, st);
+}
+
 cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     if (quad_applicable(a.nx, a.d)) return quad_launch_sweep(a, st);
     const int kc = a.d / 64;
@@ -1287,6 +1385,7 @@ cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     p.out = a.out; p.ldo = a.ldo; p.partial = a.partial;
     p.dev_status = a.dev_status;
     p.gate = a.gate;
+    if (a.mode == SWEEP_DP && a.slot_l) { p.slot_m = a.slot_m; p.slot_l = a.slot_l; p.nslots = a.slots; }
     CUtensorMap mo;
     const bool ok_map = a.groups == 1 ? make_out_map(&mo, a.out, a.nx, a.d, a.ldo, 1)
                                       : make_out_map(&mo, a.partial, a.nx, a.d, a.d, a.groups);
