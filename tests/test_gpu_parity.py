@@ -346,6 +346,32 @@ def test_bad_positives_are_flagged_not_fatal(binding, oracle):
     assert int(st.item()) == (binding.GC_DEV_POS_RANGE | binding.GC_DEV_POS_MASKED)
 
 
+@pytest.mark.parametrize("d", [128, 768])
+def test_bad_positives_with_a_fixed_row_scale(binding, oracle, d):
+    """The bf16 builds that scale each row's weights by its positive logit (narrow rows, and rows
+    of two column halves): a row whose pos_idx is unusable has no positive logit to scale by; it
+    is flagged, gets no one-hot term, and every other row still matches the oracle."""
+    B, N = 200, 300
+    prob = inputs.random_problem(B, N, d, "bf16", seed=31, tau=0.5, scale=d ** -0.5,
+                                 mask_mode=inputs.MASK_SELF)
+    pos = prob.pos_idx.copy()
+    pos[7] = N
+    pos[130] = -3
+    pos[150] = 150                                                  # the masked column
+    Q, P, _ = to_device(prob)
+    out = binding.build_cache(Q, P, torch.from_numpy(pos).cuda(), prob.tau, prob.mask_mode)
+    torch.cuda.synchronize()
+    assert int(out.dev_status.item()) == (binding.GC_DEV_POS_RANGE | binding.GC_DEV_POS_MASKED)
+    pl = out.pos_logit.cpu().numpy()
+    assert pl[7] == 0 and pl[130] == 0 and pl[150] == 0
+    good = np.array([i for i in range(B) if i not in (7, 130, 150)])
+    ref = oracle.query_rows(prob.Q, prob.P, prob.pos_idx, good, prob.tau, prob.mask_mode)
+    lse = out.row_lse.cpu().numpy()[good]
+    assert np.abs(lse - ref["row_lse"]).max() <= TOL["bf16"]["lse"] * np.abs(ref["row_lse"]).max()
+    assert grad_err(out.dQ[torch.from_numpy(good).cuda()].cpu().numpy(), ref["dQ"]) <= TOL["bf16"]["grad"]
+    assert bool(torch.isfinite(out.dQ).all()) and bool(torch.isfinite(out.dP).all())
+
+
 @pytest.mark.parametrize("index", [1, 2, 3])
 def test_deterministic(binding, index):
     prob = inputs.config(index)
