@@ -156,6 +156,40 @@ int gc_cache_apply(const float* U, int64_t ldu, const void* X, int64_t ldx, int6
                    void* ws, size_t ws_bytes, int* dev_status, void* cuda_stream);
 
 /*
+ * Section 3.4 (multi-GPU training): after the all-gather every GPU holds all representations,
+ * the loss is defined over all of them, and "the n-th GPU only computes gradient of its local
+ * representations".  These two calls are that rank-local part of Step 2 for a rank that owns
+ * query rows [q0, q0 + q_count) and passage rows [p0, p0 + p_count) of the gathered Q [B x d] and
+ * P [N x d] (pos_idx [B] indexes rows of the gathered P).  Unlike the paper's scheme a rank does
+ * not redo the whole forward: it needs lse_i of its own queries for dQ and, for dP, lse_i of all
+ * queries, which the ranks exchange between the two calls (B floats).
+ *
+ *   gc_shard_fwd_dq  forward (Eq. 1) and dQ (Eq. 5) of the local queries against all passages.
+ *       Writes row_lse[q0 .. q0 + q_count) (row_lse and pos_logit point at entry 0 of arrays of
+ *       length B), dQ [q_count x d], and *loss_part = (1/B) sum over the local queries of
+ *       (lse_i - S_{i,r_i}): the loss of Eq. 1 is the sum of loss_part over the ranks.
+ *   gc_shard_dp      dP (Eq. 6-7) of the local passages against all queries, given row_lse of
+ *       ALL B queries.  Writes dP [p_count x d].
+ *
+ * Both scale by 1/B with B the whole batch, so concatenating the ranks' dQ and dP gives exactly
+ * what gc_build_cache gives on one GPU (up to rounding order).  GC_MASK_NONE only (the paper's
+ * loss; anything else is GC_ERR_MASK); a range outside the matrices is GC_ERR_SHAPE.  Workspace:
+ * gc_shard_workspace_bytes, which covers either call.  The collectives are the caller's (the
+ * Python package's `sharded` module runs them with torch.distributed).
+ */
+size_t gc_shard_workspace_bytes(int64_t B, int64_t N, int d, int dtype, int64_t q_count,
+                                int64_t p_count);
+int gc_shard_fwd_dq(const void* Q, int64_t ldq, const void* P, int64_t ldp, const int32_t* pos_idx,
+                    int64_t B, int64_t N, int d, float tau, int mask_mode, int dtype,
+                    int64_t q0, int64_t q_count, float* loss_part, float* row_lse,
+                    float* pos_logit, float* dQ, int64_t lddq,
+                    void* ws, size_t ws_bytes, int* dev_status, void* cuda_stream);
+int gc_shard_dp(const void* Q, int64_t ldq, const void* P, int64_t ldp, const int32_t* pos_idx,
+                int64_t B, int64_t N, int d, float tau, int mask_mode, int dtype,
+                const float* row_lse, int64_t p0, int64_t p_count, float* dP, int64_t lddp,
+                void* ws, size_t ws_bytes, int* dev_status, void* cuda_stream);
+
+/*
  * Forward with library-owned scratch (no counterpart in the paper: it exists for the sake of
  * callers, not of the method).  Same inputs, outputs and results as gc_loss_fwd, but the caller
  * passes no workspace.  It is meant for callers that cannot obtain device memory at the point of

@@ -22,7 +22,8 @@ EXPORTS = ("gc_workspace_bytes", "gc_plan_name", "gc_kernel_launches", "gc_loss_
            "gc_loss_bwd", "gc_build_cache", "gc_build_cache_stored", "gc_status_string",
            "gc_profile_enable",
            "gc_profile_read", "gc_static_scratch_need", "gc_loss_fwd_static",
-           "gc_cache_apply_workspace_bytes", "gc_cache_apply")
+           "gc_cache_apply_workspace_bytes", "gc_cache_apply", "gc_shard_workspace_bytes",
+           "gc_shard_fwd_dq", "gc_shard_dp")
 GC_STATIC_SCRATCH_BYTES = 2 << 20
 
 
@@ -67,6 +68,13 @@ def _load() -> ctypes.CDLL:
     lib.gc_cache_apply.restype = i32
     lib.gc_cache_apply.argtypes = [vp, i64, vp, i64, i64, i32, i32, i32, vp, i64, i32, vp,
                                    ctypes.c_size_t, vp, vp]
+    lib.gc_shard_workspace_bytes.restype = ctypes.c_size_t
+    lib.gc_shard_workspace_bytes.argtypes = [i64, i64, i32, i32, i64, i64]
+    lib.gc_shard_fwd_dq.restype = i32
+    lib.gc_shard_fwd_dq.argtypes = common + [i64, i64, vp, vp, vp, vp, i64, vp, ctypes.c_size_t,
+                                             vp, vp]
+    lib.gc_shard_dp.restype = i32
+    lib.gc_shard_dp.argtypes = common + [vp, i64, i64, vp, i64, vp, ctypes.c_size_t, vp, vp]
     lib.gc_profile_enable.restype = i32
     lib.gc_profile_enable.argtypes = [i32]
     lib.gc_profile_read.restype = i32
@@ -222,6 +230,38 @@ def gc_cache_apply(U, X, dW, accumulate: bool, ws=None, dev_status=None):
                              _ptr(ws), ws.numel(), _ptr(dev_status), _stream())
     if rc != 0:
         raise GradCacheError(rc, "gc_cache_apply")
+
+
+def gc_shard_workspace_bytes(B: int, N: int, d: int, dtype: int, q_count: int, p_count: int) -> int:
+    return int(_lib.gc_shard_workspace_bytes(B, N, d, dtype, q_count, p_count))
+
+
+def gc_shard_fwd_dq(Q, P, pos_idx, tau, q0, q_count, loss_part, row_lse, dQ, pos_logit=None,
+                    ws=None, dev_status=None):
+    """Section 3.4, local queries [q0, q0 + q_count) of the gathered batch: writes their entries
+    of row_lse[B], dQ[q_count x d] and loss_part[1] (this rank's share of the loss of Eq. 1)."""
+    args, B, N, d, code = _common(Q, P, pos_idx, tau, GC_MASK_NONE)
+    if ws is None:
+        ws = torch.empty(max(gc_shard_workspace_bytes(B, N, d, code, q_count, N), 256),
+                         dtype=torch.uint8, device=Q.device)
+    rc = _lib.gc_shard_fwd_dq(*args, q0, q_count, _ptr(loss_part), _ptr(row_lse), _ptr(pos_logit),
+                              _ptr(dQ), dQ.stride(0), _ptr(ws), ws.numel(), _ptr(dev_status),
+                              _stream())
+    if rc != 0:
+        raise GradCacheError(rc, "gc_shard_fwd_dq")
+
+
+def gc_shard_dp(Q, P, pos_idx, tau, row_lse, p0, p_count, dP, ws=None, dev_status=None):
+    """Section 3.4, local passages [p0, p0 + p_count) of the gathered batch, given row_lse of all
+    B queries: writes dP[p_count x d]."""
+    args, B, N, d, code = _common(Q, P, pos_idx, tau, GC_MASK_NONE)
+    if ws is None:
+        ws = torch.empty(max(gc_shard_workspace_bytes(B, N, d, code, B, p_count), 256),
+                         dtype=torch.uint8, device=Q.device)
+    rc = _lib.gc_shard_dp(*args, _ptr(row_lse), p0, p_count, _ptr(dP), dP.stride(0), _ptr(ws),
+                          ws.numel(), _ptr(dev_status), _stream())
+    if rc != 0:
+        raise GradCacheError(rc, "gc_shard_dp")
 
 
 def gc_profile_enable(on: bool) -> None:

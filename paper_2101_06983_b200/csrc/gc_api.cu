@@ -173,10 +173,16 @@ Problem make_problem(const void* Q, int64_t ldq, const void* P, int64_t ldp,
     Problem p;
     p.Q = Q; p.P = P; p.pos_idx = pos_idx; p.ldq = ldq; p.ldp = ldp; p.B = B; p.N = N; p.d = d;
     p.tau = tau; p.mask_mode = mask_mode; p.dtype = dtype;
+    p.b_total = 0;
     return p;
 }
 
 constexpr Gate kOpen = {nullptr, 0};
+
+// 1 / (B tau) of Eq. 4-7, with B the whole batch when the call covers a slice of the queries
+float grad_scale(const Problem& p) {
+    return 1.f / ((float)(p.b_total > 0 ? p.b_total : p.B) * p.tau);
+}
 
 int run_fwd(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_lse,
             float* pos_logit, int* dev_status, cudaStream_t st, Gate gate = kOpen) {
@@ -196,7 +202,7 @@ int run_fwd(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, gate, st);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, gate, st, p.b_total);
     return e == cudaSuccess ? GC_OK : GC_ERR_CUDA;
 }
 
@@ -216,7 +222,7 @@ int run_sweep(const Problem& p, const Plan& pl, char* ws, int mode, const float*
     sa.mask_mode = p.mask_mode;
     sa.dtype = p.dtype;
     sa.inv_tau = 1.f / p.tau;
-    sa.out_scale = 1.f / ((float)p.B * p.tau);
+    sa.out_scale = grad_scale(p);
     sa.row_lse = row_lse;
     sa.pos_idx = p.pos_idx;
     sa.out = out;
@@ -259,11 +265,11 @@ int run_fused_fwd_dq(const Problem& p, const Plan& pl, char* ws, float* loss, fl
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, gate, st);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, gate, st, p.b_total);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_fused_dq_finalize(partial, pl.g_dq, fa.part_m, nullptr, row_lse, fa.pos_logit,
                                  p.pos_idx, p.P, p.ldp, p.B, p.N, p.d, p.mask_mode,
-                                 1.f / ((float)p.B * p.tau), dQ, lddq, gate, st);
+                                 grad_scale(p), dQ, lddq, gate, st);
     return e == cudaSuccess ? GC_OK : GC_ERR_CUDA;
 }
 
@@ -271,7 +277,7 @@ int run_fused_fwd_dq(const Problem& p, const Plan& pl, char* ws, float* loss, fl
 // rows), dQ, dP.  With a gate every kernel of it is gated.
 int run_online_sweeps(const Problem& p, const Plan& pl, char* w, float* loss, float* row_lse,
                       float* pos_logit, float* dQ, int64_t lddq, float* dP, int64_t lddp,
-                      int* dev_status, cudaStream_t st, Gate gate = kOpen) {
+                      int* dev_status, cudaStream_t st, Gate gate = kOpen, bool want_dp = true) {
     int rc;
     if (pl.fused) {
         if ((rc = run_fused_fwd_dq(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dev_status, st,
@@ -283,6 +289,7 @@ int run_online_sweeps(const Problem& p, const Plan& pl, char* w, float* loss, fl
                             gate.flag == nullptr)))
             return rc;
     }
+    if (!want_dp) return GC_OK;
     return run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, dev_status, st, gate,
                      gate.flag == nullptr);
 }
@@ -330,7 +337,7 @@ SideStream* side_stream() {
 // dQ and dP sweeps as the gated fallback.
 int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_lse,
                        float* pos_logit, float* dQ, int64_t lddq, float* dP, int64_t lddp,
-                       int* dev_status, cudaStream_t st) {
+                       int* dev_status, cudaStream_t st, bool want_dp = true) {
     float* ref2 = reinterpret_cast<float*>(ws + pl.off_ref);
     int* flag = reinterpret_cast<int*>(ws + pl.off_flag);
     const Gate in_range = {flag, 0}, out_of_range = {flag, 1};
@@ -357,31 +364,30 @@ int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, 
     // Wide rows: a sweep step is long enough to hide the slot merge of the streamed queries,
     // so the dP sweep does not wait for the combine.  Narrow rows have short steps: there the
     // combine stays on the caller's stream and the dP sweep reads row_lse.
-    const bool dp_merges = side && pl.anchored == 1;
+    const bool dp_merges = side && pl.anchored == 1 && want_dp;
     cudaStream_t comb = dp_merges ? aux : st;
     if (dp_merges && (cudaEventRecord(side->ev[0], st) != cudaSuccess ||
                       cudaStreamWaitEvent(aux, side->ev[0], 0) != cudaSuccess))
         return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, in_range,
-                           comb);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, in_range, comb, p.b_total);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     if (side && !dp_merges && (cudaEventRecord(side->ev[0], st) != cudaSuccess ||
                                cudaStreamWaitEvent(aux, side->ev[0], 0) != cudaSuccess))
         return GC_ERR_CUDA;
     e = launch_fused_dq_finalize(partial, pl.g_dq, nullptr, ref2, row_lse, fa.pos_logit, p.pos_idx,
                                  p.P, p.ldp, p.B, p.N, p.d, p.mask_mode,
-                                 1.f / ((float)p.B * p.tau), dQ, lddq, in_range, aux);
+                                 grad_scale(p), dQ, lddq, in_range, aux);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     int rc;
     if (side) {
         if ((rc = run_online_sweeps(p, pl, ws, loss, row_lse, pos_logit, dQ, lddq, dP, lddp,
-                                    dev_status, aux, out_of_range)))
+                                    dev_status, aux, out_of_range, want_dp)))
             return rc;
         if (dp_merges)
             rc = run_sweep(p, pl, ws, SWEEP_DP, row_lse, dP, lddp, dev_status, st, in_range, true,
                            fa.part_m, fa.part_l, fa.groups);
-        else
+        else if (want_dp)
             rc = run_sweep(p, pl, ws, SWEEP_DP, row_lse, dP, lddp, dev_status, st, in_range);
         if (rc) return rc;
         if (cudaEventRecord(side->ev[2], aux) != cudaSuccess ||
@@ -389,18 +395,21 @@ int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, 
             return GC_ERR_CUDA;
         return GC_OK;
     }
-    if ((rc = run_sweep(p, pl, ws, SWEEP_DP, row_lse, dP, lddp, dev_status, st, in_range))) return rc;
+    if (want_dp &&
+        (rc = run_sweep(p, pl, ws, SWEEP_DP, row_lse, dP, lddp, dev_status, st, in_range)))
+        return rc;
     return run_online_sweeps(p, pl, ws, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status, st,
-                             out_of_range);
+                             out_of_range, want_dp);
 }
 
 int run_build_sweeps(const Problem& p, const Plan& pl, char* w, float* loss, float* row_lse,
                      float* pos_logit, float* dQ, int64_t lddq, float* dP, int64_t lddp,
-                     int* dev_status, cudaStream_t st) {
+                     int* dev_status, cudaStream_t st, bool want_dp = true) {
     if (pl.anchored)
         return run_anchored_build(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status,
-                                  st);
-    return run_online_sweeps(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status, st);
+                                  st, want_dp);
+    return run_online_sweeps(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status, st,
+                             kOpen, want_dp);
 }
 
 // gc_build_cache with stored weights (Eq. 1, 5, 6-7 without recomputing a logit):
@@ -422,7 +431,7 @@ int run_build_stored(const Problem& p, const Plan& pl, char* w, float* loss, flo
     void* weights = w + pl.off_w;
     float* partq = reinterpret_cast<float*>(w + pl.off_accq);
     float* partp = reinterpret_cast<float*>(w + pl.off_accp);
-    const float scale = 1.f / ((float)p.B * p.tau);
+    const float scale = grad_scale(p);
     cudaError_t e = launch_pos_anchor(p.Q, p.ldq, p.P, p.ldp, p.pos_idx, p.B, p.N, p.d, p.mask_mode,
                                       1.4426950408889634f / p.tau, ref2, flag, st);
     if (e != cudaSuccess) return GC_ERR_CUDA;
@@ -440,7 +449,7 @@ int run_build_stored(const Problem& p, const Plan& pl, char* w, float* loss, flo
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, kOpen, st);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, kOpen, st, p.b_total);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_scale_rows(p.Q, p.ldq, p.B, p.d, ref2, row_lse, qs, st);
     if (e != cudaSuccess) return GC_ERR_CUDA;
@@ -625,6 +634,63 @@ int gc_build_cache_stored(const void* Q, int64_t ldq, const void* P, int64_t ldp
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
     return run_build_stored(p, pl, static_cast<char*>(ws), loss, row_lse, pos_logit, dQ, lddq, dP,
                             lddp, dev_status, st);
+}
+
+size_t gc_shard_workspace_bytes(int64_t B, int64_t N, int d, int dtype, int64_t q_count,
+                                int64_t p_count) {
+    if (B <= 0 || N <= 0 || d <= 0 || q_count <= 0 || p_count <= 0 || q_count > B || p_count > N)
+        return 0;
+    if (dtype != GC_F32 && dtype != GC_BF16) return 0;
+    const size_t a = make_plan(q_count, N, d, dtype).total;
+    const size_t b = make_plan(B, p_count, d, dtype).total + align256(sizeof(int32_t) * (size_t)B);
+    return a > b ? a : b;
+}
+
+int gc_shard_fwd_dq(const void* Q, int64_t ldq, const void* P, int64_t ldp, const int32_t* pos_idx,
+                    int64_t B, int64_t N, int d, float tau, int mask_mode, int dtype, int64_t q0,
+                    int64_t q_count, float* loss_part, float* row_lse, float* pos_logit, float* dQ,
+                    int64_t lddq, void* ws, size_t ws_bytes, int* dev_status, void* cuda_stream) {
+    int rc = check_common(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
+    if (rc) return rc;
+    if (mask_mode != GC_MASK_NONE) return GC_ERR_MASK;
+    if (q0 < 0 || q_count <= 0 || q0 + q_count > B) return GC_ERR_SHAPE;
+    if (!loss_part || !row_lse || !dQ) return GC_ERR_NULL;
+    if ((rc = check_grad_out(dQ, lddq, d))) return rc;
+    Plan pl = make_plan(q_count, N, d, dtype);
+    if ((rc = check_ws(ws, ws_bytes, pl.total))) return rc;
+    if ((rc = check_device())) return rc;
+    const char* q_first = static_cast<const char*>(Q) + (size_t)q0 * (size_t)ldq * elem_size(dtype);
+    Problem p = make_problem(q_first, ldq, P, ldp, pos_idx + q0, q_count, N, d, tau, mask_mode, dtype);
+    p.b_total = B;
+    return run_build_sweeps(p, pl, static_cast<char*>(ws), loss_part, row_lse + q0,
+                            pos_logit ? pos_logit + q0 : nullptr, dQ, lddq, nullptr, 0, dev_status,
+                            static_cast<cudaStream_t>(cuda_stream), false);
+}
+
+int gc_shard_dp(const void* Q, int64_t ldq, const void* P, int64_t ldp, const int32_t* pos_idx,
+                int64_t B, int64_t N, int d, float tau, int mask_mode, int dtype,
+                const float* row_lse, int64_t p0, int64_t p_count, float* dP, int64_t lddp, void* ws,
+                size_t ws_bytes, int* dev_status, void* cuda_stream) {
+    int rc = check_common(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
+    if (rc) return rc;
+    if (mask_mode != GC_MASK_NONE) return GC_ERR_MASK;
+    if (p0 < 0 || p_count <= 0 || p0 + p_count > N) return GC_ERR_SHAPE;
+    if (!row_lse || !dP) return GC_ERR_NULL;
+    if ((rc = check_grad_out(dP, lddp, d))) return rc;
+    Plan pl = make_plan(B, p_count, d, dtype);
+    const size_t need = pl.total + align256(sizeof(int32_t) * (size_t)B);
+    if ((rc = check_ws(ws, ws_bytes, need))) return rc;
+    if ((rc = check_device())) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+    char* w = static_cast<char*>(ws);
+    // positives counted from the slice's first passage; those outside the slice match no row
+    int32_t* pos_local = reinterpret_cast<int32_t*>(w + pl.total);
+    if (dev_status && launch_pos_check(pos_idx, B, N, mask_mode, dev_status, st) != cudaSuccess)
+        return GC_ERR_CUDA;
+    if (launch_shift_pos(pos_idx, B, p0, p_count, pos_local, st) != cudaSuccess) return GC_ERR_CUDA;
+    const char* p_first = static_cast<const char*>(P) + (size_t)p0 * (size_t)ldp * elem_size(dtype);
+    Problem p = make_problem(Q, ldq, p_first, ldp, pos_local, B, p_count, d, tau, mask_mode, dtype);
+    return run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, dev_status, st);
 }
 
 int gc_profile_enable(int on) {

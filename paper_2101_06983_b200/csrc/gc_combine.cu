@@ -29,7 +29,7 @@ lse_combine_kernel(const float* __restrict__ part_m, const float* __restrict__ p
                    const float* __restrict__ pos_ws, const int32_t* __restrict__ pos_idx,
                    int groups, int64_t B, int64_t N, int mask_mode, float* __restrict__ row_lse,
                    float* __restrict__ pos_logit, float* __restrict__ loss, float* red,
-                   int* __restrict__ dev_status, const Gate gate) {
+                   int* __restrict__ dev_status, const Gate gate, int64_t mean_over) {
     if (gate_closed(gate)) return;
     __shared__ float warp_sum[kCombineThreads / 32];
     __shared__ int warp_flag[kCombineThreads / 32];
@@ -74,7 +74,7 @@ lse_combine_kernel(const float* __restrict__ part_m, const float* __restrict__ p
         for (int b = lane; b < (int)gridDim.x; b += 32) v += __ldcg(red + kRedPartials + b);
         for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
         if (lane == 0) {
-            *loss = v / (float)B;
+            *loss = v / (float)mean_over;
             *reinterpret_cast<int*>(red) = 0;
         }
     }
@@ -337,14 +337,36 @@ cudaError_t launch_fused_dq_finalize(const float* partial, int groups, const flo
 cudaError_t launch_lse_combine(const float* part_m, const float* part_l, const float* pos_ws,
                                const int32_t* pos_idx, int groups, int64_t B, int64_t N,
                                int mask_mode, float* row_lse, float* pos_logit, float* loss,
-                               float* red, int* dev_status, Gate gate, cudaStream_t st) {
+                               float* red, int* dev_status, Gate gate, cudaStream_t st,
+                               int64_t mean_over) {
     int64_t blocks = (B + kCombineThreads - 1) / kCombineThreads;
     if (blocks > sm_count()) blocks = sm_count();
     if (blocks > 256) blocks = 256;          // the scratch holds this many block sums
     lse_combine_kernel<<<(int)blocks, kCombineThreads, 0, st>>>(part_m, part_l, pos_ws, pos_idx,
                                                                groups, B, N, mask_mode, row_lse,
                                                                pos_logit, loss, red, dev_status,
-                                                               gate);
+                                                               gate, mean_over > 0 ? mean_over : B);
+    return cudaGetLastError();
+}
+
+namespace {
+// out[i] = pos_idx[i] - first when that lies in [0, count), else -1 (matches no row).
+__global__ void __launch_bounds__(256)
+shift_pos_kernel(const int32_t* __restrict__ pos_idx, int64_t B, int64_t first, int64_t count,
+                 int32_t* __restrict__ out) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < B;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = (int64_t)pos_idx[i] - first;
+        out[i] = (r >= 0 && r < count) ? (int32_t)r : -1;
+    }
+}
+}  // namespace
+
+cudaError_t launch_shift_pos(const int32_t* pos_idx, int64_t B, int64_t first, int64_t count,
+                             int32_t* out, cudaStream_t st) {
+    int64_t blocks = (B + 255) / 256;
+    if (blocks > 4 * sm_count()) blocks = 4 * sm_count();
+    shift_pos_kernel<<<(int)blocks, 256, 0, st>>>(pos_idx, B, first, count, out);
     return cudaGetLastError();
 }
 

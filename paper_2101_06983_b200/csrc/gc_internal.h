@@ -47,6 +47,8 @@ struct Problem {
     float tau;
     int mask_mode;
     int dtype;
+    int64_t b_total;        // rows of the whole batch when Q holds a slice of it (0: B): the mean
+                            // of Eq. 1 and the 1/B of Eq. 4 run over this many queries
 };
 
 // The two tile sweeps share one shape: a stationary row tile X, a streamed row tile Y,
@@ -120,7 +122,10 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored = false);
 cudaError_t launch_lse_combine(const float* part_m, const float* part_l, const float* pos_ws,
                                const int32_t* pos_idx, int groups, int64_t B, int64_t N,
                                int mask_mode, float* row_lse, float* pos_logit, float* loss,
-                               float* red, int* dev_status, Gate gate, cudaStream_t st);
+                               float* red, int* dev_status, Gate gate, cudaStream_t st,
+                               int64_t mean_over = 0);
+cudaError_t launch_shift_pos(const int32_t* pos_idx, int64_t B, int64_t first, int64_t count,
+                             int32_t* out, cudaStream_t st);
 cudaError_t launch_pos_check(const int32_t* pos_idx, int64_t B, int64_t N, int mask_mode,
                              int* dev_status, cudaStream_t st);
 cudaError_t launch_fused_dq_finalize(const float* partial, int groups, const float* part_m,

@@ -1,0 +1,90 @@
+"""The multi-GPU variant of Step 2 (Section 3.4) on CPU: two gloo ranks run the host-side
+plumbing of `sharded.sharded_build_cache` (row ranges, the all-gather of representations, the
+exchange of row logsumexps, the loss all-reduce) with the two compute steps supplied by the CPU
+oracle.  The ranks' results, put together, must be the oracle's full-batch results."""
+import os
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+B, N, D, TAU = 37, 75, 24, 0.5          # ragged: 19 + 18 queries, 38 + 37 passages
+
+
+class OracleKernels:
+    """Stand-in for the library's rank-local calls, written from their documented contract."""
+
+    def fwd_dq(self, Q_all, P_all, pos_all, tau, q0, q_count, loss_part, row_lse, dQ):
+        import oracle
+        rows = np.arange(q0, q0 + q_count)
+        out = oracle.query_rows(Q_all.numpy(), P_all.numpy(), pos_all.numpy(), rows, tau, 0)
+        row_lse[q0:q0 + q_count] = torch.from_numpy(out["row_lse"]).float()
+        dQ.copy_(torch.from_numpy(out["dQ"]).float())
+        loss_part[0] = float((out["row_lse"] - out["pos_logit"]).sum() / Q_all.shape[0])
+
+    def dp(self, Q_all, P_all, pos_all, tau, row_lse, p0, p_count, dP):
+        import oracle
+        rows = np.arange(p0, p0 + p_count)
+        out = oracle.passage_rows(Q_all.numpy(), P_all.numpy(), pos_all.numpy(),
+                                  row_lse.double().numpy(), rows, tau, 0)
+        dP.copy_(torch.from_numpy(out).float())
+
+
+def _problem():
+    from paper_2101_06983_b200 import inputs
+    return inputs.random_problem(B, N, D, "f32", seed=77, tau=TAU, scale=0.3)
+
+
+def _worker(rank, world, port, out_dir):
+    os.environ["MASTER_ADDR"] = "127.0.0.1"
+    os.environ["MASTER_PORT"] = str(port)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2101_06983_b200 import sharded
+    prob = _problem()
+    (q0, b), (p0, n) = sharded.row_ranges(B, world)[rank], sharded.row_ranges(N, world)[rank]
+    Ql = torch.from_numpy(prob.Q[q0:q0 + b].copy())
+    Pl = torch.from_numpy(prob.P[p0:p0 + n].copy())
+    posl = torch.from_numpy(prob.pos_idx[q0:q0 + b].copy())
+    loss, lse, dQ, dP = sharded.sharded_build_cache(Ql, Pl, posl, TAU, B, N,
+                                                    kernels=OracleKernels())
+    torch.save(dict(loss=float(loss), lse=lse, dQ=dQ, dP=dP, q=(q0, b), p=(p0, n)),
+               os.path.join(out_dir, f"r{rank}.pt"))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+@pytest.mark.timeout(180)
+def test_two_ranks_reproduce_the_full_batch(tmp_path, oracle):
+    world, port = 2, 29600 + os.getpid() % 1000
+    mp.spawn(_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    r = [torch.load(tmp_path / f"r{k}.pt") for k in range(world)]
+    prob = _problem()
+    ref = oracle.build_cache(prob.Q, prob.P, prob.pos_idx, TAU, 0)
+    assert r[0]["q"] == (0, 19) and r[1]["q"] == (19, 18)
+    assert r[0]["p"] == (0, 38) and r[1]["p"] == (38, 37)
+    for k in range(world):
+        assert abs(r[k]["loss"] - ref["loss"]) <= 1e-5 * abs(ref["loss"])   # same on every rank
+        np.testing.assert_allclose(r[k]["lse"].numpy(), ref["row_lse"], rtol=1e-6)
+    dQ = torch.cat([r[0]["dQ"], r[1]["dQ"]]).numpy()
+    dP = torch.cat([r[0]["dP"], r[1]["dP"]]).numpy()
+    assert np.abs(dQ - ref["dQ"]).max() <= 1e-6 * np.abs(ref["dQ"]).max()
+    # dP on each rank used the exchanged float32 row_lse of the other rank's queries
+    assert np.abs(dP - ref["dP"]).max() <= 1e-5 * np.abs(ref["dP"]).max()
+
+
+def test_row_ranges_cover_everything_once():
+    from paper_2101_06983_b200 import sharded
+    for total, world in ((37, 2), (8, 8), (5, 3), (4096, 7), (3, 4)):
+        rr = sharded.row_ranges(total, world)
+        assert len(rr) == world and rr[0][0] == 0
+        assert all(rr[i][0] + rr[i][1] == rr[i + 1][0] for i in range(world - 1))
+        assert rr[-1][0] + rr[-1][1] == total
+        assert max(c for _, c in rr) - min(c for _, c in rr) <= 1
+
+
+def test_single_process_needs_no_group():
+    from paper_2101_06983_b200 import sharded
+    x = torch.arange(12.0).reshape(4, 3)
+    assert sharded.gather_rows(x, [4]) is x
