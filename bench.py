@@ -377,6 +377,62 @@ def run_ours(args, rank, local_rank, world):
         dist.destroy_process_group()
 
 
+def run_sharded(args, rank, local_rank, world):
+    """Non-default multi-GPU mode (--parallel shard): ONE global batch of the chosen workload is
+    split over the ranks as Section 3.4 describes (all-gather of representations, rank-local
+    forward + dQ and dP, exchange of row_lse, loss all-reduce).  Strong scaling: the value is the
+    whole batch's useful FLOP over the slowest rank's time, collectives included."""
+    import torch
+    import torch.distributed as dist
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    from paper_2101_06983_b200 import binding, inputs, replicas, sharded
+    prob = inputs.config(args.config)
+    if prob.mask_mode != inputs.MASK_NONE:
+        raise SystemExit("--parallel shard covers the unmasked loss only")
+    B, N, d = prob.B, prob.N, prob.d
+    Q, P, pos = binding.problem_tensors(prob, dev)
+    (q0, b), (p0, n) = sharded.row_ranges(B, world)[rank], sharded.row_ranges(N, world)[rank]
+    Ql, Pl, posl = Q[q0:q0 + b].contiguous(), P[p0:p0 + n].contiguous(), pos[q0:q0 + b].contiguous()
+    del Q, P, pos
+
+    def step():
+        return sharded.sharded_build_cache(Ql, Pl, posl, prob.tau, B, N)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    a, bev = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(args.steps):
+        loss = step()[0]
+    bev.record()
+    barrier()
+    ms = replicas.max_over_ranks([a.elapsed_time(bev) / args.steps], dev)[0]
+    if rank == 0:
+        flop = useful_flop(B, N, d)
+        print(json.dumps({
+            "metric": METRIC, "value": flop / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+            "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+            "dtype": "bf16" if prob.dtype == "bf16" else "f32", "data": "synthetic",
+            "config": {"workload": prob.name, "B": B, "N": N, "d": d,
+                       "parallelism": f"rows sharded over {world} rank(s), Section 3.4",
+                       "l2": "back to back, no flush (collectives between the kernels)"},
+            "loss": float(loss.item()), "gpu_launches": None}), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
 def run_apply(args):
     """Side measurement (not the headline metric): gc_cache_apply, Step 3 for a linear encoder,
     dW (+)= U^T X over one sub-batch of --apply-rows rows with d = d_in = 768.  HBM-bound by its
@@ -452,6 +508,9 @@ def main():
                     help="build: gc_build_cache, the headline; apply: the side measurement of "
                          "gc_cache_apply (one GPU)")
     ap.add_argument("--apply-rows", type=int, default=4096)
+    ap.add_argument("--parallel", default="replicas", choices=["replicas", "shard"],
+                    help="N > 1: independent replicas (default, weak scaling, no collective), or "
+                         "one batch sharded over the ranks as in Section 3.4 of the paper")
     args = ap.parse_args()
     if args.op == "apply":
         if int(os.environ.get("RANK", "0")) == 0:
@@ -467,6 +526,9 @@ def main():
         return
     if args.ref_rows is None:
         args.ref_rows = 4096
+    if args.parallel == "shard":
+        run_sharded(args, rank, local_rank, world)
+        return
     run_ours(args, rank, local_rank, world)
 
 
