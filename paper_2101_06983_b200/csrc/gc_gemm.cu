@@ -263,7 +263,11 @@ cudaError_t launch_gemm(const CUtensorMap& ma, const CUtensorMap& mb, const CUte
     if (nb > MAX_B_STAGES) nb = MAX_B_STAGES;
     p.nb = nb;
     const size_t dynamic_bytes = 1024 + (size_t)p.na * A_STAGE_BYTES + (size_t)nb * b_stage;
-    static bool configured = false;
+    // the attribute belongs to the (kernel, device) pair
+    static bool configured_on[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    bool& configured = configured_on[dev];
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(gemm_kernel<A_MN, PAIR>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize,

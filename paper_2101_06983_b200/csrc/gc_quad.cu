@@ -703,7 +703,11 @@ cudaError_t launch_quad(const CUtensorMap& mx, const CUtensorMap& my, const CUte
     if (ns > MAX_STAGES) ns = MAX_STAGES;
     p.nstage = ns;
     const size_t dynamic_bytes = fixed + (size_t)ns * CHUNK_BYTES;
-    static bool configured = false;
+    // the attribute belongs to the (kernel, device) pair
+    static bool configured_on[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    bool& configured = configured_on[dev];
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(quad_kernel<MODE>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -1127,7 +1127,11 @@ cudaError_t launch_one(const CUtensorMap& mx, const CUtensorMap& my, const CUten
                        const CUtensorMap& mo, const TcParams& p, int64_t ctas, cudaStream_t st) {
     constexpr bool WBUFS = (PAIR && NBUF == 1 && MODE != MODE_FWD) || MODE == MODE_FS;
     SmemPlan sp = smem_plan(p.kc, PAIR, WBUFS);
-    static bool configured = false;
+    // the attribute belongs to the (kernel, device) pair
+    static bool configured_on[64] = {false};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    bool& configured = configured_on[dev];
     if (!configured) {
         cudaError_t e = cudaFuncSetAttribute(tc_kernel<MODE, SN, NBUF, PAIR>,
                                              cudaFuncAttributeMaxDynamicSharedMemorySize,
