@@ -343,9 +343,6 @@ int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, 
     const Gate in_range = {flag, 0}, out_of_range = {flag, 1};
     SideStream* side = side_stream();
     cudaStream_t aux = side ? side->st : st;
-    cudaError_t e = launch_pos_anchor(p.Q, p.ldq, p.P, p.ldp, p.pos_idx, p.B, p.N, p.d, p.mask_mode,
-                                      1.4426950408889634f / p.tau, ref2, flag, st);
-    if (e != cudaSuccess) return GC_ERR_CUDA;
     FwdArgs fa{};
     fa.p = p;
     fa.part_m = reinterpret_cast<float*>(ws + pl.off_m);
@@ -355,10 +352,19 @@ int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, 
     fa.groups = (pl.anchored == 1 ? 4 : 2) * pl.g_dq;
     fa.dev_status = dev_status;
     float* partial = reinterpret_cast<float*>(ws + pl.off_accq);
+    // The fused sweep is launched with programmatic serialization: it starts (loads, first S
+    // tiles) while the anchor kernel still runs, and only its softmax warps wait for the
+    // anchors.  Per-kernel timing (gc_profile_enable) records an event between the two launches,
+    // which serialises them, so the overlap is left out while it is on.
+    const bool overlap = !g_prof.on;
+    cudaError_t e = launch_pos_anchor(p.Q, p.ldq, p.P, p.ldp, p.pos_idx, p.B, p.N, p.d, p.mask_mode,
+                                      1.4426950408889634f / p.tau, ref2, flag, st);
+    if (e != cudaSuccess) return GC_ERR_CUDA;
     {
         KernelTimer t(1, st);
-        e = pl.anchored == 1 ? quad_launch_fused_dq(fa, partial, pl.g_dq, ref2, flag, st)
-                             : tc_launch_anchored_dq(fa, partial, pl.g_dq, ref2, flag, st);
+        e = pl.anchored == 1
+                ? quad_launch_fused_dq(fa, partial, pl.g_dq, ref2, flag, st, overlap)
+                : tc_launch_anchored_dq(fa, partial, pl.g_dq, ref2, flag, st, overlap);
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     // Wide rows: a sweep step is long enough to hide the slot merge of the streamed queries,

@@ -172,6 +172,7 @@ pos_anchor_kernel(const __nv_bfloat16* __restrict__ Q, int64_t ldq,
                   const __nv_bfloat16* __restrict__ P, int64_t ldp,
                   const int32_t* __restrict__ pos_idx, int64_t B, int64_t N, int d, int mask_mode,
                   float c1, float* __restrict__ ref2, int* __restrict__ range_flag) {
+    dep_release();      // the sweep that follows may start; it waits for this grid before it reads ref2
     if (blockIdx.x == 0 && threadIdx.x == 0) *range_flag = 0;
     const int lane = threadIdx.x & 31;
     for (int64_t i = blockIdx.x * 8 + (threadIdx.x >> 5); i < B; i += (int64_t)gridDim.x * 8) {

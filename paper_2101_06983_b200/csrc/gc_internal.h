@@ -16,6 +16,14 @@ struct Gate {
     int want;
 };
 #ifdef __CUDACC__
+// Programmatic dependent launch: a kernel launched with the programmatic-serialization attribute
+// may start while the kernel before it in the stream still runs; dep_wait() returns once that
+// kernel has completed and its writes are visible (at once for an ordinary launch);
+// dep_release() in the earlier kernel lets the later one be scheduled early.
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dep_release() {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
 __device__ __forceinline__ bool gate_closed(const Gate& g) {
     return g.flag && ((*g.flag != 0) != (g.want != 0));
 }
@@ -161,7 +169,8 @@ int tc_fwd_groups(int64_t B, int64_t N, int d);
 bool tc_fused_applicable(int d);
 bool tc_anchor_applicable(int d);
 cudaError_t tc_launch_anchored_dq(const FwdArgs& a, float* partial, int groups,
-                                  const float* row_ref, int* range_flag, cudaStream_t st);
+                                  const float* row_ref, int* range_flag, cudaStream_t st,
+                                  bool overlap_prev = false);
 cudaError_t tc_launch_fused_dq(const FwdArgs& a, float* partial, int groups, cudaStream_t st);
 int tc_sweep_groups(int64_t nx, int64_t ny, int d);
 cudaError_t tc_launch_fwd_store(const FwdArgs& a, void* weights, int64_t ldw, const float* row_ref,
@@ -172,7 +181,7 @@ bool quad_applicable(int64_t nx, int d);
 int quad_groups(int64_t nx, int64_t ny);
 cudaError_t quad_launch_sweep(const SweepArgs& a, cudaStream_t st);
 cudaError_t quad_launch_fused_dq(const FwdArgs& a, float* partial, int groups, const float* row_ref,
-                                 int* range_flag, cudaStream_t st);
+                                 int* range_flag, cudaStream_t st, bool overlap_prev = false);
 
 // gc_gemm.cu
 int gemm_groups(int64_t m_rows, int64_t k_len, int d);

@@ -458,6 +458,9 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
         const bool sev = (q == 0 && half == 0);
         long long ph[7] = {0, 0, 0, 0, 0, 0, 0};
 #endif
+        // FA may have been launched ahead of the anchor kernel's completion: row_ref, the range
+        // flag and everything this role writes come after it
+        if (MODE == QMODE_FA) dep_wait();
         if (MODE != QMODE_DP && x < p.nx) {
             lse2_x = (MODE == QMODE_FA) ? p.row_ref[x] : p.row_lse[x] * 1.4426950408889634f;
             pos_x = p.pos_idx[x];
@@ -697,7 +700,8 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
 
 template <int MODE>
 cudaError_t launch_quad(const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& myh,
-                        const CUtensorMap& mo, QuadParams p, int64_t clusters, cudaStream_t st) {
+                        const CUtensorMap& mo, QuadParams p, int64_t clusters, cudaStream_t st,
+                        bool overlap_prev = false) {
     const size_t fixed = 1024 + (size_t)Q_XRES * X_CHUNK_BYTES + 2 * 32768;
     int ns = (int)((SMEM_LIMIT - SMEM_STATIC_RESERVE - fixed) / CHUNK_BYTES);
     if (ns > MAX_STAGES) ns = MAX_STAGES;
@@ -720,13 +724,15 @@ cudaError_t launch_quad(const CUtensorMap& mx, const CUtensorMap& my, const CUte
     cfg.blockDim = dim3(NTHREADS);
     cfg.dynamicSmemBytes = dynamic_bytes;
     cfg.stream = st;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 4;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = overlap_prev ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, quad_kernel<MODE>, mx, my, myh, mo, p);
 }
 
@@ -790,7 +796,7 @@ cudaError_t quad_launch_sweep(const SweepArgs& a, cudaStream_t st) {
 // pos_logit and the unscaled accumulators partial[groups][B][d] of sum_j 2^(s2_ij - ref_i) P_j
 // over all allowed columns but the positive one; raises *range_flag when a weight exceeds 2^100.
 cudaError_t quad_launch_fused_dq(const FwdArgs& a, float* partial, int groups, const float* row_ref,
-                                 int* range_flag, cudaStream_t st) {
+                                 int* range_flag, cudaStream_t st, bool overlap_prev) {
     const Problem& pr = a.p;
     const int kc = pr.d / 64;
     CUtensorMap mx, my, myh, mo;
@@ -813,7 +819,7 @@ cudaError_t quad_launch_fused_dq(const FwdArgs& a, float* partial, int groups, c
     p.gate = a.gate;
     p.zero_me = reinterpret_cast<int*>(a.red);
     const int64_t clusters = (((pr.B + XROWS - 1) / XROWS + 1) / 2) * groups;
-    return launch_quad<QMODE_FA>(mx, my, myh, mo, p, clusters, st);
+    return launch_quad<QMODE_FA>(mx, my, myh, mo, p, clusters, st, overlap_prev);
 }
 
 }  // namespace gc

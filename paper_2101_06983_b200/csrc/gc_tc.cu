@@ -873,6 +873,8 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             // per-row constants (DQ: the row is a query)
             float lse2_x = 0.f, l_sum = 0.f, wmax = 0.f;
             int32_t pos_x = -1;
+            // DA may have been launched ahead of the anchor kernel's completion
+            if (MODE == MODE_DA) dep_wait();
             if ((MODE == MODE_DQ || MODE == MODE_DA) && x < p.nx) {
                 lse2_x = (MODE == MODE_DA) ? p.row_ref[x] : p.row_lse[x] * 1.4426950408889634f;
                 pos_x = p.pos_idx[x];
@@ -1124,7 +1126,8 @@ SmemPlan smem_plan(int kc, bool pair = false, bool ws = false) {
 
 template <int MODE, int SN, int NBUF, bool PAIR>
 cudaError_t launch_one(const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& myh,
-                       const CUtensorMap& mo, const TcParams& p, int64_t ctas, cudaStream_t st) {
+                       const CUtensorMap& mo, const TcParams& p, int64_t ctas, cudaStream_t st,
+                       bool overlap_prev = false) {
     constexpr bool WBUFS = (PAIR && NBUF == 1 && MODE != MODE_FWD) || MODE == MODE_FS;
     SmemPlan sp = smem_plan(p.kc, PAIR, WBUFS);
     // the attribute belongs to the (kernel, device) pair
@@ -1147,14 +1150,16 @@ cudaError_t launch_one(const CUtensorMap& mx, const CUtensorMap& my, const CUten
     TcParams pp = p;
     pp.nstage = sp.nstage;
     pp.xres = sp.xres;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = PAIR ? 2 : 1;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
-    if (!PAIR) {
+    cfg.numAttrs = overlap_prev ? 2 : 1;
+    if (!PAIR && !overlap_prev) {
         tc_kernel<MODE, SN, NBUF, false><<<(unsigned)ctas, NTHREADS, sp.dynamic_bytes, st>>>(
             mx, my, myh, mo, pp);
         return cudaGetLastError();
@@ -1184,11 +1189,12 @@ int64_t cta_count(int mode, int kc, int64_t nx, int64_t ny, int parts, int group
 
 template <int MODE, int SN, int NBUF>
 cudaError_t launch(const CUtensorMap& mx, const CUtensorMap& my, const CUtensorMap& myh,
-                   const CUtensorMap& mo, const TcParams& p, cudaStream_t st) {
+                   const CUtensorMap& mo, const TcParams& p, cudaStream_t st,
+                   bool overlap_prev = false) {
     const int64_t ctas = cta_count(MODE, p.kc, p.nx, p.ny, p.dparts, p.groups);
     if (use_pair(MODE, p.kc, p.nx, p.ny))
-        return launch_one<MODE, SN, NBUF, true>(mx, my, myh, mo, p, ctas, st);
-    return launch_one<MODE, SN, NBUF, false>(mx, my, myh, mo, p, ctas, st);
+        return launch_one<MODE, SN, NBUF, true>(mx, my, myh, mo, p, ctas, st, overlap_prev);
+    return launch_one<MODE, SN, NBUF, false>(mx, my, myh, mo, p, ctas, st, overlap_prev);
 }
 
 }  // namespace
@@ -1337,7 +1343,8 @@ bool tc_anchor_applicable(int d) { return sweep_nbuf(d / 64) == 2; }
 // pos_logit and the unscaled accumulators partial[groups][B][d] of sum_j 2^(s2_ij - ref_i) P_j
 // over all allowed columns but the positive one; raises *range_flag when a weight exceeds 2^100.
 cudaError_t tc_launch_anchored_dq(const FwdArgs& a, float* partial, int groups,
-                                  const float* row_ref, int* range_flag, cudaStream_t st) {
+                                  const float* row_ref, int* range_flag, cudaStream_t st,
+                                  bool overlap_prev) {
     const Problem& pr = a.p;
     constexpr int SN = 128;
     const int kc = pr.d / 64;
@@ -1364,7 +1371,7 @@ cudaError_t tc_launch_anchored_dq(const FwdArgs& a, float* partial, int groups,
     p.zero_me = reinterpret_cast<int*>(a.red);
     p.dev_status = a.dev_status;
     p.gate = a.gate;
-    return launch<MODE_DA, SN, 2>(mx, my, myh, mo, p, st);
+    return launch<MODE_DA, SN, 2>(mx, my, myh, mo, p, st, overlap_prev);
 }
 
 cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
