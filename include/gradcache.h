@@ -34,6 +34,10 @@
  *     is read out of bounds and nothing traps.  GC_DEV_WAIT_LIMIT means a bounded on-chip wait
  *     gave up; outputs are then undefined.  The caller zeroes *dev_status beforehand.
  *   - Results are deterministic: no floating-point atomics, fixed reduction order.
+ *   - Host threads: the library keeps small per-device records (SM count, kernel attributes, one
+ *     side stream with its events) that are created on first use without locking.  Make calls
+ *     from one host thread at a time.  Calls on different streams of one device are allowed; the
+ *     work they put on the side stream is serialised there.
  */
 #ifndef GRADCACHE_H_
 #define GRADCACHE_H_

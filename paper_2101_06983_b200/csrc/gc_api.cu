@@ -59,7 +59,8 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored) {
     pl.off_pos = off;  off += align256(sizeof(float) * (size_t)B);
     pl.off_red = off;  off += 2048;      // loss reduction: block ticket + up to 256 block sums
     pl.off_accq = off;
-    if (pl.g_dq > 1 || pl.fused || pl.anchored) off += align256(sizeof(float) * (size_t)pl.g_dq * (size_t)B * dpad);
+    if (pl.g_dq > 1 || pl.fused || pl.anchored)
+        off += align256(sizeof(float) * (size_t)pl.g_dq * (size_t)B * dpad);
     pl.off_accp = off;
     if (pl.g_dp > 1) off += align256(sizeof(float) * (size_t)pl.g_dp * (size_t)N * dpad);
     pl.launches_fwd = 2;  // sweep + combine
@@ -202,7 +203,8 @@ int run_fwd(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, gate, st, p.b_total);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status,
+                           gate, st, p.b_total);
     return e == cudaSuccess ? GC_OK : GC_ERR_CUDA;
 }
 
@@ -265,7 +267,8 @@ int run_fused_fwd_dq(const Problem& p, const Plan& pl, char* ws, float* loss, fl
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, gate, st, p.b_total);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status,
+                           gate, st, p.b_total);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_fused_dq_finalize(partial, pl.g_dq, fa.part_m, nullptr, row_lse, fa.pos_logit,
                                  p.pos_idx, p.P, p.ldp, p.B, p.N, p.d, p.mask_mode,
@@ -376,7 +379,8 @@ int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, 
                       cudaStreamWaitEvent(aux, side->ev[0], 0) != cudaSuccess))
         return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, in_range, comb, p.b_total);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status,
+                           in_range, comb, p.b_total);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     if (side && !dp_merges && (cudaEventRecord(side->ev[0], st) != cudaSuccess ||
                                cudaStreamWaitEvent(aux, side->ev[0], 0) != cudaSuccess))
@@ -455,7 +459,8 @@ int run_build_stored(const Problem& p, const Plan& pl, char* w, float* loss, flo
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
-                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status, kOpen, st, p.b_total);
+                           p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status,
+                           kOpen, st, p.b_total);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_scale_rows(p.Q, p.ldq, p.B, p.d, ref2, row_lse, qs, st);
     if (e != cudaSuccess) return GC_ERR_CUDA;
