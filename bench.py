@@ -31,7 +31,7 @@ NOMINAL_BF16_TFLOPS = 2250.0      # public dense bf16 figure for B200, context o
 # ncu capture summarised in profiles/quad_kernel_cfg2_B4096_N8192_d768.txt.  Reported only while
 # the kernel source still has the hash it had when the counters were taken.
 NCU_TRAFFIC_BYTES = 19.1e6
-NCU_TRAFFIC_SOURCE_SHA1 = "502a9f7cd1fe23b2413012fd5dc559175f624525"
+NCU_TRAFFIC_SOURCE_SHA1 = "916b6c4e7d6d270f2504571c26c0464f8ffcd291"
 
 
 def ncu_traffic(workload: str):
