@@ -883,8 +883,8 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 const int b = t & (NBUF - 1);
                 const int64_t y0 = (lo + t) * SN;
                 // DP: the columns are queries; lane j holds lse / pos of column 32 cb + j
-                float lse2_y[CB_PER];
-                int32_t pos_y[CB_PER];
+                float lse2_y[CB_PER] = {};
+                int32_t pos_y[CB_PER] = {};
                 if (MODE == MODE_DP) {
 #pragma unroll
                     for (int j = 0; j < CB_PER; ++j) {
@@ -907,11 +907,16 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 const uint32_t sbuf = tmem + lane_addr + S_COL0 + b * SN;
                 // W of this half goes to the first columns of the half's own S region (already
                 // read by this warp): columns half * SN/2 + 16 j for block j.
-                // both 32-column blocks are requested before the single wait
-                uint32_t vv[CB_PER][32];
+                // WS: both 32-column blocks are requested before the single wait, so that the S
+                // tile can be released.  Otherwise one block at a time in a loop that is not
+                // unrolled (W block j overwrites logits this thread has already read): half the
+                // registers and half the instruction footprint.
+                uint32_t vv[WS ? CB_PER : 1][32];
+                if (WS) {
 #pragma unroll
-                for (int j = 0; j < CB_PER; ++j) tmem_ld32(sbuf + (cb0 + j) * 32, vv[j]);
-                tmem_ld_wait();
+                    for (int j = 0; j < CB_PER; ++j) tmem_ld32(sbuf + (cb0 + j) * 32, vv[WS ? j : 0]);
+                    tmem_ld_wait();
+                }
                 if (WS) {
                     // the S tile may be overwritten; W buffer t & 1 must have been consumed
                     tc_fence_before();
@@ -924,10 +929,16 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     }
                     if (q == 0 && half == 0) EV(2, ev_s, 12, t);
                 }
-#pragma unroll
+#pragma unroll(WS ? CB_PER : 1)
                 for (int j = 0; j < CB_PER; ++j) {
                     const int cb = cb0 + j;
-                    uint32_t (&v)[32] = vv[j];
+                    uint32_t (&v)[32] = vv[WS ? j : 0];
+                    if (!WS) {
+                        tmem_ld32(sbuf + cb * 32, v);
+                        tmem_ld_wait();
+                    }
+                    const float lse2_yj = j == 0 ? lse2_y[0] : lse2_y[CB_PER - 1];
+                    const int32_t pos_yj = j == 0 ? pos_y[0] : pos_y[CB_PER - 1];
                     const int64_t yb = y0 + cb * 32;
                     float w[32];
                     if (MODE == MODE_DQ) {
@@ -988,12 +999,12 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     } else {
 #pragma unroll
                         for (int c = 0; c < 32; ++c) {
-                            const float ls = __shfl_sync(0xffffffffu, lse2_y[j], c);
+                            const float ls = __shfl_sync(0xffffffffu, lse2_yj, c);
                             w[c] = ex2(fmaf(__uint_as_float(v[c]), p.c1, -ls));   // OOB: ex2(-inf)
                         }
                         // one-hot: column c's query has its positive at row pos - x0 of this tile
-                        const int64_t rel_row = (int64_t)pos_y[j] - x0;
-                        const bool mine = (pos_y[j] >= 0) && rel_row >= q * 32 && rel_row < q * 32 + 32;
+                        const int64_t rel_row = (int64_t)pos_yj - x0;
+                        const bool mine = (pos_yj >= 0) && rel_row >= q * 32 && rel_row < q * 32 + 32;
                         unsigned hits = __ballot_sync(0xffffffffu, mine);
                         while (hits) {
                             const int col = __ffs(hits) - 1;
