@@ -52,7 +52,7 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored) {
     size_t slots = (size_t)pl.g_fwd;
     if (pl.fused && (size_t)(2 * pl.g_dq) > slots) slots = (size_t)(2 * pl.g_dq);
     if (pl.anchored == 1 && (size_t)(4 * pl.g_dq) > slots) slots = (size_t)(4 * pl.g_dq);
-    if (pl.anchored == 2 && (size_t)(2 * pl.g_dq) > slots) slots = (size_t)(2 * pl.g_dq);
+    if (pl.anchored == 2 && (size_t)(4 * pl.g_dq) > slots) slots = (size_t)(4 * pl.g_dq);
     size_t off = 0;
     pl.off_m = off;    off += align256(sizeof(float) * slots * (size_t)B);
     pl.off_l = off;    off += align256(sizeof(float) * slots * (size_t)B);
@@ -352,7 +352,7 @@ int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, 
     fa.part_l = reinterpret_cast<float*>(ws + pl.off_l);
     fa.pos_logit = reinterpret_cast<float*>(ws + pl.off_pos);
     fa.red = reinterpret_cast<float*>(ws + pl.off_red);
-    fa.groups = (pl.anchored == 1 ? 4 : 2) * pl.g_dq;
+    fa.groups = 4 * pl.g_dq;      // per part: two duty pairs, or two softmax groups, x two column halves
     fa.dev_status = dev_status;
     float* partial = reinterpret_cast<float*>(ws + pl.off_accq);
     // The fused sweep is launched with programmatic serialization: it starts (loads, first S

@@ -130,8 +130,21 @@ struct Bars {
 // MMAs), which halves the Y traffic into shared memory.  "Full" barriers live in the leader and
 // count the bytes landing in both CTAs; "empty", s_full and acc_full are signalled in both CTAs by
 // multicast commits; the softmax warps of both CTAs arrive on the leader's w_full.
+// Narrow-row gradient sweeps (two S buffers, one CTA per tile) run two groups of softmax warps:
+// group 0 takes the even tiles (S buffer 0), group 1 the odd ones (buffer 1).  A tile keeps the
+// eight warps of its group busy for about three times as long as its MMAs take, so one group
+// caps the sweep at one tile per softmax pass however many buffers there are.
+template <int MODE, int NBUF, bool PAIR>
+__host__ __device__ constexpr bool two_softmax_groups() {
+    return NBUF == 2 && !PAIR && (MODE == MODE_DQ || MODE == MODE_DP || MODE == MODE_DA);
+}
+template <int MODE, int NBUF, bool PAIR>
+__host__ __device__ constexpr int tc_threads() {
+    return two_softmax_groups<MODE, NBUF, PAIR>() ? NTHREADS + 32 * NSOFT : NTHREADS;
+}
+
 template <int MODE, int SN, int NBUF, bool PAIR>
-__global__ void __launch_bounds__(NTHREADS, 1)
+__global__ void __launch_bounds__((tc_threads<MODE, NBUF, PAIR>()), 1)
 tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
           const __grid_constant__ CUtensorMap mapYh, const __grid_constant__ CUtensorMap mapO,
           const TcParams p) {
@@ -514,8 +527,11 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
         }
     } else {
         // ------------------------------ softmax / epilogue warps --------------------------------
+        constexpr bool GROUPS2 = two_softmax_groups<MODE, NBUF, PAIR>();
+        const int sw = warp - (NPROD + 1);             // 0..7, or 0..15 with two groups
+        const int grp = GROUPS2 ? (sw >> 3) : 0;       // softmax group: tiles grp, grp + 2, ...
         const int q = warp & 3;                        // tensor-memory lane quarter of this warp
-        const int half = (warp - (NPROD + 1)) >> 2;    // which half of the tile's columns
+        const int half = (sw & 7) >> 2;                // which half of the tile's columns
         constexpr int CB_PER = SN / 64;                // 32-column blocks per half
         const int cb0 = half * CB_PER;
         const int row = q * 32 + lane;
@@ -879,7 +895,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 lse2_x = (MODE == MODE_DA) ? p.row_ref[x] : p.row_lse[x] * 1.4426950408889634f;
                 pos_x = p.pos_idx[x];
             }
-            for (int t = 0; t < T; ++t) {
+            for (int t = grp; t < T; t += (GROUPS2 ? 2 : 1)) {
                 const int b = t & (NBUF - 1);
                 const int64_t y0 = (lo + t) * SN;
                 // DP: the columns are queries; lane j holds lse / pos of column 32 cb + j
@@ -1041,8 +1057,9 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             }
             if (q == 0 && half == 0) EV_END(2, ev_s);
             if (MODE == MODE_DA && ok && x < p.nx) {
-                // one (scale, sum) slot per row, part of the streamed range and column half
-                const int64_t slot = (int64_t)(2 * g + half) * p.nq + x;
+                // one (scale, sum) slot per row, part of the streamed range, softmax group and
+                // column half
+                const int64_t slot = (int64_t)((2 * g + grp) * 2 + half) * p.nq + x;
                 p.part_m[slot] = lse2_x * 0.69314718055994531f;
                 p.part_l[slot] = l_sum;
                 // weights beyond 2^100 (or not finite) cannot be accumulated safely
@@ -1052,6 +1069,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             // dealt alternately to the two warps of a lane quarter); final values are scaled,
             // partial sums of a split sweep are not
             TR_BEGIN(tr_epi);
+            if (grp != 0) ok = false;      // the first group writes the accumulators
             if (ok) ok = mbar_wait(smem_u32(&bars.acc_full), 0, abort_flag);
             if (ok) {
                 tc_fence_after();
@@ -1155,7 +1173,7 @@ cudaError_t launch_one(const CUtensorMap& mx, const CUtensorMap& my, const CUten
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)ctas);
-    cfg.blockDim = dim3(NTHREADS);
+    cfg.blockDim = dim3(tc_threads<MODE, NBUF, PAIR>());
     cfg.dynamicSmemBytes = sp.dynamic_bytes;
     cfg.stream = st;
     TcParams pp = p;
@@ -1171,7 +1189,8 @@ cudaError_t launch_one(const CUtensorMap& mx, const CUtensorMap& my, const CUten
     cfg.attrs = attr;
     cfg.numAttrs = overlap_prev ? 2 : 1;
     if (!PAIR && !overlap_prev) {
-        tc_kernel<MODE, SN, NBUF, false><<<(unsigned)ctas, NTHREADS, sp.dynamic_bytes, st>>>(
+        tc_kernel<MODE, SN, NBUF, false><<<(unsigned)ctas, tc_threads<MODE, NBUF, false>(),
+                                           sp.dynamic_bytes, st>>>(
             mx, my, myh, mo, pp);
         return cudaGetLastError();
     }
@@ -1350,7 +1369,7 @@ cudaError_t tc_launch_fused_dq(const FwdArgs& a, float* partial, int groups, cud
 bool tc_anchor_applicable(int d) { return sweep_nbuf(d / 64) == 2; }
 
 // Forward fused into the dQ sweep of narrow rows with row_ref (log2 domain) as each row's fixed
-// scale: writes (scale, sum) slots [2 groups][B] (scale = row_ref in natural-log units),
+// scale: writes (scale, sum) slots [4 groups][B] (scale = row_ref in natural-log units),
 // pos_logit and the unscaled accumulators partial[groups][B][d] of sum_j 2^(s2_ij - ref_i) P_j
 // over all allowed columns but the positive one; raises *range_flag when a weight exceeds 2^100.
 cudaError_t tc_launch_anchored_dq(const FwdArgs& a, float* partial, int groups,
