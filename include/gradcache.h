@@ -220,15 +220,21 @@ int gc_loss_fwd_static(const void* Q, int64_t ldq, const void* P, int64_t ldp,
                        int* dev_status, void* cuda_stream);
 
 /*
- * Measurement aid (not part of the paper's method).  After gc_profile_enable(1) every call
- * brackets its three main kernels - the forward sweep, the dQ sweep (Eq. 5) and the dP sweep
- * (Eq. 6-7) - with CUDA events recorded on the call's own stream.  gc_profile_read waits for
- * the most recent call's events and returns each kernel's duration in milliseconds (0 for a
- * kernel that call did not launch).  Host pointers.  One set of events per process: enable it
- * for single-stream measurement runs only.  Events are created on the first enable.
+ * Measurement aid (not part of the paper's method).  After gc_profile_enable(sets) with sets >= 1
+ * every call brackets its three main kernels - the forward sweep, the dQ sweep (Eq. 5) and the
+ * dP sweep (Eq. 6-7) - with CUDA events recorded on the call's own stream; gc_profile_enable(0)
+ * switches it off.  Call number c since the enable (0, 1, ...) uses event set c % sets, so up to
+ * `sets` calls (at most 256, else GC_ERR_LIMIT) can be queued back to back and read afterwards:
+ * gc_profile_read_call(c, ...) waits for that call's events and returns each kernel's duration
+ * in milliseconds (0 for a kernel the call did not launch; GC_ERR_LIMIT when call c was never
+ * made or its set has been reused); gc_profile_read does the same for the most recent call.
+ * Host pointers.  One series of event sets per process: use it for single-stream measurement
+ * runs only.  While it is on, the event between the anchor kernel and the fused sweep keeps
+ * the sweep from starting early (see gc_build_cache).
  */
-int gc_profile_enable(int on);
+int gc_profile_enable(int sets);
 int gc_profile_read(float* ms_fwd, float* ms_dq, float* ms_dp);
+int gc_profile_read_call(int64_t call, float* ms_fwd, float* ms_dq, float* ms_dp);
 
 /* Human-readable name of a gc_status value.  Static string. */
 const char* gc_status_string(int status);

@@ -21,7 +21,7 @@ GC_DEV_POS_RANGE, GC_DEV_POS_MASKED, GC_DEV_WAIT_LIMIT = 1, 2, 4
 EXPORTS = ("gc_workspace_bytes", "gc_plan_name", "gc_kernel_launches", "gc_loss_fwd",
            "gc_loss_bwd", "gc_build_cache", "gc_build_cache_stored", "gc_status_string",
            "gc_profile_enable",
-           "gc_profile_read", "gc_static_scratch_need", "gc_loss_fwd_static",
+           "gc_profile_read", "gc_profile_read_call", "gc_static_scratch_need", "gc_loss_fwd_static",
            "gc_cache_apply_workspace_bytes", "gc_cache_apply", "gc_shard_workspace_bytes",
            "gc_shard_fwd_dq", "gc_shard_dp")
 GC_STATIC_SCRATCH_BYTES = 2 << 20
@@ -79,6 +79,8 @@ def _load() -> ctypes.CDLL:
     lib.gc_profile_enable.argtypes = [i32]
     lib.gc_profile_read.restype = i32
     lib.gc_profile_read.argtypes = [ctypes.POINTER(f32)] * 3
+    lib.gc_profile_read_call.restype = i32
+    lib.gc_profile_read_call.argtypes = [i64] + [ctypes.POINTER(f32)] * 3
     return lib
 
 
@@ -264,16 +266,21 @@ def gc_shard_dp(Q, P, pos_idx, tau, row_lse, p0, p_count, dP, ws=None, dev_statu
         raise GradCacheError(rc, "gc_shard_dp")
 
 
-def gc_profile_enable(on: bool) -> None:
-    rc = _lib.gc_profile_enable(1 if on else 0)
+def gc_profile_enable(sets) -> None:
+    """Per-kernel timing on (sets >= 1 event sets, True = 1) or off (0 / False)."""
+    rc = _lib.gc_profile_enable(int(sets))
     if rc != 0:
         raise GradCacheError(rc, "gc_profile_enable")
 
 
-def gc_profile_read() -> tuple[float, float, float]:
-    """Milliseconds of the last call's forward sweep, dQ sweep and dP sweep kernels."""
+def gc_profile_read(call: int | None = None) -> tuple[float, float, float]:
+    """Milliseconds of the forward sweep, dQ sweep and dP sweep kernels of call number `call`
+    since the enable (default: the most recent call)."""
     a, b, c = ctypes.c_float(), ctypes.c_float(), ctypes.c_float()
-    rc = _lib.gc_profile_read(ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
+    if call is None:
+        rc = _lib.gc_profile_read(ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
+    else:
+        rc = _lib.gc_profile_read_call(int(call), ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
     if rc != 0:
         raise GradCacheError(rc, "gc_profile_read")
     return a.value, b.value, c.value

@@ -106,23 +106,41 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored) {
 
 namespace {
 
-// Optional per-kernel timing (gc_profile_enable): events 2k / 2k+1 bracket kernel k.
+// Optional per-kernel timing (gc_profile_enable): in the event set of the current call, events
+// 2k / 2k+1 bracket kernel k.  Call number c since the enable uses set c % sets, so that a run of
+// up to `sets` calls can be queued without a host synchronisation in between and read afterwards.
+constexpr int kMaxProfileSets = 256;
 struct Profile {
     bool on = false;
-    bool created = false;
-    cudaEvent_t ev[6];
-    bool used[3] = {false, false, false};
+    int sets = 0;               // sets in use
+    int created = 0;            // sets whose events exist
+    int64_t calls = 0;          // calls begun since the enable
+    cudaEvent_t ev[kMaxProfileSets][6];
+    bool used[kMaxProfileSets][3];
 };
 Profile g_prof;
+
+// Every entry point that times kernels begins with this.
+void profile_begin_call() {
+    if (!g_prof.on) return;
+    const int set = (int)(g_prof.calls % g_prof.sets);
+    for (int k = 0; k < 3; ++k) g_prof.used[set][k] = false;
+    ++g_prof.calls;
+}
+int profile_set() { return (int)((g_prof.calls - 1) % g_prof.sets); }
 
 struct KernelTimer {
     int k;
     cudaStream_t st;
     KernelTimer(int kernel, cudaStream_t s) : k(kernel), st(s) {   // kernel < 0: not timed
-        if (g_prof.on && k >= 0) { cudaEventRecord(g_prof.ev[2 * k], st); g_prof.used[k] = true; }
+        if (g_prof.on && g_prof.calls > 0 && k >= 0) {
+            cudaEventRecord(g_prof.ev[profile_set()][2 * k], st);
+            g_prof.used[profile_set()][k] = true;
+        }
     }
     ~KernelTimer() {
-        if (g_prof.on && k >= 0) cudaEventRecord(g_prof.ev[2 * k + 1], st);
+        if (g_prof.on && g_prof.calls > 0 && k >= 0)
+            cudaEventRecord(g_prof.ev[profile_set()][2 * k + 1], st);
     }
 };
 
@@ -560,6 +578,7 @@ int gc_loss_fwd(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
     Plan pl = make_plan(B, N, d, dtype);
     if ((rc = check_ws(ws, ws_bytes, pl.total))) return rc;
     if ((rc = check_device())) return rc;
+    profile_begin_call();
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
     return run_fwd(p, pl, static_cast<char*>(ws), loss, row_lse, pos_logit, dev_status,
                    static_cast<cudaStream_t>(cuda_stream));
@@ -582,6 +601,7 @@ int gc_loss_fwd_static(const void* Q, int64_t ldq, const void* P, int64_t ldp,
     if ((rc = check_device())) return rc;
     void* scratch = static_scratch_ptr();
     if (!scratch) return GC_ERR_CUDA;
+    profile_begin_call();
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
     return run_fwd(p, pl, static_cast<char*>(scratch), loss, row_lse, pos_logit, dev_status,
                    static_cast<cudaStream_t>(cuda_stream));
@@ -599,6 +619,7 @@ int gc_loss_bwd(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
     Plan pl = make_plan(B, N, d, dtype);
     if ((rc = check_ws(ws, ws_bytes, pl.total))) return rc;
     if ((rc = check_device())) return rc;
+    profile_begin_call();
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
     if (dev_status && launch_pos_check(pos_idx, B, N, mask_mode, dev_status, st) != cudaSuccess)
@@ -621,6 +642,7 @@ int gc_build_cache(const void* Q, int64_t ldq, const void* P, int64_t ldp, const
     Plan pl = make_plan(B, N, d, dtype);
     if ((rc = check_ws(ws, ws_bytes, pl.total))) return rc;
     if ((rc = check_device())) return rc;
+    profile_begin_call();
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
     char* w = static_cast<char*>(ws);
@@ -641,6 +663,7 @@ int gc_build_cache_stored(const void* Q, int64_t ldq, const void* P, int64_t ldp
     if (!pl.mat) return GC_ERR_LIMIT;       // not a tcgen05 shape, or the weights exceed the limit
     if ((rc = check_ws(ws, ws_bytes, pl.total))) return rc;
     if ((rc = check_device())) return rc;
+    profile_begin_call();
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
     return run_build_stored(p, pl, static_cast<char*>(ws), loss, row_lse, pos_logit, dQ, lddq, dP,
@@ -670,6 +693,7 @@ int gc_shard_fwd_dq(const void* Q, int64_t ldq, const void* P, int64_t ldp, cons
     Plan pl = make_plan(q_count, N, d, dtype);
     if ((rc = check_ws(ws, ws_bytes, pl.total))) return rc;
     if ((rc = check_device())) return rc;
+    profile_begin_call();
     const char* q_first = static_cast<const char*>(Q) + (size_t)q0 * (size_t)ldq * elem_size(dtype);
     Problem p = make_problem(q_first, ldq, P, ldp, pos_idx + q0, q_count, N, d, tau, mask_mode, dtype);
     p.b_total = B;
@@ -692,6 +716,7 @@ int gc_shard_dp(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
     const size_t need = pl.total + align256(sizeof(int32_t) * (size_t)B);
     if ((rc = check_ws(ws, ws_bytes, need))) return rc;
     if ((rc = check_device())) return rc;
+    profile_begin_call();
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     char* w = static_cast<char*>(ws);
     // positives counted from the slice's first passage; those outside the slice match no row
@@ -704,29 +729,43 @@ int gc_shard_dp(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
     return run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, dev_status, st);
 }
 
-int gc_profile_enable(int on) {
-    if (on && !g_prof.created) {
+int gc_profile_enable(int sets) {
+    if (sets < 0 || sets > kMaxProfileSets) return GC_ERR_LIMIT;
+    for (; g_prof.created < sets; ++g_prof.created)
         for (int i = 0; i < 6; ++i)
-            if (cudaEventCreate(&g_prof.ev[i]) != cudaSuccess) return GC_ERR_CUDA;
-        g_prof.created = true;
+            if (cudaEventCreate(&g_prof.ev[g_prof.created][i]) != cudaSuccess) return GC_ERR_CUDA;
+    g_prof.on = sets > 0;
+    g_prof.sets = sets;
+    g_prof.calls = 0;
+    for (int s = 0; s < sets; ++s)
+        for (int k = 0; k < 3; ++k) g_prof.used[s][k] = false;
+    return GC_OK;
+}
+
+int gc_profile_read_call(int64_t call, float* ms_fwd, float* ms_dq, float* ms_dp) {
+    if (!ms_fwd || !ms_dq || !ms_dp) return GC_ERR_NULL;
+    float* dst[3] = {ms_fwd, ms_dq, ms_dp};
+    for (int k = 0; k < 3; ++k) *dst[k] = 0.f;
+    if (g_prof.sets == 0 || call < 0 || call >= g_prof.calls || call < g_prof.calls - g_prof.sets)
+        return GC_ERR_LIMIT;                 // never made, or its event set has been reused
+    const int set = (int)(call % g_prof.sets);
+    for (int k = 0; k < 3; ++k) {
+        if (!g_prof.used[set][k]) continue;
+        if (cudaEventSynchronize(g_prof.ev[set][2 * k + 1]) != cudaSuccess) return GC_ERR_CUDA;
+        if (cudaEventElapsedTime(dst[k], g_prof.ev[set][2 * k], g_prof.ev[set][2 * k + 1]) !=
+            cudaSuccess)
+            return GC_ERR_CUDA;
     }
-    g_prof.on = (on != 0);
-    for (int k = 0; k < 3; ++k) g_prof.used[k] = false;
     return GC_OK;
 }
 
 int gc_profile_read(float* ms_fwd, float* ms_dq, float* ms_dp) {
     if (!ms_fwd || !ms_dq || !ms_dp) return GC_ERR_NULL;
-    float* dst[3] = {ms_fwd, ms_dq, ms_dp};
-    for (int k = 0; k < 3; ++k) {
-        *dst[k] = 0.f;
-        if (!g_prof.created || !g_prof.used[k]) continue;
-        if (cudaEventSynchronize(g_prof.ev[2 * k + 1]) != cudaSuccess) return GC_ERR_CUDA;
-        if (cudaEventElapsedTime(dst[k], g_prof.ev[2 * k], g_prof.ev[2 * k + 1]) != cudaSuccess)
-            return GC_ERR_CUDA;
-        g_prof.used[k] = false;
+    if (g_prof.calls == 0) {
+        *ms_fwd = *ms_dq = *ms_dp = 0.f;
+        return GC_OK;
     }
-    return GC_OK;
+    return gc_profile_read_call(g_prof.calls - 1, ms_fwd, ms_dq, ms_dp);
 }
 
 const char* gc_status_string(int status) {
