@@ -398,3 +398,27 @@ def test_workspace_canaries(binding):
                            out.dP, out.pos_logit, ws, out.dev_status)
     torch.cuda.synchronize()
     assert bool((buf[:off] == 0xA5).all()) and bool((buf[off + need:] == 0xA5).all())
+
+
+def test_per_call_kernel_timing(binding):
+    """gc_profile_enable(n) keeps one event set per call: n queued calls can be read afterwards,
+    each with positive sweep durations; a call that was never made is refused."""
+    prob = inputs.random_problem(300, 520, 768, "bf16", seed=2, tau=0.5, scale=768 ** -0.5)
+    Q, P, pos = to_device(prob)
+    out = binding.Outputs(prob.B, prob.N, prob.d, binding.GC_BF16)
+    binding.gc_profile_enable(3)
+    try:
+        for _ in range(3):
+            binding.gc_build_cache(Q, P, pos, prob.tau, prob.mask_mode, out.loss, out.row_lse,
+                                   out.dQ, out.dP, out.pos_logit, out.ws, out.dev_status)
+        torch.cuda.synchronize()
+        for call in range(3):
+            fwd, dq, dp = binding.gc_profile_read(call)
+            assert fwd == 0.0 and 0.0 < dq < 50.0 and 0.0 < dp < 50.0      # milliseconds
+        assert binding.gc_profile_read() == binding.gc_profile_read(2)
+        with pytest.raises(binding.GradCacheError) as e:
+            binding.gc_profile_read(3)
+        assert e.value.status == 9
+    finally:
+        binding.gc_profile_enable(0)
+    assert int(out.dev_status.item()) == 0
