@@ -31,6 +31,9 @@ NOMINAL_BF16_TFLOPS = 2250.0      # public dense bf16 figure for B200, context o
 # ncu capture summarised in profiles/quad_kernel_cfg2_B4096_N8192_d768.txt.  Reported only while
 # the kernel source still has the hash it had when the counters were taken.
 NCU_TRAFFIC_BYTES = 19.1e6
+# the same for config 4, from profiles/quad_kernel_cfg4_B65536_N131072_d768.txt (average of the two
+# sweep launches, reads + writes)
+NCU_TRAFFIC_BYTES_CFG4 = 2.07e9
 NCU_TRAFFIC_SOURCE_SHA1 = "916b6c4e7d6d270f2504571c26c0464f8ffcd291"
 
 
@@ -42,7 +45,11 @@ def ncu_traffic(workload: str):
             same = hashlib.sha1(fh.read()).hexdigest() == NCU_TRAFFIC_SOURCE_SHA1
     except OSError:
         same = False
-    return NCU_TRAFFIC_BYTES if same and workload.startswith("cfg2_") else None
+    if not same:
+        return None
+    if workload.startswith("cfg2_"):
+        return NCU_TRAFFIC_BYTES
+    return NCU_TRAFFIC_BYTES_CFG4 if workload.startswith("cfg4_") else None
 
 
 def load_peaks():
