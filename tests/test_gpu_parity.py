@@ -422,3 +422,42 @@ def test_per_call_kernel_timing(binding):
     finally:
         binding.gc_profile_enable(0)
     assert int(out.dev_status.item()) == 0
+
+
+def _guarded(need, pad=4096):
+    buf = torch.full((need + 2 * pad,), 0xA5, dtype=torch.uint8, device="cuda")
+    off = (-buf.data_ptr()) % 256 + 256
+    return buf, off, buf[off:off + need]
+
+
+@pytest.mark.parametrize("B,N,d", [(300, 500, 128), (300, 520, 768), (130, 90, 1024)])
+def test_workspace_canaries_of_every_bf16_plan(binding, B, N, d):
+    """Narrow rows with a fixed row scale, four-CTA sweeps, paired wide rows: gc_build_cache,
+    the rank-local calls and gc_cache_apply stay inside the workspace sizes they report."""
+    prob = inputs.random_problem(B, N, d, "bf16", seed=B, tau=0.5, scale=d ** -0.5)
+    Q, P, pos = to_device(prob)
+    code = binding.GC_BF16
+    out = binding.Outputs(B, N, d, code)
+    buf, off, ws = _guarded(binding.gc_workspace_bytes(binding.GC_OP_BUILD, B, N, d, code))
+    binding.gc_build_cache(Q, P, pos, prob.tau, prob.mask_mode, out.loss, out.row_lse, out.dQ,
+                           out.dP, out.pos_logit, ws, out.dev_status)
+    torch.cuda.synchronize()
+    assert bool((buf[:off] == 0xA5).all()) and bool((buf[off + ws.numel():] == 0xA5).all())
+
+    q0, b, p0, n = B // 3, B - B // 3, 0, N // 2
+    buf, off, ws = _guarded(binding.gc_shard_workspace_bytes(B, N, d, code, b, n))
+    part = torch.zeros(1, device="cuda")
+    lse = out.row_lse.clone()
+    binding.gc_shard_fwd_dq(Q, P, pos, prob.tau, q0, b, part, lse, out.dQ[q0:q0 + b], ws=ws)
+    binding.gc_shard_dp(Q, P, pos, prob.tau, out.row_lse, p0, n, out.dP[p0:p0 + n], ws=ws)
+    torch.cuda.synchronize()
+    assert bool((buf[:off] == 0xA5).all()) and bool((buf[off + ws.numel():] == 0xA5).all())
+
+    d_in = 192
+    X = torch.zeros(B, d_in, dtype=torch.bfloat16, device="cuda")
+    dW = torch.zeros(d, d_in, device="cuda")
+    buf, off, ws = _guarded(binding.gc_cache_apply_workspace_bytes(B, d, d_in))
+    binding.gc_cache_apply(out.dQ, X, dW, False, ws=ws)
+    torch.cuda.synchronize()
+    assert bool((buf[:off] == 0xA5).all()) and bool((buf[off + ws.numel():] == 0xA5).all())
+    assert int(out.dev_status.item()) == 0
