@@ -103,8 +103,9 @@ int gc_loss_bwd(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
 
 /*
  * Step 2 of Section 3.3 in one call: loss, row_lse, (pos_logit) and the cache dQ, dP.  Nothing of
- * size B x N is written to global memory.  For bf16 rows wider than 256 the forward runs inside
- * the dQ sweep.  Part of the work may be queued on a stream the library owns, between a fork from
+ * size B x N is written to global memory.  For bf16 rows (d a multiple of 64) the forward runs
+ * inside the dQ sweep; where each row's weights are scaled by its positive logit, the anchor
+ * kernel that computes those logits and the sweep overlap (programmatic dependent launch).  Part of the work may be queued on a stream the library owns, between a fork from
  * and a join back into `cuda_stream`: the call is asynchronous on `cuda_stream` alone, but the
  * first such call on a device creates that stream and belongs outside any stream capture.
  */
