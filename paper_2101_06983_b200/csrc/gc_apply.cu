@@ -6,13 +6,14 @@
 //
 // as one tensor-core GEMM with fp32 accumulation.  The cache is fp32 and the tensor cores take
 // bf16, so every u is split into two bf16 terms, hi = rn(u) and lo = rn(u - hi), whose sum
-// misses u by at most 2^-17 |u|; the two terms are stacked along the contraction:
+// misses u by at most 2^-17 |u|; the two terms sit side by side as 2 d output rows:
 //
-//     Ucat = [hi(U); lo(U)]  (2 rows x d),  Xcat = [X; X]  (2 rows x d_in),  dW = Ucat^T Xcat
+//     Ucat = [hi(U) | lo(U)]  (rows x 2 d),   T = Ucat^T X  (2 d x d_in),   dW = T[0:d] + T[d:2d]
 //
 // which is the transposed-A product of gc_gemm.cu (MN-major A, contraction split over CTAs,
-// unscaled fp32 partials).  A last kernel sums the partials in part order and either overwrites
-// dW (first sub-batch) or adds to it (the outer sum of Eq. 8).  No atomics: deterministic.
+// unscaled fp32 partials) reading X as it is.  A last kernel adds the two halves of every
+// partial in part order and either overwrites dW (first sub-batch) or adds to it (the outer sum
+// of Eq. 8).  No atomics: deterministic.
 #include <cuda_bf16.h>
 
 #include "gc_internal.h"
@@ -23,50 +24,42 @@ namespace {
 
 size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
 
-// One thread per 4 columns of a U row (hi / lo split) or per 8 columns of an X row (two copies).
+// One thread per 4 columns of a U row: hi at column c, lo at column d + c of the 2 d wide row.
 __global__ void __launch_bounds__(256)
-apply_prep_kernel(const float* __restrict__ U, int64_t ldu, const __nv_bfloat16* __restrict__ X,
-                  int64_t ldx, int64_t rows, int d, int d_in, __nv_bfloat16* __restrict__ Ucat,
-                  __nv_bfloat16* __restrict__ Xcat) {
-    const int64_t u_items = rows * (d / 4);
-    const int64_t x_items = rows * (d_in / 8);
-    for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < u_items + x_items;
+apply_prep_kernel(const float* __restrict__ U, int64_t ldu, int64_t rows, int d,
+                  __nv_bfloat16* __restrict__ Ucat) {
+    const int64_t items = rows * (d / 4);
+    for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < items;
          e += (int64_t)gridDim.x * blockDim.x) {
-        if (e < u_items) {
-            const int64_t i = e / (d / 4);
-            const int c = 4 * (int)(e - i * (d / 4));
-            const float4 u = *reinterpret_cast<const float4*>(U + i * ldu + c);
-            const float v[4] = {u.x, u.y, u.z, u.w};
-            __nv_bfloat16 hi[4], lo[4];
+        const int64_t i = e / (d / 4);
+        const int c = 4 * (int)(e - i * (d / 4));
+        const float4 u = *reinterpret_cast<const float4*>(U + i * ldu + c);
+        const float v[4] = {u.x, u.y, u.z, u.w};
+        __nv_bfloat16 hi[4], lo[4];
 #pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                hi[k] = __float2bfloat16_rn(v[k]);
-                lo[k] = __float2bfloat16_rn(v[k] - __bfloat162float(hi[k]));
-            }
-            *reinterpret_cast<uint2*>(Ucat + i * d + c) = *reinterpret_cast<const uint2*>(hi);
-            *reinterpret_cast<uint2*>(Ucat + (rows + i) * d + c) = *reinterpret_cast<const uint2*>(lo);
-        } else {
-            const int64_t f = e - u_items;
-            const int64_t i = f / (d_in / 8);
-            const int c = 8 * (int)(f - i * (d_in / 8));
-            const uint4 x = *reinterpret_cast<const uint4*>(X + i * ldx + c);
-            *reinterpret_cast<uint4*>(Xcat + i * d_in + c) = x;
-            *reinterpret_cast<uint4*>(Xcat + (rows + i) * d_in + c) = x;
+        for (int k = 0; k < 4; ++k) {
+            hi[k] = __float2bfloat16_rn(v[k]);
+            lo[k] = __float2bfloat16_rn(v[k] - __bfloat162float(hi[k]));
         }
+        __nv_bfloat16* row = Ucat + i * (2 * (int64_t)d);
+        *reinterpret_cast<uint2*>(row + c) = *reinterpret_cast<const uint2*>(hi);
+        *reinterpret_cast<uint2*>(row + d + c) = *reinterpret_cast<const uint2*>(lo);
     }
 }
 
-// dW[a][b] = (accumulate ? dW[a][b] : 0) + sum_g partial[g][a][b], parts in index order.
+// dW[a][b] = (accumulate ? dW[a][b] : 0) + sum_g (partial[g][a][b] + partial[g][d + a][b]), parts
+// in index order; a partial plane is [2 d][d_in].
 __global__ void __launch_bounds__(256)
 apply_reduce_kernel(const float4* __restrict__ partial, int groups, int d, int d_in4,
                     float* __restrict__ dW, int64_t lddw, int accumulate) {
     const int64_t total = (int64_t)d * d_in4;
     for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total;
          e += (int64_t)gridDim.x * blockDim.x) {
-        float4 s = partial[e];
-        for (int g = 1; g < groups; ++g) {
-            const float4 v = partial[(int64_t)g * total + e];
-            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int g = 0; g < groups; ++g) {
+            const float4 h = partial[(int64_t)g * 2 * total + e];
+            const float4 l = partial[(int64_t)g * 2 * total + total + e];
+            s.x += h.x + l.x; s.y += h.y + l.y; s.z += h.z + l.z; s.w += h.w + l.w;
         }
         const int64_t a = e / d_in4;
         const int b = 4 * (int)(e - a * d_in4);
@@ -81,16 +74,15 @@ apply_reduce_kernel(const float4* __restrict__ partial, int groups, int d, int d
 
 struct ApplyPlan {
     int groups;
-    size_t off_u, off_x, off_part, total;
+    size_t off_u, off_part, total;
 };
 
 ApplyPlan make_apply_plan(int64_t rows, int d, int d_in) {
     ApplyPlan pl{};
-    pl.groups = gemm_groups(d, 2 * rows, d_in);
+    pl.groups = gemm_groups(2 * (int64_t)d, rows, d_in);
     size_t off = 0;
     pl.off_u = off;    off += align256((size_t)2 * rows * d * sizeof(__nv_bfloat16));
-    pl.off_x = off;    off += align256((size_t)2 * rows * d_in * sizeof(__nv_bfloat16));
-    pl.off_part = off; off += align256((size_t)pl.groups * d * d_in * sizeof(float));
+    pl.off_part = off; off += align256((size_t)pl.groups * 2 * d * d_in * sizeof(float));
     pl.total = off;
     return pl;
 }
@@ -134,18 +126,16 @@ int gc_cache_apply(const float* U, int64_t ldu, const void* X, int64_t ldx, int6
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     char* w = static_cast<char*>(ws);
     __nv_bfloat16* Ucat = reinterpret_cast<__nv_bfloat16*>(w + pl.off_u);
-    __nv_bfloat16* Xcat = reinterpret_cast<__nv_bfloat16*>(w + pl.off_x);
     float* partial = reinterpret_cast<float*>(w + pl.off_part);
 
-    const int64_t items = rows * (d / 4) + rows * (d_in / 8);
+    const int64_t items = rows * (d / 4);
     int blocks = (int)((items + 255) / 256);
     if (blocks > 8 * sm_count()) blocks = 8 * sm_count();
-    apply_prep_kernel<<<blocks, 256, 0, st>>>(U, ldu, static_cast<const __nv_bfloat16*>(X), ldx,
-                                              rows, d, d_in, Ucat, Xcat);
+    apply_prep_kernel<<<blocks, 256, 0, st>>>(U, ldu, rows, d, Ucat);
     if (cudaGetLastError() != cudaSuccess) return GC_ERR_CUDA;
-    // Ucat is the [B x N] = [2 rows x d] operand read transposed: output rows are its columns
-    if (launch_weight_gemm(Ucat, d, 2 * rows, d, 1, Xcat, d_in, d_in, pl.groups, 1.f, nullptr, 0,
-                           partial, dev_status, st) != cudaSuccess)
+    // Ucat is the [B x N] = [rows x 2 d] operand read transposed: output rows are its columns
+    if (launch_weight_gemm(Ucat, 2 * (int64_t)d, rows, 2 * (int64_t)d, 1, X, ldx, d_in, pl.groups,
+                           1.f, nullptr, 0, partial, dev_status, st) != cudaSuccess)
         return GC_ERR_CUDA;
     const int64_t total = (int64_t)d * (d_in / 4);
     blocks = (int)((total + 255) / 256);
