@@ -11,9 +11,10 @@
  * Parity pins (see tests/test_oracle_pins.py): central finite differences of the loss, row
  * sums of softmax-minus-onehot, closed forms for identical representations and for the 1x2
  * logistic case, scale and permutation symmetries, and the paper's exactness claim on a linear
- * encoder; gco_cache_apply (Step 3 for a linear encoder) by the finite-difference gradient with
- * respect to the encoder matrix and a hand-worked example.  No function here is "parity
- * unpinned".
+ * encoder; gco_query_rows and gco_passage_rows by the same hand-worked example, finite
+ * differences and closed form, row for row; gco_cache_apply (Step 3 for a linear encoder) by the
+ * finite-difference gradient with respect to the encoder matrix and a hand-worked example.  No
+ * function here is "parity unpinned".
  *
  * Notation (paper, Section 3.1-3.2): Q row i is f(s_i), P row j is g(t_j), pos_idx[i] is r_i,
  * tau the temperature, S_ij = <f(s_i), g(t_j)> / tau.

@@ -27,6 +27,23 @@ MUTANTS = {
     "G read transposed in dP": ("double g = G[i * N + j];\n                    const double* q", "double g = G[(j % B) * N + (i % N)];\n                    const double* q"),
     "positive index off by one": ("total += lse[i] - S[i * N + pos_idx[i]];", "total += lse[i] - S[i * N + (pos_idx[i] + 1) % N];"),
     "max instead of logsumexp": ("return m + log(sum);", "return m;"),
+    "query_rows: dQ rows not divided by tau": (
+        "for (int64_t k = 0; k < d; ++k) out[k] /= tau;\n            }\n        }\n        free(S_row);",
+        "}\n        }\n        free(S_row);"),
+    "query_rows: one-hot on the wrong column": (
+        "double g = (p - ((j == pos_idx[i]) ? 1.0 : 0.0)) / (double)B;\n                    const double* pj",
+        "double g = (p - ((j == (pos_idx[i] + 1) % N) ? 1.0 : 0.0)) / (double)B;\n                    const double* pj"),
+    "query_rows: lse of the wrong row": (
+        "double lse = lse_row(S_row, i, N, mask_mode);", "double lse = lse_row(S_row, (i + 1) % B, N, mask_mode);"),
+    "passage_rows: row_lse read at the wrong index": (
+        "double p = allowed(mask_mode, i, j) ? exp(s - row_lse[i]) : 0.0;",
+        "double p = allowed(mask_mode, i, j) ? exp(s - row_lse[(i + 1) % B]) : 0.0;"),
+    "passage_rows: mask leaks": (
+        "double p = allowed(mask_mode, i, j) ? exp(s - row_lse[i]) : 0.0;", "double p = exp(s - row_lse[i]);"),
+    "passage_rows: logits not divided by tau": ("s /= tau;", ""),
+    "passage_rows: one-hot dropped": (
+        "double g = (p - ((j == pos_idx[i]) ? 1.0 : 0.0)) / (double)B;\n            for",
+        "double g = p / (double)B;\n            for"),
     "cache_apply reads U transposed": ("s += U[i * d + a] * X[i * d_in + b];",
                                        "s += U[(a % rows) * d + (i % d)] * X[i * d_in + b];"),
     "cache_apply overwrites instead of accumulating": ("if (accumulate) dW[a * d_in + b] += s;",
@@ -70,6 +87,46 @@ def _wrap(libpath):
             raise ValueError(f"rejected ({rc})")
         return dict(loss=float(loss.value), row_lse=lse, pos_logit=pl, dQ=dQ, dP=dP)
 
+    ip = ctypes.POINTER(ctypes.c_int32)
+    lp = ctypes.POINTER(ctypes.c_int64)
+    i64 = ctypes.c_int64
+    lib.gco_query_rows.restype = ctypes.c_int
+    lib.gco_query_rows.argtypes = [dp, dp, ip, i64, i64, i64, ctypes.c_double, ctypes.c_int, lp, i64,
+                                   dp, dp, dp]
+    lib.gco_passage_rows.restype = ctypes.c_int
+    lib.gco_passage_rows.argtypes = [dp, dp, ip, i64, i64, i64, ctypes.c_double, ctypes.c_int, dp, lp,
+                                     i64, dp]
+
+    def query_rows(Q, P, pos_idx, rows, tau=1.0, mask_mode=0, grads=True):
+        Q, P, pos = real._prep(Q, P, pos_idx)
+        B, d = Q.shape
+        rows = np.ascontiguousarray(rows, dtype=np.int64)
+        n = rows.shape[0]
+        lse, pl, dQ = np.empty(n), np.empty(n), np.empty((n, d))
+        rc = lib.gco_query_rows(real._ptr(Q, ctypes.c_double), real._ptr(P, ctypes.c_double),
+                                real._ptr(pos, ctypes.c_int32), B, P.shape[0], d, float(tau),
+                                int(mask_mode), real._ptr(rows, ctypes.c_int64), n,
+                                real._ptr(lse, ctypes.c_double), real._ptr(pl, ctypes.c_double),
+                                real._ptr(dQ, ctypes.c_double))
+        if rc != 0:
+            raise ValueError(f"rejected ({rc})")
+        return dict(row_lse=lse, pos_logit=pl, dQ=dQ)
+
+    def passage_rows(Q, P, pos_idx, row_lse, rows, tau=1.0, mask_mode=0):
+        Q, P, pos = real._prep(Q, P, pos_idx)
+        B, d = Q.shape
+        lse = real._f64(row_lse)
+        rows = np.ascontiguousarray(rows, dtype=np.int64)
+        n = rows.shape[0]
+        dP = np.empty((n, d))
+        rc = lib.gco_passage_rows(real._ptr(Q, ctypes.c_double), real._ptr(P, ctypes.c_double),
+                                  real._ptr(pos, ctypes.c_int32), B, P.shape[0], d, float(tau),
+                                  int(mask_mode), real._ptr(lse, ctypes.c_double),
+                                  real._ptr(rows, ctypes.c_int64), n, real._ptr(dP, ctypes.c_double))
+        if rc != 0:
+            raise ValueError(f"rejected ({rc})")
+        return dP
+
     lib.gco_cache_apply.restype = ctypes.c_int
     lib.gco_cache_apply.argtypes = [dp, dp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_int, dp]
@@ -88,7 +145,8 @@ def _wrap(libpath):
         return dW
 
     return types.SimpleNamespace(
-        build_cache=build_cache, cache_apply=cache_apply,
+        build_cache=build_cache, cache_apply=cache_apply, query_rows=query_rows,
+        passage_rows=passage_rows,
         loss_only=lambda Q, P, pos, tau=1.0, mask=0: build_cache(Q, P, pos, tau, mask)["loss"])
 
 
@@ -101,6 +159,10 @@ def _pins(o):
     yield lambda: pins.test_one_query_two_passages_is_logistic_loss(o)
     yield lambda: pins.test_scale_and_permutation_symmetry(o)
     yield lambda: pins.test_duplicate_positives_sum_in_epsilon(o)
+    yield lambda: pins.test_row_sampled_entry_points_on_the_hand_worked_example(o)
+    yield lambda: pins.test_row_sampled_entry_points_match_finite_differences(o, 0.1, 1)
+    yield lambda: pins.test_row_sampled_entry_points_match_finite_differences(o, 1.0, 0)
+    yield lambda: pins.test_row_sampled_entry_points_identical_representations(o)
     yield lambda: pins.test_cache_apply_hand_worked_example(o)
     yield lambda: pins.test_cache_apply_chunks_reproduce_full_batch_parameter_gradient(o)
 

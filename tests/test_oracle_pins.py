@@ -222,6 +222,74 @@ def test_against_autograd_cross_entropy(oracle, mask):
     np.testing.assert_allclose(dp, p.grad.numpy()[prow], rtol=1e-10, atol=1e-14)
 
 
+# ---- the row-sampled entry points (query_rows, passage_rows) -----------------------------------
+def test_row_sampled_entry_points_on_the_hand_worked_example(oracle):
+    """Same rational instance as above, read off the fixture: query_rows must give rows of G (P is
+    the identity) and passage_rows the hand-derived combinations of the query rows."""
+    g = _golden()
+    ln = math.log
+    Q = np.array([[ln(1), ln(2), ln(3)], [ln(4), ln(1), ln(1)]])
+    P = np.eye(3)
+    pos = np.array([2, 0], np.int32)
+    G = np.array(g["G_times_12"]).reshape(2, 3) / 12.0
+    C = np.array(g["dP_coeff_times_12"]).reshape(3, 2) / 12.0
+    rows = np.array([1, 0, 1], np.int64)
+    qr = oracle.query_rows(Q, P, pos, rows, 1.0, 0)
+    np.testing.assert_allclose(qr["dQ"], G[rows], rtol=0, atol=1e-15)
+    np.testing.assert_allclose(qr["row_lse"], [ln(6)] * 3, rtol=1e-15)
+    np.testing.assert_allclose(qr["pos_logit"], [ln(4), ln(3), ln(4)], rtol=1e-15)
+    prow = np.array([2, 0, 1, 2], np.int64)
+    dp = oracle.passage_rows(Q, P, pos, np.array([ln(6), ln(6)]), prow, 1.0, 0)
+    np.testing.assert_allclose(dp, (C @ Q)[prow], rtol=0, atol=1e-15)
+
+
+@pytest.mark.parametrize("tau", [1.0, 0.1])
+@pytest.mark.parametrize("mask", [0, 1])
+def test_row_sampled_entry_points_match_finite_differences(oracle, tau, mask):
+    """Rows of dQ from query_rows and rows of dP from passage_rows (fed the lse that query_rows
+    itself returns for every query) against central finite differences of the loss of Eq. 1, and
+    row for row against build_cache.  Rows are listed out of order and with a repeat."""
+    B, N, d = 4, 8, 5
+    Q, P, pos = _rand(11 + B + 7 * N, B, N, d, mask)
+    Q *= 0.7
+    P *= 0.7
+    gq = _fd_grad(lambda: oracle.loss_only(Q, P, pos, tau, mask), Q)
+    gp = _fd_grad(lambda: oracle.loss_only(Q, P, pos, tau, mask), P)
+    scale = max(np.abs(gq).max(), np.abs(gp).max(), 1.0)
+    all_rows = oracle.query_rows(Q, P, pos, np.arange(B, dtype=np.int64), tau, mask)
+    rows = np.array([3, 0, 2, 3], np.int64)
+    qr = oracle.query_rows(Q, P, pos, rows, tau, mask)
+    assert np.abs(qr["dQ"] - gq[rows]).max() <= 1e-7 * scale
+    prow = np.array([7, 1, 0, 4, 1], np.int64)
+    dp = oracle.passage_rows(Q, P, pos, all_rows["row_lse"], prow, tau, mask)
+    assert np.abs(dp - gp[prow]).max() <= 1e-7 * scale
+    full = oracle.build_cache(Q, P, pos, tau, mask)
+    np.testing.assert_allclose(qr["dQ"], full["dQ"][rows], rtol=0, atol=1e-14)
+    np.testing.assert_allclose(qr["row_lse"], full["row_lse"][rows], rtol=0, atol=1e-14)
+    np.testing.assert_allclose(qr["pos_logit"], full["pos_logit"][rows], rtol=0, atol=1e-14)
+    np.testing.assert_allclose(dp, full["dP"][prow], rtol=0, atol=1e-14)
+
+
+def test_row_sampled_entry_points_identical_representations(oracle):
+    """All logits equal: lse = log N, dQ rows vanish, dP_j = (B/N - c_j) q / (B tau)."""
+    B, N, tau = 6, 10, 0.25
+    q = np.array([0.3, -0.2, 0.5, 0.1])
+    Q = np.tile(q, (B, 1))
+    P = np.tile(q, (N, 1))
+    pos = np.array([0, 0, 3, 4, 9, 9], np.int32)
+    rows = np.array([5, 0, 2], np.int64)
+    qr = oracle.query_rows(Q, P, pos, rows, tau, 0)
+    s = float(q @ q) / tau
+    np.testing.assert_allclose(qr["row_lse"], s + math.log(N), rtol=1e-14)
+    np.testing.assert_allclose(qr["pos_logit"], s, rtol=1e-14)
+    assert np.abs(qr["dQ"]).max() <= 1e-16
+    c = np.bincount(pos, minlength=N)
+    expect = ((B / N - c) / (B * tau))[:, None] * q[None, :]
+    prow = np.array([9, 0, 1, 3], np.int64)
+    dp = oracle.passage_rows(Q, P, pos, np.full(B, s + math.log(N)), prow, tau, 0)
+    np.testing.assert_allclose(dp, expect[prow], rtol=0, atol=1e-15)
+
+
 # ---- the paper's exactness claim on a linear encoder (Eq. 2, Eq. 8-9) -------------------------
 def test_cached_chunked_gradient_equals_full_batch_gradient(oracle):
     """f(s) = W_f s, g(t) = W_g t.  Full-batch dL/dW_f (by finite differences on W_f) equals the
