@@ -76,7 +76,8 @@ size_t gc_workspace_bytes(int op, int64_t B, int64_t N, int d, int dtype);
 /* Name of the kernel plan the library will use for these sizes: "tcgen05" (TMA + tcgen05 MMA
  * with TMEM accumulators; bf16, d a multiple of 64 up to 4096; one CTA, a CTA pair or a cluster
  * of four per tile, by shape) or "simt" (fp32 FMA tiles; every other case, including all fp32
- * inputs).  Static string. */
+ * inputs); "invalid" for an unknown op, non-positive sizes, or a problem GC_OP_BUILD_STORED refuses.
+ * Static string. */
 const char* gc_plan_name(int op, int64_t B, int64_t N, int d, int dtype);
 
 /* Number of kernels one call launches for these sizes (for launch accounting). */
@@ -162,8 +163,8 @@ int gc_cache_apply(const float* U, int64_t ldu, const void* X, int64_t ldx, int6
 
 /*
  * Section 3.4 (multi-GPU training): after the all-gather every GPU holds all representations,
- * the loss is defined over all of them, and "the n-th GPU only computes gradient of its local
- * representations".  These two calls are that rank-local part of Step 2 for a rank that owns
+ * the loss is defined over all of them, and each rank forms the gradients of its own
+ * representations only.  These two calls are that rank-local part of Step 2 for a rank that owns
  * query rows [q0, q0 + q_count) and passage rows [p0, p0 + p_count) of the gathered Q [B x d] and
  * P [N x d] (pos_idx [B] indexes rows of the gathered P).  Unlike the paper's scheme a rank does
  * not redo the whole forward: it needs lse_i of its own queries for dQ and, for dP, lse_i of all
@@ -206,7 +207,8 @@ int gc_shard_dp(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
  * The scratch (per-part row maxima, row sums and the gathered positive logits) lives in a
  * fixed array of GC_STATIC_SCRATCH_BYTES inside the library image, so every GPU that loads the
  * library carries that much extra memory until the process exits.  Problems whose forward
- * scratch (gc_static_scratch_need) exceeds it are refused with GC_ERR_LIMIT and nothing is
+ * scratch (gc_static_scratch_need: the slots the forward sweep itself writes, not the larger
+ * workspace of the other calls) exceeds it are refused with GC_ERR_LIMIT and nothing is
  * launched.  The first call on each device looks up the array's device address (once, with that
  * device current); make that first call outside any stream capture.  All calls on a device
  * share the one array, and it keeps whatever the previous call left: the kernels overwrite
@@ -236,6 +238,19 @@ int gc_loss_fwd_static(const void* Q, int64_t ldq, const void* P, int64_t ldp,
 int gc_profile_enable(int sets);
 int gc_profile_read(float* ms_fwd, float* ms_dq, float* ms_dp);
 int gc_profile_read_call(int64_t call, float* ms_fwd, float* ms_dq, float* ms_dp);
+
+/*
+ * Test aid (no counterpart in the paper).  Every wait a tensor-core kernel of this library makes
+ * on an on-chip barrier is bounded: when the limit passes, the CTA stops waiting, ORs
+ * GC_DEV_WAIT_LIMIT into *dev_status and returns, and the context stays usable.  This call
+ * launches one small CTA that runs that same wait helper, with a limit of limit_ns nanoseconds
+ * (1 .. 1e8, else GC_ERR_LIMIT), on a barrier that nothing arrives on, so that the give-up path
+ * can be observed without any fault: afterwards *dev_status has GC_DEV_WAIT_LIMIT set and
+ * *waited_ns (device pointer, may be NULL) holds how long the wait lasted.  Asynchronous on
+ * cuda_stream.
+ */
+int gc_selftest_wait_limit(uint64_t limit_ns, int* dev_status, unsigned long long* waited_ns,
+                           void* cuda_stream);
 
 /* Human-readable name of a gc_status value.  Static string. */
 const char* gc_status_string(int status);

@@ -23,7 +23,7 @@ EXPORTS = ("gc_workspace_bytes", "gc_plan_name", "gc_kernel_launches", "gc_loss_
            "gc_profile_enable",
            "gc_profile_read", "gc_profile_read_call", "gc_static_scratch_need", "gc_loss_fwd_static",
            "gc_cache_apply_workspace_bytes", "gc_cache_apply", "gc_shard_workspace_bytes",
-           "gc_shard_fwd_dq", "gc_shard_dp")
+           "gc_shard_fwd_dq", "gc_shard_dp", "gc_selftest_wait_limit")
 GC_STATIC_SCRATCH_BYTES = 2 << 20
 
 
@@ -75,6 +75,8 @@ def _load() -> ctypes.CDLL:
                                              vp, vp]
     lib.gc_shard_dp.restype = i32
     lib.gc_shard_dp.argtypes = common + [vp, i64, i64, vp, i64, vp, ctypes.c_size_t, vp, vp]
+    lib.gc_selftest_wait_limit.restype = i32
+    lib.gc_selftest_wait_limit.argtypes = [ctypes.c_uint64, vp, vp, vp]
     lib.gc_profile_enable.restype = i32
     lib.gc_profile_enable.argtypes = [i32]
     lib.gc_profile_read.restype = i32
@@ -264,6 +266,15 @@ def gc_shard_dp(Q, P, pos_idx, tau, row_lse, p0, p_count, dP, ws=None, dev_statu
                           ws.numel(), _ptr(dev_status), _stream())
     if rc != 0:
         raise GradCacheError(rc, "gc_shard_dp")
+
+
+def gc_selftest_wait_limit(limit_ns: int, dev_status, waited_ns=None) -> None:
+    """Runs the library's bounded on-chip wait with a limit of `limit_ns` on a barrier nothing
+    arrives on: ORs GC_DEV_WAIT_LIMIT into dev_status[0] (int32) and writes the time waited to
+    waited_ns[0] (int64 tensor, optional)."""
+    rc = _lib.gc_selftest_wait_limit(int(limit_ns), _ptr(dev_status), _ptr(waited_ns), _stream())
+    if rc != 0:
+        raise GradCacheError(rc, "gc_selftest_wait_limit")
 
 
 def gc_profile_enable(sets) -> None:

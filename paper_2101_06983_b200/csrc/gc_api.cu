@@ -521,6 +521,18 @@ static __device__ __align__(256) unsigned char g_static_scratch[GC_STATIC_SCRATC
 
 namespace {
 
+// The forward sweep alone writes g_fwd (scale, sum) slots per row: lays those regions, the
+// gathered positive logits and the loss scratch out back to back (the workspace layout of the
+// other calls reserves the slots of the widest build plan) and returns the bytes they take.
+size_t forward_layout(Plan* pl, int64_t B) {
+    size_t off = 0;
+    pl->off_m = off;    off += align256(sizeof(float) * (size_t)pl->g_fwd * (size_t)B);
+    pl->off_l = off;    off += align256(sizeof(float) * (size_t)pl->g_fwd * (size_t)B);
+    pl->off_pos = off;  off += align256(sizeof(float) * (size_t)B);
+    pl->off_red = off;  off += 2048;
+    return off;
+}
+
 // Device address of g_static_scratch on the current device, or nullptr on failure.
 void* static_scratch_ptr() {
     static void* cached[64] = {nullptr};
@@ -553,8 +565,8 @@ size_t gc_workspace_bytes(int op, int64_t B, int64_t N, int d, int dtype) {
 }
 
 const char* gc_plan_name(int op, int64_t B, int64_t N, int d, int dtype) {
-    (void)op;
-    if (B <= 0 || N <= 0 || d <= 0) return "invalid";
+    if (op < GC_OP_FWD || op > GC_OP_BUILD_STORED || B <= 0 || N <= 0 || d <= 0) return "invalid";
+    if (op == GC_OP_BUILD_STORED && !make_plan(B, N, d, dtype, true).mat) return "invalid";
     return tc_supported(B, N, d, dtype) ? "tcgen05" : "simt";
 }
 
@@ -586,7 +598,8 @@ int gc_loss_fwd(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
 
 size_t gc_static_scratch_need(int64_t B, int64_t N, int d, int dtype) {
     if (B <= 0 || N <= 0 || d <= 0 || (dtype != GC_F32 && dtype != GC_BF16)) return 0;
-    return make_plan(B, N, d, dtype).off_accq;   // the forward part of the workspace layout
+    Plan pl = make_plan(B, N, d, dtype);
+    return forward_layout(&pl, B);
 }
 
 int gc_loss_fwd_static(const void* Q, int64_t ldq, const void* P, int64_t ldp,
@@ -597,7 +610,7 @@ int gc_loss_fwd_static(const void* Q, int64_t ldq, const void* P, int64_t ldp,
     if (rc) return rc;
     if (!loss || !row_lse) return GC_ERR_NULL;
     Plan pl = make_plan(B, N, d, dtype);
-    if (pl.off_accq > (size_t)GC_STATIC_SCRATCH_BYTES) return GC_ERR_LIMIT;
+    if (forward_layout(&pl, B) > (size_t)GC_STATIC_SCRATCH_BYTES) return GC_ERR_LIMIT;
     if ((rc = check_device())) return rc;
     void* scratch = static_scratch_ptr();
     if (!scratch) return GC_ERR_CUDA;

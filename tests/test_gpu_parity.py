@@ -207,18 +207,18 @@ def _check_properties(prob, out, Q, P, units=4):
 
 
 def test_config2_headline_full_size(binding, oracle):
+    """Headline workload, every element of the loss, row_lse, pos_logit, dQ and dP against the full
+    oracle (a few seconds on the host)."""
     prob = inputs.config(2)
     assert binding.gc_plan_name(binding.GC_OP_BUILD, prob.B, prob.N, prob.d, binding.GC_BF16) \
         == "tcgen05"
     Q, P, pos = to_device(prob)
     out = binding.build_cache(Q, P, pos, prob.tau, prob.mask_mode)
     torch.cuda.synchronize()
-    assert int(out.dev_status.item()) == 0
-    fwd = oracle.build_cache(prob.Q, prob.P, prob.pos_idx, prob.tau, prob.mask_mode, grads=False)
-    assert rel_err_scalar(out.loss.item(), fwd["loss"]) <= TOL["bf16"]["loss"]
+    ref = _oracle_full(oracle, prob)
+    check_against_oracle(prob, out, ref)
     lse = out.row_lse.cpu().numpy().astype(np.float64)
-    assert np.abs(lse - fwd["row_lse"]).max() <= 1e-4 * np.abs(fwd["row_lse"]).max()
-    _check_sampled(oracle, prob, out, 96, 48, full_lse=fwd["row_lse"], seed=2)
+    assert np.abs(lse - ref["row_lse"]).max() <= 1e-4 * np.abs(ref["row_lse"]).max()
     _check_properties(prob, out, Q, P)
 
 
@@ -235,7 +235,18 @@ def test_config4_extreme_batch_never_stores_S(binding, oracle):
     grown = torch.cuda.max_memory_allocated() - before
     assert grown < 2 * ((prob.B + prob.N) * prob.d * 4) + need + (64 << 20)
     assert int(out.dev_status.item()) == 0
-    _check_sampled(oracle, prob, out, 40, 0, seed=4)
+    # 256 sampled query rows (lse, positive logit, dQ) against the oracle.  Rows of dP need the
+    # logsumexp of all 65536 queries, which the oracle would take minutes to produce; the library's
+    # row_lse stands in for it here, after the sampled rows of it have just matched the oracle.
+    _check_sampled(oracle, prob, out, 256, 0, seed=4)
+    gpu_lse = out.row_lse.cpu().numpy().astype(np.float64)
+    rng = np.random.default_rng(44)
+    prow = np.unique(np.r_[0, 1, prob.N - 1, rng.integers(0, prob.N, 64)]).astype(np.int64)
+    assert prow.size >= 64
+    dp_ref = oracle.passage_rows(prob.Q, prob.P, prob.pos_idx, gpu_lse, prow, prob.tau,
+                                 prob.mask_mode)
+    dp = out.dP[torch.from_numpy(prow).cuda()].cpu().numpy()
+    assert grad_err(dp, dp_ref) <= TOL["bf16"]["grad"]
     _check_properties(prob, out, Q, P)
     # the loss is the mean of (lse - positive logit); spot rows already match the oracle
     lse = out.row_lse.double()

@@ -6,7 +6,9 @@ Collected last on purpose (file name): a run that stops at the first failure has
 exercised every other test.  Each case calls the entry point through the C ABI twice in a row -
 the second call finds the array full of the first call's values - and compares with gc_loss_fwd
 given an ordinary workspace.  Both run the same kernels, so the results must agree bit for bit,
-which is well inside the tolerances the parity tests use."""
+which is well inside the tolerances the parity tests use; the CPU oracle is compared as well, at
+the tolerances of the parity tests, so that the check does not rest on the CUDA path alone."""
+import numpy as np
 import pytest
 import torch
 
@@ -31,8 +33,12 @@ def _problems():
     yield inputs.random_problem(129, 130, 40, "f32", seed=4, tau=0.5, scale=0.5)
 
 
-def test_static_scratch_forward_matches_workspace_forward(binding):
+def test_static_scratch_forward_matches_workspace_forward(binding, oracle):
+    from gpu_util import TOL
     for prob in _problems():
+        want = oracle.build_cache(prob.Q, prob.P, prob.pos_idx, prob.tau, prob.mask_mode,
+                                  grads=False)
+        tol = TOL[prob.dtype]
         Q, P, pos = binding.problem_tensors(prob)
         code = binding._dtype_code(Q)
         assert binding.gc_static_scratch_need(prob.B, prob.N, prob.d, code) \
@@ -55,6 +61,13 @@ def test_static_scratch_forward_matches_workspace_forward(binding):
             assert torch.equal(lse, ref.row_lse), (prob.name, call)
             assert torch.equal(pl, ref.pos_logit), (prob.name, call)
             torch.testing.assert_close(loss, ref.loss, rtol=1e-5, atol=0)
+            assert abs(loss.item() - want["loss"]) <= tol["loss"] * abs(want["loss"])
+            got_lse = lse.cpu().numpy().astype(np.float64)
+            assert np.abs(got_lse - want["row_lse"]).max() \
+                <= tol["lse"] * max(1.0, np.abs(want["row_lse"]).max())
+            got_pl = pl.cpu().numpy().astype(np.float64)
+            assert np.abs(got_pl - want["pos_logit"]).max() \
+                <= tol["lse"] * max(1.0, np.abs(want["pos_logit"]).max())
 
 
 def test_static_scratch_refuses_oversized_problems(binding):
