@@ -18,11 +18,13 @@
 // and a later pass adds it to the piece that began at the row's first tile.
 //
 // Hand-off: a ring slot holds one W tile as eight 16 KB chunk images (2 CTAs x 4 chunks of 128
-// rows x 64 columns) in the layout the MMA reads from shared memory.  The S pair's softmax warps
-// store 4 KB pieces with bulk tensor stores and then add 1 to the slot's ready counter (release);
-// the acc pairs poll it (acquire, bounded), load the chunks with bulk tensor loads and add 1 to
-// the slot's consumed counter once they have landed; the S pair reuses a slot after both acc
-// pairs have consumed it.  Tiles are produced and consumed in one global order, so no wait can
+// rows x 64 columns, rows of 128 bytes).  The S pair's softmax warps write their rows straight
+// from registers (32 bytes per store) and, a little later, fence and add 1 to the slot's ready
+// counter (release); the acc pairs poll it (acquire, bounded), load the chunks with bulk tensor
+// loads and add 1 to the slot's consumed counter once they have landed; the S pair reuses a slot
+// after both acc pairs have consumed it.  Shared memory holds nothing but the operand rings: a
+// load takes about 3 K cycles to come back when every SM streams, so the bytes in flight, not the
+// request rate, are what sustains the operand bandwidth.  Tiles are produced and consumed in one global order, so no wait can
 // be cyclic; all CTAs of the launch must be resident at once (the host sizes the grid for that).
 // Every wait is bounded.
 #include "tc_common.cuh"
@@ -35,19 +37,25 @@ enum { DMODE_DQ = 1, DMODE_DP = 2, DMODE_FA = 3 };
 
 constexpr int DUO_TILE = 256;                  // x rows of a pair = y rows of a tile
 constexpr int DUO_RING = 4;                    // W slots per S pair
-constexpr int S_STAGES = 5;                    // S role: stages of one X chunk + one Y chunk
+constexpr int S_STAGES = 6;                    // S role: stages of one X chunk + one Y chunk
 constexpr uint32_t S_STAGE_BYTES = 2 * CHUNK_BYTES;
-constexpr int A_STAGES = 6;                    // acc role: W chunks (16 KB)
+constexpr int A_STAGES = 4;                    // acc role: W chunks (16 KB)
 constexpr int B_STAGES = 4;                    // acc role: 64 y rows x this CTA's columns
 constexpr uint32_t B_ATOM_BYTES = 8192;        // 64 rows x 64 columns
 constexpr uint32_t B_STAGE_BYTES = 3 * B_ATOM_BYTES;
-constexpr uint32_t STG_BYTES = NSOFT * 4096;   // one 4 KB staging buffer per softmax / epilogue warp
 constexpr uint32_t TAB_BYTES = NSOFT * 1024;   // DP: per warp, lse and pos_idx of its 128 queries
-constexpr size_t DUO_SMEM_S = (size_t)S_STAGES * S_STAGE_BYTES + STG_BYTES + TAB_BYTES;
+constexpr size_t DUO_SMEM_S = (size_t)S_STAGES * S_STAGE_BYTES + TAB_BYTES;
+constexpr uint32_t STG_BYTES = NSOFT * 8192;   // acc role: two 4 KB staging buffers per epilogue warp
 constexpr size_t DUO_SMEM_A = (size_t)A_STAGES * CHUNK_BYTES + (size_t)B_STAGES * B_STAGE_BYTES +
                               STG_BYTES;
 constexpr size_t DUO_SMEM = 1024 + (DUO_SMEM_S > DUO_SMEM_A ? DUO_SMEM_S : DUO_SMEM_A);
 static_assert(DUO_SMEM <= SMEM_LIMIT - SMEM_STATIC_RESERVE, "shared memory budget");
+// Warps: 0..2 issue the bulk loads (S role: 0 and 1; warp 2 publishes finished W tiles), 3 issues
+// the MMAs, 4..11 are the softmax / epilogue warps (twelve warps: registers are handed out to
+// four warps at a time, a thirteenth would cost as much as sixteen).
+constexpr int DPROD = 3;
+constexpr int DMMA_WARP = DPROD;
+constexpr int DTHREADS = 32 * (DPROD + 1 + NSOFT);
 constexpr int DUO_FLAG_WORDS = 64;             // words before the counters (word 0: abort)
 
 struct DuoParams {
@@ -69,19 +77,24 @@ struct DuoParams {
     float* pos_logit;         // FA
     int* range_flag;          // FA
     int* flags;               // word 0: abort; then ready[S pair][slot][rank], consumed[S pair][slot]
+    uint8_t* ring;            // W ring
+    float* out_main;          // [nx][ld_main]: pieces that begin at the first tile of their x pair
+    int64_t ld_main;
+    float* extra;             // [nteams][256][d]: the other pieces, one plane per team
     int* dev_status;
     Gate gate;
     int* zero_me;
 };
 
 struct DuoBars {
-    uint64_t full[A_STAGES];       // S role: ring stage filled (in the leader, both CTAs' bytes);
-    uint64_t empty[A_STAGES];      //   acc role: W chunk ring
+    uint64_t full[S_STAGES];       // S role: ring stage filled (in the leader, both CTAs' bytes);
+    uint64_t empty[S_STAGES];      //   acc role: W chunk ring
     uint64_t b_full[B_STAGES];     // acc role: Y ring
     uint64_t b_empty[B_STAGES];
     uint64_t t_full[2];            // S role: S tile b complete; acc role: [0] accumulator complete
     uint64_t t_free[2];            // this CTA's eight warps have read it
     uint64_t t_free_peer[2];       // leader: the same of the second CTA, forwarded by its idle MMA warp
+    uint64_t w_stored[DUO_RING];   // S role: the eight softmax warps have written their rows of a slot
 };
 
 // ---- schedule: tile s = xp * YT + yt; team t owns the contiguous range [lo, hi) -----------------
@@ -104,6 +117,9 @@ __device__ __forceinline__ int ld_acquire_gpu(const int* p) {
 }
 __device__ __forceinline__ void red_release_gpu(int* p, int v) {
     asm volatile("red.release.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void red_relaxed_gpu(int* p, int v) {
+    asm volatile("red.relaxed.gpu.global.add.s32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void fence_proxy_async_all() {
     asm volatile("fence.proxy.async;" ::: "memory");
@@ -147,11 +163,11 @@ __device__ __forceinline__ void mma_pair(uint32_t d_tmem, uint32_t a_lo, uint32_
 }
 
 template <int MODE>
-__global__ void __launch_bounds__(NTHREADS, 1)
+__global__ void __launch_bounds__(DTHREADS, 1)
 duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapYs,
-           const __grid_constant__ CUtensorMap mapYa, const __grid_constant__ CUtensorMap mapWst,
-           const __grid_constant__ CUtensorMap mapWld, const __grid_constant__ CUtensorMap mapMain,
-           const __grid_constant__ CUtensorMap mapExtra, const DuoParams p) {
+           const __grid_constant__ CUtensorMap mapYa, const __grid_constant__ CUtensorMap mapWld,
+           const __grid_constant__ CUtensorMap mapMain, const __grid_constant__ CUtensorMap mapExtra,
+           const DuoParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) DuoBars bars;
     __shared__ uint32_t tmem_base_s;
@@ -187,7 +203,7 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
 
     if (threadIdx.x == 0) {
         abort_s = 0;
-        for (int s = 0; s < A_STAGES; ++s) {
+        for (int s = 0; s < S_STAGES; ++s) {
             mbar_init(smem_u32(&bars.full[s]), 1);
             mbar_init(smem_u32(&bars.empty[s]), 1);
         }
@@ -200,9 +216,10 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
             mbar_init(smem_u32(&bars.t_free[b]), NSOFT);
             mbar_init(smem_u32(&bars.t_free_peer[b]), 1);
         }
+        for (int b = 0; b < DUO_RING; ++b) mbar_init(smem_u32(&bars.w_stored[b]), NSOFT);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == MMA_WARP) {
+    if (warp == DMMA_WARP) {
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
                      ::"r"(smem_u32(&tmem_base_s)), "r"((uint32_t)TMEM_COLS) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
@@ -219,10 +236,23 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
         // S role
         // =========================================================================================
         const uint32_t ring_smem = base;
-        const uint32_t stg_smem = base + S_STAGES * S_STAGE_BYTES;
-        const uint32_t tab_smem = stg_smem + STG_BYTES;
+        const uint32_t tab_smem = base + S_STAGES * S_STAGE_BYTES;
         const int sp = 2 * team + sidx;
-        if (warp < NPROD) {
+        if (warp == 2) {
+            // ------------------------------ publisher ------------------------------------------
+            // The softmax warps' stores of a tile become visible to the acc pairs here: one fence
+            // after all eight warps have arrived covers their stores (release is cumulative), and
+            // it stalls this warp instead of theirs.
+            const int nj = (nk - sidx + 1) / 2;
+            for (int j = 0; j < nj; ++j) {
+                const int slot = j % DUO_RING;
+                if (!mbar_wait(smem_u32(&bars.w_stored[slot]), (uint32_t)((j / DUO_RING) & 1), abort_flag))
+                    break;
+                __threadfence();
+                if (lane == 0) red_release_gpu(ready + (sp * DUO_RING + slot) * 2 + (int)rank, NSOFT);
+                __syncwarp();
+            }
+        } else if (warp < 2) {
             // ------------------------------ TMA producers -------------------------------------
             int stage = 0, item = 0;
             uint32_t phase = 0;
@@ -236,7 +266,7 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
                     const int st = stage;
                     const uint32_t ph = phase;
                     if (++stage == S_STAGES) { stage = 0; phase ^= 1u; }
-                    if ((item & (NPROD - 1)) != warp) continue;
+                    if ((item & 1) != warp) continue;
                     if (!mbar_wait(smem_u32(&bars.empty[st]), ph ^ 1u, abort_flag)) {
                         ok = false;
                         break;
@@ -251,7 +281,7 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
                     }
                 }
             }
-        } else if (warp == MMA_WARP) {
+        } else if (warp == DMMA_WARP) {
             if (leader) {
                 // ------------------------------ MMA issuer --------------------------------------
                 const uint32_t idesc_s = instr_desc(DUO_TILE, false, 2 * XROWS);
@@ -305,20 +335,19 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
             }
         } else {
             // ------------------------------ softmax warps ---------------------------------------
-            const int sw = warp - (NPROD + 1);             // 0..7
+            const int sw = warp - (DPROD + 1);             // 0..7
             const int q = warp & 3;                        // tensor-memory lane quarter
             const int half = sw >> 2;                      // columns [128 half, 128 half + 128)
             const int row = q * 32 + lane;
             const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
             const bool self_mask = (p.mask_mode == GC_MASK_SELF);
-            const uint32_t stg = stg_smem + (uint32_t)sw * 4096u;
             // DP: logsumexp (log2 domain) and positive of the 128 streamed queries of this warp's
             // column half, private to the warp so that no block-wide barrier is needed
             float* const lse_tab = reinterpret_cast<float*>(smem_raw + (tab_smem - smem_u32(smem_raw))) +
                                    sw * 256;
             int32_t* const pos_tab = reinterpret_cast<int32_t*>(lse_tab + 128);
             bool ok = true;
-            float lse2_x = 0.f, l = 0.f, wmax = 0.f;
+            float lse2_x = 0.f, l = 0.f;
             int32_t pos_x = -1;
             int64_t cur_xp = -1, x = 0;
             // FA may have been launched ahead of the anchor kernel's completion: row_ref, the
@@ -330,7 +359,9 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
                 const int64_t slot = (int64_t)((rel * 2 + sidx) * 2 + half) * p.nq + x;
                 p.part_m[slot] = lse2_x * 0.69314718055994531f;
                 p.part_l[slot] = l;
-                if (!(wmax <= 1.2676506e30f)) *p.range_flag = 1;   // beyond 2^100, or not finite
+                // weights are >= 0, so a row sum within 2^100 bounds every weight of the row; one
+                // beyond it (or not finite) cannot be accumulated safely
+                if (!(l <= 1.2676506e30f)) *p.range_flag = 1;
             };
             int j = 0;
             for (int k = sidx; k < nk; k += 2, ++j) {
@@ -344,7 +375,6 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
                     cur_xp = xp;
                     x = x0 + row;
                     l = 0.f;
-                    wmax = 0.f;
                     lse2_x = 0.f;
                     pos_x = -1;
                     if (MODE != DMODE_DP && x < p.nx) {
@@ -374,145 +404,137 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
                     fence_proxy_async_all();
                 }
                 const uint32_t sbuf = tmem + lane_addr + (uint32_t)b * DUO_TILE;
-#pragma unroll 1
-                for (int ch = 0; ch < 2; ++ch) {
-                    const int chunk = half * 2 + ch;       // 64-column chunk of the tile
-                    uint32_t keep[2][16];
-#pragma unroll
-                    for (int blk = 0; blk < 2; ++blk) {
-                        const int cb = chunk * 2 + blk;    // 32-column block of the tile
-                        uint32_t v[32];
-                        tmem_ld32(sbuf + cb * 32, v);
-                        tmem_ld_wait();
-                        if (ch == 1 && blk == 1) {         // the S tile may be overwritten
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(smem_u32(&bars.t_free[b]));
-                        }
-                        const int64_t yb = y0 + cb * 32;
-                        float w[32];
-                        if (MODE == DMODE_FA) {
-                            const bool has_pos = pos_x >= yb && pos_x < yb + 32 && pos_x < p.ny &&
-                                                 !(self_mask && x == pos_x);
-                            if (has_pos) {
-                                const int rel = (int)(pos_x - yb);
-                                float spv = 0.f;
-#pragma unroll
-                                for (int c = 0; c < 32; ++c)
-                                    if (c == rel) spv = __uint_as_float(v[c]);
-                                p.pos_logit[x] = spv * p.inv_tau;
-                            }
+                // weights of one 32-column block: v (logits, fp32 bits) -> 32 bf16 = 64 bytes of
+                // this thread's row of the chunk image, written as two 32-byte stores
+                auto weights = [&](uint32_t (&v)[32], int cb, int lb, uint8_t* dst) {
+                    const int64_t yb = y0 + cb * 32;
+                    float w[32];
+                    if (MODE == DMODE_FA) {
+                        const bool has_pos = pos_x >= yb && pos_x < yb + 32 && pos_x < p.ny &&
+                                             !(self_mask && x == pos_x);
+                        if (has_pos) {
+                            const int rel = (int)(pos_x - yb);
+                            float spv = 0.f;
 #pragma unroll
                             for (int c = 0; c < 32; ++c)
-                                w[c] = ex2(fmaf(__uint_as_float(v[c]), p.c1, -lse2_x));
-                            if (yb + 32 > p.ny) {
+                                if (c == rel) spv = __uint_as_float(v[c]);
+                            p.pos_logit[x] = spv * p.inv_tau;
+                        }
 #pragma unroll
-                                for (int c = 0; c < 32; ++c)
-                                    if (yb + c >= p.ny) w[c] = 0.f;
-                            }
-                            if (self_mask && x >= yb && x < yb + 32) {
-                                const int rel = (int)(x - yb);
-#pragma unroll
-                                for (int c = 0; c < 32; ++c)
-                                    if (c == rel) w[c] = 0.f;
-                            }
-                            float s0 = 0.f, s1 = 0.f, m0 = 0.f;
-#pragma unroll
-                            for (int c = 0; c < 32; c += 2) {
-                                s0 += w[c];
-                                s1 += w[c + 1];
-                                m0 = fmaxf(m0, fmaxf(w[c], w[c + 1]));
-                            }
-                            l += s0 + s1;
-                            wmax = fmaxf(wmax, m0);
-                            if (pos_x >= yb && pos_x < yb + 32) {      // positive: fp32, later
-                                const int rel = (int)(pos_x - yb);
-#pragma unroll
-                                for (int c = 0; c < 32; ++c)
-                                    if (c == rel) w[c] = 0.f;
-                            }
-                        } else if (MODE == DMODE_DQ) {
+                        for (int c = 0; c < 32; ++c)
+                            w[c] = ex2(fmaf(__uint_as_float(v[c]), p.c1, -lse2_x));
+                        if (yb + 32 > p.ny) {
 #pragma unroll
                             for (int c = 0; c < 32; ++c)
-                                w[c] = ex2(fmaf(__uint_as_float(v[c]), p.c1, -lse2_x));
-                            if (pos_x >= yb && pos_x < yb + 32) {
-                                const int rel = (int)(pos_x - yb);
-#pragma unroll
-                                for (int c = 0; c < 32; ++c)
-                                    if (c == rel) w[c] -= 1.f;
-                            }
-                            if (yb + 32 > p.ny) {
-#pragma unroll
-                                for (int c = 0; c < 32; ++c)
-                                    if (yb + c >= p.ny) w[c] = 0.f;
-                            }
-                        } else {
-                            const int lb = (ch * 2 + blk) * 32;    // block within the warp's half
-                            const float4* lt = reinterpret_cast<const float4*>(lse_tab + lb);
-#pragma unroll
-                            for (int c = 0; c < 32; c += 4) {
-                                const float4 l4 = lt[c >> 2];          // OOB query: ex2(-inf) = 0
-                                w[c] = ex2(fmaf(__uint_as_float(v[c]), p.c1, -l4.x));
-                                w[c + 1] = ex2(fmaf(__uint_as_float(v[c + 1]), p.c1, -l4.y));
-                                w[c + 2] = ex2(fmaf(__uint_as_float(v[c + 2]), p.c1, -l4.z));
-                                w[c + 3] = ex2(fmaf(__uint_as_float(v[c + 3]), p.c1, -l4.w));
-                            }
-                            // one-hot: column c's query has its positive at row pos - x0 of this CTA
-                            const int32_t pos_yj = pos_tab[lb + lane];
-                            const int64_t rel_row = (int64_t)pos_yj - x0;
-                            const bool mine = (pos_yj >= 0) && rel_row >= q * 32 && rel_row < q * 32 + 32;
-                            unsigned hits = __ballot_sync(0xffffffffu, mine);
-                            while (hits) {
-                                const int col = __ffs(hits) - 1;
-                                hits &= hits - 1;
-                                const int target = (int)__shfl_sync(0xffffffffu, (int)rel_row, col) - q * 32;
-                                if (lane == target) {
-#pragma unroll
-                                    for (int c = 0; c < 32; ++c)
-                                        if (c == col) w[c] -= 1.f;
-                                }
-                            }
+                                if (yb + c >= p.ny) w[c] = 0.f;
                         }
-                        if (MODE != DMODE_FA && self_mask && x >= yb && x < yb + 32) {
+                        if (self_mask && x >= yb && x < yb + 32) {
                             const int rel = (int)(x - yb);
 #pragma unroll
                             for (int c = 0; c < 32; ++c)
                                 if (c == rel) w[c] = 0.f;
                         }
+                        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
 #pragma unroll
-                        for (int r = 0; r < 16; ++r) {
-                            __nv_bfloat162 h = __floats2bfloat162_rn(w[2 * r], w[2 * r + 1]);
-                            keep[blk][r] = *reinterpret_cast<uint32_t*>(&h);
+                        for (int c = 0; c < 32; c += 4) {
+                            s0 += w[c];
+                            s1 += w[c + 1];
+                            s2 += w[c + 2];
+                            s3 += w[c + 3];
+                        }
+                        l += (s0 + s1) + (s2 + s3);
+                        if (pos_x >= yb && pos_x < yb + 32) {      // positive: fp32, later
+                            const int rel = (int)(pos_x - yb);
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (c == rel) w[c] = 0.f;
+                        }
+                    } else if (MODE == DMODE_DQ) {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c)
+                            w[c] = ex2(fmaf(__uint_as_float(v[c]), p.c1, -lse2_x));
+                        if (pos_x >= yb && pos_x < yb + 32) {
+                            const int rel = (int)(pos_x - yb);
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (c == rel) w[c] -= 1.f;
+                        }
+                        if (yb + 32 > p.ny) {
+#pragma unroll
+                            for (int c = 0; c < 32; ++c)
+                                if (yb + c >= p.ny) w[c] = 0.f;
+                        }
+                    } else {
+                        const float4* lt = reinterpret_cast<const float4*>(lse_tab + lb);
+#pragma unroll
+                        for (int c = 0; c < 32; c += 4) {
+                            const float4 l4 = lt[c >> 2];          // OOB query: ex2(-inf) = 0
+                            w[c] = ex2(fmaf(__uint_as_float(v[c]), p.c1, -l4.x));
+                            w[c + 1] = ex2(fmaf(__uint_as_float(v[c + 1]), p.c1, -l4.y));
+                            w[c + 2] = ex2(fmaf(__uint_as_float(v[c + 2]), p.c1, -l4.z));
+                            w[c + 3] = ex2(fmaf(__uint_as_float(v[c + 3]), p.c1, -l4.w));
+                        }
+                        // one-hot: column c's query has its positive at row pos - x0 of this CTA
+                        const int32_t pos_yj = pos_tab[lb + lane];
+                        const int64_t rel_row = (int64_t)pos_yj - x0;
+                        const bool mine = (pos_yj >= 0) && rel_row >= q * 32 && rel_row < q * 32 + 32;
+                        unsigned hits = __ballot_sync(0xffffffffu, mine);
+                        while (hits) {
+                            const int col = __ffs(hits) - 1;
+                            hits &= hits - 1;
+                            const int target = (int)__shfl_sync(0xffffffffu, (int)rel_row, col) - q * 32;
+                            if (lane == target) {
+#pragma unroll
+                                for (int c = 0; c < 32; ++c)
+                                    if (c == col) w[c] -= 1.f;
+                            }
                         }
                     }
-                    // this warp's 32 rows of the chunk: 4 KB in the swizzled image, one bulk store
-                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                    __syncwarp();
+                    if (MODE != DMODE_FA && self_mask && x >= yb && x < yb + 32) {
+                        const int rel = (int)(x - yb);
 #pragma unroll
-                    for (int blk = 0; blk < 2; ++blk) {
-                        const uint32_t line = stg + lane * 128;
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            const uint32_t addr = line + (((4 * blk + i) ^ (lane & 7)) << 4);
-                            asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
-                                         ::"r"(addr), "r"(keep[blk][4 * i]), "r"(keep[blk][4 * i + 1]),
-                                           "r"(keep[blk][4 * i + 2]), "r"(keep[blk][4 * i + 3])
-                                         : "memory");
-                        }
+                        for (int c = 0; c < 32; ++c)
+                            if (c == rel) w[c] = 0.f;
                     }
-                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                    __syncwarp();
-                    if (lane == 0)
-                        tma_store_2d(&mapWst, stg, 0, ring_row(sp, slot, (int)rank, chunk) + q * 32);
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) {
+                        __nv_bfloat162 h = __floats2bfloat162_rn(w[2 * r], w[2 * r + 1]);
+                        pk[r] = *reinterpret_cast<uint32_t*>(&h);
+                    }
+#pragma unroll
+                    for (int i = 0; i < 2; ++i)
+                        asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                                     ::"l"(dst + 32 * i), "r"(pk[8 * i]), "r"(pk[8 * i + 1]),
+                                       "r"(pk[8 * i + 2]), "r"(pk[8 * i + 3]), "r"(pk[8 * i + 4]),
+                                       "r"(pk[8 * i + 5]), "r"(pk[8 * i + 6]), "r"(pk[8 * i + 7])
+                                     : "memory");
+                };
+                // The loads of the next chunk's two blocks are issued as soon as the registers of
+                // the current ones are free, so that only the first load of a tile is waited for.
+                uint32_t va[32], vb[32];
+                tmem_ld32(sbuf + (half * 4) * 32, va);
+                tmem_ld32(sbuf + (half * 4 + 1) * 32, vb);
+#pragma unroll 1
+                for (int ch = 0; ch < 2; ++ch) {
+                    const int chunk = half * 2 + ch;       // 64-column chunk of the tile
+                    // this thread's 128-byte row of the chunk image in the ring
+                    uint8_t* const dst = p.ring +
+                        ((size_t)ring_row(sp, slot, (int)rank, chunk) + (size_t)row) * 128;
+                    tmem_ld_wait();
+                    if (ch == 1) {                         // the S tile may be overwritten
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(smem_u32(&bars.t_free[b]));
+                    }
+                    weights(va, chunk * 2, ch * 64, dst);
+                    if (ch == 0) tmem_ld32(sbuf + (half * 4 + 2) * 32, va);
+                    weights(vb, chunk * 2 + 1, ch * 64 + 32, dst + 64);
+                    if (ch == 0) tmem_ld32(sbuf + (half * 4 + 3) * 32, vb);
                 }
-                // the tile's two pieces of this warp are in the ring: publish
-                if (lane == 0) {
-                    asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-                    fence_proxy_async_all();
-                    __threadfence();
-                    red_release_gpu(ready + (sp * DUO_RING + slot) * 2 + (int)rank, 1);
-                }
+                // this warp's rows of the tile are on their way: tell the publisher
                 __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars.w_stored[slot]));
             }
             if (ok) flush_slots();
         }
@@ -557,8 +579,8 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
                     __syncwarp();
                 }
             }
-        } else if (warp == 1) {
-            // ------------------------------ Y tiles, 64 rows at a time --------------------------
+        } else if (warp < DPROD) {
+            // ------------------------------ Y tiles, 64 rows at a time (two warps) --------------
             // Columns of this CTA: the N = 256 instruction takes columns [0, 128) of its 256 from
             // rank 0 and [128, 256) from rank 1; the N = 128 one that follows takes 64 from each.
             int stage = 0;
@@ -571,6 +593,7 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
                     const int st = stage;
                     const uint32_t ph = phase;
                     if (++stage == B_STAGES) { stage = 0; phase ^= 1u; }
+                    if ((c & 1) != warp - 1) continue;
                     if (!mbar_wait(smem_u32(&bars.b_empty[st]), ph ^ 1u, abort_flag)) {
                         ok = false;
                         break;
@@ -590,7 +613,7 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
                     }
                 }
             }
-        } else if (warp == MMA_WARP) {
+        } else if (warp == DMMA_WARP) {
             if (leader) {
                 // ------------------------------ MMA issuer --------------------------------------
                 const uint32_t idesc256 = instr_desc(256, true, 2 * XROWS);
@@ -631,7 +654,9 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
                             tc_commit_pair(smem_u32(&bars.b_empty[sb]));
                             if (c == 3) {       // all four chunks of the tile have left the ring
                                 const int sp = 2 * team + (k & 1), j = k >> 1;
-                                red_release_gpu(consumed + sp * DUO_RING + (j % DUO_RING), 1);
+                                // (the loads have completed: nothing of this thread's needs
+                                // publishing, and a release here would stall the issuing thread)
+                                red_relaxed_gpu(consumed + sp * DUO_RING + (j % DUO_RING), 1);
                             }
                         }
                         if (++sa == A_STAGES) { sa = 0; pa ^= 1u; }
@@ -650,11 +675,12 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
             }
         } else {
             // ------------------------------ epilogue warps --------------------------------------
-            const int sw = warp - (NPROD + 1);
+            const int sw = warp - (DPROD + 1);
             const int q = warp & 3;
             const int half = sw >> 2;                      // alternate 32-column blocks
             const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
-            const uint32_t buf = stg_smem + (uint32_t)sw * 4096u;
+            const uint32_t buf0 = stg_smem + (uint32_t)sw * 8192u;
+            int nst = 0;                                   // bulk stores issued by this warp
             for (int i = 0; i < npieces; ++i) {
                 if (!mbar_wait(smem_u32(&bars.t_full[0]), (uint32_t)(i & 1), abort_flag)) break;
                 tc_fence_after();
@@ -665,12 +691,14 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
                 const int row0 = (main_piece ? (int)(xp * DUO_TILE) : 0) + (int)rank * 128 + q * 32;
                 const int plane = main_piece ? 0 : team;
                 const float sc = (main_piece && MODE != DMODE_FA) ? p.out_scale : 1.f;
-                for (int cb = half; cb < c_count * 2; cb += 2) {
+                for (int cb = half; cb < c_count * 2; cb += 2, ++nst) {
                     uint32_t v[32];
                     tmem_ld32(tmem + lane_addr + cb * 32, v);
-                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    // the store issued two blocks ago has finished reading this buffer
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
                     __syncwarp();
                     tmem_ld_wait();
+                    const uint32_t buf = buf0 + (uint32_t)(nst & 1) * 4096u;
                     stage_block(buf, v, sc, lane);
                     __syncwarp();
                     if (lane == 0) tma_store_3d(map, buf, c_begin * 64 + cb * 32, row0, plane);
@@ -697,7 +725,7 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
         __syncthreads();
     }
     cluster_sync_all();   // no MMA, load or arrival of the other CTA touches this one any more
-    if (warp == MMA_WARP) {
+    if (warp == DMMA_WARP) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;"
                      ::"r"(tmem), "r"((uint32_t)TMEM_COLS) : "memory");
@@ -705,30 +733,43 @@ duo_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUt
 }
 
 // Adds the extra planes to the rows whose x pair was split between teams: out[row] += scale *
-// extra[t][row - first row of the pair], teams in index order (one thread owns an element, so
-// the sum does not depend on timing).
+// extra[t][row - first row of the pair].  blockIdx.y = team; a team whose extra plane belongs to
+// the same x pair as the team before it leaves its plane to the first such team, which adds the
+// planes of the whole run in team order (one thread owns an element, so the sum does not depend on
+// timing).
 __global__ void __launch_bounds__(256)
 duo_fixup_kernel(const float4* __restrict__ extra, int64_t nx, int d4, int64_t YT, int64_t total,
                  int nteams, float scale, float* __restrict__ out, int64_t ldo, const Gate gate) {
     if (gate_closed(gate)) return;
+    const int t0 = (int)blockIdx.y + 1;
+    int64_t lo, hi;
+    team_range(total, nteams, t0, &lo, &hi);
+    if (lo % YT == 0) return;                              // this team has no extra plane
+    const int64_t xp = lo / YT;
+    if (t0 > 1) {
+        int64_t plo, phi;
+        team_range(total, nteams, t0 - 1, &plo, &phi);
+        if (plo % YT != 0 && plo / YT == xp) return;       // the run began earlier
+    }
     const int64_t per_plane = (int64_t)DUO_TILE * d4;
     for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < per_plane;
          e += (int64_t)gridDim.x * blockDim.x) {
         const int r = (int)(e / d4);
         const int c = 4 * (int)(e - (int64_t)r * d4);
-        for (int t = 1; t < nteams; ++t) {
-            int64_t lo, hi;
-            team_range(total, nteams, t, &lo, &hi);
-            if (lo % YT == 0) continue;
-            const int64_t row = (lo / YT) * DUO_TILE + r;
-            if (row >= nx) continue;
+        const int64_t row = xp * DUO_TILE + r;
+        if (row >= nx) continue;
+        float4* dst = reinterpret_cast<float4*>(out + row * ldo + c);
+        float4 o = *dst;
+        for (int t = t0; t < nteams; ++t) {
+            if (t > t0) {
+                team_range(total, nteams, t, &lo, &hi);
+                if (lo % YT == 0 || lo / YT != xp) break;
+            }
             const float4 v = extra[(int64_t)t * per_plane + e];
-            float4* dst = reinterpret_cast<float4*>(out + row * ldo + c);
-            float4 o = *dst;
             o.x = fmaf(v.x, scale, o.x); o.y = fmaf(v.y, scale, o.y);
             o.z = fmaf(v.z, scale, o.z); o.w = fmaf(v.w, scale, o.w);
-            *dst = o;
         }
+        *dst = o;
     }
 }
 
@@ -798,7 +839,7 @@ int duo_resident_clusters() {
         }
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3(2 * 74);
-        cfg.blockDim = dim3(NTHREADS);
+        cfg.blockDim = dim3(DTHREADS);
         cfg.dynamicSmemBytes = DUO_SMEM;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeClusterDimension;
@@ -819,13 +860,12 @@ int duo_resident_clusters() {
 
 template <int MODE>
 cudaError_t launch_duo(const CUtensorMap& mx, const CUtensorMap& mys, const CUtensorMap& mya,
-                       const CUtensorMap& mwst, const CUtensorMap& mwld, const CUtensorMap& mmain,
-                       const CUtensorMap& mextra, const DuoParams& p, cudaStream_t st,
-                       bool overlap_prev) {
+                       const CUtensorMap& mwld, const CUtensorMap& mmain, const CUtensorMap& mextra,
+                       const DuoParams& p, cudaStream_t st, bool overlap_prev) {
     if (duo_resident_clusters<MODE>() < 4 * p.nteams) return cudaErrorLaunchOutOfResources;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)(p.nteams * 8));
-    cfg.blockDim = dim3(NTHREADS);
+    cfg.blockDim = dim3(DTHREADS);
     cfg.dynamicSmemBytes = DUO_SMEM;
     cfg.stream = st;
     cudaLaunchAttribute attr[2];
@@ -837,7 +877,7 @@ cudaError_t launch_duo(const CUtensorMap& mx, const CUtensorMap& mys, const CUte
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = overlap_prev ? 2 : 1;
-    return cudaLaunchKernelEx(&cfg, duo_kernel<MODE>, mx, mys, mya, mwst, mwld, mmain, mextra, p);
+    return cudaLaunchKernelEx(&cfg, duo_kernel<MODE>, mx, mys, mya, mwld, mmain, mextra, p);
 }
 
 int64_t tiles_of(int64_t n) { return (n + DUO_TILE - 1) / DUO_TILE; }
@@ -891,7 +931,7 @@ size_t duo_extra_bytes(int nteams, int d) { return (size_t)nteams * DUO_TILE * (
 
 namespace {
 
-struct DuoMaps { CUtensorMap mx, mys, mya, mwst, mwld, mmain, mextra; };
+struct DuoMaps { CUtensorMap mx, mys, mya, mwld, mmain, mextra; };
 
 bool duo_setup(DuoParams* p, DuoMaps* m, const void* X, int64_t ldx, int64_t nx, const void* Y,
                int64_t ldy, int64_t ny, int d, const DuoScratch& ws, float* main_out, int64_t ld_main) {
@@ -902,10 +942,13 @@ bool duo_setup(DuoParams* p, DuoMaps* m, const void* X, int64_t ldx, int64_t nx,
     p->kc = d / 64;
     p->dpc = chunks_per_part(p->kc);
     p->flags = ws.flags;
+    p->ring = static_cast<uint8_t*>(ws.ring);
+    p->out_main = main_out;
+    p->ld_main = ld_main;
+    p->extra = ws.extra;
     const int64_t ring_rows = (int64_t)p->nteams * 2 * DUO_RING * 8 * 128;
     return make_map(&m->mx, X, nx, d, ldx, XROWS) && make_map(&m->mys, Y, ny, d, ldy, 128) &&
-           make_map(&m->mya, Y, ny, d, ldy, 64) && make_ring_map(&m->mwst, ws.ring, ring_rows, 32) &&
-           make_ring_map(&m->mwld, ws.ring, ring_rows, 128) &&
+           make_map(&m->mya, Y, ny, d, ldy, 64) && make_ring_map(&m->mwld, ws.ring, ring_rows, 128) &&
            make_out_map(&m->mmain, main_out, nx, d, ld_main, 1) &&
            make_out_map(&m->mextra, ws.extra, DUO_TILE, d, d, p->nteams);
 }
@@ -927,12 +970,12 @@ cudaError_t duo_launch_sweep(const SweepArgs& a, const DuoScratch& ws, cudaStrea
     p.dev_status = a.dev_status;
     p.gate = a.gate;
     cudaError_t e = a.mode == SWEEP_DQ
-        ? launch_duo<DMODE_DQ>(m.mx, m.mys, m.mya, m.mwst, m.mwld, m.mmain, m.mextra, p, st, false)
-        : launch_duo<DMODE_DP>(m.mx, m.mys, m.mya, m.mwst, m.mwld, m.mmain, m.mextra, p, st, false);
+        ? launch_duo<DMODE_DQ>(m.mx, m.mys, m.mya, m.mwld, m.mmain, m.mextra, p, st, false)
+        : launch_duo<DMODE_DP>(m.mx, m.mys, m.mya, m.mwld, m.mmain, m.mextra, p, st, false);
     if (e != cudaSuccess || p.nteams < 2) return e;
     const int d4 = a.d / 4;
-    int64_t blocks = ((int64_t)DUO_TILE * d4 + 255) / 256;
-    duo_fixup_kernel<<<(unsigned)blocks, 256, 0, st>>>(reinterpret_cast<const float4*>(ws.extra), a.nx,
+    const int64_t blocks = ((int64_t)DUO_TILE * d4 + 255) / 256;
+    duo_fixup_kernel<<<dim3((unsigned)blocks, (unsigned)(p.nteams - 1)), 256, 0, st>>>(reinterpret_cast<const float4*>(ws.extra), a.nx,
                                                       d4, p.YT, p.total, p.nteams, a.out_scale, a.out,
                                                       a.ldo, a.gate);
     return cudaGetLastError();
@@ -963,8 +1006,7 @@ cudaError_t duo_launch_fused_dq(const FwdArgs& a, float* main_plane, const DuoSc
     p.dev_status = a.dev_status;
     p.gate = a.gate;
     p.zero_me = reinterpret_cast<int*>(a.red);
-    return launch_duo<DMODE_FA>(m.mx, m.mys, m.mya, m.mwst, m.mwld, m.mmain, m.mextra, p, st,
-                                overlap_prev);
+    return launch_duo<DMODE_FA>(m.mx, m.mys, m.mya, m.mwld, m.mmain, m.mextra, p, st, overlap_prev);
 }
 
 cudaError_t duo_launch_dq_finalize(const float* main_plane, const DuoScratch& ws, const float* row_ref2,
