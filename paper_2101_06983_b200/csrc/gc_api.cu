@@ -43,21 +43,15 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored) {
         pl.g_dp = simt_sweep_groups(N, B, d);
     }
     pl.fused = (pl.tc && tc_fused_applicable(d)) ? 1 : 0;
-    // two-role sweeps for rows of two column halves: the dQ-side sweeps stream N passages past B
-    // queries, the dP sweep B queries past N passages
-    pl.duo_q = (pl.tc && duo_applicable(B, d)) ? duo_teams(B, N) : 0;
-    pl.duo_p = (pl.tc && duo_applicable(N, d)) ? duo_teams(N, B) : 0;
-    if (pl.duo_p) pl.g_dp = 1;          // the two-role dP sweep writes its output itself
-    pl.duo_slots = pl.duo_q ? 4 * duo_max_pieces(B, N) : 0;
-    // 1: two-role sweeps (rows of two column halves); 2: narrow rows (two S buffers)
-    pl.anchored = (pl.fused && pl.duo_q) ? 1
+    // 1: four-CTA sweeps (rows of two column halves); 2: narrow rows (two S buffers)
+    pl.anchored = (pl.fused && quad_applicable(B, d)) ? 1
                   : (pl.tc && !pl.fused && tc_anchor_applicable(d)) ? 2 : 0;
     size_t dpad = (size_t)((d + 3) & ~3);
     // (max, sum) slots: the forward sweep writes g_fwd of them per row, the fused sweep 2 g_dq,
     // the anchored fused sweep 4 g_dq
     size_t slots = (size_t)pl.g_fwd;
     if (pl.fused && (size_t)(2 * pl.g_dq) > slots) slots = (size_t)(2 * pl.g_dq);
-    if (pl.anchored == 1 && (size_t)pl.duo_slots > slots) slots = (size_t)pl.duo_slots;
+    if (pl.anchored == 1 && (size_t)(4 * pl.g_dq) > slots) slots = (size_t)(4 * pl.g_dq);
     if (pl.anchored == 2 && (size_t)(4 * pl.g_dq) > slots) slots = (size_t)(4 * pl.g_dq);
     size_t off = 0;
     pl.off_m = off;    off += align256(sizeof(float) * slots * (size_t)B);
@@ -72,12 +66,7 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored) {
     pl.launches_fwd = 2;  // sweep + combine
     pl.launches_bwd = 2 + (pl.g_dq > 1 ? 1 : 0) + (pl.g_dp > 1 ? 1 : 0);
     pl.launches_build = pl.fused ? 4 + (pl.g_dp > 1 ? 1 : 0) : pl.launches_fwd + pl.launches_bwd;
-    // counter clearing, anchor, fused sweep, combine, finalize, dP sweep (+ fix-up), fallback
-    if (pl.anchored == 1)
-        pl.launches_build = 6 + (pl.duo_p > 1 ? 1 : 0) + pl.launches_build +
-                            ((pl.duo_p > 1) ? 1 : 0);
-    else if (pl.duo_q || pl.duo_p)
-        pl.launches_build += 1;
+    if (pl.anchored == 1) pl.launches_build = 1 + 2 * pl.launches_build;   // anchor, sequence, fallback
     // anchor, fused sweep, combine, finalize, dP sweep (+ reduce), then the gated forward + sweeps
     if (pl.anchored == 2)
         pl.launches_build = 5 + (pl.g_dp > 1 ? 1 : 0) + pl.launches_fwd + pl.launches_bwd;
@@ -110,16 +99,6 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored) {
         // anchor, sweep, combine, row scaling, dQ GEMM, dQ finalize, dP GEMM (+ reduce),
         // positive terms, then the gated fallback sequence
         pl.launches_build = 8 + (pl.g_mp > 1 ? 1 : 0) + pl.launches_build;
-    }
-    // scratch of the two-role sweeps, after every region the other plans may have moved
-    if (pl.duo_q || pl.duo_p) {
-        const int most = pl.duo_q > pl.duo_p ? pl.duo_q : pl.duo_p;
-        pl.flag_bytes = align256(duo_flag_bytes(most));
-        pl.off_flags = off;    off += 2 * pl.flag_bytes;       // dQ-side sweep, dP sweep
-        pl.off_ring = off;     off += align256(duo_ring_bytes(most));
-        pl.off_extra_q = off;  off += align256(duo_extra_bytes(pl.duo_q, d));
-        pl.off_extra_p = off;  off += align256(duo_extra_bytes(pl.duo_p, d));
-        pl.launches_bwd += 1 + (pl.duo_q > 1 ? 1 : 0) + (pl.duo_p > 1 ? 1 : 0);
     }
     pl.total = off;
     return pl;
@@ -219,21 +198,6 @@ Problem make_problem(const void* Q, int64_t ldq, const void* P, int64_t ldp,
 
 constexpr Gate kOpen = {nullptr, 0};
 
-// Scratch of the two-role sweeps: side 0 = the dQ-side sweep of a call, 1 = its dP sweep.  The ring
-// is shared (the two sweeps of a call run one after the other); counters and extra planes are not.
-DuoScratch duo_scratch(const Plan& pl, char* ws, int side) {
-    DuoScratch s;
-    s.ring = ws + pl.off_ring;
-    s.flags = reinterpret_cast<int*>(ws + pl.off_flags + (side ? pl.flag_bytes : 0));
-    s.extra = reinterpret_cast<float*>(ws + (side ? pl.off_extra_p : pl.off_extra_q));
-    return s;
-}
-// The counters of both sides start a call at zero.
-cudaError_t duo_clear(const Plan& pl, char* ws, cudaStream_t st) {
-    if (!pl.duo_q && !pl.duo_p) return cudaSuccess;
-    return cudaMemsetAsync(ws + pl.off_flags, 0, 2 * pl.flag_bytes, st);
-}
-
 // 1 / (B tau) of Eq. 4-7, with B the whole batch when the call covers a slice of the queries
 float grad_scale(const Problem& p) {
     return 1.f / ((float)(p.b_total > 0 ? p.b_total : p.B) * p.tau);
@@ -285,10 +249,6 @@ int run_sweep(const Problem& p, const Plan& pl, char* ws, int mode, const float*
     sa.ldo = ldo;
     sa.groups = dq ? pl.g_dq : pl.g_dp;
     sa.partial = reinterpret_cast<float*>(ws + (dq ? pl.off_accq : pl.off_accp));
-    if (pl.tc && (dq ? pl.duo_q : pl.duo_p)) {      // two-role sweep: writes `out` itself
-        sa.groups = 1;
-        sa.duo = duo_scratch(pl, ws, dq ? 0 : 1);
-    }
     sa.dev_status = dev_status;
     cudaError_t e;
     {
@@ -382,17 +342,20 @@ SideStream* side_stream() {
     return s.ok ? &s : nullptr;
 }
 
-// gc_build_cache for bf16 rows whose forward runs inside the dQ sweep with the positive logit as
-// each row's fixed scale (anchor kernel), so that no running maximum has to be tracked: rows of
-// two column halves (two-role sweeps) and narrow rows (one-CTA sweeps with two S buffers).  A
-// weight beyond 2^100 raises the range flag; the kernels after the fused sweep run only while it is
-// down, and the online-maximum sequence, which is always launched, runs only when it is up and
-// then produces every output.
+// gc_build_cache for rows of two column halves (four-CTA sweeps).  The forward is fused into the
+// dQ sweep with the positive logit as each row's fixed scale (anchor kernel), so no running
+// maximum has to be agreed across the cluster.  A weight beyond 2^100 raises the range flag; the
+// kernels after the fused sweep run only while it is down, and the online-maximum sequence, which
+// is always launched, runs only when it is up and then produces every output.
 //
-//   caller's stream:  anchor, fused sweep, combine (row_lse, loss), dP sweep (+ fix-up / reduce)
-//   side stream:      after the combine: dQ finalize, then the gated online-maximum sequence
+//   caller's stream:  anchor, fused sweep, dP sweep (+ reduce), which merges the forward slots
+//                     of its streamed queries itself
+//   side stream:      after the fused sweep: combine (row_lse, loss), dQ finalize, then the
+//                     gated online-maximum sequence
 // Both are joined back before the call returns.  Without a side stream everything is queued on
-// the caller's stream in dependency order.
+// the caller's stream in dependency order with the combine before the dP sweep.  Narrow rows
+// (two S buffers in tensor memory) take the same sequence with the one-CTA sweeps, and forward,
+// dQ and dP sweeps as the gated fallback.
 int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_lse,
                        float* pos_logit, float* dQ, int64_t lddq, float* dP, int64_t lddp,
                        int* dev_status, cudaStream_t st, bool want_dp = true) {
@@ -401,16 +364,13 @@ int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, 
     const Gate in_range = {flag, 0}, out_of_range = {flag, 1};
     SideStream* side = side_stream();
     cudaStream_t aux = side ? side->st : st;
-    const bool duo = pl.anchored == 1;
     FwdArgs fa{};
     fa.p = p;
     fa.part_m = reinterpret_cast<float*>(ws + pl.off_m);
     fa.part_l = reinterpret_cast<float*>(ws + pl.off_l);
     fa.pos_logit = reinterpret_cast<float*>(ws + pl.off_pos);
     fa.red = reinterpret_cast<float*>(ws + pl.off_red);
-    // slots per row: (team of the x pair, S pair, column half), or per part two softmax groups x
-    // two column halves
-    fa.groups = duo ? pl.duo_slots : 4 * pl.g_dq;
+    fa.groups = 4 * pl.g_dq;      // per part: two duty pairs, or two softmax groups, x two column halves
     fa.dev_status = dev_status;
     float* partial = reinterpret_cast<float*>(ws + pl.off_accq);
     // The fused sweep is launched with programmatic serialization: it starts (loads, first S
@@ -419,37 +379,45 @@ int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, 
     // which serialises them, so the overlap is left out while it is on.
     const bool overlap = !g_prof.on;
     cudaError_t e = launch_pos_anchor(p.Q, p.ldq, p.P, p.ldp, p.pos_idx, p.B, p.N, p.d, p.mask_mode,
-                                      1.4426950408889634f / p.tau, ref2, flag, st,
-                                      duo ? fa.part_m : nullptr, duo ? fa.groups : 0);
+                                      1.4426950408889634f / p.tau, ref2, flag, st);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     {
         KernelTimer t(1, st);
-        e = duo ? duo_launch_fused_dq(fa, partial, duo_scratch(pl, ws, 0), ref2, flag, st, overlap)
+        e = pl.anchored == 1
+                ? quad_launch_fused_dq(fa, partial, pl.g_dq, ref2, flag, st, overlap)
                 : tc_launch_anchored_dq(fa, partial, pl.g_dq, ref2, flag, st, overlap);
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
+    // Wide rows: a sweep step is long enough to hide the slot merge of the streamed queries,
+    // so the dP sweep does not wait for the combine.  Narrow rows have short steps: there the
+    // combine stays on the caller's stream and the dP sweep reads row_lse.
+    const bool dp_merges = side && pl.anchored == 1 && want_dp;
+    cudaStream_t comb = dp_merges ? aux : st;
+    if (dp_merges && (cudaEventRecord(side->ev[0], st) != cudaSuccess ||
+                      cudaStreamWaitEvent(aux, side->ev[0], 0) != cudaSuccess))
+        return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
                            p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status,
-                           in_range, st, p.b_total);
+                           in_range, comb, p.b_total);
     if (e != cudaSuccess) return GC_ERR_CUDA;
-    if (side && (cudaEventRecord(side->ev[0], st) != cudaSuccess ||
-                 cudaStreamWaitEvent(aux, side->ev[0], 0) != cudaSuccess))
+    if (side && !dp_merges && (cudaEventRecord(side->ev[0], st) != cudaSuccess ||
+                               cudaStreamWaitEvent(aux, side->ev[0], 0) != cudaSuccess))
         return GC_ERR_CUDA;
-    e = duo ? duo_launch_dq_finalize(partial, duo_scratch(pl, ws, 0), ref2, row_lse, fa.pos_logit,
-                                     p.pos_idx, p.P, p.ldp, p.B, p.N, p.d, p.mask_mode,
-                                     grad_scale(p), dQ, lddq, in_range, aux)
-            : launch_fused_dq_finalize(partial, pl.g_dq, nullptr, ref2, row_lse, fa.pos_logit,
-                                       p.pos_idx, p.P, p.ldp, p.B, p.N, p.d, p.mask_mode,
-                                       grad_scale(p), dQ, lddq, in_range, aux);
+    e = launch_fused_dq_finalize(partial, pl.g_dq, nullptr, ref2, row_lse, fa.pos_logit, p.pos_idx,
+                                 p.P, p.ldp, p.B, p.N, p.d, p.mask_mode,
+                                 grad_scale(p), dQ, lddq, in_range, aux);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     int rc;
     if (side) {
         if ((rc = run_online_sweeps(p, pl, ws, loss, row_lse, pos_logit, dQ, lddq, dP, lddp,
                                     dev_status, aux, out_of_range, want_dp)))
             return rc;
-        if (want_dp &&
-            (rc = run_sweep(p, pl, ws, SWEEP_DP, row_lse, dP, lddp, dev_status, st, in_range)))
-            return rc;
+        if (dp_merges)
+            rc = run_sweep(p, pl, ws, SWEEP_DP, row_lse, dP, lddp, dev_status, st, in_range, true,
+                           fa.part_m, fa.part_l, fa.groups);
+        else if (want_dp)
+            rc = run_sweep(p, pl, ws, SWEEP_DP, row_lse, dP, lddp, dev_status, st, in_range);
+        if (rc) return rc;
         if (cudaEventRecord(side->ev[2], aux) != cudaSuccess ||
             cudaStreamWaitEvent(st, side->ev[2], 0) != cudaSuccess)
             return GC_ERR_CUDA;
@@ -670,7 +638,6 @@ int gc_loss_bwd(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
     if (dev_status && launch_pos_check(pos_idx, B, N, mask_mode, dev_status, st) != cudaSuccess)
         return GC_ERR_CUDA;
     char* w = static_cast<char*>(ws);
-    if (duo_clear(pl, w, st) != cudaSuccess) return GC_ERR_CUDA;
     if (dQ && (rc = run_sweep(p, pl, w, SWEEP_DQ, row_lse, dQ, lddq, dev_status, st))) return rc;
     if (dP && (rc = run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, dev_status, st))) return rc;
     return GC_OK;
@@ -692,7 +659,6 @@ int gc_build_cache(const void* Q, int64_t ldq, const void* P, int64_t ldp, const
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
     char* w = static_cast<char*>(ws);
-    if (duo_clear(pl, w, st) != cudaSuccess) return GC_ERR_CUDA;
     return run_build_sweeps(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status, st);
 }
 
@@ -713,7 +679,6 @@ int gc_build_cache_stored(const void* Q, int64_t ldq, const void* P, int64_t ldp
     profile_begin_call();
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
-    if (duo_clear(pl, static_cast<char*>(ws), st) != cudaSuccess) return GC_ERR_CUDA;
     return run_build_stored(p, pl, static_cast<char*>(ws), loss, row_lse, pos_logit, dQ, lddq, dP,
                             lddp, dev_status, st);
 }
@@ -745,8 +710,6 @@ int gc_shard_fwd_dq(const void* Q, int64_t ldq, const void* P, int64_t ldp, cons
     const char* q_first = static_cast<const char*>(Q) + (size_t)q0 * (size_t)ldq * elem_size(dtype);
     Problem p = make_problem(q_first, ldq, P, ldp, pos_idx + q0, q_count, N, d, tau, mask_mode, dtype);
     p.b_total = B;
-    if (duo_clear(pl, static_cast<char*>(ws), static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
-        return GC_ERR_CUDA;
     return run_build_sweeps(p, pl, static_cast<char*>(ws), loss_part, row_lse + q0,
                             pos_logit ? pos_logit + q0 : nullptr, dQ, lddq, nullptr, 0, dev_status,
                             static_cast<cudaStream_t>(cuda_stream), false);
@@ -769,7 +732,6 @@ int gc_shard_dp(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
     profile_begin_call();
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     char* w = static_cast<char*>(ws);
-    if (duo_clear(pl, w, st) != cudaSuccess) return GC_ERR_CUDA;
     // positives counted from the slice's first passage; those outside the slice match no row
     int32_t* pos_local = reinterpret_cast<int32_t*>(w + pl.total);
     if (dev_status && launch_pos_check(pos_idx, B, N, mask_mode, dev_status, st) != cudaSuccess)

@@ -171,14 +171,9 @@ __global__ void __launch_bounds__(256)
 pos_anchor_kernel(const __nv_bfloat16* __restrict__ Q, int64_t ldq,
                   const __nv_bfloat16* __restrict__ P, int64_t ldp,
                   const int32_t* __restrict__ pos_idx, int64_t B, int64_t N, int d, int mask_mode,
-                  float c1, float* __restrict__ ref2, int* __restrict__ range_flag,
-                  float* __restrict__ clear_m, int64_t clear_count) {
+                  float c1, float* __restrict__ ref2, int* __restrict__ range_flag) {
     dep_release();      // the sweep that follows may start; it waits for this grid before it reads ref2
     if (blockIdx.x == 0 && threadIdx.x == 0) *range_flag = 0;
-    // (scale, sum) slots that the sweep may leave unwritten read as empty
-    for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < clear_count;
-         e += (int64_t)gridDim.x * blockDim.x)
-        clear_m[e] = -INFINITY;
     const int lane = threadIdx.x & 31;
     for (int64_t i = blockIdx.x * 8 + (threadIdx.x >> 5); i < B; i += (int64_t)gridDim.x * 8) {
         const int32_t r = pos_idx[i];
@@ -289,16 +284,14 @@ dp_positive_kernel(const int32_t* __restrict__ pos_idx, int64_t B, int64_t N, in
 
 cudaError_t launch_pos_anchor(const void* Q, int64_t ldq, const void* P, int64_t ldp,
                               const int32_t* pos_idx, int64_t B, int64_t N, int d, int mask_mode,
-                              float c1, float* ref2, int* range_flag, cudaStream_t st,
-                              float* clear_m, int clear_slots) {
+                              float c1, float* ref2, int* range_flag, cudaStream_t st) {
     int64_t blocks = (B + 7) / 8;
     int cap = sm_count() * 8;
     if (blocks > cap) blocks = cap;
     pos_anchor_kernel<<<(int)blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(Q), ldq,
                                                   static_cast<const __nv_bfloat16*>(P), ldp,
                                                   pos_idx, B, N, d, mask_mode, c1, ref2,
-                                                  range_flag, clear_m,
-                                                  clear_m ? (int64_t)clear_slots * B : 0);
+                                                  range_flag);
     return cudaGetLastError();
 }
 

@@ -66,14 +66,6 @@ struct Problem {
 // In both, W = 0 for the masked pair (query index == passage index under GC_MASK_SELF).
 enum SweepMode { SWEEP_DQ = 0, SWEEP_DP = 1 };
 
-// Scratch of the two-role sweeps (gc_duo.cu): the W ring, its counters (zero before a launch) and
-// the extra accumulator planes of x pairs that are split between teams.
-struct DuoScratch {
-    void* ring;
-    int* flags;
-    float* extra;
-};
-
 struct SweepArgs {
     const void* X;          // stationary rows  [nx x d]
     const void* Y;          // streamed rows    [ny x d]
@@ -98,7 +90,6 @@ struct SweepArgs {
     const float* slot_m;
     const float* slot_l;
     int slots;
-    DuoScratch duo;         // ring != NULL: the sweep runs as the two-role kernel
 };
 
 struct FwdArgs {
@@ -124,10 +115,6 @@ struct Plan {
     int anchored;           // 1: ... with the positive logit as the fixed scale of each row (four-
                             // CTA sweep); the online-maximum sweep then is its gated fallback
     int launches_build;
-    // Two-role sweeps (rows of two column halves): teams of the dQ-side and dP-side sweeps (0:
-    // the sweep runs another kernel), slots of row sums per query in the fused sweep, scratch
-    int duo_q, duo_p, duo_slots;
-    size_t off_ring, off_flags, off_extra_q, off_extra_p, flag_bytes;
     // Stored-weights plan of gc_build_cache (tcgen05 only): one forward sweep keeps the bf16
     // weights, two GEMMs form the gradients; the sweeps above stay as its fallback.
     int mat;
@@ -160,8 +147,7 @@ cudaError_t launch_partial_reduce(const float* partial, int groups, int64_t rows
                                   cudaStream_t st);
 cudaError_t launch_pos_anchor(const void* Q, int64_t ldq, const void* P, int64_t ldp,
                               const int32_t* pos_idx, int64_t B, int64_t N, int d, int mask_mode,
-                              float c1, float* ref2, int* range_flag, cudaStream_t st,
-                              float* clear_m = nullptr, int clear_slots = 0);
+                              float c1, float* ref2, int* range_flag, cudaStream_t st);
 cudaError_t launch_scale_rows(const void* Q, int64_t ldq, int64_t B, int d, const float* ref2,
                               const float* row_lse, void* Qs, cudaStream_t st);
 cudaError_t launch_dp_positive(const int32_t* pos_idx, int64_t B, int64_t N, int mask_mode,
@@ -190,23 +176,12 @@ int tc_sweep_groups(int64_t nx, int64_t ny, int d);
 cudaError_t tc_launch_fwd_store(const FwdArgs& a, void* weights, int64_t ldw, const float* row_ref,
                                 int* range_flag, cudaStream_t st);
 
-// gc_duo.cu
-bool duo_applicable(int64_t nx, int d);
-int duo_max_teams();
-int duo_teams(int64_t nx, int64_t ny);
-int duo_max_pieces(int64_t nx, int64_t ny);
-size_t duo_ring_bytes(int nteams);
-size_t duo_flag_bytes(int nteams);
-size_t duo_extra_bytes(int nteams, int d);
-cudaError_t duo_launch_sweep(const SweepArgs& a, const DuoScratch& ws, cudaStream_t st);
-cudaError_t duo_launch_fused_dq(const FwdArgs& a, float* main_plane, const DuoScratch& ws,
-                                const float* row_ref, int* range_flag, cudaStream_t st,
-                                bool overlap_prev = false);
-cudaError_t duo_launch_dq_finalize(const float* main_plane, const DuoScratch& ws,
-                                   const float* row_ref2, const float* row_lse, const float* pos_ws,
-                                   const int32_t* pos_idx, const void* P, int64_t ldp, int64_t B,
-                                   int64_t N, int d, int mask_mode, float scale, float* out,
-                                   int64_t ldo, Gate gate, cudaStream_t st);
+// gc_quad.cu
+bool quad_applicable(int64_t nx, int d);
+int quad_groups(int64_t nx, int64_t ny);
+cudaError_t quad_launch_sweep(const SweepArgs& a, cudaStream_t st);
+cudaError_t quad_launch_fused_dq(const FwdArgs& a, float* partial, int groups, const float* row_ref,
+                                 int* range_flag, cudaStream_t st, bool overlap_prev = false);
 
 // gc_gemm.cu
 int gemm_groups(int64_t m_rows, int64_t k_len, int d);

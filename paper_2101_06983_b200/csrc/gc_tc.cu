@@ -18,8 +18,8 @@
 //   FS   (Eq. 1)    forward that also stores the bf16 weights 2^(s2 - ref2_x) of all pairs (the
 //                   stored-weights comparison plan).
 //
-// Rows of two column halves with more than one x tile are served by the two-role sweeps of
-// gc_duo.cu instead; there FQ remains as the gated fallback.
+// Rows of two column halves with more than one x tile are served by the four-CTA sweeps of
+// gc_quad.cu instead; there FQ and DP remain as the gated fallback.
 //
 // The stationary tile X (128 x d) stays resident in shared memory when d <= 512; for wider rows
 // only its first chunks stay (6, or 2 beside shared-memory W buffers) and the others are
@@ -1264,6 +1264,7 @@ int tc_fwd_groups(int64_t B, int64_t N, int d) {
 }
 
 int tc_sweep_groups(int64_t nx, int64_t ny, int d) {
+    if (quad_applicable(nx, d)) return quad_groups(nx, ny);
     int kc = d / 64;
     int64_t units = ((nx + XROWS - 1) / XROWS) * parts_for(kc);
     int64_t steps = (ny + 127) / 128;
@@ -1404,7 +1405,7 @@ cudaError_t tc_launch_anchored_dq(const FwdArgs& a, float* partial, int groups,
 }
 
 cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
-    if (a.duo.ring) return duo_launch_sweep(a, a.duo, st);
+    if (quad_applicable(a.nx, a.d)) return quad_launch_sweep(a, st);
     const int kc = a.d / 64;
     constexpr int SN = 128;
     CUtensorMap mx, my, myh;
