@@ -5,8 +5,11 @@
 
 One "step" is one gc_build_cache call over one synthetic batch.  The default workload is the
 headline configuration B = 4096, N = 8192, d = 768, bf16 inputs.  The metric is useful TFLOP/s
-counting 3 GEMMs of 2 B N d each.  With N > 1 (torchrun) every rank runs an independent replica
-of the same batch shape; there is no collective on the data path.
+counting 3 GEMMs of 2 B N d each.  With N > 1 the ONE batch is split over the ranks the way
+Section 3.4 of the paper describes (all-gather of the representations, rank-local gradients,
+exchange of the row logsumexps): strong scaling, collectives inside the timed region.
+`--parallel replicas` runs N independent batches instead (weak scaling, no collective).
+`--gpus N` without a torchrun environment starts the N ranks itself.
 
 Prints ONE JSON line on rank 0.  `--impl reference` times the CPU oracle instead (a deliberately
 plain program; see oracle/).
@@ -24,32 +27,43 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
-METRIC = "gc_build_cache TFLOP/s (3 GEMMs of 2*B*N*d) at B=4096,N=8192,d=768"
 UNIT = "TFLOP/s"
+
+
+def metric_name(B, N, d):
+    return f"gc_build_cache TFLOP/s (3 GEMMs of 2*B*N*d) at B={B},N={N},d={d}"
+
+
 NOMINAL_BF16_TFLOPS = 2250.0      # public dense bf16 figure for B200, context only
-# dram__bytes_read.sum + dram__bytes_write.sum per sweep launch at the headline shape, from the
-# ncu capture summarised in profiles/quad_kernel_cfg2_B4096_N8192_d768.txt.  Reported only while
-# the kernel source still has the hash it had when the counters were taken.
-NCU_TRAFFIC_BYTES = 19.1e6
-# the same for config 4, from profiles/quad_kernel_cfg4_B65536_N131072_d768.txt (average of the two
-# sweep launches, reads + writes)
-NCU_TRAFFIC_BYTES_CFG4 = 2.07e9
-NCU_TRAFFIC_SOURCE_SHA1 = "916b6c4e7d6d270f2504571c26c0464f8ffcd291"
+# dram__bytes_read.sum + dram__bytes_write.sum of ONE STEP (every launch of a gc_build_cache
+# call summed) from the ncu captures summarised under profiles/ (step_traffic_*.txt).  Reported
+# only while the kernel sources still have the hash they had when the counters were taken.
+NCU_STEP_TRAFFIC = {"cfg2_": None, "cfg4_": None}
+NCU_TRAFFIC_SOURCE_SHA1 = ""
+FP32_LANES_PER_SM = 128           # fp32 FMA lanes of one SM (2 FLOP per lane and clock)
+
+
+def sources_sha1():
+    import glob
+    import hashlib
+    h = hashlib.sha1()
+    for f in sorted(glob.glob(os.path.join(ROOT, "paper_2101_06983_b200", "csrc", "*"))):
+        with open(f, "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()
 
 
 def ncu_traffic(workload: str):
-    import hashlib
-    src = os.path.join(ROOT, "paper_2101_06983_b200", "csrc", "gc_quad.cu")
     try:
-        with open(src, "rb") as fh:
-            same = hashlib.sha1(fh.read()).hexdigest() == NCU_TRAFFIC_SOURCE_SHA1
+        same = sources_sha1() == NCU_TRAFFIC_SOURCE_SHA1
     except OSError:
         same = False
     if not same:
         return None
-    if workload.startswith("cfg2_"):
-        return NCU_TRAFFIC_BYTES
-    return NCU_TRAFFIC_BYTES_CFG4 if workload.startswith("cfg4_") else None
+    for prefix, val in NCU_STEP_TRAFFIC.items():
+        if workload.startswith(prefix):
+            return val
+    return None
 
 
 def load_peaks():
@@ -168,7 +182,8 @@ def run_reference(args, rank, world):
     sample = (f"first {rows} of {prob.B} query rows against all {prob.N} passages "
               f"(loss, dQ rows, dP contributions), double precision, per step")
     line = {
-        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+        "impl": "reference", "metric": metric_name(prob.B, prob.N, prob.d), "value": value,
+        "unit": UNIT, "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
@@ -271,6 +286,28 @@ def run_ours(args, rank, local_rank, world):
     barrier()
     warm_ms = a.elapsed_time(b) / args.steps
 
+    # ---- sustained: at least a second of back-to-back steps, clocks sampled meanwhile -------------
+    # A short timed region runs at boost clocks; under a second of tensor work the power cap
+    # settles the SM clock lower.  time x median MHz lets runs at different clocks be compared.
+    sustained = None
+    if not args.no_sustained:
+        n_sus = max(args.steps, int(1.2 / max(warm_ms * 1e-3, 1e-6)))
+        sus_sampler = ClockSampler(physical_gpu_index(local_rank), period=0.005)
+        barrier()
+        sus_sampler.start()
+        a.record()
+        for _ in range(n_sus):
+            step()
+        b.record()
+        barrier()
+        sus_clocks = sus_sampler.result()
+        sus_ms = a.elapsed_time(b) / n_sus
+        sustained = {"steps": n_sus, "ms_per_step": sus_ms,
+                     "value": world * flop / (sus_ms * 1e-3) / 1e12, "unit": UNIT,
+                     "sm_mhz_median": sus_clocks["sm_mhz"], "reasons": sus_clocks["reasons"],
+                     "ms_x_mhz": None if sus_clocks["sm_mhz"] is None
+                     else sus_ms * sus_clocks["sm_mhz"]}
+
     # ---- end to end through the C ABI with host buffers ------------------------------------------
     # Every step copies its inputs from pinned host memory, calls gc_build_cache and copies the
     # cache (dQ, dP) and the loss back.  Two sets of device buffers and three streams (upload,
@@ -353,15 +390,37 @@ def run_ours(args, rank, local_rank, world):
             sweep_flop = (6.0 if fused else 4.0) * B * N * d / 2.0      # per launch, averaged
         achieved = sweep_flop / (sweep_ms * 1e-3) / 1e12 if sweep_ms > 0 else 0.0
         value = replicas.whole_job_rate(flop, world, ms_per_step) / 1e12
+        if plan.startswith("tcgen05"):
+            roof = {"bound": "tensor", "kernel": f"{plan} sweeps (the tensor-core launches of a step)",
+                    "achieved": achieved, "peak": pk["tf_burst"], "unit": "TFLOP/s",
+                    "frac": achieved / pk["tf_burst"], "peak_source": pk["source"]}
+        else:
+            # fp32 FMA tiles: bound by the fp32 pipes, SMs x 128 lanes x 2 FLOP x the maximum SM
+            # clock; the launches of a step executed (fwd 2 + dQ 4 + dP 4) B N d
+            alu_ms = (kern[0] + kern[1] + kern[2]) / args.steps
+            executed = 10.0 * B * N * d / (alu_ms * 1e-3) / 1e12 if alu_ms > 0 else 0.0
+            sms = torch.cuda.get_device_properties(dev).multi_processor_count
+            mhz = clocks["sm_max_mhz"] or 1965
+            alu_peak = sms * FP32_LANES_PER_SM * 2 * mhz * 1e6 / 1e12
+            roof = {"bound": "alu", "kernel": "fp32 FMA tile kernels (forward, dQ and dP sweeps)",
+                    "achieved": executed, "peak": alu_peak, "unit": "TFLOP/s",
+                    "frac": executed / alu_peak,
+                    "peak_source": "derived: SMs x 128 fp32 lanes x 2 x max SM clock"}
+        step_traffic = None if stored else ncu_traffic(prob.name)
+        roof["traffic"] = step_traffic
+        roof["traffic_scope"] = "dram bytes of one step, all launches (ncu)"
+        roof["algorithmic_bytes_per_step"] = (B + N) * d * (2 if prob.dtype == "bf16" else 4) + \
+            (B + N) * d * 4
         line = {
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "metric": metric_name(B, N, d), "value": value, "unit": UNIT, "n_gpus": world,
+            "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16" if prob.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": prob.name, "B": B, "N": N, "d": d, "tau": prob.tau,
                        "mask": "self" if prob.mask_mode else "none", "plan": plan,
                        "l2": "flushed before every timed step (256 MiB write)",
-                       "parallelism": f"{world} independent replica(s)"},
+                       "parallelism": f"{world} independent replica(s), no collective"},
             "rows_per_s": world * (B + N) / (ms_per_step * 1e-3),
             "pct_of_bf16_peak": {"burst_measured": 100 * value / world / pk["tf_burst"],
                                  "sustained_measured": 100 * value / world / pk["tf_sustained"],
@@ -373,11 +432,8 @@ def run_ours(args, rank, local_rank, world):
                           "dp_sweep": kern[2] / args.steps,
                           "pass": "second pass of the same flushed steps, per-kernel CUDA events",
                           "ms_per_step_with_events": profiled_ms / args.steps},
-            "roofline": {"bound": "tensor",
-                         "kernel": f"{plan} sweeps (the tensor-core launches of a step)",
-                         "achieved": achieved, "peak": pk["tf_burst"], "unit": "TFLOP/s",
-                         "frac": achieved / pk["tf_burst"], "peak_source": pk["source"],
-                         "traffic": None if stored else ncu_traffic(prob.name)},
+            "sustained": sustained,
+            "roofline": roof,
             "e2e": {"value": world * flop / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
                     "ms_per_step": e2e_ms, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                     "loss_read_back": e2e_loss,
@@ -405,10 +461,10 @@ def run_ours(args, rank, local_rank, world):
 
 
 def run_sharded(args, rank, local_rank, world):
-    """Non-default multi-GPU mode (--parallel shard): ONE global batch of the chosen workload is
-    split over the ranks as Section 3.4 describes (all-gather of representations, rank-local
-    forward + dQ and dP, exchange of row_lse, loss all-reduce).  Strong scaling: the value is the
-    whole batch's useful FLOP over the slowest rank's time, collectives included."""
+    """Multi-GPU mode (default for N > 1): ONE global batch of the chosen workload is split over
+    the ranks as Section 3.4 describes (all-gather of representations, rank-local forward + dQ
+    and dP, exchange of row_lse, loss all-reduce).  Strong scaling: the value is the whole batch's
+    useful FLOP over the slowest rank's time, collectives included."""
     import torch
     import torch.distributed as dist
     if not torch.cuda.is_available():
@@ -418,44 +474,71 @@ def run_sharded(args, rank, local_rank, world):
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
     from paper_2101_06983_b200 import binding, inputs, replicas, sharded
-    prob = inputs.config(args.config)
-    if prob.mask_mode != inputs.MASK_NONE:
-        raise SystemExit("--parallel shard covers the unmasked loss only")
-    B, N, d = prob.B, prob.N, prob.d
-    Q, P, pos = binding.problem_tensors(prob, dev)
-    (q0, b), (p0, n) = sharded.row_ranges(B, world)[rank], sharded.row_ranges(N, world)[rank]
-    Ql, Pl, posl = Q[q0:q0 + b].contiguous(), P[p0:p0 + n].contiguous(), pos[q0:q0 + b].contiguous()
-    del Q, P, pos
 
-    def step():
-        return sharded.sharded_build_cache(Ql, Pl, posl, prob.tau, B, N)
+    def measure(index, steps, warmup):
+        prob = inputs.config(index)
+        B, N, d = prob.B, prob.N, prob.d
+        Q, P, pos = binding.problem_tensors(prob, dev)
+        (q0, b), (p0, n) = sharded.row_ranges(B, world)[rank], sharded.row_ranges(N, world)[rank]
+        Ql, Pl = Q[q0:q0 + b].contiguous(), P[p0:p0 + n].contiguous()
+        posl = pos[q0:q0 + b].contiguous()
+        del Q, P, pos
+        step = sharded.ShardedStep(B, N, d, Ql.dtype, dev, mask_mode=prob.mask_mode)
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
+        def barrier():
+            if world > 1:
+                dist.barrier()
+            torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
-        step()
-    barrier()
-    a, bev = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record()
-    for _ in range(args.steps):
-        loss = step()[0]
-    bev.record()
-    barrier()
-    ms = replicas.max_over_ranks([a.elapsed_time(bev) / args.steps], dev)[0]
+        for _ in range(max(warmup, 3)):
+            step.run(Ql, Pl, posl, prob.tau)
+        barrier()
+        a, bev = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(steps):
+            loss = step.run(Ql, Pl, posl, prob.tau)[0]
+        bev.record()
+        barrier()
+        ms = replicas.max_over_ranks([a.elapsed_time(bev) / steps], dev)[0]
+        # where the time goes: one more pass with every section synchronised (diagnostic)
+        parts = {"gather_reps_s": 0.0, "fwd_dq_s": 0.0, "lse_and_loss_s": 0.0, "dp_s": 0.0}
+        for _ in range(3):
+            step.run(Ql, Pl, posl, prob.tau, measure=True)
+            for k in parts:
+                parts[k] += step.timings[k] / 3
+        keys = sorted(parts)
+        worst = replicas.max_over_ranks([parts[k] for k in keys], dev)
+        comm = sum(v for k, v in zip(keys, worst) if k in ("gather_reps_s", "lse_and_loss_s"))
+        comp = sum(v for k, v in zip(keys, worst) if k in ("fwd_dq_s", "dp_s"))
+        return prob, ms, float(loss.item()), {"communication_ms": comm * 1e3,
+                                              "compute_ms": comp * 1e3,
+                                              "note": "sections synchronised one by one, max over ranks"}
+
+    prob, ms, loss, split = measure(args.config, args.steps, args.warmup)
+    also = None
+    if world > 1 and args.config != 4 and not args.no_also:
+        p4, ms4, loss4, split4 = measure(4, max(3, min(args.steps, 5)), 3)
+        also = {"workload": p4.name, "ms_per_step": ms4,
+                "value": useful_flop(p4.B, p4.N, p4.d) / (ms4 * 1e-3) / 1e12, "unit": UNIT,
+                "loss": loss4, "split": split4}
     if rank == 0:
+        B, N, d = prob.B, prob.N, prob.d
         flop = useful_flop(B, N, d)
         print(json.dumps({
-            "metric": METRIC, "value": flop / (ms * 1e-3) / 1e12, "unit": UNIT, "n_gpus": world,
-            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
+            "metric": metric_name(B, N, d), "value": flop / (ms * 1e-3) / 1e12, "unit": UNIT,
+            "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms,
             "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
             "dtype": "bf16" if prob.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": prob.name, "B": B, "N": N, "d": d,
-                       "parallelism": f"rows sharded over {world} rank(s), Section 3.4",
+                       "parallelism": f"query and passage rows sharded over {world} rank(s), "
+                                      "Section 3.4: all-gather of Q, P, pos_idx; all-gather of "
+                                      "row_lse; all-reduce of the loss",
                        "l2": "back to back, no flush (collectives between the kernels)"},
-            "loss": float(loss.item()), "gpu_launches": None}), flush=True)
+            "split": split, "also": also, "loss": loss,
+            "gpu_launches": args.steps * (
+                binding.gc_kernel_launches(binding.GC_OP_BUILD, max(1, B // world), N, d,
+                                           binding.GC_BF16 if prob.dtype == "bf16" else binding.GC_F32)
+                + 3)}), flush=True)
     if world > 1:
         dist.destroy_process_group()
 
@@ -541,10 +624,35 @@ def main():
                     help="build: gc_build_cache, the headline; apply: the side measurement of "
                          "gc_cache_apply (one GPU)")
     ap.add_argument("--apply-rows", type=int, default=4096)
-    ap.add_argument("--parallel", default="replicas", choices=["replicas", "shard"],
-                    help="N > 1: independent replicas (default, weak scaling, no collective), or "
-                         "one batch sharded over the ranks as in Section 3.4 of the paper")
+    ap.add_argument("--parallel", default=None, choices=["replicas", "shard"],
+                    help="shard (default for N > 1): one batch split over the ranks as in Section "
+                         "3.4 of the paper, strong scaling; replicas (default for N = 1): "
+                         "independent batches, weak scaling, no collective")
+    ap.add_argument("--no-sustained", action="store_true",
+                    help="skip the second-long back-to-back measurement")
+    ap.add_argument("--no-also", action="store_true",
+                    help="sharded mode: skip the B=65536 workload measured beside the chosen one")
     args = ap.parse_args()
+    env_world = os.environ.get("WORLD_SIZE")
+    if env_world is not None and int(env_world) != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} contradicts WORLD_SIZE={env_world}")
+    if args.gpus > 1 and env_world is None and args.impl == "ours" and args.op == "build":
+        # not under torchrun: start the ranks ourselves, one per GPU of this node
+        import torch
+        have = torch.cuda.device_count() if torch.cuda.is_available() else 0
+        if have < args.gpus:
+            raise SystemExit(f"--gpus {args.gpus} needs {args.gpus} CUDA devices on this node, "
+                             f"found {have}: refusing to run fewer ranks")
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        os.execv(sys.executable, [sys.executable, "-m", "torch.distributed.run", "--nnodes=1",
+                                  f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1",
+                                  "--master-port", str(port), os.path.abspath(__file__),
+                                  *sys.argv[1:]])
+    if args.parallel is None:
+        args.parallel = "shard" if args.gpus > 1 else "replicas"
     if args.op == "apply":
         if int(os.environ.get("RANK", "0")) == 0:
             run_apply(args)

@@ -178,8 +178,9 @@ int gc_cache_apply(const float* U, int64_t ldu, const void* X, int64_t ldx, int6
  *       ALL B queries.  Writes dP [p_count x d].
  *
  * Both scale by 1/B with B the whole batch, so concatenating the ranks' dQ and dP gives exactly
- * what gc_build_cache gives on one GPU (up to rounding order).  GC_MASK_NONE only (the paper's
- * loss; anything else is GC_ERR_MASK); a range outside the matrices is GC_ERR_SHAPE.  Workspace:
+ * what gc_build_cache gives on one GPU (up to rounding order).  GC_MASK_SELF drops the pair of
+ * query i and passage i of the WHOLE batch, wherever the rank's rows lie in it; a range outside the
+ * matrices is GC_ERR_SHAPE.  Workspace:
  * gc_shard_workspace_bytes, which covers either call.  The collectives are the caller's (the
  * Python package's `sharded` module runs them with torch.distributed).
  */

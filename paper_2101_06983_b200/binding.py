@@ -241,10 +241,10 @@ def gc_shard_workspace_bytes(B: int, N: int, d: int, dtype: int, q_count: int, p
 
 
 def gc_shard_fwd_dq(Q, P, pos_idx, tau, q0, q_count, loss_part, row_lse, dQ, pos_logit=None,
-                    ws=None, dev_status=None):
+                    ws=None, dev_status=None, mask_mode=GC_MASK_NONE):
     """Section 3.4, local queries [q0, q0 + q_count) of the gathered batch: writes their entries
     of row_lse[B], dQ[q_count x d] and loss_part[1] (this rank's share of the loss of Eq. 1)."""
-    args, B, N, d, code = _common(Q, P, pos_idx, tau, GC_MASK_NONE)
+    args, B, N, d, code = _common(Q, P, pos_idx, tau, mask_mode)
     if ws is None:
         ws = torch.empty(max(gc_shard_workspace_bytes(B, N, d, code, q_count, N), 256),
                          dtype=torch.uint8, device=Q.device)
@@ -255,10 +255,11 @@ def gc_shard_fwd_dq(Q, P, pos_idx, tau, q0, q_count, loss_part, row_lse, dQ, pos
         raise GradCacheError(rc, "gc_shard_fwd_dq")
 
 
-def gc_shard_dp(Q, P, pos_idx, tau, row_lse, p0, p_count, dP, ws=None, dev_status=None):
+def gc_shard_dp(Q, P, pos_idx, tau, row_lse, p0, p_count, dP, ws=None, dev_status=None,
+                mask_mode=GC_MASK_NONE):
     """Section 3.4, local passages [p0, p0 + p_count) of the gathered batch, given row_lse of all
     B queries: writes dP[p_count x d]."""
-    args, B, N, d, code = _common(Q, P, pos_idx, tau, GC_MASK_NONE)
+    args, B, N, d, code = _common(Q, P, pos_idx, tau, mask_mode)
     if ws is None:
         ws = torch.empty(max(gc_shard_workspace_bytes(B, N, d, code, B, p_count), 256),
                          dtype=torch.uint8, device=Q.device)

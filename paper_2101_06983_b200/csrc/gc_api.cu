@@ -193,6 +193,7 @@ Problem make_problem(const void* Q, int64_t ldq, const void* P, int64_t ldp,
     p.Q = Q; p.P = P; p.pos_idx = pos_idx; p.ldq = ldq; p.ldp = ldp; p.B = B; p.N = N; p.d = d;
     p.tau = tau; p.mask_mode = mask_mode; p.dtype = dtype;
     p.b_total = 0;
+    p.mask_shift = 0;
     return p;
 }
 
@@ -222,7 +223,7 @@ int run_fwd(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
                            p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status,
-                           gate, st, p.b_total);
+                           gate, st, p.b_total, p.mask_shift);
     return e == cudaSuccess ? GC_OK : GC_ERR_CUDA;
 }
 
@@ -240,6 +241,7 @@ int run_sweep(const Problem& p, const Plan& pl, char* ws, int mode, const float*
     sa.d = p.d;
     sa.mode = mode;
     sa.mask_mode = p.mask_mode;
+    sa.mask_delta = dq ? p.mask_shift : -p.mask_shift;
     sa.dtype = p.dtype;
     sa.inv_tau = 1.f / p.tau;
     sa.out_scale = grad_scale(p);
@@ -286,11 +288,11 @@ int run_fused_fwd_dq(const Problem& p, const Plan& pl, char* ws, float* loss, fl
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
                            p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status,
-                           gate, st, p.b_total);
+                           gate, st, p.b_total, p.mask_shift);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_fused_dq_finalize(partial, pl.g_dq, fa.part_m, nullptr, row_lse, fa.pos_logit,
                                  p.pos_idx, p.P, p.ldp, p.B, p.N, p.d, p.mask_mode,
-                                 grad_scale(p), dQ, lddq, gate, st);
+                                 grad_scale(p), dQ, lddq, gate, st, p.mask_shift);
     return e == cudaSuccess ? GC_OK : GC_ERR_CUDA;
 }
 
@@ -379,7 +381,7 @@ int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, 
     // which serialises them, so the overlap is left out while it is on.
     const bool overlap = !g_prof.on;
     cudaError_t e = launch_pos_anchor(p.Q, p.ldq, p.P, p.ldp, p.pos_idx, p.B, p.N, p.d, p.mask_mode,
-                                      1.4426950408889634f / p.tau, ref2, flag, st);
+                                      1.4426950408889634f / p.tau, ref2, flag, st, p.mask_shift);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     {
         KernelTimer t(1, st);
@@ -398,14 +400,14 @@ int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, 
         return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
                            p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status,
-                           in_range, comb, p.b_total);
+                           in_range, comb, p.b_total, p.mask_shift);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     if (side && !dp_merges && (cudaEventRecord(side->ev[0], st) != cudaSuccess ||
                                cudaStreamWaitEvent(aux, side->ev[0], 0) != cudaSuccess))
         return GC_ERR_CUDA;
     e = launch_fused_dq_finalize(partial, pl.g_dq, nullptr, ref2, row_lse, fa.pos_logit, p.pos_idx,
                                  p.P, p.ldp, p.B, p.N, p.d, p.mask_mode,
-                                 grad_scale(p), dQ, lddq, in_range, aux);
+                                 grad_scale(p), dQ, lddq, in_range, aux, p.mask_shift);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     int rc;
     if (side) {
@@ -461,7 +463,7 @@ int run_build_stored(const Problem& p, const Plan& pl, char* w, float* loss, flo
     float* partp = reinterpret_cast<float*>(w + pl.off_accp);
     const float scale = grad_scale(p);
     cudaError_t e = launch_pos_anchor(p.Q, p.ldq, p.P, p.ldp, p.pos_idx, p.B, p.N, p.d, p.mask_mode,
-                                      1.4426950408889634f / p.tau, ref2, flag, st);
+                                      1.4426950408889634f / p.tau, ref2, flag, st, p.mask_shift);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     FwdArgs fa{};
     fa.p = p;
@@ -478,7 +480,7 @@ int run_build_stored(const Problem& p, const Plan& pl, char* w, float* loss, flo
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_lse_combine(fa.part_m, fa.part_l, fa.pos_logit, p.pos_idx, fa.groups, p.B, p.N,
                            p.mask_mode, row_lse, pos_logit, loss, fa.red, dev_status,
-                           kOpen, st, p.b_total);
+                           kOpen, st, p.b_total, p.mask_shift);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_scale_rows(p.Q, p.ldq, p.B, p.d, ref2, row_lse, qs, st);
     if (e != cudaSuccess) return GC_ERR_CUDA;
@@ -490,7 +492,7 @@ int run_build_stored(const Problem& p, const Plan& pl, char* w, float* loss, flo
     if (e != cudaSuccess) return GC_ERR_CUDA;
     e = launch_fused_dq_finalize(partq, pl.g_mq, nullptr, ref2, row_lse, fa.pos_logit, p.pos_idx,
                                  p.P, p.ldp, p.B, p.N, p.d, p.mask_mode, scale, dQ, lddq, kOpen,
-                                 st);
+                                 st, p.mask_shift);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     {
         KernelTimer t(2, st);
@@ -503,7 +505,7 @@ int run_build_stored(const Problem& p, const Plan& pl, char* w, float* loss, flo
         if (e != cudaSuccess) return GC_ERR_CUDA;
     }
     e = launch_dp_positive(p.pos_idx, p.B, p.N, p.mask_mode, fa.pos_logit, row_lse, p.Q, p.ldq, p.d,
-                           scale, dP, lddp, st);
+                           scale, dP, lddp, st, p.mask_shift);
     if (e != cudaSuccess) return GC_ERR_CUDA;
     const Gate out_of_range = {flag, 1};
     return run_online_sweeps(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status, st,
@@ -699,7 +701,6 @@ int gc_shard_fwd_dq(const void* Q, int64_t ldq, const void* P, int64_t ldp, cons
                     int64_t lddq, void* ws, size_t ws_bytes, int* dev_status, void* cuda_stream) {
     int rc = check_common(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
     if (rc) return rc;
-    if (mask_mode != GC_MASK_NONE) return GC_ERR_MASK;
     if (q0 < 0 || q_count <= 0 || q0 + q_count > B) return GC_ERR_SHAPE;
     if (!loss_part || !row_lse || !dQ) return GC_ERR_NULL;
     if ((rc = check_grad_out(dQ, lddq, d))) return rc;
@@ -710,6 +711,7 @@ int gc_shard_fwd_dq(const void* Q, int64_t ldq, const void* P, int64_t ldp, cons
     const char* q_first = static_cast<const char*>(Q) + (size_t)q0 * (size_t)ldq * elem_size(dtype);
     Problem p = make_problem(q_first, ldq, P, ldp, pos_idx + q0, q_count, N, d, tau, mask_mode, dtype);
     p.b_total = B;
+    p.mask_shift = q0;             // local query i is query q0 + i of the batch
     return run_build_sweeps(p, pl, static_cast<char*>(ws), loss_part, row_lse + q0,
                             pos_logit ? pos_logit + q0 : nullptr, dQ, lddq, nullptr, 0, dev_status,
                             static_cast<cudaStream_t>(cuda_stream), false);
@@ -721,7 +723,6 @@ int gc_shard_dp(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
                 size_t ws_bytes, int* dev_status, void* cuda_stream) {
     int rc = check_common(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
     if (rc) return rc;
-    if (mask_mode != GC_MASK_NONE) return GC_ERR_MASK;
     if (p0 < 0 || p_count <= 0 || p0 + p_count > N) return GC_ERR_SHAPE;
     if (!row_lse || !dP) return GC_ERR_NULL;
     if ((rc = check_grad_out(dP, lddp, d))) return rc;
@@ -739,6 +740,7 @@ int gc_shard_dp(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
     if (launch_shift_pos(pos_idx, B, p0, p_count, pos_local, st) != cudaSuccess) return GC_ERR_CUDA;
     const char* p_first = static_cast<const char*>(P) + (size_t)p0 * (size_t)ldp * elem_size(dtype);
     Problem p = make_problem(Q, ldq, p_first, ldp, pos_local, B, p_count, d, tau, mask_mode, dtype);
+    p.mask_shift = -p0;            // local passage j is passage p0 + j of the batch
     return run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, dev_status, st);
 }
 

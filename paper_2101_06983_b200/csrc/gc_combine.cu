@@ -14,9 +14,10 @@ constexpr int kCombineThreads = 256;
 constexpr int kRedPartials = 64;     // float offset of the per-block sums in the scratch
 
 // pos_idx[i] outside [0, N) or on the masked diagonal: flags for *dev_status, 0 when usable.
-__device__ __forceinline__ int pos_flags(int32_t r, int64_t i, int64_t N, int mask_mode) {
+__device__ __forceinline__ int pos_flags(int32_t r, int64_t i, int64_t N, int mask_mode,
+                                         int64_t shift) {
     if (r < 0 || (int64_t)r >= N) return GC_DEV_POS_RANGE;
-    if (mask_mode == GC_MASK_SELF && (int64_t)r == i) return GC_DEV_POS_MASKED;
+    if (mask_mode == GC_MASK_SELF && (int64_t)r == i + shift) return GC_DEV_POS_MASKED;
     return 0;
 }
 
@@ -29,7 +30,8 @@ lse_combine_kernel(const float* __restrict__ part_m, const float* __restrict__ p
                    const float* __restrict__ pos_ws, const int32_t* __restrict__ pos_idx,
                    int groups, int64_t B, int64_t N, int mask_mode, float* __restrict__ row_lse,
                    float* __restrict__ pos_logit, float* __restrict__ loss, float* red,
-                   int* __restrict__ dev_status, const Gate gate, int64_t mean_over) {
+                   int* __restrict__ dev_status, const Gate gate, int64_t mean_over,
+                   int64_t mask_shift) {
     if (gate_closed(gate)) return;
     __shared__ float warp_sum[kCombineThreads / 32];
     __shared__ int warp_flag[kCombineThreads / 32];
@@ -40,7 +42,7 @@ lse_combine_kernel(const float* __restrict__ part_m, const float* __restrict__ p
          i += (int64_t)gridDim.x * kCombineThreads) {
         const float lse = combined_lse(part_m, part_l, groups, B, i);
         row_lse[i] = lse;
-        int f = pos_flags(pos_idx[i], i, N, mask_mode);
+        int f = pos_flags(pos_idx[i], i, N, mask_mode, mask_shift);
         float pl = f ? 0.f : pos_ws[i];
         if (pos_logit) pos_logit[i] = pl;
         flags |= f;
@@ -82,11 +84,11 @@ lse_combine_kernel(const float* __restrict__ part_m, const float* __restrict__ p
 
 __global__ void __launch_bounds__(256)
 pos_check_kernel(const int32_t* __restrict__ pos_idx, int64_t B, int64_t N, int mask_mode,
-                 int* __restrict__ dev_status) {
+                 int* __restrict__ dev_status, int64_t mask_shift) {
     int flags = 0;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < B;
          i += (int64_t)gridDim.x * blockDim.x)
-        flags |= pos_flags(pos_idx[i], i, N, mask_mode);
+        flags |= pos_flags(pos_idx[i], i, N, mask_mode, mask_shift);
     flags = __reduce_or_sync(0xffffffffu, flags);
     if ((threadIdx.x & 31) == 0 && flags) atomicOr(dev_status, flags);
 }
@@ -133,7 +135,7 @@ fused_dq_finalize_kernel(const float4* __restrict__ partial, int groups,
                          const float* __restrict__ pos_ws, const int32_t* __restrict__ pos_idx,
                          const __nv_bfloat16* __restrict__ P, int64_t ldp, int64_t B, int64_t N,
                          int d4, int mask_mode, float scale, float* __restrict__ out,
-                         int64_t ldo, const Gate gate) {
+                         int64_t ldo, const Gate gate, int64_t mask_shift) {
     if (gate_closed(gate)) return;
     int64_t total = B * d4;
     for (int64_t e = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; e < total;
@@ -150,7 +152,7 @@ fused_dq_finalize_kernel(const float4* __restrict__ partial, int groups,
             acc.z = fmaf(v.z, w, acc.z); acc.w = fmaf(v.w, w, acc.w);
         }
         const int32_t r = pos_idx[i];
-        if (pos_flags(r, i, N, mask_mode) == 0) {
+        if (pos_flags(r, i, N, mask_mode, mask_shift) == 0) {
             const float pm1 = expf(pos_ws[i] - lse) - 1.f;
             const __nv_bfloat16* pr = P + (int64_t)r * ldp + c;
             acc.x = fmaf(pm1, __bfloat162float(pr[0]), acc.x);
@@ -171,14 +173,15 @@ __global__ void __launch_bounds__(256)
 pos_anchor_kernel(const __nv_bfloat16* __restrict__ Q, int64_t ldq,
                   const __nv_bfloat16* __restrict__ P, int64_t ldp,
                   const int32_t* __restrict__ pos_idx, int64_t B, int64_t N, int d, int mask_mode,
-                  float c1, float* __restrict__ ref2, int* __restrict__ range_flag) {
+                  float c1, float* __restrict__ ref2, int* __restrict__ range_flag,
+                  int64_t mask_shift) {
     dep_release();      // the sweep that follows may start; it waits for this grid before it reads ref2
     if (blockIdx.x == 0 && threadIdx.x == 0) *range_flag = 0;
     const int lane = threadIdx.x & 31;
     for (int64_t i = blockIdx.x * 8 + (threadIdx.x >> 5); i < B; i += (int64_t)gridDim.x * 8) {
         const int32_t r = pos_idx[i];
         float acc = 0.f;
-        if (pos_flags(r, i, N, mask_mode) == 0) {
+        if (pos_flags(r, i, N, mask_mode, mask_shift) == 0) {
             const uint4* q = reinterpret_cast<const uint4*>(Q + i * ldq);
             const uint4* pp = reinterpret_cast<const uint4*>(P + (int64_t)r * ldp);
             for (int c = lane; c < d / 8; c += 32) {        // 8 elements per load; d % 8 == 0
@@ -231,7 +234,7 @@ __global__ void __launch_bounds__(1024)
 dp_positive_kernel(const int32_t* __restrict__ pos_idx, int64_t B, int64_t N, int mask_mode,
                    const float* __restrict__ pos_ws, const float* __restrict__ row_lse,
                    const __nv_bfloat16* __restrict__ Q, int64_t ldq, int d, float scale,
-                   float* __restrict__ out, int64_t ldo) {
+                   float* __restrict__ out, int64_t ldo, int64_t mask_shift) {
     __shared__ int list_i[1024];
     __shared__ int list_w[1024];
     __shared__ int warp_count[32];
@@ -243,7 +246,7 @@ dp_positive_kernel(const int32_t* __restrict__ pos_idx, int64_t B, int64_t N, in
         int32_t r = 0;
         if (i < B) {
             r = pos_idx[i];
-            match = pos_flags(r, i, N, mask_mode) == 0 && r >= j0 && r < j0 + kPosTile;
+            match = pos_flags(r, i, N, mask_mode, mask_shift) == 0 && r >= j0 && r < j0 + kPosTile;
         }
         const unsigned ballot = __ballot_sync(0xffffffffu, match);
         if (lane == 0) warp_count[warp] = __popc(ballot);
@@ -284,14 +287,15 @@ dp_positive_kernel(const int32_t* __restrict__ pos_idx, int64_t B, int64_t N, in
 
 cudaError_t launch_pos_anchor(const void* Q, int64_t ldq, const void* P, int64_t ldp,
                               const int32_t* pos_idx, int64_t B, int64_t N, int d, int mask_mode,
-                              float c1, float* ref2, int* range_flag, cudaStream_t st) {
+                              float c1, float* ref2, int* range_flag, cudaStream_t st,
+                              int64_t mask_shift) {
     int64_t blocks = (B + 7) / 8;
     int cap = sm_count() * 8;
     if (blocks > cap) blocks = cap;
     pos_anchor_kernel<<<(int)blocks, 256, 0, st>>>(static_cast<const __nv_bfloat16*>(Q), ldq,
                                                   static_cast<const __nv_bfloat16*>(P), ldp,
                                                   pos_idx, B, N, d, mask_mode, c1, ref2,
-                                                  range_flag);
+                                                  range_flag, mask_shift);
     return cudaGetLastError();
 }
 
@@ -310,11 +314,11 @@ cudaError_t launch_scale_rows(const void* Q, int64_t ldq, int64_t B, int d, cons
 cudaError_t launch_dp_positive(const int32_t* pos_idx, int64_t B, int64_t N, int mask_mode,
                                const float* pos_ws, const float* row_lse, const void* Q,
                                int64_t ldq, int d, float scale, float* out, int64_t ldo,
-                               cudaStream_t st) {
+                               cudaStream_t st, int64_t mask_shift) {
     const int64_t blocks = (N + kPosTile - 1) / kPosTile;
     dp_positive_kernel<<<(unsigned)blocks, 1024, 0, st>>>(pos_idx, B, N, mask_mode, pos_ws, row_lse,
                                                          static_cast<const __nv_bfloat16*>(Q), ldq,
-                                                         d, scale, out, ldo);
+                                                         d, scale, out, ldo, mask_shift);
     return cudaGetLastError();
 }
 
@@ -323,7 +327,7 @@ cudaError_t launch_fused_dq_finalize(const float* partial, int groups, const flo
                                      const float* pos_ws, const int32_t* pos_idx, const void* P,
                                      int64_t ldp, int64_t B, int64_t N, int d, int mask_mode,
                                      float scale, float* out, int64_t ldo, Gate gate,
-                                     cudaStream_t st) {
+                                     cudaStream_t st, int64_t mask_shift) {
     int64_t total = B * (d / 4);
     int64_t blocks = (total + 255) / 256;
     int cap = sm_count() * 8;
@@ -331,7 +335,7 @@ cudaError_t launch_fused_dq_finalize(const float* partial, int groups, const flo
     fused_dq_finalize_kernel<<<(int)blocks, 256, 0, st>>>(
         reinterpret_cast<const float4*>(partial), groups, part_m, row_ref2, row_lse, pos_ws,
         pos_idx, static_cast<const __nv_bfloat16*>(P), ldp, B, N, d / 4, mask_mode, scale, out, ldo,
-        gate);
+        gate, mask_shift);
     return cudaGetLastError();
 }
 
@@ -339,14 +343,15 @@ cudaError_t launch_lse_combine(const float* part_m, const float* part_l, const f
                                const int32_t* pos_idx, int groups, int64_t B, int64_t N,
                                int mask_mode, float* row_lse, float* pos_logit, float* loss,
                                float* red, int* dev_status, Gate gate, cudaStream_t st,
-                               int64_t mean_over) {
+                               int64_t mean_over, int64_t mask_shift) {
     int64_t blocks = (B + kCombineThreads - 1) / kCombineThreads;
     if (blocks > sm_count()) blocks = sm_count();
     if (blocks > 256) blocks = 256;          // the scratch holds this many block sums
     lse_combine_kernel<<<(int)blocks, kCombineThreads, 0, st>>>(part_m, part_l, pos_ws, pos_idx,
                                                                groups, B, N, mask_mode, row_lse,
                                                                pos_logit, loss, red, dev_status,
-                                                               gate, mean_over > 0 ? mean_over : B);
+                                                               gate, mean_over > 0 ? mean_over : B,
+                                                               mask_shift);
     return cudaGetLastError();
 }
 
@@ -372,10 +377,10 @@ cudaError_t launch_shift_pos(const int32_t* pos_idx, int64_t B, int64_t first, i
 }
 
 cudaError_t launch_pos_check(const int32_t* pos_idx, int64_t B, int64_t N, int mask_mode,
-                             int* dev_status, cudaStream_t st) {
+                             int* dev_status, cudaStream_t st, int64_t mask_shift) {
     int blocks = (int)((B + 255) / 256);
     if (blocks > 1024) blocks = 1024;
-    pos_check_kernel<<<blocks, 256, 0, st>>>(pos_idx, B, N, mask_mode, dev_status);
+    pos_check_kernel<<<blocks, 256, 0, st>>>(pos_idx, B, N, mask_mode, dev_status, mask_shift);
     return cudaGetLastError();
 }
 

@@ -57,6 +57,9 @@ struct Problem {
     int dtype;
     int64_t b_total;        // rows of the whole batch when Q holds a slice of it (0: B): the mean
                             // of Eq. 1 and the 1/B of Eq. 4 run over this many queries
+    int64_t mask_shift;     // GC_MASK_SELF drops the pair (query i, passage j) with j == i +
+                            // mask_shift: 0 for whole matrices, first query row minus first
+                            // passage row (in the whole batch) when Q or P is a slice
 };
 
 // The two tile sweeps share one shape: a stationary row tile X, a streamed row tile Y,
@@ -74,6 +77,7 @@ struct SweepArgs {
     int d;
     int mode;               // SweepMode
     int mask_mode;
+    int64_t mask_delta;     // masked pair: y == x + mask_delta (+mask_shift for x = query, - for x = passage)
     int dtype;
     float inv_tau;
     float out_scale;        // 1 / (B * tau), applied where the final value is written
@@ -131,29 +135,30 @@ cudaError_t launch_lse_combine(const float* part_m, const float* part_l, const f
                                const int32_t* pos_idx, int groups, int64_t B, int64_t N,
                                int mask_mode, float* row_lse, float* pos_logit, float* loss,
                                float* red, int* dev_status, Gate gate, cudaStream_t st,
-                               int64_t mean_over = 0);
+                               int64_t mean_over = 0, int64_t mask_shift = 0);
 cudaError_t launch_shift_pos(const int32_t* pos_idx, int64_t B, int64_t first, int64_t count,
                              int32_t* out, cudaStream_t st);
 cudaError_t launch_pos_check(const int32_t* pos_idx, int64_t B, int64_t N, int mask_mode,
-                             int* dev_status, cudaStream_t st);
+                             int* dev_status, cudaStream_t st, int64_t mask_shift = 0);
 cudaError_t launch_fused_dq_finalize(const float* partial, int groups, const float* part_m,
                                      const float* row_ref2, const float* row_lse,
                                      const float* pos_ws, const int32_t* pos_idx, const void* P,
                                      int64_t ldp, int64_t B, int64_t N, int d, int mask_mode,
                                      float scale, float* out, int64_t ldo, Gate gate,
-                                     cudaStream_t st);
+                                     cudaStream_t st, int64_t mask_shift = 0);
 cudaError_t launch_partial_reduce(const float* partial, int groups, int64_t rows, int d,
                                   float scale, float* out, int64_t ldo, Gate gate,
                                   cudaStream_t st);
 cudaError_t launch_pos_anchor(const void* Q, int64_t ldq, const void* P, int64_t ldp,
                               const int32_t* pos_idx, int64_t B, int64_t N, int d, int mask_mode,
-                              float c1, float* ref2, int* range_flag, cudaStream_t st);
+                              float c1, float* ref2, int* range_flag, cudaStream_t st,
+                              int64_t mask_shift = 0);
 cudaError_t launch_scale_rows(const void* Q, int64_t ldq, int64_t B, int d, const float* ref2,
                               const float* row_lse, void* Qs, cudaStream_t st);
 cudaError_t launch_dp_positive(const int32_t* pos_idx, int64_t B, int64_t N, int mask_mode,
                                const float* pos_ws, const float* row_lse, const void* Q,
                                int64_t ldq, int d, float scale, float* out, int64_t ldo,
-                               cudaStream_t st);
+                               cudaStream_t st, int64_t mask_shift = 0);
 
 // gc_simt.cu
 cudaError_t simt_launch_fwd(const FwdArgs& a, cudaStream_t st);

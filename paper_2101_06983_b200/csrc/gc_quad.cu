@@ -50,6 +50,7 @@ struct QuadParams {
     float* pos_logit;         // FA
     int* range_flag;          // FA
     int* dev_status;
+    int64_t mask_delta;       // GC_MASK_SELF drops the pair (x, y) with y == x + mask_delta
     Gate gate;
     int* zero_me;
 };
@@ -433,6 +434,7 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
         const int cb0 = half * CB_PER;
         const int row = q * 32 + lane;
         const int64_t x = x0 + row;
+        const int64_t xm = x + p.mask_delta;     // the streamed index masked for this row
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         const bool self_mask = (p.mask_mode == GC_MASK_SELF);
         bool ok = true;
@@ -522,7 +524,7 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                 float w[32];
                 if (MODE == QMODE_FA) {
                     const bool has_pos = pos_x >= yb && pos_x < yb + 32 && pos_x < p.ny &&
-                                         !(self_mask && x == pos_x);
+                                         !(self_mask && xm == pos_x);
                     if (has_pos) {
                         const int rel = (int)(pos_x - yb);
                         float sp = 0.f;
@@ -542,8 +544,8 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                         for (int c = 0; c < 32; ++c)
                             if (yb + c >= p.ny) w[c] = 0.f;
                     }
-                    if (self_mask && x >= yb && x < yb + 32) {
-                        const int rel = (int)(x - yb);
+                    if (self_mask && xm >= yb && xm < yb + 32) {
+                        const int rel = (int)(xm - yb);
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
                             if (c == rel) w[c] = 0.f;
@@ -598,8 +600,8 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                         }
                     }
                 }
-                if (MODE != QMODE_FA && self_mask && x >= yb && x < yb + 32) {
-                    const int rel = (int)(x - yb);
+                if (MODE != QMODE_FA && self_mask && xm >= yb && xm < yb + 32) {
+                    const int rel = (int)(xm - yb);
 #pragma unroll
                     for (int c = 0; c < 32; ++c)
                         if (c == rel) w[c] = 0.f;
@@ -774,6 +776,7 @@ cudaError_t quad_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     p.nx = a.nx; p.ny = a.ny;
     p.kc = kc; p.dpc = chunks_per_part(kc); p.groups = a.groups;
     p.mask_mode = a.mask_mode;
+    p.mask_delta = a.mask_delta;
     p.inv_tau = a.inv_tau;
     p.c1 = 1.4426950408889634f * a.inv_tau;
     p.out_scale = a.out_scale;
@@ -809,6 +812,7 @@ cudaError_t quad_launch_fused_dq(const FwdArgs& a, float* partial, int groups, c
     p.nx = pr.B; p.ny = pr.N; p.nq = pr.B;
     p.kc = kc; p.dpc = chunks_per_part(kc); p.groups = groups;
     p.mask_mode = pr.mask_mode;
+    p.mask_delta = pr.mask_shift;
     p.inv_tau = 1.f / pr.tau;
     p.c1 = 1.4426950408889634f / pr.tau;
     p.pos_idx = pr.pos_idx;

@@ -150,7 +150,7 @@ __global__ void __launch_bounds__(THREADS) simt_fwd_kernel(FwdArgs a) {
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 int64_t j = j0 + tx * 4 + c;
-                bool ok = (j < p.N) && !(p.mask_mode == GC_MASK_SELF && i == j);
+                bool ok = (j < p.N) && !(p.mask_mode == GC_MASK_SELF && i + p.mask_shift == j);
                 v[c] = ok ? acc[r][c] * inv_tau : -INFINITY;
                 tile_max = fmaxf(tile_max, v[c]);
                 if (ok && i < p.B && j == (int64_t)pos[r]) a.pos_logit[i] = v[c];
@@ -238,7 +238,7 @@ __global__ void __launch_bounds__(THREADS) simt_sweep_kernel(SweepArgs a) {
             for (int c = 0; c < 4; ++c) {
                 int64_t y = y0 + tx * 4 + c;
                 float w = 0.f;
-                bool live = (x < a.nx) && (y < a.ny) && !(a.mask_mode == GC_MASK_SELF && x == y);
+                bool live = (x < a.nx) && (y < a.ny) && !(a.mask_mode == GC_MASK_SELF && x + a.mask_delta == y);
                 if (live) {
                     float lse = dq ? lse_x[r] : lse_y[c];
                     bool hit = dq ? (y == (int64_t)pos_x[r]) : (x == (int64_t)pos_y[c]);

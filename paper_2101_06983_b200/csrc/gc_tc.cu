@@ -104,6 +104,7 @@ struct TcParams {
     const float* slot_m;      // DP with nslots > 0: forward slots [nslots][ny] to merge instead of
     const float* slot_l;      //   reading row_lse
     int nslots;
+    int64_t mask_delta;       // GC_MASK_SELF drops the pair (x, y) with y == x + mask_delta
     Gate gate;                // closed: the kernel returns at once
     int* zero_me;             // forward sweeps: the ticket word of the reduction that follows
 };
@@ -536,6 +537,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
         const int cb0 = half * CB_PER;
         const int row = q * 32 + lane;
         const int64_t x = x0 + row;
+        const int64_t xm = x + p.mask_delta;     // the streamed index masked for this row
         const uint32_t lane_addr = (uint32_t)(q * 32) << 16;
         const bool self_mask = (p.mask_mode == GC_MASK_SELF);
         bool ok = true;
@@ -580,7 +582,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     tmem_ld_wait();
                     const int64_t yb = y0 + cb * 32;
                     if (yb >= p.ny) continue;
-                    if (pos_x >= yb && pos_x < yb + 32 && !(self_mask && x == pos_x)) {
+                    if (pos_x >= yb && pos_x < yb + 32 && !(self_mask && xm == pos_x)) {
                         const int rel = (int)(pos_x - yb);
                         float s = 0.f;
 #pragma unroll
@@ -596,8 +598,8 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         for (int c = 0; c < 32; ++c)
                             if (yb + c >= p.ny) s2[c] = -INFINITY;
                     }
-                    if (self_mask && x >= yb && x < yb + 32) {
-                        const int rel = (int)(x - yb);
+                    if (self_mask && xm >= yb && xm < yb + 32) {
+                        const int rel = (int)(xm - yb);
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
                             if (c == rel) s2[c] = -INFINITY;
@@ -661,7 +663,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 for (int j = 0; j < CB_PER; ++j) {
                     const int64_t yb = y0 + (cb0 + j) * 32;
                     const bool has_pos = pos_x >= yb && pos_x < yb + 32 && pos_x < p.ny &&
-                                         !(self_mask && x == pos_x);
+                                         !(self_mask && xm == pos_x);
                     if (has_pos) {
                         const int rel = (int)(pos_x - yb);
                         float sp = 0.f;
@@ -675,8 +677,8 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         for (int c = 0; c < 32; ++c)
                             if (yb + c >= p.ny) vv[j][c] = __float_as_uint(-INFINITY);
                     }
-                    if (self_mask && x >= yb && x < yb + 32) {
-                        const int rel = (int)(x - yb);
+                    if (self_mask && xm >= yb && xm < yb + 32) {
+                        const int rel = (int)(xm - yb);
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
                             if (c == rel) vv[j][c] = __float_as_uint(-INFINITY);
@@ -759,7 +761,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 for (int j = 0; j < CB_PER; ++j) {
                     const int64_t yb = y0 + (cb0 + j) * 32;
                     const bool has_pos = pos_x >= yb && pos_x < yb + 32 && pos_x < p.ny &&
-                                         !(self_mask && x == pos_x);
+                                         !(self_mask && xm == pos_x);
                     if (has_pos) {
                         const int rel = (int)(pos_x - yb);
                         float sp = 0.f;
@@ -773,8 +775,8 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         for (int c = 0; c < 32; ++c)
                             if (yb + c >= p.ny) vv[j][c] = __float_as_uint(-INFINITY);
                     }
-                    if (self_mask && x >= yb && x < yb + 32) {
-                        const int rel = (int)(x - yb);
+                    if (self_mask && xm >= yb && xm < yb + 32) {
+                        const int rel = (int)(xm - yb);
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
                             if (c == rel) vv[j][c] = __float_as_uint(-INFINITY);
@@ -974,7 +976,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         }
                     } else if (MODE == MODE_DA) {
                         const bool has_pos = pos_x >= yb && pos_x < yb + 32 && pos_x < p.ny &&
-                                             !(self_mask && x == pos_x);
+                                             !(self_mask && xm == pos_x);
                         if (has_pos) {
                             const int rel = (int)(pos_x - yb);
                             float sp = 0.f;
@@ -991,8 +993,8 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                             for (int c = 0; c < 32; ++c)
                                 if (yb + c >= p.ny) w[c] = 0.f;
                         }
-                        if (self_mask && x >= yb && x < yb + 32) {
-                            const int rel = (int)(x - yb);
+                        if (self_mask && xm >= yb && xm < yb + 32) {
+                            const int rel = (int)(xm - yb);
 #pragma unroll
                             for (int c = 0; c < 32; ++c)
                                 if (c == rel) w[c] = 0.f;
@@ -1033,8 +1035,8 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                             }
                         }
                     }
-                    if (self_mask && x >= yb && x < yb + 32) {
-                        const int rel = (int)(x - yb);
+                    if (self_mask && xm >= yb && xm < yb + 32) {
+                        const int rel = (int)(xm - yb);
 #pragma unroll
                         for (int c = 0; c < 32; ++c)
                             if (c == rel) w[c] = 0.f;
@@ -1290,6 +1292,7 @@ cudaError_t tc_launch_fwd(const FwdArgs& a, cudaStream_t st) {
     p.xres = smem_plan(p.kc).xres;
     p.ipc = smem_plan(p.kc).ipc;
     p.mask_mode = pr.mask_mode;
+    p.mask_delta = pr.mask_shift;
     p.inv_tau = 1.f / pr.tau;
     p.c1 = 1.4426950408889634f / pr.tau;
     p.pos_idx = pr.pos_idx;
@@ -1322,6 +1325,7 @@ cudaError_t tc_launch_fwd_store(const FwdArgs& a, void* weights, int64_t ldw, co
     p.xres = sp.xres;
     p.ipc = sp.ipc;
     p.mask_mode = pr.mask_mode;
+    p.mask_delta = pr.mask_shift;
     p.inv_tau = 1.f / pr.tau;
     p.c1 = 1.4426950408889634f / pr.tau;
     p.pos_idx = pr.pos_idx;
@@ -1353,6 +1357,7 @@ cudaError_t tc_launch_fused_dq(const FwdArgs& a, float* partial, int groups, cud
     p.xres = smem_plan(kc).xres;
     p.ipc = smem_plan(kc).ipc;
     p.mask_mode = pr.mask_mode;
+    p.mask_delta = pr.mask_shift;
     p.inv_tau = 1.f / pr.tau;
     p.c1 = 1.4426950408889634f / pr.tau;
     p.pos_idx = pr.pos_idx;
@@ -1391,6 +1396,7 @@ cudaError_t tc_launch_anchored_dq(const FwdArgs& a, float* partial, int groups,
     p.xres = smem_plan(kc).xres;
     p.ipc = smem_plan(kc).ipc;
     p.mask_mode = pr.mask_mode;
+    p.mask_delta = pr.mask_shift;
     p.inv_tau = 1.f / pr.tau;
     p.c1 = 1.4426950408889634f / pr.tau;
     p.pos_idx = pr.pos_idx;
@@ -1419,6 +1425,7 @@ cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     p.xres = smem_plan(kc).xres;
     p.ipc = smem_plan(kc).ipc;
     p.mask_mode = a.mask_mode;
+    p.mask_delta = a.mask_delta;
     p.inv_tau = a.inv_tau;
     p.c1 = 1.4426950408889634f * a.inv_tau;
     p.out_scale = a.out_scale;

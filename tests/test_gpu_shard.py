@@ -59,6 +59,62 @@ def test_ranks_together_reproduce_the_full_batch(binding, oracle, B, N, d, dtype
     assert grad_err(dP.cpu().numpy(), ref["dP"], floor) <= tol["grad"]
 
 
+MASKED = [
+    # rows (Q = P = the same rows), d, dtype, world: the self mask with shared rows, as in the
+    # two-view workload; the masked pair of a rank's row lies wherever that row sits in the batch
+    (60, 40, "f32", 3),
+    (300, 128, "bf16", 2),
+    (520, 768, "bf16", 3),
+    (1000, 128, "bf16", 4),
+]
+
+
+@pytest.mark.parametrize("n,d,dtype,world", MASKED)
+def test_self_mask_follows_the_rank_ranges(binding, oracle, n, d, dtype, world):
+    prob = inputs.random_problem(n, n, d, dtype, seed=n + d, tau=0.2, mask_mode=inputs.MASK_SELF,
+                                 scale=d ** -0.5, shared=True)
+    ref = oracle.build_cache(prob.Q, prob.P, prob.pos_idx, prob.tau, prob.mask_mode)
+    Q, P, pos = to_device(prob)
+    row_lse = torch.zeros(n, device="cuda")
+    dQ = torch.empty(n, d, device="cuda")
+    dP = torch.empty(n, d, device="cuda")
+    loss = torch.zeros(1, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    part = torch.zeros(1, device="cuda")
+    for q0, b in sharded.row_ranges(n, world):
+        binding.gc_shard_fwd_dq(Q, P, pos, prob.tau, q0, b, part, row_lse, dQ[q0:q0 + b],
+                                dev_status=status, mask_mode=prob.mask_mode)
+        loss += part
+    for p0, m in sharded.row_ranges(n, world):
+        binding.gc_shard_dp(Q, P, pos, prob.tau, row_lse, p0, m, dP[p0:p0 + m], dev_status=status,
+                            mask_mode=prob.mask_mode)
+    torch.cuda.synchronize()
+    tol = TOL[dtype]
+    assert int(status.item()) == 0
+    assert abs(loss.item() - ref["loss"]) <= tol["loss"] * abs(ref["loss"])
+    lse = row_lse.cpu().numpy().astype(np.float64)
+    assert np.abs(lse - ref["row_lse"]).max() <= tol["lse"] * max(1.0, np.abs(ref["row_lse"]).max())
+    floor = grad_floor(prob)
+    assert grad_err(dQ.cpu().numpy(), ref["dQ"], floor) <= tol["grad"]
+    assert grad_err(dP.cpu().numpy(), ref["dP"], floor) <= tol["grad"]
+
+
+def test_sharded_step_object_on_one_gpu(binding, oracle):
+    """`sharded.ShardedStep` (preallocated buffers, library kernels) as a world of one rank, twice
+    in a row on the same buffers."""
+    prob = inputs.random_problem(300, 520, 768, "bf16", seed=12, tau=0.5, scale=768 ** -0.5)
+    ref = oracle.build_cache(prob.Q, prob.P, prob.pos_idx, prob.tau, prob.mask_mode)
+    Q, P, pos = to_device(prob)
+    step = sharded.ShardedStep(prob.B, prob.N, prob.d, Q.dtype, Q.device)
+    for _ in range(2):
+        loss, lse, dQ, dP = step.run(Q, P, pos, prob.tau, measure=True)
+        torch.cuda.synchronize()
+        assert abs(loss.item() - ref["loss"]) <= TOL["bf16"]["loss"] * abs(ref["loss"])
+        assert grad_err(dQ.cpu().numpy(), ref["dQ"]) <= TOL["bf16"]["grad"]
+        assert grad_err(dP.cpu().numpy(), ref["dP"]) <= TOL["bf16"]["grad"]
+    assert set(step.timings) == {"gather_reps_s", "fwd_dq_s", "lse_and_loss_s", "dp_s"}
+
+
 def test_one_rank_is_the_whole_batch(binding):
     """world = 1: the two calls together are gc_loss_fwd + gc_loss_bwd on the same kernels."""
     prob = inputs.random_problem(140, 270, 64, "bf16", seed=5, tau=0.7, scale=0.125)
