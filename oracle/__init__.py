@@ -51,6 +51,9 @@ def _load():
         lib.gco_passage_rows.restype = ctypes.c_int
         lib.gco_passage_rows.argtypes = [dp, dp, ip, i64, i64, i64, ctypes.c_double, ctypes.c_int,
                                          dp, lp, i64, dp]
+        lib.gco_build_variant.restype = ctypes.c_int
+        lib.gco_build_variant.argtypes = [dp, dp, lp, ip, i64, i64, i64, ctypes.c_double,
+                                          ctypes.c_int, ctypes.c_int, ctypes.c_int, dp, dp, dp, dp]
         lib.gco_cache_apply.restype = ctypes.c_int
         lib.gco_cache_apply.argtypes = [dp, dp, i64, i64, i64, ctypes.c_int, dp]
         _lib = lib
@@ -140,6 +143,37 @@ def passage_rows(Q, P, pos_idx, row_lse, rows, tau=1.0, mask_mode=0):
     if rc != 0:
         raise ValueError(f"oracle rejected the problem (code {rc})")
     return dP
+
+
+def build_variant(Q, P, positives, tau=1.0, mask_mode=0, cosine=False, two_direction=False):
+    """Loss variants of Section 3.3's Step 2 remark: cosine similarity (gradients with respect to
+    the un-normalised rows), several positives per query (`positives`: a list of index lists, or a
+    1-D array for one positive each), the two-direction loss, and dL/dtau.
+    Returns dict(loss, dQ, dP, dtau) in float64."""
+    Q = _f64(Q)
+    P = _f64(P)
+    B, d = Q.shape
+    N = P.shape[0]
+    if isinstance(positives, np.ndarray) and positives.ndim == 1:
+        lists = [[int(v)] for v in positives]
+    else:
+        lists = [[int(v) for v in row] for row in positives]
+    if len(lists) != B or P.shape[1] != d:
+        raise ValueError("shape mismatch")
+    ptr = np.zeros(B + 1, np.int64)
+    ptr[1:] = np.cumsum([len(r) for r in lists])
+    flat = np.ascontiguousarray([v for r in lists for v in r], dtype=np.int32)
+    loss, dtau = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    dQ = np.empty((B, d), np.float64)
+    dP = np.empty((N, d), np.float64)
+    rc = _load().gco_build_variant(
+        _ptr(Q, ctypes.c_double), _ptr(P, ctypes.c_double), _ptr(ptr, ctypes.c_int64),
+        _ptr(flat, ctypes.c_int32), B, N, d, float(tau), int(mask_mode), int(bool(cosine)),
+        int(bool(two_direction)), ctypes.byref(loss), _ptr(dQ, ctypes.c_double),
+        _ptr(dP, ctypes.c_double), ctypes.byref(dtau))
+    if rc != 0:
+        raise ValueError(f"oracle rejected the problem (code {rc})")
+    return dict(loss=float(loss.value), dQ=dQ, dP=dP, dtau=float(dtau.value))
 
 
 def cache_apply(U, X, dW=None):

@@ -13,8 +13,9 @@
  * logistic case, scale and permutation symmetries, and the paper's exactness claim on a linear
  * encoder; gco_query_rows and gco_passage_rows by the same hand-worked example, finite
  * differences and closed form, row for row; gco_cache_apply (Step 3 for a linear encoder) by the
- * finite-difference gradient with respect to the encoder matrix and a hand-worked example.  No
- * function here is "parity unpinned".
+ * finite-difference gradient with respect to the encoder matrix and a hand-worked example;
+ * gco_build_variant (cosine similarity, several positives, two-direction loss, dL/dtau) in
+ * tests/test_oracle_variants.py.  No function here is "parity unpinned".
  *
  * Notation (paper, Section 3.1-3.2): Q row i is f(s_i), P row j is g(t_j), pos_idx[i] is r_i,
  * tau the temperature, S_ij = <f(s_i), g(t_j)> / tau.
@@ -260,5 +261,157 @@ int gco_cache_apply(const double* U, const double* X, int64_t rows, int64_t d, i
             else dW[a * d_in + b] = s;
         }
     }
+    return 0;
+}
+
+/*
+ * Variants of the loss that the paper leaves to automatic differentiation (Section 3.3, Step 2:
+ * any loss on the stored representations works).  Still Step 2: the loss over all B x N pairs
+ * and its gradient with respect to every representation, plus the derivative with respect to the
+ * temperature.  Everything explicit, in double; S and G stored whole.
+ *
+ *   cosine != 0      similarity is the cosine: S_ij = <q_i/|q_i|, p_j/|p_j|> / tau.  dQ, dP are
+ *                    the gradients with respect to the UN-normalised rows (the Jacobian of the
+ *                    normalisation, (I - n n^T)/|x| with n = x/|x|, applied to the gradient with
+ *                    respect to the unit rows).
+ *   positives        CSR: query i has the positives pos_list[pos_ptr[i] .. pos_ptr[i+1]) (at least
+ *                    one, distinct, none on the masked diagonal).  Loss of query i = mean over its
+ *                    positives of -log p_ir, so G_ij = (p_ij - [j in R_i]/|R_i|)/B.  One positive
+ *                    per query is Eq. 1.
+ *   two_direction    (needs exactly one positive per query) L = (L_row + L_col)/2 with L_row =
+ *                    Eq. 1 and L_col its mirror image over the same B positive pairs: passage r_i
+ *                    is the anchor, the B queries are its candidates,
+ *                        L_col = (1/B) sum_i (log sum_{i'} exp(S_{i' r_i}) - S_{i r_i}),
+ *                    the sum over i' running over the allowed pairs.  N may exceed B: passages
+ *                    that are nobody's positive only appear in the row softmax.
+ *   dtau             dL/dtau = -(1/tau) sum_ij G_ij S_ij  (S = <.,.>/tau).
+ * Outputs may be NULL.  Returns 0, a positive code for bad arguments, -1 when out of memory.
+ * Pinned in tests/test_oracle_variants.py by finite differences with respect to every input and
+ * tau, Euler's identity for the joint scaling of Q and tau, orthogonality of the cosine
+ * gradients to their rows, the role-swap symmetry of the two-direction loss and reduction to
+ * gco_build_cache.
+ */
+int gco_build_variant(const double* Q, const double* P, const int64_t* pos_ptr,
+                      const int32_t* pos_list, int64_t B, int64_t N, int64_t d, double tau,
+                      int mask_mode, int cosine, int two_direction, double* loss, double* dQ,
+                      double* dP, double* dtau) {
+    if (B <= 0 || N <= 0 || d <= 0) return 1;
+    if (!(tau > 0.0) || !isfinite(tau)) return 2;
+    if (mask_mode != GCO_MASK_NONE && mask_mode != GCO_MASK_SELF) return 3;
+    if (pos_ptr[0] != 0) return 4;
+    for (int64_t i = 0; i < B; ++i) {
+        int64_t n = pos_ptr[i + 1] - pos_ptr[i];
+        if (n < 1) return 4;
+        if (two_direction && n != 1) return 7;
+        for (int64_t a = pos_ptr[i]; a < pos_ptr[i + 1]; ++a) {
+            if (pos_list[a] < 0 || pos_list[a] >= N) return 4;
+            if (!allowed(mask_mode, i, pos_list[a])) return 5;
+            for (int64_t b = pos_ptr[i]; b < a; ++b)
+                if (pos_list[b] == pos_list[a]) return 6;
+        }
+    }
+    double* Qn = (double*)malloc(sizeof(double) * (size_t)B * (size_t)d);
+    double* Pn = (double*)malloc(sizeof(double) * (size_t)N * (size_t)d);
+    double* qnorm = (double*)malloc(sizeof(double) * (size_t)B);
+    double* pnorm = (double*)malloc(sizeof(double) * (size_t)N);
+    double* S = (double*)malloc(sizeof(double) * (size_t)B * (size_t)N);
+    double* G = (double*)malloc(sizeof(double) * (size_t)B * (size_t)N);
+    double* gQ = (double*)malloc(sizeof(double) * (size_t)B * (size_t)d);
+    double* gP = (double*)malloc(sizeof(double) * (size_t)N * (size_t)d);
+    if (!Qn || !Pn || !qnorm || !pnorm || !S || !G || !gQ || !gP) {
+        free(Qn); free(Pn); free(qnorm); free(pnorm); free(S); free(G); free(gQ); free(gP);
+        return -1;
+    }
+    /* the rows the similarity is taken of: the inputs, or their unit vectors */
+    for (int64_t i = 0; i < B; ++i) {
+        double s = 0.0;
+        for (int64_t k = 0; k < d; ++k) s += Q[i * d + k] * Q[i * d + k];
+        qnorm[i] = cosine ? sqrt(s) : 1.0;
+        for (int64_t k = 0; k < d; ++k) Qn[i * d + k] = Q[i * d + k] / qnorm[i];
+    }
+    for (int64_t j = 0; j < N; ++j) {
+        double s = 0.0;
+        for (int64_t k = 0; k < d; ++k) s += P[j * d + k] * P[j * d + k];
+        pnorm[j] = cosine ? sqrt(s) : 1.0;
+        for (int64_t k = 0; k < d; ++k) Pn[j * d + k] = P[j * d + k] / pnorm[j];
+    }
+    for (int64_t i = 0; i < B; ++i) logits_row(Qn, Pn, i, N, d, tau, S + i * N);
+
+    /* row direction: every query against all passages */
+    double total = 0.0;
+    for (int64_t i = 0; i < B; ++i) {
+        const double lse = lse_row(S + i * N, i, N, mask_mode);
+        const int64_t np = pos_ptr[i + 1] - pos_ptr[i];
+        for (int64_t j = 0; j < N; ++j)
+            G[i * N + j] = (allowed(mask_mode, i, j) ? exp(S[i * N + j] - lse) : 0.0) / (double)B;
+        for (int64_t a = pos_ptr[i]; a < pos_ptr[i + 1]; ++a) {
+            total += (lse - S[i * N + pos_list[a]]) / (double)np;
+            G[i * N + pos_list[a]] -= 1.0 / ((double)np * (double)B);
+        }
+    }
+    double L = total / (double)B;
+
+    if (two_direction) {
+        /* column direction: the positive passage of query i against all queries */
+        double total_c = 0.0;
+        for (int64_t i = 0; i < B; ++i) {
+            const int64_t j = pos_list[pos_ptr[i]];
+            double m = -INFINITY;
+            for (int64_t k = 0; k < B; ++k)
+                if (allowed(mask_mode, k, j) && S[k * N + j] > m) m = S[k * N + j];
+            double sum = 0.0;
+            for (int64_t k = 0; k < B; ++k)
+                if (allowed(mask_mode, k, j)) sum += exp(S[k * N + j] - m);
+            const double lse_c = m + log(sum);
+            total_c += lse_c - S[i * N + j];
+            /* d/dS of this term: softmax over the column, minus one at (i, j); both halves
+             * of the loss weigh 1/2 */
+            for (int64_t k = 0; k < B; ++k) {
+                double pc = allowed(mask_mode, k, j) ? exp(S[k * N + j] - lse_c) : 0.0;
+                G[k * N + j] += pc / (double)B;
+            }
+            G[i * N + j] -= 1.0 / (double)B;
+        }
+        L = 0.5 * (L + total_c / (double)B);
+        for (int64_t e = 0; e < B * N; ++e) G[e] *= 0.5;
+    }
+    if (loss) *loss = L;
+
+    /* gradients with respect to the rows the similarity saw, and with respect to tau */
+    for (int64_t i = 0; i < B; ++i)
+        for (int64_t k = 0; k < d; ++k) {
+            double s = 0.0;
+            for (int64_t j = 0; j < N; ++j) s += G[i * N + j] * Pn[j * d + k];
+            gQ[i * d + k] = s / tau;
+        }
+    for (int64_t j = 0; j < N; ++j)
+        for (int64_t k = 0; k < d; ++k) {
+            double s = 0.0;
+            for (int64_t i = 0; i < B; ++i) s += G[i * N + j] * Qn[i * d + k];
+            gP[j * d + k] = s / tau;
+        }
+    if (dtau) {
+        double s = 0.0;
+        for (int64_t e = 0; e < B * N; ++e) s += G[e] * S[e];
+        *dtau = -s / tau;
+    }
+    /* back through the normalisation: dx = (g - n <n, g>) / |x| */
+    if (dQ)
+        for (int64_t i = 0; i < B; ++i) {
+            double dot = 0.0;
+            for (int64_t k = 0; k < d; ++k) dot += Qn[i * d + k] * gQ[i * d + k];
+            for (int64_t k = 0; k < d; ++k)
+                dQ[i * d + k] = cosine ? (gQ[i * d + k] - Qn[i * d + k] * dot) / qnorm[i]
+                                       : gQ[i * d + k];
+        }
+    if (dP)
+        for (int64_t j = 0; j < N; ++j) {
+            double dot = 0.0;
+            for (int64_t k = 0; k < d; ++k) dot += Pn[j * d + k] * gP[j * d + k];
+            for (int64_t k = 0; k < d; ++k)
+                dP[j * d + k] = cosine ? (gP[j * d + k] - Pn[j * d + k] * dot) / pnorm[j]
+                                       : gP[j * d + k];
+        }
+    free(Qn); free(Pn); free(qnorm); free(pnorm); free(S); free(G); free(gQ); free(gP);
     return 0;
 }

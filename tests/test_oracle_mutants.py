@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 
 import test_oracle_pins as pins
+import test_oracle_variants as vpins
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 SRC = open(os.path.join(ROOT, "oracle", "gc_oracle.c")).read()
@@ -44,6 +45,25 @@ MUTANTS = {
     "passage_rows: one-hot dropped": (
         "double g = (p - ((j == pos_idx[i]) ? 1.0 : 0.0)) / (double)B;\n            for",
         "double g = p / (double)B;\n            for"),
+    "variant: 1/|R_i| missing in G": (
+        "G[i * N + pos_list[a]] -= 1.0 / ((double)np * (double)B);",
+        "G[i * N + pos_list[a]] -= 1.0 / (double)B;"),
+    "variant: 1/|R_i| missing in the loss": (
+        "total += (lse - S[i * N + pos_list[a]]) / (double)np;", "total += (lse - S[i * N + pos_list[a]]);"),
+    "variant: projection dropped from the cosine Jacobian": (
+        "dQ[i * d + k] = cosine ? (gQ[i * d + k] - Qn[i * d + k] * dot) / qnorm[i]",
+        "dQ[i * d + k] = cosine ? gQ[i * d + k] / qnorm[i]"),
+    "variant: 1/|p| dropped from the cosine Jacobian": (
+        "dP[j * d + k] = cosine ? (gP[j * d + k] - Pn[j * d + k] * dot) / pnorm[j]",
+        "dP[j * d + k] = cosine ? (gP[j * d + k] - Pn[j * d + k] * dot)"),
+    "variant: wrong sign of dtau": ("*dtau = -s / tau;", "*dtau = s / tau;"),
+    "variant: dtau without 1/tau": ("*dtau = -s / tau;", "*dtau = -s;"),
+    "variant: halves not averaged": ("for (int64_t e = 0; e < B * N; ++e) G[e] *= 0.5;", ""),
+    "variant: column softmax minus one at the wrong query": (
+        "G[i * N + j] -= 1.0 / (double)B;\n        }\n        L = 0.5",
+        "G[((i + 1) % B) * N + j] -= 1.0 / (double)B;\n        }\n        L = 0.5"),
+    "variant: column logsumexp ignores the mask": (
+        "if (allowed(mask_mode, k, j)) sum += exp(S[k * N + j] - m);", "sum += exp(S[k * N + j] - m);"),
     "cache_apply reads U transposed": ("s += U[i * d + a] * X[i * d_in + b];",
                                        "s += U[(a % rows) * d + (i % d)] * X[i * d_in + b];"),
     "cache_apply overwrites instead of accumulating": ("if (accumulate) dW[a * d_in + b] += s;",
@@ -127,6 +147,33 @@ def _wrap(libpath):
             raise ValueError(f"rejected ({rc})")
         return dP
 
+    lib.gco_build_variant.restype = ctypes.c_int
+    lib.gco_build_variant.argtypes = [dp, dp, lp, ip, i64, i64, i64, ctypes.c_double, ctypes.c_int,
+                                      ctypes.c_int, ctypes.c_int, dp, dp, dp, dp]
+
+    def build_variant(Q, P, positives, tau=1.0, mask_mode=0, cosine=False, two_direction=False):
+        Q, P = real._f64(Q), real._f64(P)
+        B, d = Q.shape
+        N = P.shape[0]
+        if isinstance(positives, np.ndarray) and positives.ndim == 1:
+            lists = [[int(v)] for v in positives]
+        else:
+            lists = [[int(v) for v in row] for row in positives]
+        ptr = np.zeros(B + 1, np.int64)
+        ptr[1:] = np.cumsum([len(r) for r in lists])
+        flat = np.ascontiguousarray([v for r in lists for v in r], dtype=np.int32)
+        loss, dtau = ctypes.c_double(0.0), ctypes.c_double(0.0)
+        dQ, dP = np.empty((B, d)), np.empty((N, d))
+        rc = lib.gco_build_variant(real._ptr(Q, ctypes.c_double), real._ptr(P, ctypes.c_double),
+                                   real._ptr(ptr, ctypes.c_int64), real._ptr(flat, ctypes.c_int32), B,
+                                   N, d, float(tau), int(mask_mode), int(bool(cosine)),
+                                   int(bool(two_direction)), ctypes.byref(loss),
+                                   real._ptr(dQ, ctypes.c_double), real._ptr(dP, ctypes.c_double),
+                                   ctypes.byref(dtau))
+        if rc != 0:
+            raise ValueError(f"rejected ({rc})")
+        return dict(loss=float(loss.value), dQ=dQ, dP=dP, dtau=float(dtau.value))
+
     lib.gco_cache_apply.restype = ctypes.c_int
     lib.gco_cache_apply.argtypes = [dp, dp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_int, dp]
@@ -146,7 +193,7 @@ def _wrap(libpath):
 
     return types.SimpleNamespace(
         build_cache=build_cache, cache_apply=cache_apply, query_rows=query_rows,
-        passage_rows=passage_rows,
+        passage_rows=passage_rows, build_variant=build_variant,
         loss_only=lambda Q, P, pos, tau=1.0, mask=0: build_cache(Q, P, pos, tau, mask)["loss"])
 
 
@@ -163,6 +210,12 @@ def _pins(o):
     yield lambda: pins.test_row_sampled_entry_points_match_finite_differences(o, 0.1, 1)
     yield lambda: pins.test_row_sampled_entry_points_match_finite_differences(o, 1.0, 0)
     yield lambda: pins.test_row_sampled_entry_points_identical_representations(o)
+    yield lambda: vpins.test_variant_gradients_match_finite_differences(o, True, False, 1, 0.2)
+    yield lambda: vpins.test_variant_gradients_match_finite_differences(o, False, True, 1, 0.2)
+    yield lambda: vpins.test_euler_identity_for_joint_scaling(o, True)
+    yield lambda: vpins.test_cosine_is_scale_invariant_and_gradients_are_tangent(o)
+    yield lambda: vpins.test_two_direction_loss_is_symmetric_under_role_swap(o)
+    yield lambda: vpins.test_two_positives_hand_worked(o)
     yield lambda: pins.test_cache_apply_hand_worked_example(o)
     yield lambda: pins.test_cache_apply_chunks_reproduce_full_batch_parameter_gradient(o)
 
