@@ -197,6 +197,35 @@ int gc_shard_dp(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
                 void* ws, size_t ws_bytes, int* dev_status, void* cuda_stream);
 
 /*
+ * Loss variants (Section 3.3, Step 2: the loss computed on the stored representations may vary,
+ * and the paper leaves its derivative to automatic differentiation; these calls supply the two
+ * derivatives that need no change to the sweeps).
+ *
+ * Cosine similarity, S_ij = <q_i/|q_i|, p_j/|p_j|> / tau:
+ *   gc_row_normalize  Xn[i] = X[i] / |X[i]| in the dtype of X (bf16: round to nearest even) and
+ *                     inv_norm[i] = 1/|X[i]| (float; the norm is accumulated in fp32; a zero row
+ *                     stays zero with inv_norm 0).  Call it on Q and on P, run gc_build_cache (or
+ *                     gc_loss_fwd / gc_loss_bwd) on the unit rows, then
+ *   gc_cosine_bwd     dX[i] = inv_norm[i] (dXn[i] - n_i <n_i, dXn[i]>), n_i = inv_norm[i] X[i] in
+ *                     fp32: the Jacobian (I - n n^T)/|x| of the normalisation applied to the cache
+ *                     rows dXn (dQ or dP of the unit rows).  dX may be the same buffer as dXn.
+ * Learnable temperature:
+ *   gc_dtau           *dtau = dL/dtau = -(1/tau) sum_i <Q_i, dQ_i>, with Q the rows the sweeps saw
+ *                     and dQ their cache rows (Eq. 5 gives <Q_i, dQ_i> = sum_j G_ij S_ij).  Rows
+ *                     are summed in a fixed order.  Workspace: gc_dtau_workspace_bytes(B).
+ * X, Xn, Q: [rows x d] of dtype (GC_F32 or GC_BF16), leading dimensions in elements, rows on
+ * 16-byte boundaries, d a multiple of 8 (else GC_ERR_LIMIT); dXn, dX, dQ float.  Device pointers,
+ * asynchronous on cuda_stream, deterministic.
+ */
+int gc_row_normalize(const void* X, int64_t ldx, int64_t rows, int d, int dtype, void* Xn,
+                     int64_t ldxn, float* inv_norm, void* cuda_stream);
+int gc_cosine_bwd(const void* X, int64_t ldx, int64_t rows, int d, int dtype, const float* inv_norm,
+                  const float* dXn, int64_t lddxn, float* dX, int64_t lddx, void* cuda_stream);
+size_t gc_dtau_workspace_bytes(int64_t B);
+int gc_dtau(const void* Q, int64_t ldq, const float* dQ, int64_t lddq, int64_t B, int d, float tau,
+            int dtype, float* dtau, void* ws, size_t ws_bytes, void* cuda_stream);
+
+/*
  * Forward with library-owned scratch (no counterpart in the paper: it exists for the sake of
  * callers, not of the method).  Same inputs, outputs and results as gc_loss_fwd, but the caller
  * passes no workspace.  It is meant for callers that cannot obtain device memory at the point of

@@ -23,7 +23,8 @@ EXPORTS = ("gc_workspace_bytes", "gc_plan_name", "gc_kernel_launches", "gc_loss_
            "gc_profile_enable",
            "gc_profile_read", "gc_profile_read_call", "gc_static_scratch_need", "gc_loss_fwd_static",
            "gc_cache_apply_workspace_bytes", "gc_cache_apply", "gc_shard_workspace_bytes",
-           "gc_shard_fwd_dq", "gc_shard_dp", "gc_selftest_wait_limit")
+           "gc_shard_fwd_dq", "gc_shard_dp", "gc_selftest_wait_limit", "gc_row_normalize",
+           "gc_cosine_bwd", "gc_dtau_workspace_bytes", "gc_dtau")
 GC_STATIC_SCRATCH_BYTES = 2 << 20
 
 
@@ -75,6 +76,14 @@ def _load() -> ctypes.CDLL:
                                              vp, vp]
     lib.gc_shard_dp.restype = i32
     lib.gc_shard_dp.argtypes = common + [vp, i64, i64, vp, i64, vp, ctypes.c_size_t, vp, vp]
+    lib.gc_row_normalize.restype = i32
+    lib.gc_row_normalize.argtypes = [vp, i64, i64, i32, i32, vp, i64, vp, vp]
+    lib.gc_cosine_bwd.restype = i32
+    lib.gc_cosine_bwd.argtypes = [vp, i64, i64, i32, i32, vp, vp, i64, vp, i64, vp]
+    lib.gc_dtau_workspace_bytes.restype = ctypes.c_size_t
+    lib.gc_dtau_workspace_bytes.argtypes = [i64]
+    lib.gc_dtau.restype = i32
+    lib.gc_dtau.argtypes = [vp, i64, vp, i64, i64, i32, f32, i32, vp, vp, ctypes.c_size_t, vp]
     lib.gc_selftest_wait_limit.restype = i32
     lib.gc_selftest_wait_limit.argtypes = [ctypes.c_uint64, vp, vp, vp]
     lib.gc_profile_enable.restype = i32
@@ -267,6 +276,38 @@ def gc_shard_dp(Q, P, pos_idx, tau, row_lse, p0, p_count, dP, ws=None, dev_statu
                           ws.numel(), _ptr(dev_status), _stream())
     if rc != 0:
         raise GradCacheError(rc, "gc_shard_dp")
+
+
+def gc_row_normalize(X, Xn, inv_norm) -> None:
+    """Xn[i] = X[i]/|X[i]| (dtype of X) and inv_norm[i] = 1/|X[i]| (float32): the unit rows of the
+    cosine-similarity loss."""
+    rows, d = X.shape
+    rc = _lib.gc_row_normalize(_ptr(X), X.stride(0), rows, d, _dtype_code(X), _ptr(Xn),
+                               Xn.stride(0), _ptr(inv_norm), _stream())
+    if rc != 0:
+        raise GradCacheError(rc, "gc_row_normalize")
+
+
+def gc_cosine_bwd(X, inv_norm, dXn, dX) -> None:
+    """dX[i] = inv_norm[i] (dXn[i] - n_i <n_i, dXn[i]>): cache rows of the unit rows taken back
+    through the normalisation (dX may be dXn)."""
+    rows, d = X.shape
+    rc = _lib.gc_cosine_bwd(_ptr(X), X.stride(0), rows, d, _dtype_code(X), _ptr(inv_norm),
+                            _ptr(dXn), dXn.stride(0), _ptr(dX), dX.stride(0), _stream())
+    if rc != 0:
+        raise GradCacheError(rc, "gc_cosine_bwd")
+
+
+def gc_dtau(Q, dQ, tau, dtau, ws=None) -> None:
+    """dtau[0] = dL/dtau = -(1/tau) sum_i <Q_i, dQ_i> (Q: the rows the sweeps saw)."""
+    B, d = Q.shape
+    if ws is None:
+        ws = torch.empty(max(int(_lib.gc_dtau_workspace_bytes(B)), 256), dtype=torch.uint8,
+                         device=Q.device)
+    rc = _lib.gc_dtau(_ptr(Q), Q.stride(0), _ptr(dQ), dQ.stride(0), B, d, float(tau),
+                      _dtype_code(Q), _ptr(dtau), _ptr(ws), ws.numel(), _stream())
+    if rc != 0:
+        raise GradCacheError(rc, "gc_dtau")
 
 
 def gc_selftest_wait_limit(limit_ns: int, dev_status, waited_ns=None) -> None:

@@ -57,27 +57,6 @@ struct QuadParams {
 
 constexpr int Q_XRES = 0;     // X chunks that stay resident (a deeper ring serves better)
 
-// Optional diagnostics (-DGC_TC_TRACE): event timeline of the two pair leaders of cluster 0 in
-// the mode g_qev_mode selects; per role (tag, low clock bits) pairs.
-#ifdef GC_TC_TRACE
-__device__ unsigned int g_qevlog[4][8192];
-__device__ int g_qev_mode = -1;
-#define QEV_DECL(cnt) int cnt = 0
-#define QEV(role, cnt, kind, idx)                                                          \
-    do {                                                                                   \
-        if (qev_on && (cnt) < 4094) {                                                      \
-            g_qevlog[role][2 * (cnt)] = ((unsigned)(kind) << 16) | ((unsigned)(idx) & 0xffffu); \
-            g_qevlog[role][2 * (cnt) + 1] = (unsigned)clock64();                           \
-            ++(cnt);                                                                       \
-        }                                                                                  \
-    } while (0)
-#define QEV_END(role, cnt) do { if (qev_on) g_qevlog[role][2 * 4095] = (unsigned)(cnt); } while (0)
-#else
-#define QEV_DECL(cnt)
-#define QEV(role, cnt, kind, idx)
-#define QEV_END(role, cnt)
-#endif
-
 struct QBars {
     uint64_t x_full;
     uint64_t y_full[MAX_STAGES];
@@ -136,9 +115,6 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
 
     const uint32_t rank = cluster_ctarank();        // 0..3
     const int pr = (int)(rank >> 1);                // pair = column half = duty parity
-#ifdef GC_TC_TRACE
-    const bool qev_on = (blockIdx.x == 0 || blockIdx.x == 2) && lane == 0 && g_qev_mode == MODE;
-#endif
     const int side = (int)(rank & 1);               // which of the two x tiles
     const bool leader = (side == 0);
     const uint32_t leader_rank = rank & ~1u;
@@ -218,9 +194,6 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
         int next = 0;
         uint32_t next_phase = 0;
         bool ok = true;
-#ifdef GC_TC_TRACE
-        int ev_p = 0;
-#endif
         auto acquire = [&]() -> int {
             const int stage = next;
             const uint32_t phase = next_phase;
@@ -230,16 +203,6 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                 ok = false;
                 return -1;
             }
-#ifdef GC_TC_TRACE
-            if (blockIdx.x == 0 && lane == 0 && g_qev_mode == MODE + 16) {
-                if (ev_p < 4094) {
-                    g_qevlog[2 + warp][2 * ev_p] = (20u << 16) | (unsigned)stage;
-                    g_qevlog[2 + warp][2 * ev_p + 1] = (unsigned)clock64();
-                    ++ev_p;
-                    g_qevlog[2 + warp][2 * 4095] = (unsigned)ev_p;
-                }
-            }
-#endif
             return stage;
         };
         // kind 0: this CTA's 64 rows of two Y chunks (S phase); kind 1: one X chunk of its 128
@@ -287,10 +250,8 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
             const uint32_t ring_lo = desc_lo(y_smem, CHUNK_BYTES);
             int next = 0;
             uint32_t next_phase = 0;
-            QEV_DECL(ev_m);
             bool ok = mbar_wait(smem_u32(&bars.x_full), 0, abort_flag);
             tc_fence_after();
-            QEV(pr, ev_m, 0, 0);
             auto next_stage = [&]() -> int {
                 const int stage = next;
                 const uint32_t phase = next_phase;
@@ -299,29 +260,17 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                     ok = false;
                     return -1;
                 }
-#ifdef GC_TC_TRACE
-                if (blockIdx.x == 0 && lane == 0 && g_qev_mode == MODE + 16) {
-                    if (ev_m < 4094) {
-                        g_qevlog[0][2 * ev_m] = (1u << 16) | (unsigned)stage;
-                        g_qevlog[0][2 * ev_m + 1] = (unsigned)clock64();
-                        ++ev_m;
-                        g_qevlog[0][2 * 4095] = (unsigned)ev_m;
-                    }
-                }
-#endif
                 return stage;
             };
             for_each_op([&](int kind, int idx) {
                 if (!ok) return;
                 if (kind == 0) {
-                    QEV(pr, ev_m, 1, idx);
                     if (idx >= 1) {     // the softmax warps have read the previous duty tile
                         ok = mbar_wait(smem_u32(&bars.s_read), (idx - 1) & 1, abort_flag) &&
                              mbar_wait(smem_u32(&bars.s_read_peer), (idx - 1) & 1, abort_flag);
                         if (!ok) return;
                         tc_fence_after();
                     }
-                    QEV(pr, ev_m, 2, idx);
                     const uint32_t d_tmem = tmem + S_COL0;
                     for (int c = 0; c < p.kc && ok; c += 2) {
                         const int ys = next_stage();
@@ -348,10 +297,8 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                         }
                     }
                     if (ok && elect_one()) tc_commit_mask(smem_u32(&bars.s_full), pair_mask);
-                    QEV(pr, ev_m, 3, idx);
                 } else {
                     const int u = idx, b = u & 1, round = u >> 1;
-                    QEV(pr, ev_m, 4, idx);
                     if (b == pr) {
                         ok = mbar_wait(smem_u32(&bars.w_done), round & 1, abort_flag) &&
                              mbar_wait(smem_u32(&bars.w_done_peer), round & 1, abort_flag);
@@ -361,7 +308,6 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                     }
                     if (!ok) return;
                     tc_fence_after();
-                    QEV(pr, ev_m, 5, idx);
                     const uint32_t w_lo = desc_lo(w_smem + b * 32768u, 0);   // K-major A operand
                     for (int a = 0; a < na && ok; ++a) {
                         const int ys = next_stage();
@@ -381,10 +327,8 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                                 tc_commit_mask(smem_u32(&bars.w_empty[b][pr]), (uint16_t)0xF);
                         }
                     }
-                    QEV(pr, ev_m, 6, idx);
                 }
             });
-            QEV_END(pr, ev_m);
             if (ok && elect_one()) tc_commit_mask(smem_u32(&bars.acc_full), pair_mask);
         } else {
             // Forwarder: the second CTA's completed phases (S tile read, W written, received W
@@ -456,10 +400,6 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
         };
         float lse2_x = 0.f, l = 0.f, wmax = 0.f;
         int32_t pos_x = -1;
-#ifdef GC_TC_TRACE
-        const bool sev = (q == 0 && half == 0);
-        long long ph[7] = {0, 0, 0, 0, 0, 0, 0};
-#endif
         // FA may have been launched ahead of the anchor kernel's completion: row_ref, the range
         // flag and everything this role writes come after it
         if (MODE == QMODE_FA) dep_wait();
@@ -484,16 +424,9 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                     pos_y[jj] = (y < p.ny) ? p.pos_idx[y] : -1;
                 }
             }
-#ifdef GC_TC_TRACE
-            const long long c0_ = clock64();
-#endif
             ok = mbar_wait(smem_u32(&bars.s_full), j & 1, abort_flag);
             if (!ok) break;
             tc_fence_after();
-#ifdef GC_TC_TRACE
-            const long long c1_ = clock64(); ph[0] += c1_ - c0_;
-            long long c2_ = c1_, c3_ = c1_;
-#endif
             const uint32_t sbuf = tmem + lane_addr + S_COL0;
             // Both 32-column blocks are read at once, so that the S tile is free again; the
             // arithmetic then takes one block at a time in a loop that is not unrolled: the body is
@@ -502,15 +435,9 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
             tmem_ld32(sbuf + cb0 * 32, va);
             tmem_ld32(sbuf + (cb0 + 1) * 32, vb);
             tmem_ld_wait();
-#ifdef GC_TC_TRACE
-            c2_ = clock64(); ph[1] += c2_ - c1_;
-#endif
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bars.s_read));  // the S tile may be overwritten
-#ifdef GC_TC_TRACE
-            c3_ = clock64(); ph[2] += c3_ - c2_;
-#endif
             uint32_t keep_a[16], keep_b[16];
 #pragma unroll 1
             for (int jj = 0; jj < CB_PER; ++jj) {
@@ -628,15 +555,9 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
             }
             put_w_block(0, keep_a);
             put_w_block(1, keep_b);
-#ifdef GC_TC_TRACE
-            const long long c5_ = clock64(); ph[4] += c5_ - c3_;
-#endif
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             tc_fence_before();
             __syncwarp();
-#ifdef GC_TC_TRACE
-            const long long c6_ = clock64(); ph[5] += c6_ - c5_;
-#endif
             if (lane == 0) mbar_arrive(smem_u32(&bars.w_done));
             if (sender) {
                 ok = mbar_wait(smem_u32(&bars.w_done), j & 1, abort_flag);
@@ -647,22 +568,7 @@ quad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CU
                 }
                 __syncwarp();
             }
-#ifdef GC_TC_TRACE
-            ph[6] += clock64() - c6_;
-            if (sev && qev_on && j < 6) {       // first tiles one by one: clocks at the phase ends
-                unsigned int* e = &g_qevlog[2 + pr][64 + 16 * j];
-                e[0] = (unsigned)c0_; e[1] = (unsigned)c1_; e[2] = (unsigned)c2_;
-                e[3] = (unsigned)c3_; e[4] = (unsigned)c5_; e[5] = (unsigned)c6_;
-                e[6] = (unsigned)clock64();
-            }
-#endif
         }
-#ifdef GC_TC_TRACE
-        if (sev && qev_on) {
-            for (int k = 0; k < 7; ++k) g_qevlog[2 + pr][2 * k + 1] = (unsigned)(ph[k] / max(nd, 1));
-            g_qevlog[2 + pr][2 * 4095] = 7;
-        }
-#endif
         if (MODE == QMODE_FA && ok && x < p.nx) {
             // one (scale, sum) slot per row, part of the streamed range, duty pair and column half
             const int64_t slot = (int64_t)((2 * g + pr) * 2 + half) * p.nq + x;
@@ -740,13 +646,6 @@ cudaError_t launch_quad(const CUtensorMap& mx, const CUtensorMap& my, const CUte
 
 }  // namespace
 
-#ifdef GC_TC_TRACE
-extern "C" int gc_debug_qevlog(unsigned int* out, int mode) {
-    if (out && cudaMemcpyFromSymbol(out, g_qevlog, sizeof(g_qevlog)) != cudaSuccess) return 1;
-    if (cudaMemcpyToSymbol(g_qev_mode, &mode, sizeof(int)) != cudaSuccess) return 1;
-    return 0;
-}
-#endif
 
 // Two column halves of an even number of chunks each, at most 384 columns per half, more than
 // one x tile.

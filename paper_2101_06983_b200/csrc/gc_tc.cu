@@ -44,39 +44,6 @@ namespace {
 // FQ: forward fused into dQ; FS: forward that also stores the bf16 weights
 enum { MODE_FWD = 0, MODE_DQ = 1, MODE_DP = 2, MODE_FQ = 3, MODE_FS = 4, MODE_DA = 5 };
 
-// Optional diagnostics (-DGC_TC_TRACE): cycles each role spends waiting, summed over CTAs.
-#ifdef GC_TC_TRACE
-enum { TR_MMA_TOTAL, TR_MMA_WAIT_Y, TR_MMA_WAIT_W, TR_SM_TOTAL, TR_SM_WAIT_S, TR_SM_EPI,
-       TR_PROD_TOTAL, TR_PROD_WAIT, TR_CTAS, TR_MMA_ISSUE, TR_MMA_COMMIT, TR_ACC_ISSUE, TR_ACC_COMMIT, TR_SFULL_COMMIT,
-       TR_CTA_LIFE, TR_SETUP, TR_T0_MIN, TR_T0_MAX, TR_T1_MIN, TR_T1_MAX, TR_COUNT };
-__device__ unsigned long long g_trace[6][TR_COUNT];
-#define TR_DECL(v) long long v = 0
-#define TR_BEGIN(v) long long v##_t0 = clock64()
-#define TR_END(v) v += clock64() - v##_t0
-#define TR_ADD(mode, slot, v) atomicAdd(&g_trace[mode][slot], (unsigned long long)(v))
-// Event timeline of CTA 0 in the mode g_ev_mode selects: per role, (tag, low clock bits) pairs.
-__device__ unsigned int g_evlog[3][16384];
-__device__ int g_ev_mode = -1;
-#define EV_DECL(cnt) int cnt = 0
-#define EV(role, cnt, kind, idx)                                                       \
-    do {                                                                               \
-        if (ev_on && (cnt) < 8190) {                                                   \
-            g_evlog[role][2 * (cnt)] = ((unsigned)(kind) << 16) | ((unsigned)(idx) & 0xffffu); \
-            g_evlog[role][2 * (cnt) + 1] = (unsigned)clock64();                        \
-            ++(cnt);                                                                   \
-        }                                                                              \
-    } while (0)
-#define EV_END(role, cnt) do { if (ev_on) g_evlog[role][2 * 8191] = (unsigned)(cnt); } while (0)
-#else
-#define EV_DECL(cnt)
-#define EV(role, cnt, kind, idx)
-#define EV_END(role, cnt)
-#define TR_DECL(v)
-#define TR_BEGIN(v)
-#define TR_END(v)
-#define TR_ADD(mode, slot, v)
-#endif
-
 struct TcParams {
     int64_t nx, ny;
     int64_t nq;               // number of queries B (pitch of the forward partial arrays)
@@ -172,15 +139,8 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     constexpr int BSH = (NBUF == 2) ? 1 : 0;            // log2(NBUF)
     constexpr int WBUF = WS ? 2 : NBUF;                 // W buffers (w_full barriers in use)
     constexpr int WSH = (WBUF == 2) ? 1 : 0;
-#ifdef GC_TC_TRACE
-    const unsigned long long cta_t0 = global_ns();
-    const long long cta_c0 = clock64();
-#endif
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);   // warp-uniform
     const int lane = threadIdx.x & 31;
-#ifdef GC_TC_TRACE
-    const bool ev_on = blockIdx.x == 0 && lane == 0 && g_ev_mode == MODE;
-#endif
 
     // work item: (x tile, column part, part of the streamed range)
     const uint32_t rank = PAIR ? cluster_ctarank() : 0u;
@@ -241,9 +201,6 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
     if (PAIR) cluster_sync_all();     // both CTAs' barriers exist before anything signals them
     tc_fence_after();
     const uint32_t tmem = tmem_base_s;
-#ifdef GC_TC_TRACE
-    if (threadIdx.x == 0) TR_ADD(MODE, TR_SETUP, clock64() - cta_c0);
-#endif
     // shared::cluster address, in the leader, of the barrier at the same offset as `local`
     auto in_leader = [&](uint32_t local) -> uint32_t { return PAIR ? mapa_u32(local, 0) : local; };
 
@@ -265,9 +222,6 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             int next = 0;
             uint32_t next_phase = 0;
             bool ok = true;
-            EV_DECL(ev_p);
-            TR_DECL(tr_wait);
-            TR_BEGIN(tr_total);
             // Claims the next ring stage if it belongs to this warp: waits until the MMAs that
             // read its previous contents have completed.  Returns the stage or -1.
             auto acquire = [&]() -> int {
@@ -275,14 +229,11 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 const uint32_t phase = next_phase;
                 if (++next == p.nstage) { next = 0; next_phase ^= 1u; }
                 if (!ok || (stage & (NPROD - 1)) != warp) return -1;
-                TR_BEGIN(tr_wait);
                 const bool got = mbar_wait(smem_u32(&bars.y_empty[stage]), phase ^ 1u, abort_flag);
-                TR_END(tr_wait);
                 if (!got) {
                     ok = false;
                     return -1;
                 }
-                if (warp == 0) EV(0, ev_p, 20, stage);
                 return stage;
             };
             // Ring items.  kind 0: Y for the S MMAs (ipc chunks; a paired CTA loads the 64 rows of
@@ -327,14 +278,6 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         load_item(2, c_begin + c, (lo + t - LAG) * SN);
                 }
             }
-            if (warp == 0) EV_END(0, ev_p);
-#ifdef GC_TC_TRACE
-            if (warp == 0 && lane == 0) {
-                TR_ADD(MODE, TR_PROD_TOTAL, clock64() - tr_total_t0);
-                TR_ADD(MODE, TR_PROD_WAIT, tr_wait);
-                TR_ADD(MODE, TR_CTAS, 1);
-            }
-#endif
         }
     } else if (warp == MMA_WARP) {
         // ------------------------------ MMA issuer ----------------------------------------------
@@ -357,42 +300,27 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             const uint32_t idesc_acc = (p.ipc == 2) ? idesc_acc128 : idesc_acc64;   // paired: ipc == 2
             int next = 0;
             uint32_t next_phase = 0;
-            TR_DECL(tr_wy);
-            TR_DECL(tr_ww);
-            TR_DECL(tr_is);
-            TR_DECL(tr_cm);
-            TR_DECL(tr_ai);
-            TR_DECL(tr_ac);
-            TR_DECL(tr_sf);
-            EV_DECL(ev_m);
-            TR_BEGIN(tr_total);
             bool ok = mbar_wait(smem_u32(&bars.x_full), 0, abort_flag);
-            EV(1, ev_m, 0, 0);
             tc_fence_after();
             // Waits for the next ring stage to be filled; returns its index or -1.
             auto next_stage = [&]() -> int {
                 const int stage = next;
                 const uint32_t phase = next_phase;
                 if (++next == p.nstage) { next = 0; next_phase ^= 1u; }
-                TR_BEGIN(tr_wy);
                 const bool got = mbar_wait(smem_u32(&bars.y_full[stage]), phase, abort_flag);
-                TR_END(tr_wy);
                 if (!got) {
                     ok = false;
                     return -1;
                 }
-                EV(1, ev_m, 1, stage);
                 return stage;   // filled by TMA (async proxy), read by the MMA: the mbarrier orders it
             };
             for (int t = 0; t < T + LAG && ok; ++t) {
                 if (t < T) {
                     const int b = t & (NBUF - 1);
                     if (WS && t >= 1) {     // the softmax warps have read S(t-1) out of the tile
-                        EV(1, ev_m, 2, t);
                         ok = mbar_wait(smem_u32(&bars.s_free), (t - 1) & 1, abort_flag);
                         if (!ok) break;
                         tc_fence_after();
-                        EV(1, ev_m, 3, t);
                     }
                     if (NOACC && t >= NBUF) {
                         ok = mbar_wait(smem_u32(&bars.w_full[b]), ((t - NBUF) >> BSH) & 1,
@@ -416,7 +344,6 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                                 if (!ok) break;
                                 xa = ring_lo + xs * stage_lo;
                             }
-                            TR_BEGIN(tr_is);
                             if (elect_one()) {
                                 if (c == 0) mma_ss<false, false>(d_tmem, xa, yb, idesc_s);
                                 else        mma_ss<true, false>(d_tmem, xa, yb, idesc_s);
@@ -432,7 +359,6 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                                 if (xs >= 0) tc_commit(smem_u32(&bars.y_empty[xs]));
                                 tc_commit(smem_u32(&bars.y_empty[ys]));
                             }
-                            TR_END(tr_is);
                         } else {
                             // paired: the Y item holds this CTA's 64 rows of two chunks (8 KB
                             // each), every streamed X chunk is an item of its own
@@ -445,7 +371,6 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                                     xa = ring_lo + xs * stage_lo;
                                 }
                                 const uint32_t yj = yb + j * YCH_LO;
-                                TR_BEGIN(tr_is);
                                 if (elect_one()) {
                                     if (c + j == 0) mma_ss<false, true>(d_tmem, xa, yj, idesc_s);
                                     else            mma_ss<true, true>(d_tmem, xa, yj, idesc_s);
@@ -455,24 +380,17 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                                     if (xs >= 0) tc_commit_pair(smem_u32(&bars.y_empty[xs]));
                                     if (j == 1) tc_commit_pair(smem_u32(&bars.y_empty[ys]));
                                 }
-                                TR_END(tr_is);
                             }
                         }
                     }
                     if (!ok) break;
-                    TR_BEGIN(tr_sf);
                     if (elect_one()) commit(smem_u32(&bars.s_full[b]));
-                    TR_END(tr_sf);
-                    EV(1, ev_m, 4, t);
                 }
                 if (!NOACC && t >= LAG) {
                     const int u = t - LAG, b = u & (WBUF - 1);
-                    TR_BEGIN(tr_ww);
                     ok = mbar_wait(smem_u32(&bars.w_full[b]), (u >> WSH) & 1, abort_flag);
-                    TR_END(tr_ww);
                     if (!ok) break;
                     tc_fence_after();
-                    EV(1, ev_m, 5, u);
                     const uint32_t w_tmem = tmem + S_COL0 + (WS ? 0 : b * SN);
                     const uint32_t w_lo = desc_lo(w_smem + b * 32768u, 0);   // WS: K-major A operand
                     // one ring item per iteration: ipc chunks = 64 * ipc accumulator columns
@@ -481,7 +399,6 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         if (!ok) break;
                         const uint32_t yb = ring_lo + ys * stage_lo;
                         const uint32_t d_tmem = tmem + c * 64;
-                        TR_BEGIN(tr_ai);
                         if (elect_one()) {
                             // k-steps of the first column half read W at columns 8 k, those of
                             // the second half at SN/2 + 8 (k - KH)
@@ -505,26 +422,11 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                             }
                             commit(smem_u32(&bars.y_empty[ys]));
                         }
-                        TR_END(tr_ai);
                     }
                     if (WS && ok && elect_one()) commit(smem_u32(&bars.w_empty[b]));
-                    EV(1, ev_m, 6, u);
                 }
             }
             if (ok && !NOACC && elect_one()) commit(smem_u32(&bars.acc_full));
-            EV_END(1, ev_m);
-#ifdef GC_TC_TRACE
-            if (lane == 0) {
-            TR_ADD(MODE, TR_MMA_TOTAL, clock64() - tr_total_t0);
-            TR_ADD(MODE, TR_MMA_WAIT_Y, tr_wy);
-            TR_ADD(MODE, TR_MMA_WAIT_W, tr_ww);
-            TR_ADD(MODE, TR_MMA_ISSUE, tr_is);
-            TR_ADD(MODE, TR_MMA_COMMIT, tr_cm);
-            TR_ADD(MODE, TR_ACC_ISSUE, tr_ai);
-            TR_ADD(MODE, TR_ACC_COMMIT, tr_ac);
-            TR_ADD(MODE, TR_SFULL_COMMIT, tr_sf);
-            }
-#endif
         }
     } else {
         // ------------------------------ softmax / epilogue warps --------------------------------
@@ -559,19 +461,13 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                                "r"(pk[4 * i + 3]) : "memory");
             }
         };
-        TR_DECL(tr_ws);
-        TR_DECL(tr_epi);
-        EV_DECL(ev_s);
-        TR_BEGIN(tr_total);
 
         if (MODE == MODE_FWD) {
             float m = -INFINITY, l = 0.f;
             const int32_t pos_x = (x < p.nx) ? p.pos_idx[x] : -1;
             for (int t = 0; t < T; ++t) {
                 const int b = t & (NBUF - 1);
-                TR_BEGIN(tr_ws);
                 ok = mbar_wait(smem_u32(&bars.s_full[b]), (t >> BSH) & 1, abort_flag);
-                TR_END(tr_ws);
                 if (!ok) break;
                 tc_fence_after();
                 const int64_t y0 = (lo + t) * SN;
@@ -641,9 +537,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             for (int t = 0; t < T; ++t) {
                 const int b = t & (NBUF - 1);
                 const int64_t y0 = (lo + t) * SN;
-                TR_BEGIN(tr_ws);
                 ok = mbar_wait(smem_u32(&bars.s_full[b]), (t >> BSH) & 1, abort_flag);
-                TR_END(tr_ws);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t sbuf = tmem + lane_addr + S_COL0 + b * SN;
@@ -740,9 +634,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             const int32_t pos_x = (x < p.nx) ? p.pos_idx[x] : -1;
             for (int t = 0; t < T; ++t) {
                 const int64_t y0 = (lo + t) * SN;
-                TR_BEGIN(tr_ws);
                 ok = mbar_wait(smem_u32(&bars.s_full[0]), t & 1, abort_flag);
-                TR_END(tr_ws);
                 if (!ok) break;
                 tc_fence_after();
                 const uint32_t sbuf = tmem + lane_addr + S_COL0;
@@ -877,7 +769,6 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 p.part_l[slot] = l;
             }
             // unscaled accumulator part -> partial buffer [g][nx][d]
-            TR_BEGIN(tr_epi);
             if (ok) ok = mbar_wait(smem_u32(&bars.acc_full), 0, abort_flag);
             if (ok) {
                 tc_fence_after();
@@ -886,7 +777,6 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 store_acc_blocks(tmem + lane_addr, c_count * 2, half, slot, 1.f, lane, &mapO,
                                  c_begin * 64, (int)x0 + q * 32, g);
             }
-            TR_END(tr_epi);
         } else {
             // per-row constants (DQ: the row is a query)
             float lse2_x = 0.f, l_sum = 0.f, wmax = 0.f;
@@ -916,12 +806,9 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                         pos_y[j] = (y < p.ny) ? p.pos_idx[y] : -1;
                     }
                 }
-                TR_BEGIN(tr_ws);
                 ok = mbar_wait(smem_u32(&bars.s_full[b]), (t >> BSH) & 1, abort_flag);
-                TR_END(tr_ws);
                 if (!ok) break;
                 tc_fence_after();
-                if (q == 0 && half == 0) EV(2, ev_s, 10, t);
                 const uint32_t sbuf = tmem + lane_addr + S_COL0 + b * SN;
                 // W of this half goes to the first columns of the half's own S region (already
                 // read by this warp): columns half * SN/2 + 16 j for block j.
@@ -940,12 +827,10 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                     tc_fence_before();
                     __syncwarp();
                     if (lane == 0) arrive_w(smem_u32(&bars.s_free));
-                    if (q == 0 && half == 0) EV(2, ev_s, 11, t);
                     if (t >= 2) {
                         ok = mbar_wait(smem_u32(&bars.w_empty[t & 1]), ((t - 2) >> 1) & 1, abort_flag);
                         if (!ok) break;
                     }
-                    if (q == 0 && half == 0) EV(2, ev_s, 12, t);
                 }
 #pragma unroll(WS ? CB_PER : 1)
                 for (int j = 0; j < CB_PER; ++j) {
@@ -1055,9 +940,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) arrive_w(smem_u32(&bars.w_full[WS ? (t & 1) : b]));
-                if (q == 0 && half == 0) EV(2, ev_s, 13, t);
             }
-            if (q == 0 && half == 0) EV_END(2, ev_s);
             if (MODE == MODE_DA && ok && x < p.nx) {
                 // one (scale, sum) slot per row, part of the streamed range, softmax group and
                 // column half
@@ -1070,7 +953,6 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             // epilogue: accumulator columns of this part -> global memory (32-column blocks are
             // dealt alternately to the two warps of a lane quarter); final values are scaled,
             // partial sums of a split sweep are not
-            TR_BEGIN(tr_epi);
             if (grp != 0) ok = false;      // the first group writes the accumulators
             if (ok) ok = mbar_wait(smem_u32(&bars.acc_full), 0, abort_flag);
             if (ok) {
@@ -1081,15 +963,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                                  final_out ? p.out_scale : 1.f, lane, &mapO, c_begin * 64,
                                  (int)x0 + q * 32, final_out ? 0 : g);
             }
-            TR_END(tr_epi);
         }
-#ifdef GC_TC_TRACE
-        if (q == 0 && half == 0 && lane == 0) {
-            TR_ADD(MODE, TR_SM_TOTAL, clock64() - tr_total_t0);
-            TR_ADD(MODE, TR_SM_WAIT_S, tr_ws);
-            TR_ADD(MODE, TR_SM_EPI, tr_epi);
-        }
-#endif
     }
 
     // ------------------------------ teardown ------------------------------------------------------
@@ -1103,16 +977,6 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
         __syncthreads();
     }
     if (PAIR) cluster_sync_all();   // the peer's MMAs, loads and arrivals no longer touch this CTA
-#ifdef GC_TC_TRACE
-    if (threadIdx.x == 0) {
-        const unsigned long long t1 = global_ns();
-        TR_ADD(MODE, TR_CTA_LIFE, clock64() - cta_c0);
-        atomicMin(&g_trace[MODE][TR_T0_MIN], cta_t0);
-        atomicMax(&g_trace[MODE][TR_T0_MAX], cta_t0);
-        atomicMin(&g_trace[MODE][TR_T1_MIN], t1);
-        atomicMax(&g_trace[MODE][TR_T1_MAX], t1);
-    }
-#endif
     if (warp == MMA_WARP) {
         tc_fence_after();
         if (PAIR)
@@ -1231,22 +1095,6 @@ cudaError_t launch(const CUtensorMap& mx, const CUtensorMap& my, const CUtensorM
 
 }  // namespace
 
-#ifdef GC_TC_TRACE
-extern "C" int gc_debug_evlog(unsigned int* out, int mode) {
-    if (out && cudaMemcpyFromSymbol(out, g_evlog, sizeof(g_evlog)) != cudaSuccess) return 1;
-    if (cudaMemcpyToSymbol(g_ev_mode, &mode, sizeof(int)) != cudaSuccess) return 1;
-    return 0;
-}
-extern "C" int gc_debug_trace(unsigned long long* out, int clear) {
-    if (out && cudaMemcpyFromSymbol(out, g_trace, sizeof(g_trace)) != cudaSuccess) return 1;
-    if (clear) {
-        static unsigned long long zero[6][TR_COUNT] = {};
-        for (int m = 0; m < 6; ++m) zero[m][TR_T0_MIN] = zero[m][TR_T1_MIN] = ~0ull;
-        if (cudaMemcpyToSymbol(g_trace, zero, sizeof(zero)) != cudaSuccess) return 1;
-    }
-    return 0;
-}
-#endif
 
 bool tc_supported(int64_t B, int64_t N, int d, int dtype) {
     (void)B; (void)N;
