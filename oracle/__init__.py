@@ -54,6 +54,10 @@ def _load():
         lib.gco_build_variant.restype = ctypes.c_int
         lib.gco_build_variant.argtypes = [dp, dp, lp, ip, i64, i64, i64, ctypes.c_double,
                                           ctypes.c_int, ctypes.c_int, ctypes.c_int, dp, dp, dp, dp]
+        lib.gco_dist_loss.restype = ctypes.c_int
+        lib.gco_dist_loss.argtypes = [dp, ip, i64, i64, ctypes.c_double, ctypes.c_int, dp, dp]
+        lib.gco_dist_w.restype = ctypes.c_int
+        lib.gco_dist_w.argtypes = [dp, ip, i64, i64, ctypes.c_double, ctypes.c_int, dp]
         lib.gco_cache_apply.restype = ctypes.c_int
         lib.gco_cache_apply.argtypes = [dp, dp, i64, i64, i64, ctypes.c_int, dp]
         _lib = lib
@@ -174,6 +178,34 @@ def build_variant(Q, P, positives, tau=1.0, mask_mode=0, cosine=False, two_direc
     if rc != 0:
         raise ValueError(f"oracle rejected the problem (code {rc})")
     return dict(loss=float(loss.value), dQ=dQ, dP=dP, dtau=float(dtau.value))
+
+
+def dist_loss(D, pos_idx, tau=1.0, mask_mode=0):
+    """Section 5: the loss of Eq. 1 as a function of the matrix of distances D [B x N] (logit of a
+    pair = d_ij / tau).  Returns dict(loss, row_lse)."""
+    D = _f64(D)
+    B, N = D.shape
+    pos = np.ascontiguousarray(pos_idx, dtype=np.int32)
+    loss = ctypes.c_double(0.0)
+    lse = np.empty(B, np.float64)
+    rc = _load().gco_dist_loss(_ptr(D, ctypes.c_double), _ptr(pos, ctypes.c_int32), B, N, float(tau),
+                               int(mask_mode), ctypes.byref(loss), _ptr(lse, ctypes.c_double))
+    if rc != 0:
+        raise ValueError(f"oracle rejected the problem (code {rc})")
+    return dict(loss=float(loss.value), row_lse=lse)
+
+
+def dist_w(D, pos_idx, tau=1.0, mask_mode=0):
+    """Section 5: the Distance Gradient Cache w_ij = dL/dd_ij as a B x N float64 matrix."""
+    D = _f64(D)
+    B, N = D.shape
+    pos = np.ascontiguousarray(pos_idx, dtype=np.int32)
+    W = np.empty((B, N), np.float64)
+    rc = _load().gco_dist_w(_ptr(D, ctypes.c_double), _ptr(pos, ctypes.c_int32), B, N, float(tau),
+                            int(mask_mode), _ptr(W, ctypes.c_double))
+    if rc != 0:
+        raise ValueError(f"oracle rejected the problem (code {rc})")
+    return W
 
 
 def cache_apply(U, X, dW=None):

@@ -15,7 +15,8 @@
  * differences and closed form, row for row; gco_cache_apply (Step 3 for a linear encoder) by the
  * finite-difference gradient with respect to the encoder matrix and a hand-worked example;
  * gco_build_variant (cosine similarity, several positives, two-direction loss, dL/dtau) in
- * tests/test_oracle_variants.py.  No function here is "parity unpinned".
+ * tests/test_oracle_variants.py; gco_dist_loss / gco_dist_w (Distance Gradient Cache, Section 5)
+ * in tests/test_oracle_distance.py.  No function here is "parity unpinned".
  *
  * Notation (paper, Section 3.1-3.2): Q row i is f(s_i), P row j is g(t_j), pos_idx[i] is r_i,
  * tau the temperature, S_ij = <f(s_i), g(t_j)> / tau.
@@ -414,4 +415,51 @@ int gco_build_variant(const double* Q, const double* P, const int64_t* pos_ptr,
         }
     free(Qn); free(Pn); free(qnorm); free(pnorm); free(S); free(G); free(gQ); free(gP);
     return 0;
+}
+
+/*
+ * Distance Gradient Cache (Section 5, Eq. 10-13).  The similarity is a general distance
+ * d_ij = Phi(f(s_i), g(t_j)); the loss is Eq. 1 with d_ij / tau as the logit of pair (i, j).
+ *
+ *   gco_dist_loss   the loss as a function of the B x N matrix of distances D, and lse_i.
+ *   gco_dist_w      the Distance Gradient Cache w_ij = dL/dd_ij = (p_ij - [j == r_i]) / (B tau),
+ *                   p the row softmax of D / tau over the allowed pairs (0 where masked).
+ * With these, Eq. 11 is dL/dOmega = sum_ij w_ij dPhi_ij/dOmega and Eq. 12-13 are u_i = sum_j w_ij
+ * dd_ij/df(s_i), v_j = sum_i w_ij dd_ij/dg(t_j); for the dot product d_ij = <f_i, g_j> they reduce
+ * to Eq. 5-7.  Pinned in tests/test_oracle_distance.py.
+ */
+int gco_dist_loss(const double* D, const int32_t* pos_idx, int64_t B, int64_t N, double tau,
+                  int mask_mode, double* loss, double* row_lse) {
+    int rc = check_args(pos_idx, B, N, 1, tau, mask_mode);
+    if (rc) return rc;
+    double total = 0.0;
+    for (int64_t i = 0; i < B; ++i) {
+        double m = -INFINITY;
+        for (int64_t j = 0; j < N; ++j)
+            if (allowed(mask_mode, i, j) && D[i * N + j] / tau > m) m = D[i * N + j] / tau;
+        double sum = 0.0;
+        for (int64_t j = 0; j < N; ++j)
+            if (allowed(mask_mode, i, j)) sum += exp(D[i * N + j] / tau - m);
+        const double lse = m + log(sum);
+        if (row_lse) row_lse[i] = lse;
+        total += lse - D[i * N + pos_idx[i]] / tau;
+    }
+    if (loss) *loss = total / (double)B;
+    return 0;
+}
+
+int gco_dist_w(const double* D, const int32_t* pos_idx, int64_t B, int64_t N, double tau,
+               int mask_mode, double* W) {
+    int rc = check_args(pos_idx, B, N, 1, tau, mask_mode);
+    if (rc) return rc;
+    double* lse = (double*)malloc(sizeof(double) * (size_t)B);
+    if (!lse) return -1;
+    rc = gco_dist_loss(D, pos_idx, B, N, tau, mask_mode, NULL, lse);
+    for (int64_t i = 0; i < B && !rc; ++i)
+        for (int64_t j = 0; j < N; ++j) {
+            double p = allowed(mask_mode, i, j) ? exp(D[i * N + j] / tau - lse[i]) : 0.0;
+            W[i * N + j] = (p - ((j == pos_idx[i]) ? 1.0 : 0.0)) / ((double)B * tau);
+        }
+    free(lse);
+    return rc;
 }

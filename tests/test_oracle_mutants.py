@@ -11,6 +11,7 @@ import pytest
 
 import test_oracle_pins as pins
 import test_oracle_variants as vpins
+import test_oracle_distance as dpins
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 SRC = open(os.path.join(ROOT, "oracle", "gc_oracle.c")).read()
@@ -64,6 +65,14 @@ MUTANTS = {
         "G[((i + 1) % B) * N + j] -= 1.0 / (double)B;\n        }\n        L = 0.5"),
     "variant: column logsumexp ignores the mask": (
         "if (allowed(mask_mode, k, j)) sum += exp(S[k * N + j] - m);", "sum += exp(S[k * N + j] - m);"),
+    "distance cache: 1/tau missing in w": (
+        "W[i * N + j] = (p - ((j == pos_idx[i]) ? 1.0 : 0.0)) / ((double)B * tau);",
+        "W[i * N + j] = (p - ((j == pos_idx[i]) ? 1.0 : 0.0)) / (double)B;"),
+    "distance cache: mask leaks into w": (
+        "double p = allowed(mask_mode, i, j) ? exp(D[i * N + j] / tau - lse[i]) : 0.0;",
+        "double p = exp(D[i * N + j] / tau - lse[i]);"),
+    "distance cache: positive distance not scaled by tau": (
+        "total += lse - D[i * N + pos_idx[i]] / tau;", "total += lse - D[i * N + pos_idx[i]];"),
     "cache_apply reads U transposed": ("s += U[i * d + a] * X[i * d_in + b];",
                                        "s += U[(a % rows) * d + (i % d)] * X[i * d_in + b];"),
     "cache_apply overwrites instead of accumulating": ("if (accumulate) dW[a * d_in + b] += s;",
@@ -174,6 +183,35 @@ def _wrap(libpath):
             raise ValueError(f"rejected ({rc})")
         return dict(loss=float(loss.value), dQ=dQ, dP=dP, dtau=float(dtau.value))
 
+    lib.gco_dist_loss.restype = ctypes.c_int
+    lib.gco_dist_loss.argtypes = [dp, ip, i64, i64, ctypes.c_double, ctypes.c_int, dp, dp]
+    lib.gco_dist_w.restype = ctypes.c_int
+    lib.gco_dist_w.argtypes = [dp, ip, i64, i64, ctypes.c_double, ctypes.c_int, dp]
+
+    def dist_loss(D, pos_idx, tau=1.0, mask_mode=0):
+        D = real._f64(D)
+        B, N = D.shape
+        pos = np.ascontiguousarray(pos_idx, dtype=np.int32)
+        loss = ctypes.c_double(0.0)
+        lse = np.empty(B)
+        rc = lib.gco_dist_loss(real._ptr(D, ctypes.c_double), real._ptr(pos, ctypes.c_int32), B, N,
+                               float(tau), int(mask_mode), ctypes.byref(loss),
+                               real._ptr(lse, ctypes.c_double))
+        if rc != 0:
+            raise ValueError(f"rejected ({rc})")
+        return dict(loss=float(loss.value), row_lse=lse)
+
+    def dist_w(D, pos_idx, tau=1.0, mask_mode=0):
+        D = real._f64(D)
+        B, N = D.shape
+        pos = np.ascontiguousarray(pos_idx, dtype=np.int32)
+        W = np.empty((B, N))
+        rc = lib.gco_dist_w(real._ptr(D, ctypes.c_double), real._ptr(pos, ctypes.c_int32), B, N,
+                            float(tau), int(mask_mode), real._ptr(W, ctypes.c_double))
+        if rc != 0:
+            raise ValueError(f"rejected ({rc})")
+        return W
+
     lib.gco_cache_apply.restype = ctypes.c_int
     lib.gco_cache_apply.argtypes = [dp, dp, ctypes.c_int64, ctypes.c_int64, ctypes.c_int64,
                                     ctypes.c_int, dp]
@@ -193,7 +231,7 @@ def _wrap(libpath):
 
     return types.SimpleNamespace(
         build_cache=build_cache, cache_apply=cache_apply, query_rows=query_rows,
-        passage_rows=passage_rows, build_variant=build_variant,
+        passage_rows=passage_rows, build_variant=build_variant, dist_loss=dist_loss, dist_w=dist_w,
         loss_only=lambda Q, P, pos, tau=1.0, mask=0: build_cache(Q, P, pos, tau, mask)["loss"])
 
 
@@ -216,6 +254,8 @@ def _pins(o):
     yield lambda: vpins.test_cosine_is_scale_invariant_and_gradients_are_tangent(o)
     yield lambda: vpins.test_two_direction_loss_is_symmetric_under_role_swap(o)
     yield lambda: vpins.test_two_positives_hand_worked(o)
+    yield lambda: dpins.test_w_is_the_derivative_of_the_loss_in_every_distance(o, 0.3, 1)
+    yield lambda: dpins.test_dot_product_links_the_two_caches(o, 1)
     yield lambda: pins.test_cache_apply_hand_worked_example(o)
     yield lambda: pins.test_cache_apply_chunks_reproduce_full_batch_parameter_gradient(o)
 
