@@ -226,6 +226,43 @@ int gc_dtau(const void* Q, int64_t ldq, const float* dQ, int64_t lddq, int64_t B
             int dtype, float* dtau, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Distance Gradient Cache (Section 5, Eq. 10-13) in tiled form.  The similarity of pair (i, j) is
+ * a distance d_ij = Phi(f(s_i), g(t_j)) computed by the caller's network; the loss is Eq. 1 with
+ * d_ij / tau as the logit.  The paper stores all B x N values w_ij = dL/dd_ij.  Here the caller
+ * walks its sub-batch pairs twice and hands over one block of distances at a time, so nothing of
+ * size B x N is kept:
+ *   gc_dist_begin       resets the per-row state run_m, run_l, pos_d (float [B] each, caller-owned)
+ *   gc_dist_accumulate  folds D_block [bq x bn] (float, leading dimension ldd; rows i0.., columns
+ *                       j0.. of the full matrix) into the running maximum and sum of its rows and
+ *                       records d_{i,r_i}/tau where column r_i lies in the block.  Blocks of the
+ *                       same rows must be accumulated one after the other (stream order does).
+ *   gc_dist_finish      row_lse[i] = log sum_j exp(d_ij / tau) over the allowed pairs, loss = Eq. 1;
+ *                       pos_idx errors go to *dev_status as in gc_loss_fwd
+ *   gc_dist_w_block     W_block[r][c] = w_ij = (exp(d_ij / tau - lse_i) - [j == r_i]) / (B tau), 0
+ *                       at the masked pair: the block of the Distance Gradient Cache that Eq. 11
+ *                       (dL/dOmega = sum w_ij dPhi_ij/dOmega) and Eq. 12-13 (u_i = sum_j w_ij
+ *                       dd_ij/df(s_i), v_j likewise) consume for this sub-batch pair
+ *   gc_dist_dot_block   D_block[r][c] = <Q[i0 + r], P[j0 + c]> for the dot-product distance (then
+ *                       Eq. 12-13 reduce to Eq. 5-7: u = W P, v = W^T Q); Q, P as in gc_loss_fwd,
+ *                       d a multiple of 8 (else GC_ERR_LIMIT)
+ * A block outside the B x N matrix is GC_ERR_SHAPE.  Device pointers, asynchronous on cuda_stream,
+ * deterministic (fixed reduction order); fp32 arithmetic.
+ */
+int gc_dist_begin(float* run_m, float* run_l, float* pos_d, int64_t B, void* cuda_stream);
+int gc_dist_accumulate(const float* D_block, int64_t ldd, int64_t i0, int64_t bq, int64_t j0,
+                       int64_t bn, const int32_t* pos_idx, int64_t B, int64_t N, float tau,
+                       int mask_mode, float* run_m, float* run_l, float* pos_d, void* cuda_stream);
+int gc_dist_finish(const float* run_m, const float* run_l, const float* pos_d,
+                   const int32_t* pos_idx, int64_t B, int64_t N, int mask_mode, float* row_lse,
+                   float* loss, int* dev_status, void* cuda_stream);
+int gc_dist_w_block(const float* D_block, int64_t ldd, int64_t i0, int64_t bq, int64_t j0,
+                    int64_t bn, const int32_t* pos_idx, const float* row_lse, int64_t B, int64_t N,
+                    float tau, int mask_mode, float* W_block, int64_t ldw, void* cuda_stream);
+int gc_dist_dot_block(const void* Q, int64_t ldq, const void* P, int64_t ldp, int64_t B, int64_t N,
+                      int d, int dtype, int64_t i0, int64_t bq, int64_t j0, int64_t bn,
+                      float* D_block, int64_t ldd, void* cuda_stream);
+
+/*
  * Forward with library-owned scratch (no counterpart in the paper: it exists for the sake of
  * callers, not of the method).  Same inputs, outputs and results as gc_loss_fwd, but the caller
  * passes no workspace.  It is meant for callers that cannot obtain device memory at the point of

@@ -24,7 +24,8 @@ EXPORTS = ("gc_workspace_bytes", "gc_plan_name", "gc_kernel_launches", "gc_loss_
            "gc_profile_read", "gc_profile_read_call", "gc_static_scratch_need", "gc_loss_fwd_static",
            "gc_cache_apply_workspace_bytes", "gc_cache_apply", "gc_shard_workspace_bytes",
            "gc_shard_fwd_dq", "gc_shard_dp", "gc_selftest_wait_limit", "gc_row_normalize",
-           "gc_cosine_bwd", "gc_dtau_workspace_bytes", "gc_dtau")
+           "gc_cosine_bwd", "gc_dtau_workspace_bytes", "gc_dtau", "gc_dist_begin",
+           "gc_dist_accumulate", "gc_dist_finish", "gc_dist_w_block", "gc_dist_dot_block")
 GC_STATIC_SCRATCH_BYTES = 2 << 20
 
 
@@ -84,6 +85,16 @@ def _load() -> ctypes.CDLL:
     lib.gc_dtau_workspace_bytes.argtypes = [i64]
     lib.gc_dtau.restype = i32
     lib.gc_dtau.argtypes = [vp, i64, vp, i64, i64, i32, f32, i32, vp, vp, ctypes.c_size_t, vp]
+    lib.gc_dist_begin.restype = i32
+    lib.gc_dist_begin.argtypes = [vp, vp, vp, i64, vp]
+    lib.gc_dist_accumulate.restype = i32
+    lib.gc_dist_accumulate.argtypes = [vp, i64, i64, i64, i64, i64, vp, i64, i64, f32, i32, vp, vp, vp, vp]
+    lib.gc_dist_finish.restype = i32
+    lib.gc_dist_finish.argtypes = [vp, vp, vp, vp, i64, i64, i32, vp, vp, vp, vp]
+    lib.gc_dist_w_block.restype = i32
+    lib.gc_dist_w_block.argtypes = [vp, i64, i64, i64, i64, i64, vp, vp, i64, i64, f32, i32, vp, i64, vp]
+    lib.gc_dist_dot_block.restype = i32
+    lib.gc_dist_dot_block.argtypes = [vp, i64, vp, i64, i64, i64, i32, i32, i64, i64, i64, i64, vp, i64, vp]
     lib.gc_selftest_wait_limit.restype = i32
     lib.gc_selftest_wait_limit.argtypes = [ctypes.c_uint64, vp, vp, vp]
     lib.gc_profile_enable.restype = i32
@@ -308,6 +319,57 @@ def gc_dtau(Q, dQ, tau, dtau, ws=None) -> None:
                       _dtype_code(Q), _ptr(dtau), _ptr(ws), ws.numel(), _stream())
     if rc != 0:
         raise GradCacheError(rc, "gc_dtau")
+
+
+class DistanceCache:
+    """Section 5 in tiled form: per-row state of the first pass over the distance blocks, then
+    row_lse / loss, then blocks of the Distance Gradient Cache w = dL/dd.  Marshalling only."""
+
+    def __init__(self, pos_idx, B, N, tau, mask_mode=GC_MASK_NONE):
+        dev = pos_idx.device
+        self.pos, self.B, self.N, self.tau, self.mask = pos_idx, B, N, float(tau), int(mask_mode)
+        self.run_m = torch.empty(B, device=dev)
+        self.run_l = torch.empty(B, device=dev)
+        self.pos_d = torch.empty(B, device=dev)
+        self.row_lse = torch.empty(B, device=dev)
+        self.loss = torch.zeros(1, device=dev)
+        self.dev_status = torch.zeros(1, dtype=torch.int32, device=dev)
+        rc = _lib.gc_dist_begin(_ptr(self.run_m), _ptr(self.run_l), _ptr(self.pos_d), B, _stream())
+        if rc != 0:
+            raise GradCacheError(rc, "gc_dist_begin")
+
+    def accumulate(self, D_block, i0, j0):
+        bq, bn = D_block.shape
+        rc = _lib.gc_dist_accumulate(_ptr(D_block), D_block.stride(0), i0, bq, j0, bn, _ptr(self.pos),
+                                     self.B, self.N, self.tau, self.mask, _ptr(self.run_m),
+                                     _ptr(self.run_l), _ptr(self.pos_d), _stream())
+        if rc != 0:
+            raise GradCacheError(rc, "gc_dist_accumulate")
+
+    def finish(self):
+        rc = _lib.gc_dist_finish(_ptr(self.run_m), _ptr(self.run_l), _ptr(self.pos_d), _ptr(self.pos),
+                                 self.B, self.N, self.mask, _ptr(self.row_lse), _ptr(self.loss),
+                                 _ptr(self.dev_status), _stream())
+        if rc != 0:
+            raise GradCacheError(rc, "gc_dist_finish")
+
+    def w_block(self, D_block, i0, j0, W_block):
+        bq, bn = D_block.shape
+        rc = _lib.gc_dist_w_block(_ptr(D_block), D_block.stride(0), i0, bq, j0, bn, _ptr(self.pos),
+                                  _ptr(self.row_lse), self.B, self.N, self.tau, self.mask,
+                                  _ptr(W_block), W_block.stride(0), _stream())
+        if rc != 0:
+            raise GradCacheError(rc, "gc_dist_w_block")
+
+
+def gc_dist_dot_block(Q, P, i0, bq, j0, bn, D_block) -> None:
+    """D_block[r][c] = <Q[i0 + r], P[j0 + c]>: a block of dot-product distances (float32)."""
+    B, d = Q.shape
+    N = P.shape[0]
+    rc = _lib.gc_dist_dot_block(_ptr(Q), Q.stride(0), _ptr(P), P.stride(0), B, N, d, _dtype_code(Q),
+                                i0, bq, j0, bn, _ptr(D_block), D_block.stride(0), _stream())
+    if rc != 0:
+        raise GradCacheError(rc, "gc_dist_dot_block")
 
 
 def gc_selftest_wait_limit(limit_ns: int, dev_status, waited_ns=None) -> None:
