@@ -152,8 +152,10 @@ int gc_build_cache_stored(const void* Q, int64_t ldq, const void* P, int64_t ldp
  * Each u is used as the sum of two bf16 terms (its rounding and the rounding of the remainder,
  * together exact to 2^-17 |u|), products are exact and accumulation is fp32 on the tensor cores.
  * Limits: d a multiple of 8, d_in a multiple of 64 and at most 4096 (else GC_ERR_LIMIT); rows of
- * U, X and dW start on 16-byte boundaries.  Workspace: gc_cache_apply_workspace_bytes (0 for
- * sizes outside the limits), 256-byte aligned, caller-owned.  Asynchronous on cuda_stream;
+ * U, X and dW start on 16-byte boundaries.  One kernel launch; the partial sums over parts of the
+ * sub-batch are exchanged through shared memory, so the workspace is nominal:
+ * gc_cache_apply_workspace_bytes returns 256 (0 for sizes outside the limits) and ws must be a
+ * 256-byte aligned, caller-owned buffer of at least that size.  Asynchronous on cuda_stream;
  * deterministic; GC_DEV_WAIT_LIMIT in *dev_status (may be NULL) as for the other calls.
  */
 size_t gc_cache_apply_workspace_bytes(int64_t rows, int d, int d_in);

@@ -124,7 +124,7 @@ def test_refusals(binding):
                                torch.zeros(64, 96, device="cuda"), False)
     assert e.value.status == 9                                # GC_ERR_LIMIT
     with pytest.raises(binding.GradCacheError) as e:
-        binding.gc_cache_apply(U, X, W, False, ws=torch.empty(256, dtype=torch.uint8, device="cuda"))
+        binding.gc_cache_apply(U, X, W, False, ws=torch.empty(64, dtype=torch.uint8, device="cuda"))
     assert e.value.status == 6                                # GC_ERR_WORKSPACE
     assert binding.gc_cache_apply_workspace_bytes(16, 64, 96) == 0
     assert binding.gc_cache_apply_workspace_bytes(16, 64, 64) > 0
