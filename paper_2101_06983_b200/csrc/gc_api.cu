@@ -517,6 +517,19 @@ int run_build_stored(const Problem& p, const Plan& pl, char* w, float* loss, flo
 
 using namespace gc;
 
+namespace {
+
+// One-tile batches: the whole call is one launch (gc_small.cu); timed as the fused sweep.
+int run_small(int op, const Problem& p, const float* row_lse_in, float* loss, float* row_lse,
+              float* pos_logit, float* dQ, int64_t lddq, float* dP, int64_t lddp, int* dev_status,
+              cudaStream_t st) {
+    KernelTimer t(1, st);
+    return launch_small(op, p, row_lse_in, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status,
+                        st) == cudaSuccess ? GC_OK : GC_ERR_CUDA;
+}
+
+}  // namespace
+
 // Scratch for gc_loss_fwd_static.  In host code this name is only a handle for the symbol: the
 // address a kernel can use comes from cudaGetSymbolAddress, looked up once per device.
 static __device__ __align__(256) unsigned char g_static_scratch[GC_STATIC_SCRATCH_BYTES];
@@ -569,11 +582,13 @@ size_t gc_workspace_bytes(int op, int64_t B, int64_t N, int d, int dtype) {
 const char* gc_plan_name(int op, int64_t B, int64_t N, int d, int dtype) {
     if (op < GC_OP_FWD || op > GC_OP_BUILD_STORED || B <= 0 || N <= 0 || d <= 0) return "invalid";
     if (op == GC_OP_BUILD_STORED && !make_plan(B, N, d, dtype, true).mat) return "invalid";
+    if (op != GC_OP_BUILD_STORED && small_applicable(B, N, d, dtype)) return "tcgen05-one-tile";
     return tc_supported(B, N, d, dtype) ? "tcgen05" : "simt";
 }
 
 int gc_kernel_launches(int op, int64_t B, int64_t N, int d, int dtype) {
     if (B <= 0 || N <= 0 || d <= 0) return 0;
+    if (op >= GC_OP_FWD && op <= GC_OP_BUILD && small_applicable(B, N, d, dtype)) return 1;
     Plan pl = make_plan(B, N, d, dtype);
     if (op == GC_OP_FWD) return pl.launches_fwd;
     if (op == GC_OP_BWD) return pl.launches_bwd + 1;   // + pos_idx validation
@@ -594,6 +609,9 @@ int gc_loss_fwd(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
     if ((rc = check_device())) return rc;
     profile_begin_call();
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
+    if (small_applicable(B, N, d, dtype))
+        return run_small(GC_OP_FWD, p, nullptr, loss, row_lse, pos_logit, nullptr, 0, nullptr, 0,
+                         dev_status, static_cast<cudaStream_t>(cuda_stream));
     return run_fwd(p, pl, static_cast<char*>(ws), loss, row_lse, pos_logit, dev_status,
                    static_cast<cudaStream_t>(cuda_stream));
 }
@@ -618,6 +636,9 @@ int gc_loss_fwd_static(const void* Q, int64_t ldq, const void* P, int64_t ldp,
     if (!scratch) return GC_ERR_CUDA;
     profile_begin_call();
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
+    if (small_applicable(B, N, d, dtype))      // one launch, no scratch at all
+        return run_small(GC_OP_FWD, p, nullptr, loss, row_lse, pos_logit, nullptr, 0, nullptr, 0,
+                         dev_status, static_cast<cudaStream_t>(cuda_stream));
     return run_fwd(p, pl, static_cast<char*>(scratch), loss, row_lse, pos_logit, dev_status,
                    static_cast<cudaStream_t>(cuda_stream));
 }
@@ -637,6 +658,9 @@ int gc_loss_bwd(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
     profile_begin_call();
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
+    if (small_applicable(B, N, d, dtype) && (dQ || dP))
+        return run_small(GC_OP_BWD, p, row_lse, nullptr, nullptr, nullptr, dQ, lddq, dP, lddp,
+                         dev_status, st);
     if (dev_status && launch_pos_check(pos_idx, B, N, mask_mode, dev_status, st) != cudaSuccess)
         return GC_ERR_CUDA;
     char* w = static_cast<char*>(ws);
@@ -661,6 +685,9 @@ int gc_build_cache(const void* Q, int64_t ldq, const void* P, int64_t ldp, const
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
     Problem p = make_problem(Q, ldq, P, ldp, pos_idx, B, N, d, tau, mask_mode, dtype);
     char* w = static_cast<char*>(ws);
+    if (small_applicable(B, N, d, dtype))
+        return run_small(GC_OP_BUILD, p, nullptr, loss, row_lse, pos_logit, dQ, lddq, dP, lddp,
+                         dev_status, st);
     return run_build_sweeps(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status, st);
 }
 

@@ -314,22 +314,6 @@ apply_kernel(const __grid_constant__ CUtensorMap mapU, const __grid_constant__ C
     }
 }
 
-// Row-major fp32 matrix [rows x d], boxes of 32 columns (128 bytes) x 32 rows, 128-byte swizzle,
-// out-of-range elements read as zero.
-bool make_map_f32(CUtensorMap* map, const void* base, int64_t rows, int d, int64_t ld) {
-    EncodeTiledFn fn = encode_fn();
-    if (!fn) return false;
-    cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
-    cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
-    cuuint32_t box[2] = {32, (cuuint32_t)AK};
-    cuuint32_t estr[2] = {1, 1};
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims,
-                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS;
-}
-
 struct ApplyPlan {
     int tiles_m, tiles_n, splits;
 };
@@ -392,7 +376,7 @@ int gc_cache_apply(const float* U, int64_t ldu, const void* X, int64_t ldx, int6
     cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
 
     CUtensorMap mu, mx;
-    if (!make_map_f32(&mu, U, rows, d, ldu) || !make_map(&mx, X, rows, d_in, ldx, AK))
+    if (!make_map_f32(&mu, U, rows, d, ldu, AK) || !make_map(&mx, X, rows, d_in, ldx, AK))
         return GC_ERR_CUDA;
     ApplyParams p{};
     p.rows = rows; p.d = d; p.d_in = d_in;

@@ -188,6 +188,12 @@ cudaError_t quad_launch_sweep(const SweepArgs& a, cudaStream_t st);
 cudaError_t quad_launch_fused_dq(const FwdArgs& a, float* partial, int groups, const float* row_ref,
                                  int* range_flag, cudaStream_t st, bool overlap_prev = false);
 
+// gc_small.cu
+bool small_applicable(int64_t B, int64_t N, int d, int dtype);
+cudaError_t launch_small(int op, const Problem& pr, const float* row_lse_in, float* loss,
+                         float* row_lse, float* pos_logit, float* dQ, int64_t lddq, float* dP,
+                         int64_t lddp, int* dev_status, cudaStream_t st);
+
 // gc_gemm.cu
 int gemm_groups(int64_t m_rows, int64_t k_len, int d);
 cudaError_t launch_weight_gemm(const void* weights, int64_t ldw, int64_t B, int64_t N, int transpose,

@@ -369,6 +369,23 @@ bool make_map(CUtensorMap* map, const void* base, int64_t rows, int d, int64_t l
     return r == CUDA_SUCCESS;
 }
 
+// Row-major fp32 matrix [rows x d], boxes of (box_rows x 32 columns = 128 bytes), 128-byte
+// swizzle, out-of-range elements read as zero.
+bool make_map_f32(CUtensorMap* map, const void* base, int64_t rows, int d, int64_t ld,
+                  int box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)ld * 4};
+    cuuint32_t box[2] = {32, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims,
+                    strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
 // fp32 destination of the accumulators as [planes][rows][d]: the output matrix itself (one plane,
 // row pitch ld) or the per-part partial sums (planes = parts of the streamed range, pitch d).
 // Boxes of 32 rows x 32 columns, 128-byte swizzle.

@@ -57,9 +57,14 @@ def test_workspace_is_linear_in_rows_not_quadratic(binding):
 
 def test_plan_names(binding):
     b = binding
-    assert b.gc_plan_name(b.GC_OP_BUILD, 64, 128, 768, b.GC_F32) == "simt"
+    # one tile: fp32 up to 128 x 128, bf16 up to 128 x 256, d a multiple of 8 up to 1024
+    assert b.gc_plan_name(b.GC_OP_BUILD, 64, 128, 768, b.GC_F32) == "tcgen05-one-tile"
+    assert b.gc_plan_name(b.GC_OP_BUILD, 128, 256, 768, b.GC_BF16) == "tcgen05-one-tile"
+    assert b.gc_kernel_launches(b.GC_OP_BUILD, 64, 128, 768, b.GC_F32) == 1
+    assert b.gc_plan_name(b.GC_OP_BUILD, 64, 129, 768, b.GC_F32) == "simt"
+    assert b.gc_plan_name(b.GC_OP_BUILD, 129, 128, 768, b.GC_BF16) == "tcgen05"
     assert b.gc_plan_name(b.GC_OP_BUILD, 64, 128, 100, b.GC_BF16) == "simt"
-    assert b.gc_kernel_launches(b.GC_OP_BUILD, 64, 128, 768, b.GC_F32) >= 4
+    assert b.gc_kernel_launches(b.GC_OP_BUILD, 64, 129, 768, b.GC_F32) >= 4
 
 
 def _call_fwd(lib, **over):
