@@ -35,6 +35,7 @@ constexpr uint32_t BF_W_OFF = SM_STAGES * BF_STAGE;          // four weight chun
 constexpr uint32_t F32_TERM_OFF = SM_STAGES * F32_STAGE;     // q1 q2 q3 p1 p2 p3 behind the ring
 constexpr size_t SM_DYN_SMEM = 1024 + (size_t)SM_STAGES * BF_STAGE + 4 * TILE;
 constexpr uint32_t COL_S = 0, COL_DQ = 256, COL_DP = 320;    // tensor-memory columns
+constexpr uint32_t COL_S2 = 384;     // fp32 inputs: the small products of S (128 columns)
 
 static_assert(SM_DYN_SMEM <= SMEM_LIMIT - SMEM_STATIC_RESERVE, "shared memory budget");
 static_assert(F32_TERM_OFF + 6 * TILE <= SM_STAGES * BF_STAGE + 4 * TILE, "fp32 layout fits");
@@ -107,6 +108,28 @@ __device__ __forceinline__ bool workers_all(bool mine) {
         : "=r"(all) : "r"(mine ? 1u : 0u), "n"(32 * SM_WORKERS) : "memory");
     return all != 0;
 }
+__device__ __forceinline__ float lg2(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+// 32 columns of this thread's row of S; fp32 inputs keep S as the sum of three accumulators.
+template <bool F32>
+__device__ __forceinline__ void load_s(uint32_t trow, int jb, float (&s)[32]) {
+    uint32_t v[32];
+    tmem_ld32(trow + COL_S + jb, v);
+    tmem_ld_wait();
+#pragma unroll
+    for (int e = 0; e < 32; ++e) s[e] = __uint_as_float(v[e]);
+    if (F32) {
+        uint32_t u[32];
+        tmem_ld32(trow + COL_S + 128 + jb, v);
+        tmem_ld32(trow + COL_S2 + jb, u);
+        tmem_ld_wait();
+#pragma unroll
+        for (int e = 0; e < 32; ++e) s[e] = (s[e] + __uint_as_float(v[e])) + __uint_as_float(u[e]);
+    }
+}
 __device__ __forceinline__ void workers_sync() {
     asm volatile("bar.sync 1, %0;" ::"n"(32 * SM_WORKERS) : "memory");
 }
@@ -114,12 +137,13 @@ __device__ __forceinline__ void workers_sync() {
 template <bool F32>
 __global__ void __launch_bounds__(SM_THREADS, 1)
 small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ CUtensorMap mapP,
+             const __grid_constant__ CUtensorMap mapDQ, const __grid_constant__ CUtensorMap mapDP,
              const SmallParams p) {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) SmallBars bars;
     __shared__ uint32_t tmem_base_s;
     __shared__ int abort_s;
-    __shared__ float x_max[2][128], x_sum[2][128];     // exchange between the two column halves
+    __shared__ float x_max[2][128], x_sum[2][128], x_pos[2][128];   // exchange between the column halves
     __shared__ float loss_part[4];
     volatile int* abort_flag = &abort_s;
 
@@ -212,13 +236,19 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
                         const uint32_t q1 = desc_lo(term_smem, 0) + k;
                         const uint32_t p1 = desc_lo(term_smem + 3 * TILE, 0) + k;
                         constexpr uint32_t T = TILE >> 4;
-                        if (t == 0 && kk == 0) mma_ss<false, false>(tmem + COL_S, q1, p1, idesc_s);
-                        else                   mma_ss<true, false>(tmem + COL_S, q1, p1, idesc_s);
-                        mma_ss<true, false>(tmem + COL_S, q1, p1 + T, idesc_s);
-                        mma_ss<true, false>(tmem + COL_S, q1 + T, p1, idesc_s);
-                        mma_ss<true, false>(tmem + COL_S, q1 + T, p1 + T, idesc_s);
-                        mma_ss<true, false>(tmem + COL_S, q1, p1 + 2 * T, idesc_s);
-                        mma_ss<true, false>(tmem + COL_S, q1 + 2 * T, p1, idesc_s);
+                        // The accumulator adds with truncation: the leading product alternates
+                        // between two accumulators and the five small ones have a third, so that
+                        // each takes few additions of its own magnitude; the softmax warps sum
+                        // the three in fp32.
+                        const uint32_t lead = tmem + COL_S + 128 * kk, rest = tmem + COL_S2;
+                        if (t == 0) mma_ss<false, false>(lead, q1, p1, idesc_s);
+                        else        mma_ss<true, false>(lead, q1, p1, idesc_s);
+                        if (t == 0 && kk == 0) mma_ss<false, false>(rest, q1, p1 + T, idesc_s);
+                        else                   mma_ss<true, false>(rest, q1, p1 + T, idesc_s);
+                        mma_ss<true, false>(rest, q1 + T, p1, idesc_s);
+                        mma_ss<true, false>(rest, q1 + T, p1 + T, idesc_s);
+                        mma_ss<true, false>(rest, q1, p1 + 2 * T, idesc_s);
+                        mma_ss<true, false>(rest, q1 + 2 * T, p1, idesc_s);
                     }
                     tc_commit(smem_u32(&bars.term_empty[h]));
                 }
@@ -305,10 +335,16 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
         const uint32_t lane_addr = (uint32_t)(32 * q) << 16;
         bool ok = true;
         if (F32) {
-            // fp32 -> three bf16 terms.  Item = 8 consecutive columns of one row (two 16-byte
-            // pieces in, one piece per term out).  Eight neighbouring threads take four items of
-            // row r and four of row r + 4, the second row fetching its two pieces in the opposite
-            // order: loads and stores both fall on distinct banks.
+            // fp32 -> three bf16 terms by truncation (t1 = the upper 16 bits of x, t2 those of
+            // x - t1, t3 those of what is left: x = t1 + t2 + t3 exactly).  Item = 8 consecutive
+            // columns of one row (two 16-byte pieces in, one piece per term out).  Eight
+            // neighbouring threads take four items of row r and four of row r + 4, the second
+            // row fetching its two pieces in the opposite order: loads and stores both fall on
+            // distinct banks.  Rows past B (N) are skipped: the term tiles start out as zeros.
+            for (int e = wt; e < (int)(6 * TILE / 16); e += 32 * SM_WORKERS) {
+                const uint32_t z[4] = {0u, 0u, 0u, 0u};
+                sts128u(term_smem + 16 * e, z);
+            }
             int stage = 0;
             uint32_t phase = 0;
             for (int t = 0; t < s_steps + g_steps; ++t) {
@@ -323,16 +359,26 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
                     const int cp = id & 3, rr = (id >> 2) & 1, b = (id >> 3) & 3, a = (id >> 5) & 15;
                     const int mat = id >> 9;
                     const int r = 8 * a + b + 4 * rr, sw = r & 7;
+                    if (r >= (mat ? p.N : p.B)) continue;
                     const uint32_t src = src0 + mat * TILE + r * 128;
                     const int first = (2 * cp) ^ rr;
                     const float4 A = lds128f(src + (uint32_t)((first ^ sw) << 4));
                     const float4 Bv = lds128f(src + (uint32_t)(((first ^ 1) ^ sw) << 4));
                     const float4 f0 = rr ? Bv : A, f1 = rr ? A : Bv;
+                    const float x[8] = {f0.x, f0.y, f0.z, f0.w, f1.x, f1.y, f1.z, f1.w};
                     uint32_t t1[4], t2[4], t3[4];
-                    split3(f0.x, f0.y, &t1[0], &t2[0], &t3[0]);
-                    split3(f0.z, f0.w, &t1[1], &t2[1], &t3[1]);
-                    split3(f1.x, f1.y, &t1[2], &t2[2], &t3[2]);
-                    split3(f1.z, f1.w, &t1[3], &t2[3], &t3[3]);
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const uint32_t a0 = __float_as_uint(x[2 * e]), a1 = __float_as_uint(x[2 * e + 1]);
+                        const float r0 = x[2 * e] - __uint_as_float(a0 & 0xffff0000u);
+                        const float r1 = x[2 * e + 1] - __uint_as_float(a1 & 0xffff0000u);
+                        const uint32_t b0 = __float_as_uint(r0), b1 = __float_as_uint(r1);
+                        const float s0 = r0 - __uint_as_float(b0 & 0xffff0000u);
+                        const float s1 = r1 - __uint_as_float(b1 & 0xffff0000u);
+                        t1[e] = __byte_perm(a0, a1, 0x7632);      // the two upper halves
+                        t2[e] = __byte_perm(b0, b1, 0x7632);
+                        t3[e] = __byte_perm(__float_as_uint(s0), __float_as_uint(s1), 0x7632);
+                    }
                     const uint32_t dst = term_smem + (uint32_t)(3 * mat) * TILE + r * 128 +
                                          (uint32_t)(((4 * h + cp) ^ sw) << 4);
                     sts128u(dst, t1);
@@ -352,6 +398,8 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
         if (workers_all(ok)) {
             tc_fence_after();
             // ------------------------------ softmax of row i over this half's columns -------------
+            // One pass over the row keeps a running (max, sum); the special columns of a block of
+            // 32 (past N, the masked pair, the positive) are patched after the plain arithmetic.
             const int ncols = F32 ? 128 : 256;
             const int j0 = half * (ncols / 2);                    // fp32: 0 or 64; bf16: 0 or 128
             const int nblk = ncols / 64;                          // blocks of 32 columns per half
@@ -365,43 +413,48 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
             const int masked = p.mask_mode == GC_MASK_SELF ? i + p.mask_shift : -1;
             float lse2, pos2 = 0.f;
             if (p.op == GC_OP_BWD) {
-                lse2 = i < p.B ? p.row_lse_in[i] * 1.4426950408889634f : 0.f;
+                lse2 = p.row_lse_in[i < p.B ? i : 0] * 1.4426950408889634f;
             } else {
-                float m = -INFINITY;
+                float m = -INFINITY, sum = 0.f;
                 for (int cb = 0; cb < nblk; ++cb) {
-                    uint32_t v[32];
-                    tmem_ld32(tmem + lane_addr + COL_S + j0 + 32 * cb, v);
-                    tmem_ld_wait();
+                    const int jb = j0 + 32 * cb;
+                    if (jb >= p.N) break;
+                    float s2[32];
+                    load_s<F32>(tmem + lane_addr, jb, s2);
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        const int j = j0 + 32 * cb + e;
-                        const float s2 = __uint_as_float(v[e]) * p.scale2;
-                        if (j == pos) pos2 = s2;
-                        if (j < p.N && j != masked) m = fmaxf(m, s2);
+                    for (int e = 0; e < 32; ++e) s2[e] *= p.scale2;
+                    if ((unsigned)(pos - jb) < 32u) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) if (e == pos - jb) pos2 = s2[e];
                     }
+                    if ((unsigned)(masked - jb) < 32u) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) if (e == masked - jb) s2[e] = -INFINITY;
+                    }
+                    if (jb + 32 > p.N) {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) if (jb + e >= p.N) s2[e] = -INFINITY;
+                    }
+                    float bm = s2[0];
+#pragma unroll
+                    for (int e = 1; e < 32; ++e) bm = fmaxf(bm, s2[e]);
+                    const float mn = fmaxf(m, bm);
+                    const float ref = mn == -INFINITY ? 0.f : mn;
+                    float part = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) part += ex2(s2[e] - ref);
+                    sum = sum * ex2(m - ref) + part;
+                    m = mn;
                 }
                 x_max[half][i] = m;
-                x_sum[half][i] = pos2;
-                workers_sync();
-                m = fmaxf(x_max[0][i], x_max[1][i]);
-                pos2 = x_sum[0][i] + x_sum[1][i];                 // the other half holds 0
-                workers_sync();
-                float sum = 0.f;
-                for (int cb = 0; cb < nblk; ++cb) {
-                    uint32_t v[32];
-                    tmem_ld32(tmem + lane_addr + COL_S + j0 + 32 * cb, v);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        const int j = j0 + 32 * cb + e;
-                        const float s2 = __uint_as_float(v[e]) * p.scale2;
-                        if (j < p.N && j != masked) sum += exp2f(s2 - m);
-                    }
-                }
                 x_sum[half][i] = sum;
+                x_pos[half][i] = pos2;
                 workers_sync();
-                sum = x_sum[0][i] + x_sum[1][i];
-                lse2 = m + log2f(sum);
+                const float m0 = x_max[0][i], m1 = x_max[1][i];
+                m = fmaxf(m0, m1);
+                sum = x_sum[0][i] * ex2(m0 - m) + x_sum[1][i] * ex2(m1 - m);
+                pos2 = x_pos[0][i] + x_pos[1][i];                 // the other half holds 0
+                lse2 = m + lg2(sum);
             }
             // ------------------------------ outputs of the forward (CTA 0) ------------------------
             if (slice == 0) {
@@ -427,23 +480,33 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
             if (do_grad) {
                 // ------------------------------ weights as MMA operands ---------------------------
                 // chunk c = 64 columns; element (i, j) in 16-byte piece ((j % 64) / 8) ^ (i % 8) of
-                // row i: a K-major A operand for dQ and, read by columns, an MN-major one for dP
+                // row i: a K-major A operand for dQ and, read by columns, an MN-major one for dP.
+                // Rows past B get lse = +inf: all their weights are 0.
+                const float neg_lse = i < p.B ? -lse2 : -INFINITY;
+                const int pos_w = i < p.B ? pos : -1;
                 for (int cb = 0; cb < nblk; ++cb) {
-                    uint32_t v[32];
-                    tmem_ld32(tmem + lane_addr + COL_S + j0 + 32 * cb, v);
-                    tmem_ld_wait();
-                    float w[32];
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) {
-                        const int j = j0 + 32 * cb + e;
-                        float x = 0.f;
-                        if (i < p.B && j < p.N && j != masked) {
-                            x = exp2f(__uint_as_float(v[e]) * p.scale2 - lse2);
-                            if (j == pos) x -= 1.f;
-                        }
-                        w[e] = x;
-                    }
                     const int jb = j0 + 32 * cb;                  // 4 pieces of 8 columns
+                    float w[32];
+                    if (jb < p.N) {
+                        load_s<F32>(tmem + lane_addr, jb, w);
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) w[e] = ex2(fmaf(w[e], p.scale2, neg_lse));
+                        if ((unsigned)(masked - jb) < 32u) {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) if (e == masked - jb) w[e] = 0.f;
+                        }
+                        if ((unsigned)(pos_w - jb) < 32u) {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) if (e == pos_w - jb) w[e] -= 1.f;
+                        }
+                        if (jb + 32 > p.N) {
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) if (jb + e >= p.N) w[e] = 0.f;
+                        }
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) w[e] = 0.f;
+                    }
                     const uint32_t row = w_smem + (uint32_t)(jb >> 6) * TILE + i * 128;
 #pragma unroll
                     for (int pc = 0; pc < 4; ++pc) {
@@ -467,28 +530,35 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&bars.w_full));
                 // ------------------------------ gradients out -------------------------------------
+                // A warp's 32 x 32 block goes through a 4 KB buffer (two per warp, over the
+                // drained pipeline buffers) and leaves with one bulk tensor store, which clips it
+                // at the matrix's last row and column.
                 if (mbar_wait(smem_u32(&bars.acc_full), 0, abort_flag)) {
                     tc_fence_after();
                     const int col = 64 * slice + 32 * half;
+                    const uint32_t slot = base + (uint32_t)(warp - SM_FIRST_WORKER) * 8192u;
+                    int n = 0;
                     for (int blk = 0; blk < 1 + ptiles; ++blk) {       // dQ, dP rows 0.., dP rows 128..
-                        const int rows = blk == 0 ? p.B : p.N - 128 * (blk - 1);
-                        float* out = blk == 0 ? p.dQ + (int64_t)i * p.lddq
-                                              : p.dP + (int64_t)(128 * (blk - 1) + i) * p.lddp;
+                        const int rows = blk == 0 ? p.B : p.N;
+                        const int row0 = (blk == 0 ? 0 : 128 * (blk - 1)) + 32 * q;
+                        const bool have = blk == 0 ? p.dQ != nullptr : p.dP != nullptr;
+                        if (!have || row0 >= rows || col >= p.d) continue;
                         uint32_t v[32];
                         tmem_ld32(tmem + lane_addr + (blk == 0 ? COL_DQ : COL_DP + 64 * (blk - 1)) +
                                       32 * half, v);
-                        tmem_ld_wait();
-                        if (i < rows && (blk == 0 ? p.dQ : p.dP) != nullptr) {
-#pragma unroll
-                            for (int e = 0; e < 8; ++e)
-                                if (col + 4 * e < p.d)
-                                    *reinterpret_cast<float4*>(out + col + 4 * e) = make_float4(
-                                        __uint_as_float(v[4 * e]) * p.out_scale,
-                                        __uint_as_float(v[4 * e + 1]) * p.out_scale,
-                                        __uint_as_float(v[4 * e + 2]) * p.out_scale,
-                                        __uint_as_float(v[4 * e + 3]) * p.out_scale);
+                        if (n >= 2) {   // the store issued two blocks ago has read this buffer
+                            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+                            __syncwarp();
                         }
+                        tmem_ld_wait();
+                        const uint32_t buf = slot + (uint32_t)(n & 1) * 4096u;
+                        stage_block(buf, v, p.out_scale, lane);
+                        __syncwarp();
+                        if (lane == 0) tma_store_3d(blk == 0 ? &mapDQ : &mapDP, buf, col, row0, 0);
+                        ++n;
                     }
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+                    __syncwarp();
                 }
             }
         }
@@ -512,8 +582,9 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
 }
 
 template <bool F32>
-cudaError_t launch_small_t(const CUtensorMap& mq, const CUtensorMap& mp, const SmallParams& p,
-                           unsigned ctas, cudaStream_t st) {
+cudaError_t launch_small_t(const CUtensorMap& mq, const CUtensorMap& mp, const CUtensorMap& mdq,
+                           const CUtensorMap& mdp, const SmallParams& p, unsigned ctas,
+                           cudaStream_t st) {
     static bool configured_on[64] = {false};      // the attribute belongs to (kernel, device)
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
@@ -524,7 +595,7 @@ cudaError_t launch_small_t(const CUtensorMap& mq, const CUtensorMap& mp, const S
         if (e != cudaSuccess) return e;
         configured_on[dev] = true;
     }
-    small_kernel<F32><<<ctas, SM_THREADS, SM_DYN_SMEM, st>>>(mq, mp, p);
+    small_kernel<F32><<<ctas, SM_THREADS, SM_DYN_SMEM, st>>>(mq, mp, mdq, mdp, p);
     return cudaGetLastError();
 }
 
@@ -546,6 +617,11 @@ cudaError_t launch_small(int op, const Problem& pr, const float* row_lse_in, flo
                         : make_map(&mq, pr.Q, pr.B, pr.d, pr.ldq, 128) &&
                               make_map(&mp, pr.P, pr.N, pr.d, pr.ldp, 128);
     if (!ok) return cudaErrorInvalidValue;
+    // gradient outputs as [1][rows][d] for the epilogue's bulk tensor stores; a missing output
+    // (gc_loss_fwd; gc_loss_bwd with one of the two) gets a map of the other, never written
+    CUtensorMap mdq = mq, mdp = mp;
+    if (dQ && !make_out_map(&mdq, dQ, pr.B, pr.d, lddq, 1)) return cudaErrorInvalidValue;
+    if (dP && !make_out_map(&mdp, dP, pr.N, pr.d, lddp, 1)) return cudaErrorInvalidValue;
     SmallParams p{};
     p.B = (int)pr.B; p.N = (int)pr.N; p.d = pr.d;
     p.op = op;
@@ -561,7 +637,8 @@ cudaError_t launch_small(int op, const Problem& pr, const float* row_lse_in, flo
     p.dQ = dQ; p.lddq = lddq; p.dP = dP; p.lddp = lddp;
     p.dev_status = dev_status;
     const unsigned ctas = op == GC_OP_FWD ? 1u : (unsigned)((pr.d + 63) / 64);
-    return f32 ? launch_small_t<true>(mq, mp, p, ctas, st) : launch_small_t<false>(mq, mp, p, ctas, st);
+    return f32 ? launch_small_t<true>(mq, mp, mdq, mdp, p, ctas, st)
+               : launch_small_t<false>(mq, mp, mdq, mdp, p, ctas, st);
 }
 
 }  // namespace gc
