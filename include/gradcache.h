@@ -228,6 +228,39 @@ int gc_dtau(const void* Q, int64_t ldq, const float* dQ, int64_t lddq, int64_t B
             int dtype, float* dtau, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /*
+ * Two more loss variants of Section 3.3, Step 2, each one call that runs gc_build_cache and adds
+ * what differs from Eq. 1 in fp32 (device pointers, asynchronous on cuda_stream, deterministic:
+ * sums into rows of dP that several queries point at are formed in ascending query order).
+ *
+ *   gc_build_cache_multi_pos   several positives per query, given as a CSR list: query i has the
+ *       positives pos_list[pos_ptr[i] .. pos_ptr[i + 1]) (int32, pos_ptr of length B + 1, n_pos =
+ *       pos_ptr[B] entries in all, at least one per query, distinct within a query).  Loss of
+ *       query i = mean over its positives of -log p_ir, so G_ij = (p_ij - [j in R_i]/|R_i|)/B;
+ *       one positive per query is gc_build_cache.  An empty or out-of-range list sets
+ *       GC_DEV_POS_RANGE, a positive on the masked diagonal GC_DEV_POS_MASKED.
+ *   gc_build_cache_two_direction   L = (L_row + L_col)/2 with L_row = Eq. 1 and L_col its mirror
+ *       image over the same B positive pairs: passage r_i is the anchor and the B queries are its
+ *       candidates, L_col = (1/B) sum_i (log sum_i' exp(S_{i' r_i}) - S_{i r_i}).  N may exceed B.
+ *       No mask (GC_MASK_NONE).  row_lse receives the row direction's logsumexp.
+ * Q, P, dQ, dP, loss, row_lse, tau, dtype as in gc_build_cache; d a multiple of 8 (else
+ * GC_ERR_LIMIT).  Workspace: gc_multi_pos_workspace_bytes / gc_two_direction_workspace_bytes
+ * (0 for invalid arguments), 256-byte aligned, caller-owned.
+ */
+size_t gc_multi_pos_workspace_bytes(int64_t B, int64_t N, int d, int dtype, int64_t n_pos);
+int gc_build_cache_multi_pos(const void* Q, int64_t ldq, const void* P, int64_t ldp,
+                             const int32_t* pos_ptr, const int32_t* pos_list, int64_t n_pos,
+                             int64_t B, int64_t N, int d, float tau, int mask_mode, int dtype,
+                             float* loss, float* row_lse, float* dQ, int64_t lddq, float* dP,
+                             int64_t lddp, void* ws, size_t ws_bytes, int* dev_status,
+                             void* cuda_stream);
+size_t gc_two_direction_workspace_bytes(int64_t B, int64_t N, int d, int dtype);
+int gc_build_cache_two_direction(const void* Q, int64_t ldq, const void* P, int64_t ldp,
+                                 const int32_t* pos_idx, int64_t B, int64_t N, int d, float tau,
+                                 int dtype, float* loss, float* row_lse, float* dQ, int64_t lddq,
+                                 float* dP, int64_t lddp, void* ws, size_t ws_bytes,
+                                 int* dev_status, void* cuda_stream);
+
+/*
  * Distance Gradient Cache (Section 5, Eq. 10-13) in tiled form.  The similarity of pair (i, j) is
  * a distance d_ij = Phi(f(s_i), g(t_j)) computed by the caller's network; the loss is Eq. 1 with
  * d_ij / tau as the logit.  The paper stores all B x N values w_ij = dL/dd_ij.  Here the caller

@@ -25,7 +25,9 @@ EXPORTS = ("gc_workspace_bytes", "gc_plan_name", "gc_kernel_launches", "gc_loss_
            "gc_cache_apply_workspace_bytes", "gc_cache_apply", "gc_shard_workspace_bytes",
            "gc_shard_fwd_dq", "gc_shard_dp", "gc_selftest_wait_limit", "gc_row_normalize",
            "gc_cosine_bwd", "gc_dtau_workspace_bytes", "gc_dtau", "gc_dist_begin",
-           "gc_dist_accumulate", "gc_dist_finish", "gc_dist_w_block", "gc_dist_dot_block")
+           "gc_dist_accumulate", "gc_dist_finish", "gc_dist_w_block", "gc_dist_dot_block",
+           "gc_multi_pos_workspace_bytes", "gc_build_cache_multi_pos",
+           "gc_two_direction_workspace_bytes", "gc_build_cache_two_direction")
 GC_STATIC_SCRATCH_BYTES = 2 << 20
 
 
@@ -85,6 +87,17 @@ def _load() -> ctypes.CDLL:
     lib.gc_dtau_workspace_bytes.argtypes = [i64]
     lib.gc_dtau.restype = i32
     lib.gc_dtau.argtypes = [vp, i64, vp, i64, i64, i32, f32, i32, vp, vp, ctypes.c_size_t, vp]
+    lib.gc_multi_pos_workspace_bytes.restype = ctypes.c_size_t
+    lib.gc_multi_pos_workspace_bytes.argtypes = [i64, i64, i32, i32, i64]
+    lib.gc_build_cache_multi_pos.restype = i32
+    lib.gc_build_cache_multi_pos.argtypes = [vp, i64, vp, i64, vp, vp, i64, i64, i64, i32, f32, i32,
+                                             i32, vp, vp, vp, i64, vp, i64, vp, ctypes.c_size_t,
+                                             vp, vp]
+    lib.gc_two_direction_workspace_bytes.restype = ctypes.c_size_t
+    lib.gc_two_direction_workspace_bytes.argtypes = [i64, i64, i32, i32]
+    lib.gc_build_cache_two_direction.restype = i32
+    lib.gc_build_cache_two_direction.argtypes = [vp, i64, vp, i64, vp, i64, i64, i32, f32, i32, vp,
+                                                 vp, vp, i64, vp, i64, vp, ctypes.c_size_t, vp, vp]
     lib.gc_dist_begin.restype = i32
     lib.gc_dist_begin.argtypes = [vp, vp, vp, i64, vp]
     lib.gc_dist_accumulate.restype = i32
@@ -319,6 +332,44 @@ def gc_dtau(Q, dQ, tau, dtau, ws=None) -> None:
                       _dtype_code(Q), _ptr(dtau), _ptr(ws), ws.numel(), _stream())
     if rc != 0:
         raise GradCacheError(rc, "gc_dtau")
+
+
+def gc_build_cache_multi_pos(Q, P, pos_ptr, pos_list, tau, mask_mode, loss, row_lse, dQ, dP,
+                             ws=None, dev_status=None) -> None:
+    """Several positives per query (CSR lists pos_ptr [B + 1], pos_list, int32): loss and cache
+    rows of the mean-over-positives loss (Section 3.3, Step 2)."""
+    B, d = Q.shape
+    N = P.shape[0]
+    n_pos = pos_list.numel()
+    code = _dtype_code(Q)
+    if ws is None:
+        ws = torch.empty(max(int(_lib.gc_multi_pos_workspace_bytes(B, N, d, code, n_pos)), 256),
+                         dtype=torch.uint8, device=Q.device)
+    rc = _lib.gc_build_cache_multi_pos(_ptr(Q), Q.stride(0), _ptr(P), P.stride(0), _ptr(pos_ptr),
+                                       _ptr(pos_list), n_pos, B, N, d, float(tau), int(mask_mode),
+                                       code, _ptr(loss), _ptr(row_lse), _ptr(dQ), dQ.stride(0),
+                                       _ptr(dP), dP.stride(0), _ptr(ws), ws.numel(),
+                                       _ptr(dev_status), _stream())
+    if rc != 0:
+        raise GradCacheError(rc, "gc_build_cache_multi_pos")
+
+
+def gc_build_cache_two_direction(Q, P, pos_idx, tau, loss, row_lse, dQ, dP, ws=None,
+                                 dev_status=None) -> None:
+    """L = (L_row + L_col) / 2 over the B positive pairs (Section 3.3, Step 2), no mask."""
+    B, d = Q.shape
+    N = P.shape[0]
+    code = _dtype_code(Q)
+    if ws is None:
+        ws = torch.empty(max(int(_lib.gc_two_direction_workspace_bytes(B, N, d, code)), 256),
+                         dtype=torch.uint8, device=Q.device)
+    rc = _lib.gc_build_cache_two_direction(_ptr(Q), Q.stride(0), _ptr(P), P.stride(0),
+                                           _ptr(pos_idx), B, N, d, float(tau), code, _ptr(loss),
+                                           _ptr(row_lse), _ptr(dQ), dQ.stride(0), _ptr(dP),
+                                           dP.stride(0), _ptr(ws), ws.numel(), _ptr(dev_status),
+                                           _stream())
+    if rc != 0:
+        raise GradCacheError(rc, "gc_build_cache_two_direction")
 
 
 class DistanceCache:

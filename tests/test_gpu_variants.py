@@ -100,3 +100,110 @@ def test_variant_calls_refuse_bad_arguments(binding):
     with pytest.raises(binding.GradCacheError) as e:
         binding.gc_dtau(Q, torch.zeros(4, 16, device="cuda"), 0.0, torch.zeros(1, device="cuda"))
     assert e.value.status == 2
+
+
+def _positive_lists(B, N, rng, mask_mode, max_pos=4):
+    """Between one and max_pos distinct positives per query, none on the masked diagonal; some
+    passages are the positive of several queries."""
+    lists = []
+    for i in range(B):
+        k = int(rng.integers(1, max_pos + 1))
+        allowed = np.array([j for j in range(N) if not (mask_mode and j == i)])
+        lists.append([int(v) for v in rng.choice(allowed, size=min(k, len(allowed)), replace=False)])
+    return lists
+
+
+@pytest.mark.parametrize("B,N,d,dtype,tau,mask", [
+    (64, 128, 768, "f32", 1.0, 0), (100, 57, 72, "f32", 0.3, 0), (128, 256, 768, "bf16", 1.0, 0),
+    (300, 300, 128, "bf16", 0.2, 1), (520, 900, 768, "bf16", 0.5, 0), (200, 200, 64, "f32", 0.5, 1),
+])
+def test_several_positives_per_query(binding, oracle, B, N, d, dtype, tau, mask):
+    prob = inputs.random_problem(B, N, d, dtype, seed=B + 3 * d, tau=tau, scale=d ** -0.5,
+                                 mask_mode=mask, shared=bool(mask))
+    rng = np.random.default_rng(B + N)
+    lists = _positive_lists(B, N, rng, mask)
+    ref = oracle.build_variant(prob.Q, prob.P, lists, prob.tau, prob.mask_mode)
+    Q, P, _ = to_device(prob)
+    ptr = np.zeros(B + 1, np.int32)
+    ptr[1:] = np.cumsum([len(r) for r in lists])
+    flat = np.array([v for r in lists for v in r], np.int32)
+    pos_ptr, pos_list = torch.from_numpy(ptr).cuda(), torch.from_numpy(flat).cuda()
+    f = dict(dtype=torch.float32, device="cuda")
+    outs = []
+    for _ in range(2):
+        loss, lse = torch.zeros(1, **f), torch.empty(B, **f)
+        dQ, dP = torch.full((B, d), float("nan"), **f), torch.full((N, d), float("nan"), **f)
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        binding.gc_build_cache_multi_pos(Q, P, pos_ptr, pos_list, prob.tau, prob.mask_mode, loss,
+                                         lse, dQ, dP, dev_status=st)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        outs.append((loss, dQ, dP))
+    loss, dQ, dP = outs[0]
+    tol = TOL[dtype]
+    assert abs(loss.item() - ref["loss"]) <= tol["loss"] * max(abs(ref["loss"]), 1e-6)
+    floor = 1e-2 * max(float(np.abs(prob.Q).max()), float(np.abs(prob.P).max())) / (B * tau)
+    assert grad_err(dQ.cpu().numpy(), ref["dQ"], floor) <= tol["grad"]
+    assert grad_err(dP.cpu().numpy(), ref["dP"], floor) <= tol["grad"]
+    assert torch.equal(dQ, outs[1][1]) and torch.equal(dP, outs[1][2])      # reproducible
+    assert torch.equal(loss, outs[1][0])
+
+
+def test_one_positive_per_query_is_the_plain_call(binding):
+    prob = inputs.random_problem(150, 260, 128, "bf16", seed=8, tau=0.4, scale=0.1)
+    Q, P, pos = to_device(prob)
+    plain = binding.build_cache(Q, P, pos, prob.tau, 0)
+    B, N, d = prob.B, prob.N, prob.d
+    f = dict(dtype=torch.float32, device="cuda")
+    loss, lse, dQ, dP = torch.zeros(1, **f), torch.empty(B, **f), torch.empty(B, d, **f), torch.empty(N, d, **f)
+    ptr = torch.arange(B + 1, dtype=torch.int32, device="cuda")
+    binding.gc_build_cache_multi_pos(Q, P, ptr, pos, prob.tau, 0, loss, lse, dQ, dP)
+    torch.cuda.synchronize()
+    assert torch.equal(loss, plain.loss) and torch.equal(dQ, plain.dQ) and torch.equal(dP, plain.dP)
+
+
+def test_bad_positive_lists_raise_the_device_flags(binding):
+    prob = inputs.random_problem(40, 60, 64, "bf16", seed=3, tau=1.0, scale=0.2)
+    Q, P, pos = to_device(prob)
+    B, N, d = prob.B, prob.N, prob.d
+    f = dict(dtype=torch.float32, device="cuda")
+    loss, lse, dQ, dP = torch.zeros(1, **f), torch.empty(B, **f), torch.empty(B, d, **f), torch.empty(N, d, **f)
+    ptr = torch.arange(B + 1, dtype=torch.int32, device="cuda")
+    ptr[5] = ptr[4]                                 # query 4 has no positive
+    bad = pos.clone()
+    bad[9] = N + 3                                  # out of range
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    binding.gc_build_cache_multi_pos(Q, P, ptr, bad, prob.tau, 0, loss, lse, dQ, dP, dev_status=st)
+    torch.cuda.synchronize()
+    assert int(st.item()) & 1                       # GC_DEV_POS_RANGE
+    assert bool(torch.isfinite(dQ).all()) and bool(torch.isfinite(dP).all())
+
+
+@pytest.mark.parametrize("B,N,d,dtype,tau", [
+    (64, 128, 768, "f32", 1.0), (100, 100, 72, "f32", 0.3), (128, 256, 768, "bf16", 1.0),
+    (300, 450, 128, "bf16", 0.2), (520, 900, 768, "bf16", 0.5), (77, 77, 64, "f32", 0.5),
+])
+def test_two_direction_loss(binding, oracle, B, N, d, dtype, tau):
+    prob = inputs.random_problem(B, N, d, dtype, seed=2 * B + d, tau=tau, scale=d ** -0.5)
+    pos_np = prob.pos_idx.copy()
+    pos_np[B // 2] = pos_np[0]                      # two queries share a positive passage
+    ref = oracle.build_variant(prob.Q, prob.P, pos_np, prob.tau, 0, two_direction=True)
+    Q, P, _ = to_device(prob)
+    pos = torch.from_numpy(pos_np).cuda()
+    f = dict(dtype=torch.float32, device="cuda")
+    outs = []
+    for _ in range(2):
+        loss, lse = torch.zeros(1, **f), torch.empty(B, **f)
+        dQ, dP = torch.full((B, d), float("nan"), **f), torch.full((N, d), float("nan"), **f)
+        st = torch.zeros(1, dtype=torch.int32, device="cuda")
+        binding.gc_build_cache_two_direction(Q, P, pos, prob.tau, loss, lse, dQ, dP, dev_status=st)
+        torch.cuda.synchronize()
+        assert int(st.item()) == 0
+        outs.append((loss, dQ, dP))
+    loss, dQ, dP = outs[0]
+    tol = TOL[dtype]
+    assert abs(loss.item() - ref["loss"]) <= tol["loss"] * max(abs(ref["loss"]), 1e-6)
+    floor = 1e-2 * max(float(np.abs(prob.Q).max()), float(np.abs(prob.P).max())) / (B * tau)
+    assert grad_err(dQ.cpu().numpy(), ref["dQ"], floor) <= tol["grad"]
+    assert grad_err(dP.cpu().numpy(), ref["dP"], floor) <= tol["grad"]
+    assert torch.equal(dQ, outs[1][1]) and torch.equal(dP, outs[1][2])
