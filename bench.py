@@ -36,33 +36,37 @@ def metric_name(B, N, d):
 
 NOMINAL_BF16_TFLOPS = 2250.0      # public dense bf16 figure for B200, context only
 # dram__bytes_read.sum + dram__bytes_write.sum of ONE STEP (every launch of a gc_build_cache
-# call summed) from the ncu captures summarised under profiles/ (step_traffic_*.txt).  Reported
-# only while the kernel sources still have the hash they had when the counters were taken.
-NCU_STEP_TRAFFIC = {"cfg2_": None, "cfg4_": None}
-NCU_TRAFFIC_SOURCE_SHA1 = ""
+# call summed) from the ncu captures summarised under profiles/ (quad_kernel_cfg2_*, quad_kernel_
+# cfg4_*, small_kernel_*).  Under ncu every launch starts from flushed caches, so a step of
+# several launches counts its inputs once per launch.  A figure is reported only while the
+# sources its kernels come from still have the hash they had when the counters were taken.
+SWEEP_SOURCES = ['gc_api.cu', 'gc_combine.cu', 'gc_internal.h', 'gc_quad.cu', 'gc_tc.cu', 'tc_common.cuh']
+ONE_TILE_SOURCES = ['gc_api.cu', 'gc_internal.h', 'gc_small.cu', 'tc_common.cuh']
+NCU_STEP_TRAFFIC = {
+    "cfg2_": (82.9e6, SWEEP_SOURCES, "84483f8f278705562c0aa3af6042063f4047ab83"),
+    "cfg4_": (4.80e9, SWEEP_SOURCES, "84483f8f278705562c0aa3af6042063f4047ab83"),
+    "cfg1_": (0.626e6, ONE_TILE_SOURCES, "5805c171fec09e6f6d30518e78491b7718936123"),
+    "cfg0_": (0.639e6, ONE_TILE_SOURCES, "5805c171fec09e6f6d30518e78491b7718936123"),
+}
 FP32_LANES_PER_SM = 128           # fp32 FMA lanes of one SM (2 FLOP per lane and clock)
 
 
-def sources_sha1():
-    import glob
+def sources_sha1(files):
     import hashlib
     h = hashlib.sha1()
-    for f in sorted(glob.glob(os.path.join(ROOT, "paper_2101_06983_b200", "csrc", "*"))):
-        with open(f, "rb") as fh:
+    for f in files:
+        with open(os.path.join(ROOT, "paper_2101_06983_b200", "csrc", f), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()
 
 
 def ncu_traffic(workload: str):
-    try:
-        same = sources_sha1() == NCU_TRAFFIC_SOURCE_SHA1
-    except OSError:
-        same = False
-    if not same:
-        return None
-    for prefix, val in NCU_STEP_TRAFFIC.items():
+    for prefix, (val, files, digest) in NCU_STEP_TRAFFIC.items():
         if workload.startswith(prefix):
-            return val
+            try:
+                return val if sources_sha1(files) == digest else None
+            except OSError:
+                return None
     return None
 
 
