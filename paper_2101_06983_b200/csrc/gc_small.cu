@@ -12,10 +12,11 @@
 // CTA 0 also writes loss, row_lse, pos_logit and the pos_idx flags.
 //
 // fp32 inputs run on the same tensor cores: converter warps split every value into three bf16
-// terms x = t1 + t2 + t3 (each the rounding of what the previous ones left, so the sum is exact
-// to 2^-24 |x|) as it arrives, S takes the six products t1 t1', t1 t2', t1 t3', t2 t1', t2 t2',
-// t3 t1' in fp32 accumulation, the weights are kept as two terms and the gradient products take
-// w1 t1 + w1 t2 + w2 t1.  Every mbarrier wait is bounded.
+// terms x = t1 + t2 + t3 (each the upper 16 bits of what the previous ones left, so the sum is
+// exact) as it arrives, S takes the six products t1 t1', t1 t2', t1 t3', t2 t1', t2 t2', t3 t1'
+// in fp32 accumulation (spread over three accumulators, see the MMA warp), the weights are kept
+// as two terms and the gradient products take w1 t1 + w1 t2 + w2 t1.  Every mbarrier wait is
+// bounded.
 #include "tc_common.cuh"
 
 namespace gc {
@@ -87,15 +88,6 @@ __device__ __forceinline__ uint32_t pack_bf16(float x, float y) {
 __device__ __forceinline__ float lo_f(uint32_t packed) { return __uint_as_float(packed << 16); }
 __device__ __forceinline__ float hi_f(uint32_t packed) {
     return __uint_as_float(packed & 0xffff0000u);
-}
-// (x, y) -> three packed bf16 pairs whose sum is (x, y) to 2^-24
-__device__ __forceinline__ void split3(float x, float y, uint32_t* t1, uint32_t* t2, uint32_t* t3) {
-    const uint32_t a = pack_bf16(x, y);
-    const float rx = x - lo_f(a), ry = y - hi_f(a);
-    const uint32_t b = pack_bf16(rx, ry);
-    *t1 = a;
-    *t2 = b;
-    *t3 = pack_bf16(rx - lo_f(b), ry - hi_f(b));
 }
 // All worker threads take a decision together (named barrier 1).
 __device__ __forceinline__ bool workers_all(bool mine) {
