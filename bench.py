@@ -45,8 +45,8 @@ ONE_TILE_SOURCES = ['gc_api.cu', 'gc_internal.h', 'gc_small.cu', 'tc_common.cuh'
 NCU_STEP_TRAFFIC = {
     "cfg2_": (82.9e6, SWEEP_SOURCES, "84483f8f278705562c0aa3af6042063f4047ab83"),
     "cfg4_": (4.80e9, SWEEP_SOURCES, "84483f8f278705562c0aa3af6042063f4047ab83"),
-    "cfg1_": (0.626e6, ONE_TILE_SOURCES, "8220e2b8fc15f752c1e880c89b323cd0306d2cac"),
-    "cfg0_": (0.639e6, ONE_TILE_SOURCES, "8220e2b8fc15f752c1e880c89b323cd0306d2cac"),
+    "cfg1_": (0.626e6, ONE_TILE_SOURCES, "d537a05746f7d575fcdb3d7bd527b6d963c777b6"),
+    "cfg0_": (0.638e6, ONE_TILE_SOURCES, "d537a05746f7d575fcdb3d7bd527b6d963c777b6"),
 }
 FP32_LANES_PER_SM = 128           # fp32 FMA lanes of one SM (2 FLOP per lane and clock)
 

@@ -15,8 +15,8 @@
 // terms x = t1 + t2 + t3 (each the upper 16 bits of what the previous ones left, so the sum is
 // exact) as it arrives, S takes the six products t1 t1', t1 t2', t1 t3', t2 t1', t2 t2', t3 t1'
 // in fp32 accumulation (spread over three accumulators, see the MMA warp), the weights are kept
-// as two terms and the gradient products take w1 t1 + w1 t2 + w2 t1.  Every mbarrier wait is
-// bounded.
+// as two terms and the gradient products take w1 (t1 + t2 + t3) + w2 (t1 + t2).  Every mbarrier
+// wait is bounded.
 #include "tc_common.cuh"
 
 namespace gc {
@@ -280,11 +280,12 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
         if (ok && do_grad) {
             tc_fence_after();
             if (elect_one()) {
-                // products (weight term, operand term): fp32 inputs take w1 t1, w1 t2, w2 t1
-                constexpr int NPROD_G = F32 ? 3 : 1;
+                // products (weight term, operand term): fp32 inputs take w1 t1, w1 t2, w1 t3, w2 t1,
+                // w2 t2 (the terms are truncations: dropping t3 would leave a one-sided 2^-16)
+                constexpr int NPROD_G = F32 ? 5 : 1;
                 constexpr uint32_t T = TILE >> 4;
-                const uint32_t w_term[3] = {0u, 0u, 2 * T};        // lo weights: 2 chunks further
-                const uint32_t o_term[3] = {0u, T, 0u};
+                const uint32_t w_term[5] = {0u, 0u, 0u, 2 * T, 2 * T};   // lo weights: 2 chunks further
+                const uint32_t o_term[5] = {0u, T, 2 * T, 0u, T};
                 // dQ slice: contraction over passages, 64 per weight chunk
                 bool first = true;
                 for (int c = 0; c < nchunks; ++c) {
