@@ -42,6 +42,10 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored) {
         pl.g_dq = simt_sweep_groups(B, N, d);
         pl.g_dp = simt_sweep_groups(N, B, d);
     }
+    // fp32 batches of a few tiles: the one-tile tcgen05 kernel per tile pair (gc_small.cu); its
+    // slots and partial planes share the regions of the plan it replaces
+    pl.tiles = small_tiled_applicable(B, N, d, dtype) ? 1 : 0;
+    const int tiles_x = pl.tiles ? small_tiles_x(B) : 0, tiles_y = pl.tiles ? small_tiles_y(N) : 0;
     pl.fused = (pl.tc && tc_fused_applicable(d)) ? 1 : 0;
     // 1: four-CTA sweeps (rows of two column halves); 2: narrow rows (two S buffers)
     pl.anchored = (pl.fused && quad_applicable(B, d)) ? 1
@@ -53,16 +57,19 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored) {
     if (pl.fused && (size_t)(2 * pl.g_dq) > slots) slots = (size_t)(2 * pl.g_dq);
     if (pl.anchored == 1 && (size_t)(4 * pl.g_dq) > slots) slots = (size_t)(4 * pl.g_dq);
     if (pl.anchored == 2 && (size_t)(4 * pl.g_dq) > slots) slots = (size_t)(4 * pl.g_dq);
+    if ((size_t)tiles_y > slots) slots = (size_t)tiles_y;
+    const int planes_q = pl.g_dq > tiles_y ? pl.g_dq : tiles_y;
+    const int planes_p = pl.g_dp > tiles_x ? pl.g_dp : tiles_x;
     size_t off = 0;
     pl.off_m = off;    off += align256(sizeof(float) * slots * (size_t)B);
     pl.off_l = off;    off += align256(sizeof(float) * slots * (size_t)B);
     pl.off_pos = off;  off += align256(sizeof(float) * (size_t)B);
     pl.off_red = off;  off += 2048;      // loss reduction: block ticket + up to 256 block sums
     pl.off_accq = off;
-    if (pl.g_dq > 1 || pl.fused || pl.anchored)
-        off += align256(sizeof(float) * (size_t)pl.g_dq * (size_t)B * dpad);
+    if (planes_q > 1 || pl.fused || pl.anchored)
+        off += align256(sizeof(float) * (size_t)planes_q * (size_t)B * dpad);
     pl.off_accp = off;
-    if (pl.g_dp > 1) off += align256(sizeof(float) * (size_t)pl.g_dp * (size_t)N * dpad);
+    if (planes_p > 1) off += align256(sizeof(float) * (size_t)planes_p * (size_t)N * dpad);
     pl.launches_fwd = 2;  // sweep + combine
     pl.launches_bwd = 2 + (pl.g_dq > 1 ? 1 : 0) + (pl.g_dp > 1 ? 1 : 0);
     pl.launches_build = pl.fused ? 4 + (pl.g_dp > 1 ? 1 : 0) : pl.launches_fwd + pl.launches_bwd;
@@ -528,6 +535,47 @@ int run_small(int op, const Problem& p, const float* row_lse_in, float* loss, fl
                         st) == cudaSuccess ? GC_OK : GC_ERR_CUDA;
 }
 
+// fp32 batches of a few tiles (gc_small.cu): forward = tile kernel + combine, gradients = tile
+// kernel + one reduce per side that has several planes.
+int run_tiles_fwd(const Problem& p, const Plan& pl, char* ws, float* loss, float* row_lse,
+                  float* pos_logit, int* dev_status, cudaStream_t st) {
+    float* part_m = reinterpret_cast<float*>(ws + pl.off_m);
+    float* part_l = reinterpret_cast<float*>(ws + pl.off_l);
+    float* pos_ws = reinterpret_cast<float*>(ws + pl.off_pos);
+    float* red = reinterpret_cast<float*>(ws + pl.off_red);
+    cudaError_t e;
+    {
+        KernelTimer t(0, st);
+        e = launch_small_tiled_fwd(p, part_m, part_l, pos_ws, red, dev_status, st);
+    }
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    e = launch_lse_combine(part_m, part_l, pos_ws, p.pos_idx, small_tiles_y(p.N), p.B, p.N,
+                           p.mask_mode, row_lse, pos_logit, loss, red, dev_status, kOpen, st,
+                           p.b_total, p.mask_shift);
+    return e == cudaSuccess ? GC_OK : GC_ERR_CUDA;
+}
+
+int run_tiles_bwd(const Problem& p, const Plan& pl, char* ws, const float* row_lse, float* dQ,
+                  int64_t lddq, float* dP, int64_t lddp, int* dev_status, cudaStream_t st) {
+    float* partial_q = reinterpret_cast<float*>(ws + pl.off_accq);
+    float* partial_p = reinterpret_cast<float*>(ws + pl.off_accp);
+    cudaError_t e;
+    {
+        KernelTimer t(1, st);
+        e = launch_small_tiled_bwd(p, row_lse, dQ, lddq, partial_q, dP, lddp, partial_p, dev_status,
+                                   st);
+    }
+    if (e != cudaSuccess) return GC_ERR_CUDA;
+    const int tx = small_tiles_x(p.B), ty = small_tiles_y(p.N);
+    if (dQ && ty > 1 &&
+        launch_partial_reduce(partial_q, ty, p.B, p.d, grad_scale(p), dQ, lddq, kOpen, st) != cudaSuccess)
+        return GC_ERR_CUDA;
+    if (dP && tx > 1 &&
+        launch_partial_reduce(partial_p, tx, p.N, p.d, grad_scale(p), dP, lddp, kOpen, st) != cudaSuccess)
+        return GC_ERR_CUDA;
+    return GC_OK;
+}
+
 }  // namespace
 
 // Scratch for gc_loss_fwd_static.  In host code this name is only a handle for the symbol: the
@@ -539,10 +587,12 @@ namespace {
 // The forward sweep alone writes g_fwd (scale, sum) slots per row: lays those regions, the
 // gathered positive logits and the loss scratch out back to back (the workspace layout of the
 // other calls reserves the slots of the widest build plan) and returns the bytes they take.
-size_t forward_layout(Plan* pl, int64_t B) {
+size_t forward_layout(Plan* pl, int64_t B, int64_t N) {
+    size_t slots = (size_t)pl->g_fwd;
+    if (pl->tiles && (size_t)small_tiles_y(N) > slots) slots = (size_t)small_tiles_y(N);
     size_t off = 0;
-    pl->off_m = off;    off += align256(sizeof(float) * (size_t)pl->g_fwd * (size_t)B);
-    pl->off_l = off;    off += align256(sizeof(float) * (size_t)pl->g_fwd * (size_t)B);
+    pl->off_m = off;    off += align256(sizeof(float) * slots * (size_t)B);
+    pl->off_l = off;    off += align256(sizeof(float) * slots * (size_t)B);
     pl->off_pos = off;  off += align256(sizeof(float) * (size_t)B);
     pl->off_red = off;  off += 2048;
     return off;
@@ -583,12 +633,19 @@ const char* gc_plan_name(int op, int64_t B, int64_t N, int d, int dtype) {
     if (op < GC_OP_FWD || op > GC_OP_BUILD_STORED || B <= 0 || N <= 0 || d <= 0) return "invalid";
     if (op == GC_OP_BUILD_STORED && !make_plan(B, N, d, dtype, true).mat) return "invalid";
     if (op != GC_OP_BUILD_STORED && small_applicable(B, N, d, dtype)) return "tcgen05-one-tile";
+    if (op != GC_OP_BUILD_STORED && small_tiled_applicable(B, N, d, dtype)) return "tcgen05-tiles";
     return tc_supported(B, N, d, dtype) ? "tcgen05" : "simt";
 }
 
 int gc_kernel_launches(int op, int64_t B, int64_t N, int d, int dtype) {
     if (B <= 0 || N <= 0 || d <= 0) return 0;
     if (op >= GC_OP_FWD && op <= GC_OP_BUILD && small_applicable(B, N, d, dtype)) return 1;
+    if (op >= GC_OP_FWD && op <= GC_OP_BUILD && small_tiled_applicable(B, N, d, dtype)) {
+        const int reduces = (small_tiles_y(N) > 1 ? 1 : 0) + (small_tiles_x(B) > 1 ? 1 : 0);
+        if (op == GC_OP_FWD) return 2;                  // tile kernel, combine
+        if (op == GC_OP_BWD) return 2 + reduces;        // pos_idx validation, tile kernel, reduces
+        return 3 + reduces;
+    }
     Plan pl = make_plan(B, N, d, dtype);
     if (op == GC_OP_FWD) return pl.launches_fwd;
     if (op == GC_OP_BWD) return pl.launches_bwd + 1;   // + pos_idx validation
@@ -612,6 +669,9 @@ int gc_loss_fwd(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
     if (small_applicable(B, N, d, dtype))
         return run_small(GC_OP_FWD, p, nullptr, loss, row_lse, pos_logit, nullptr, 0, nullptr, 0,
                          dev_status, static_cast<cudaStream_t>(cuda_stream));
+    if (pl.tiles)
+        return run_tiles_fwd(p, pl, static_cast<char*>(ws), loss, row_lse, pos_logit, dev_status,
+                             static_cast<cudaStream_t>(cuda_stream));
     return run_fwd(p, pl, static_cast<char*>(ws), loss, row_lse, pos_logit, dev_status,
                    static_cast<cudaStream_t>(cuda_stream));
 }
@@ -619,7 +679,7 @@ int gc_loss_fwd(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
 size_t gc_static_scratch_need(int64_t B, int64_t N, int d, int dtype) {
     if (B <= 0 || N <= 0 || d <= 0 || (dtype != GC_F32 && dtype != GC_BF16)) return 0;
     Plan pl = make_plan(B, N, d, dtype);
-    return forward_layout(&pl, B);
+    return forward_layout(&pl, B, N);
 }
 
 int gc_loss_fwd_static(const void* Q, int64_t ldq, const void* P, int64_t ldp,
@@ -630,7 +690,7 @@ int gc_loss_fwd_static(const void* Q, int64_t ldq, const void* P, int64_t ldp,
     if (rc) return rc;
     if (!loss || !row_lse) return GC_ERR_NULL;
     Plan pl = make_plan(B, N, d, dtype);
-    if (forward_layout(&pl, B) > (size_t)GC_STATIC_SCRATCH_BYTES) return GC_ERR_LIMIT;
+    if (forward_layout(&pl, B, N) > (size_t)GC_STATIC_SCRATCH_BYTES) return GC_ERR_LIMIT;
     if ((rc = check_device())) return rc;
     void* scratch = static_scratch_ptr();
     if (!scratch) return GC_ERR_CUDA;
@@ -639,6 +699,9 @@ int gc_loss_fwd_static(const void* Q, int64_t ldq, const void* P, int64_t ldp,
     if (small_applicable(B, N, d, dtype))      // one launch, no scratch at all
         return run_small(GC_OP_FWD, p, nullptr, loss, row_lse, pos_logit, nullptr, 0, nullptr, 0,
                          dev_status, static_cast<cudaStream_t>(cuda_stream));
+    if (pl.tiles)
+        return run_tiles_fwd(p, pl, static_cast<char*>(scratch), loss, row_lse, pos_logit,
+                             dev_status, static_cast<cudaStream_t>(cuda_stream));
     return run_fwd(p, pl, static_cast<char*>(scratch), loss, row_lse, pos_logit, dev_status,
                    static_cast<cudaStream_t>(cuda_stream));
 }
@@ -664,6 +727,8 @@ int gc_loss_bwd(const void* Q, int64_t ldq, const void* P, int64_t ldp, const in
     if (dev_status && launch_pos_check(pos_idx, B, N, mask_mode, dev_status, st) != cudaSuccess)
         return GC_ERR_CUDA;
     char* w = static_cast<char*>(ws);
+    if (pl.tiles && (dQ || dP))
+        return run_tiles_bwd(p, pl, w, row_lse, dQ, lddq, dP, lddp, dev_status, st);
     if (dQ && (rc = run_sweep(p, pl, w, SWEEP_DQ, row_lse, dQ, lddq, dev_status, st))) return rc;
     if (dP && (rc = run_sweep(p, pl, w, SWEEP_DP, row_lse, dP, lddp, dev_status, st))) return rc;
     return GC_OK;
@@ -688,6 +753,10 @@ int gc_build_cache(const void* Q, int64_t ldq, const void* P, int64_t ldp, const
     if (small_applicable(B, N, d, dtype))
         return run_small(GC_OP_BUILD, p, nullptr, loss, row_lse, pos_logit, dQ, lddq, dP, lddp,
                          dev_status, st);
+    if (pl.tiles) {
+        if ((rc = run_tiles_fwd(p, pl, w, loss, row_lse, pos_logit, dev_status, st))) return rc;
+        return run_tiles_bwd(p, pl, w, row_lse, dQ, lddq, dP, lddp, dev_status, st);
+    }
     return run_build_sweeps(p, pl, w, loss, row_lse, pos_logit, dQ, lddq, dP, lddp, dev_status, st);
 }
 

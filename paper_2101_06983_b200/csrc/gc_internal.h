@@ -111,6 +111,7 @@ struct FwdArgs {
 // How one call is carried out for given sizes on the current device.
 struct Plan {
     int tc;                 // 1: tcgen05 kernels, 0: SIMT kernels
+    int tiles;              // 1: fp32 batch of a few tiles on the one-tile tcgen05 kernel
     int g_fwd, g_dq, g_dp;  // split factors of the streamed range
     size_t off_m, off_l, off_pos, off_red, off_accq, off_accp;
     size_t total;           // workspace bytes (multiple of 256)
@@ -193,6 +194,15 @@ bool small_applicable(int64_t B, int64_t N, int d, int dtype);
 cudaError_t launch_small(int op, const Problem& pr, const float* row_lse_in, float* loss,
                          float* row_lse, float* pos_logit, float* dQ, int64_t lddq, float* dP,
                          int64_t lddp, int* dev_status, cudaStream_t st);
+
+bool small_tiled_applicable(int64_t B, int64_t N, int d, int dtype);
+int small_tiles_x(int64_t B);
+int small_tiles_y(int64_t N);
+cudaError_t launch_small_tiled_fwd(const Problem& pr, float* part_m, float* part_l, float* pos_ws,
+                                   float* red, int* dev_status, cudaStream_t st);
+cudaError_t launch_small_tiled_bwd(const Problem& pr, const float* row_lse, float* dQ, int64_t lddq,
+                                   float* partial_q, float* dP, int64_t lddp, float* partial_p,
+                                   int* dev_status, cudaStream_t st);
 
 // gc_gemm.cu
 int gemm_groups(int64_t m_rows, int64_t k_len, int d);

@@ -47,10 +47,22 @@ struct SmallParams {
     int mask_mode;
     int mask_shift;           // masked pair: j == i + mask_shift
     float scale2;             // log2(e) / tau
+    float inv_tau;
     float out_scale;          // 1 / (B tau)
     float inv_mean;           // 1 / B
     const int32_t* pos_idx;
     const float* row_lse_in;  // GC_OP_BWD
+    // Several tiles (grid y = query tiles of 128, grid z = passage tiles): the forward writes one
+    // (max, sum) slot per passage tile and row, slot t at [t * B + i] (natural-log units), and the
+    // positive's logit, for the combine kernel that follows; the gradients of a tile pair go to
+    // plane (passage tile) of the dQ partials and plane (query tile) of the dP partials.
+    int tiled;
+    int plane_q, plane_p;     // the gradient of that side goes to a plane of partials
+    float out_scale_q, out_scale_p;
+    float* part_m;
+    float* part_l;
+    float* pos_ws;
+    int* zero_me;             // block ticket of the loss reduction that follows: cleared here
     float* loss;
     float* row_lse;
     float* pos_logit;         // may be NULL
@@ -100,11 +112,6 @@ __device__ __forceinline__ bool workers_all(bool mine) {
         : "=r"(all) : "r"(mine ? 1u : 0u), "n"(32 * SM_WORKERS) : "memory");
     return all != 0;
 }
-__device__ __forceinline__ float lg2(float x) {
-    float y;
-    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
 // 32 columns of this thread's row of S; fp32 inputs keep S as the sum of three accumulators.
 template <bool F32>
 __device__ __forceinline__ void load_s(uint32_t trow, int jb, float (&s)[32]) {
@@ -143,13 +150,17 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
     const int lane = threadIdx.x & 31;
     const int slice = blockIdx.x;
     const bool do_grad = p.op != GC_OP_FWD;
+    // this CTA's tile pair: rows x0 .. of Q, rows y0 .. of P; B_ and N_ are the rows it holds
+    constexpr int YT = F32 ? 128 : 256;
+    const int x0 = 128 * (int)blockIdx.y, y0 = YT * (int)blockIdx.z;
+    const int B_ = min(128, p.B - x0), N_ = min(YT, p.N - y0);
     // steps of the S loop: 64 columns (bf16) or 32 columns (fp32, an even number of them so that
     // a slice's first half always lands in the first half of the term tiles; a step past d reads
     // zeros); then the CTA's own slice
     const int s_steps = F32 ? 2 * ((p.d + 63) / 64) : (p.d + 63) / 64;
     const int g_steps = do_grad ? (F32 ? 2 : 1) : 0;
-    const int n_pad = (p.N + 15) & ~15;
-    const int ptiles = p.N > 128 ? 2 : 1;
+    const int n_pad = (N_ + 15) & ~15;
+    const int ptiles = N_ > 128 ? 2 : 1;
 
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     constexpr uint32_t STAGE = F32 ? F32_STAGE : BF_STAGE;
@@ -196,13 +207,13 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
             if (elect_one()) {
                 if (F32) {
                     mbar_expect_tx(full, 2 * TILE);
-                    tma_load_2d(dst, &mapQ, col, 0, full);
-                    tma_load_2d(dst + TILE, &mapP, col, 0, full);
+                    tma_load_2d(dst, &mapQ, col, x0, full);
+                    tma_load_2d(dst + TILE, &mapP, col, y0, full);
                 } else {
                     mbar_expect_tx(full, (uint32_t)(1 + ptiles) * TILE);
-                    tma_load_2d(dst, &mapQ, col, 0, full);
-                    tma_load_2d(dst + TILE, &mapP, col, 0, full);
-                    if (ptiles == 2) tma_load_2d(dst + 2 * TILE, &mapP, col, 128, full);
+                    tma_load_2d(dst, &mapQ, col, x0, full);
+                    tma_load_2d(dst + TILE, &mapP, col, y0, full);
+                    if (ptiles == 2) tma_load_2d(dst + 2 * TILE, &mapP, col, y0 + 128, full);
                 }
             }
             if (++stage == SM_STAGES) { stage = 0; phase ^= 1u; }
@@ -212,7 +223,7 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
         const uint32_t idesc_s = instr_desc(n_pad, false, XROWS, false);
         const uint32_t idesc_dq = instr_desc(64, true, XROWS, false);    // A = W, K-major
         const uint32_t idesc_dp = instr_desc(64, true, XROWS, true);     // A = W^T: MN-major
-        const int nchunks = (p.N + 63) / 64;
+        const int nchunks = (N_ + 63) / 64;
         bool ok = true;
         uint32_t q_tile = 0, p_tile = 0;       // the CTA's own slices as MN-major B operands
         if (F32) {
@@ -352,7 +363,7 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
                     const int cp = id & 3, rr = (id >> 2) & 1, b = (id >> 3) & 3, a = (id >> 5) & 15;
                     const int mat = id >> 9;
                     const int r = 8 * a + b + 4 * rr, sw = r & 7;
-                    if (r >= (mat ? p.N : p.B)) continue;
+                    if (r >= (mat ? N_ : B_)) continue;
                     const uint32_t src = src0 + mat * TILE + r * 128;
                     const int first = (2 * cp) ^ rr;
                     const float4 A = lds128f(src + (uint32_t)((first ^ sw) << 4));
@@ -396,47 +407,50 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
             const int ncols = F32 ? 128 : 256;
             const int j0 = half * (ncols / 2);                    // fp32: 0 or 64; bf16: 0 or 128
             const int nblk = ncols / 64;                          // blocks of 32 columns per half
-            const int32_t r_i = i < p.B ? p.pos_idx[i] : -1;
+            // columns are counted within the tile: the positive and the masked pair of row i fall
+            // into it or not
+            const int32_t r_i = i < B_ ? p.pos_idx[x0 + i] : -1;
             int flags = 0;
-            if (i < p.B) {
+            if (i < B_) {
                 if (r_i < 0 || r_i >= p.N) flags = GC_DEV_POS_RANGE;
-                else if (p.mask_mode == GC_MASK_SELF && r_i == i + p.mask_shift) flags = GC_DEV_POS_MASKED;
+                else if (p.mask_mode == GC_MASK_SELF && r_i == x0 + i + p.mask_shift) flags = GC_DEV_POS_MASKED;
             }
-            const int pos = flags ? -1 : r_i;
-            const int masked = p.mask_mode == GC_MASK_SELF ? i + p.mask_shift : -1;
-            float lse2, pos2 = 0.f;
+            const int pos = (flags || r_i < y0 || r_i >= y0 + N_) ? -1 : r_i - y0;
+            const int masked = p.mask_mode == GC_MASK_SELF ? x0 + i + p.mask_shift - y0 : -1;
+            float lse2, pos2 = 0.f, lse_nat = 0.f, m_row = 0.f, lnsum_row = 0.f;
             if (p.op == GC_OP_BWD) {
-                lse2 = p.row_lse_in[i < p.B ? i : 0] * 1.4426950408889634f;
+                lse2 = p.row_lse_in[i < B_ ? x0 + i : 0] * 1.4426950408889634f;
             } else {
-                float m = -INFINITY, sum = 0.f;
+                // The running maximum is kept in units of <q, p> (unscaled), so that the row's
+                // logsumexp and its positive logit come out of the same product with 1/tau:
+                // lse_i - S_{i,r_i} is exactly 0 when the positive is the only column.
+                float m = -INFINITY, sum = 0.f, lnsum = 0.f;
                 for (int cb = 0; cb < nblk; ++cb) {
                     const int jb = j0 + 32 * cb;
-                    if (jb >= p.N) break;
-                    float s2[32];
-                    load_s<F32>(tmem + lane_addr, jb, s2);
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) s2[e] *= p.scale2;
+                    if (jb >= N_) break;
+                    float sr[32];
+                    load_s<F32>(tmem + lane_addr, jb, sr);
                     if ((unsigned)(pos - jb) < 32u) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) if (e == pos - jb) pos2 = s2[e];
+                        for (int e = 0; e < 32; ++e) if (e == pos - jb) pos2 = sr[e];
                     }
                     if ((unsigned)(masked - jb) < 32u) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) if (e == masked - jb) s2[e] = -INFINITY;
+                        for (int e = 0; e < 32; ++e) if (e == masked - jb) sr[e] = -INFINITY;
                     }
-                    if (jb + 32 > p.N) {
+                    if (jb + 32 > N_) {
 #pragma unroll
-                        for (int e = 0; e < 32; ++e) if (jb + e >= p.N) s2[e] = -INFINITY;
+                        for (int e = 0; e < 32; ++e) if (jb + e >= N_) sr[e] = -INFINITY;
                     }
-                    float bm = s2[0];
+                    float bm = sr[0];
 #pragma unroll
-                    for (int e = 1; e < 32; ++e) bm = fmaxf(bm, s2[e]);
+                    for (int e = 1; e < 32; ++e) bm = fmaxf(bm, sr[e]);
                     const float mn = fmaxf(m, bm);
                     const float ref = mn == -INFINITY ? 0.f : mn;
-                    float part = 0.f;
+                    float part = 0.f;      // (s - max) first: the largest term is exactly 2^0
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) part += ex2(s2[e] - ref);
-                    sum = sum * ex2(m - ref) + part;
+                    for (int e = 0; e < 32; ++e) part += ex2((sr[e] - ref) * p.scale2);
+                    sum = sum * ex2((m - ref) * p.scale2) + part;
                     m = mn;
                 }
                 x_max[half][i] = m;
@@ -445,19 +459,35 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
                 workers_sync();
                 const float m0 = x_max[0][i], m1 = x_max[1][i];
                 m = fmaxf(m0, m1);
-                sum = x_sum[0][i] * ex2(m0 - m) + x_sum[1][i] * ex2(m1 - m);
+                const float mref = m == -INFINITY ? 0.f : m;                // all columns masked
+                sum = x_sum[0][i] * ex2((m0 - mref) * p.scale2) +
+                      x_sum[1][i] * ex2((m1 - mref) * p.scale2);
                 pos2 = x_pos[0][i] + x_pos[1][i];                 // the other half holds 0
-                lse2 = m + lg2(sum);
+                const float lg = log2f(sum);          // once per row: the accurate one
+                lse2 = m * p.scale2 + lg;
+                lnsum = lg * 0.6931471805599453f;
+                if (p.tiled) {
+                    // one slot per passage tile; the combine kernel merges them
+                    if (half == 0 && i < B_) {
+                        p.part_m[(int64_t)blockIdx.z * p.B + x0 + i] = m * p.inv_tau;
+                        p.part_l[(int64_t)blockIdx.z * p.B + x0 + i] = sum;
+                        if (pos >= 0) p.pos_ws[x0 + i] = pos2 * p.inv_tau;
+                    }
+                    if (blockIdx.y == 0 && blockIdx.z == 0 && wt == 0 && p.zero_me) *p.zero_me = 0;
+                }
+                lse_nat = m * p.inv_tau + lnsum;
+                m_row = m;
+                lnsum_row = lnsum;
             }
             // ------------------------------ outputs of the forward (CTA 0) ------------------------
-            if (slice == 0) {
-                const float ln2 = 0.6931471805599453f;
+            if (slice == 0 && !p.tiled) {
                 float term = 0.f;
-                if (half == 0 && i < p.B) {
+                if (half == 0 && i < B_) {
                     if (p.op != GC_OP_BWD) {
-                        p.row_lse[i] = lse2 * ln2;
-                        if (p.pos_logit) p.pos_logit[i] = pos2 * ln2;
-                        term = (lse2 - pos2) * ln2;
+                        const float pl = pos2 * p.inv_tau;
+                        p.row_lse[i] = lse_nat;
+                        if (p.pos_logit) p.pos_logit[i] = pl;
+                        term = (m_row - pos2) * p.inv_tau + lnsum_row;   // no cancellation of two roundings
                     }
                     if (flags && p.dev_status) atomicOr(p.dev_status, flags);
                 }
@@ -475,12 +505,12 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
                 // chunk c = 64 columns; element (i, j) in 16-byte piece ((j % 64) / 8) ^ (i % 8) of
                 // row i: a K-major A operand for dQ and, read by columns, an MN-major one for dP.
                 // Rows past B get lse = +inf: all their weights are 0.
-                const float neg_lse = i < p.B ? -lse2 : -INFINITY;
-                const int pos_w = i < p.B ? pos : -1;
+                const float neg_lse = i < B_ ? -lse2 : -INFINITY;
+                const int pos_w = i < B_ ? pos : -1;
                 for (int cb = 0; cb < nblk; ++cb) {
                     const int jb = j0 + 32 * cb;                  // 4 pieces of 8 columns
                     float w[32];
-                    if (jb < p.N) {
+                    if (jb < N_) {
                         load_s<F32>(tmem + lane_addr, jb, w);
 #pragma unroll
                         for (int e = 0; e < 32; ++e) w[e] = ex2(fmaf(w[e], p.scale2, neg_lse));
@@ -492,9 +522,9 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
 #pragma unroll
                             for (int e = 0; e < 32; ++e) if (e == pos_w - jb) w[e] -= 1.f;
                         }
-                        if (jb + 32 > p.N) {
+                        if (jb + 32 > N_) {
 #pragma unroll
-                            for (int e = 0; e < 32; ++e) if (jb + e >= p.N) w[e] = 0.f;
+                            for (int e = 0; e < 32; ++e) if (jb + e >= N_) w[e] = 0.f;
                         }
                     } else {
 #pragma unroll
@@ -533,7 +563,7 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
                     int n = 0;
                     for (int blk = 0; blk < 1 + ptiles; ++blk) {       // dQ, dP rows 0.., dP rows 128..
                         const int rows = blk == 0 ? p.B : p.N;
-                        const int row0 = (blk == 0 ? 0 : 128 * (blk - 1)) + 32 * q;
+                        const int row0 = (blk == 0 ? x0 : y0 + 128 * (blk - 1)) + 32 * q;
                         const bool have = blk == 0 ? p.dQ != nullptr : p.dP != nullptr;
                         if (!have || row0 >= rows || col >= p.d) continue;
                         uint32_t v[32];
@@ -545,9 +575,13 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
                         }
                         tmem_ld_wait();
                         const uint32_t buf = slot + (uint32_t)(n & 1) * 4096u;
-                        stage_block(buf, v, p.out_scale, lane);
+                        stage_block(buf, v, blk == 0 ? p.out_scale_q : p.out_scale_p, lane);
                         __syncwarp();
-                        if (lane == 0) tma_store_3d(blk == 0 ? &mapDQ : &mapDP, buf, col, row0, 0);
+                        // several tiles: plane = the tile of the other side (unscaled partials)
+                        if (lane == 0)
+                            tma_store_3d(blk == 0 ? &mapDQ : &mapDP, buf, col, row0,
+                                         blk == 0 ? (p.plane_q ? (int)blockIdx.z : 0)
+                                                  : (p.plane_p ? (int)blockIdx.y : 0));
                         ++n;
                     }
                     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
@@ -576,7 +610,7 @@ small_kernel(const __grid_constant__ CUtensorMap mapQ, const __grid_constant__ C
 
 template <bool F32>
 cudaError_t launch_small_t(const CUtensorMap& mq, const CUtensorMap& mp, const CUtensorMap& mdq,
-                           const CUtensorMap& mdp, const SmallParams& p, unsigned ctas,
+                           const CUtensorMap& mdp, const SmallParams& p, dim3 grid,
                            cudaStream_t st) {
     static bool configured_on[64] = {false};      // the attribute belongs to (kernel, device)
     int dev = 0;
@@ -588,7 +622,7 @@ cudaError_t launch_small_t(const CUtensorMap& mq, const CUtensorMap& mp, const C
         if (e != cudaSuccess) return e;
         configured_on[dev] = true;
     }
-    small_kernel<F32><<<ctas, SM_THREADS, SM_DYN_SMEM, st>>>(mq, mp, mdq, mdp, p);
+    small_kernel<F32><<<grid, SM_THREADS, SM_DYN_SMEM, st>>>(mq, mp, mdq, mdp, p);
     return cudaGetLastError();
 }
 
@@ -621,17 +655,100 @@ cudaError_t launch_small(int op, const Problem& pr, const float* row_lse_in, flo
     p.mask_mode = pr.mask_mode;
     p.mask_shift = (int)pr.mask_shift;
     p.scale2 = 1.4426950408889634f / pr.tau;
+    p.inv_tau = 1.f / pr.tau;
     const float batch = (float)(pr.b_total > 0 ? pr.b_total : pr.B);
     p.out_scale = 1.f / (batch * pr.tau);
+    p.out_scale_q = p.out_scale_p = p.out_scale;
     p.inv_mean = 1.f / batch;
     p.pos_idx = pr.pos_idx;
     p.row_lse_in = row_lse_in;
     p.loss = loss; p.row_lse = row_lse; p.pos_logit = pos_logit;
     p.dQ = dQ; p.lddq = lddq; p.dP = dP; p.lddp = lddp;
     p.dev_status = dev_status;
-    const unsigned ctas = op == GC_OP_FWD ? 1u : (unsigned)((pr.d + 63) / 64);
-    return f32 ? launch_small_t<true>(mq, mp, mdq, mdp, p, ctas, st)
-               : launch_small_t<false>(mq, mp, mdq, mdp, p, ctas, st);
+    const dim3 grid(op == GC_OP_FWD ? 1u : (unsigned)((pr.d + 63) / 64));
+    return f32 ? launch_small_t<true>(mq, mp, mdq, mdp, p, grid, st)
+               : launch_small_t<false>(mq, mp, mdq, mdp, p, grid, st);
+}
+
+// fp32 batches of a few tiles (query tiles of 128 x passage tiles of 128) run the same kernel
+// once per tile pair and column slice: the forward launch leaves one (max, sum) slot per passage
+// tile and row for the combine kernel, the gradient launch (row_lse given) writes every tile
+// pair's slices as planes of partial sums that a reduce kernel adds in index order.  Every CTA
+// of a tile pair forms that pair's logits, so the work grows with d / 64: a plan for batches
+// where launches, not arithmetic, set the time.
+bool small_tiled_applicable(int64_t B, int64_t N, int d, int dtype) {
+    if (dtype != GC_F32 || d % 8 != 0 || d > 4096 || small_applicable(B, N, d, dtype)) return false;
+    const int64_t xt = (B + 127) / 128, yt = (N + 127) / 128;
+    return xt * yt <= 64 && xt * yt * ((d + 63) / 64) <= 2048;
+}
+int small_tiles_x(int64_t B) { return (int)((B + 127) / 128); }
+int small_tiles_y(int64_t N) { return (int)((N + 127) / 128); }
+
+// Forward of the tiled plan: slots part_m / part_l [tiles_y][B], pos_ws [B]; `red` is the scratch
+// of the combine kernel that follows.
+cudaError_t launch_small_tiled_fwd(const Problem& pr, float* part_m, float* part_l, float* pos_ws,
+                                   float* red, int* dev_status, cudaStream_t st) {
+    CUtensorMap mq, mp;
+    if (!make_map_f32(&mq, pr.Q, pr.B, pr.d, pr.ldq, 128) ||
+        !make_map_f32(&mp, pr.P, pr.N, pr.d, pr.ldp, 128))
+        return cudaErrorInvalidValue;
+    SmallParams p{};
+    p.B = (int)pr.B; p.N = (int)pr.N; p.d = pr.d;
+    p.op = GC_OP_FWD;
+    p.mask_mode = pr.mask_mode;
+    p.mask_shift = (int)pr.mask_shift;
+    p.scale2 = 1.4426950408889634f / pr.tau;
+    p.inv_tau = 1.f / pr.tau;
+    p.pos_idx = pr.pos_idx;
+    p.tiled = 1;
+    p.part_m = part_m; p.part_l = part_l; p.pos_ws = pos_ws;
+    p.zero_me = reinterpret_cast<int*>(red);
+    p.dev_status = dev_status;
+    const dim3 grid(1u, (unsigned)small_tiles_x(pr.B), (unsigned)small_tiles_y(pr.N));
+    return launch_small_t<true>(mq, mp, mq, mp, p, grid, st);
+}
+
+// Gradients of the tiled plan from row_lse.  With one passage tile dQ is final (scaled) in dQ,
+// otherwise plane t of partial_q [tiles_y][B][d] holds passage tile t's unscaled share; likewise
+// dP / partial_p [tiles_x][N][d].  Either output may be NULL.
+cudaError_t launch_small_tiled_bwd(const Problem& pr, const float* row_lse, float* dQ, int64_t lddq,
+                                   float* partial_q, float* dP, int64_t lddp, float* partial_p,
+                                   int* dev_status, cudaStream_t st) {
+    const int xt = small_tiles_x(pr.B), yt = small_tiles_y(pr.N);
+    CUtensorMap mq, mp;
+    if (!make_map_f32(&mq, pr.Q, pr.B, pr.d, pr.ldq, 128) ||
+        !make_map_f32(&mp, pr.P, pr.N, pr.d, pr.ldp, 128))
+        return cudaErrorInvalidValue;
+    CUtensorMap mdq = mq, mdp = mp;
+    if (dQ) {
+        const bool ok = yt == 1 ? make_out_map(&mdq, dQ, pr.B, pr.d, lddq, 1)
+                                : make_out_map(&mdq, partial_q, pr.B, pr.d, pr.d, yt);
+        if (!ok) return cudaErrorInvalidValue;
+    }
+    if (dP) {
+        const bool ok = xt == 1 ? make_out_map(&mdp, dP, pr.N, pr.d, lddp, 1)
+                                : make_out_map(&mdp, partial_p, pr.N, pr.d, pr.d, xt);
+        if (!ok) return cudaErrorInvalidValue;
+    }
+    SmallParams p{};
+    p.B = (int)pr.B; p.N = (int)pr.N; p.d = pr.d;
+    p.op = GC_OP_BWD;
+    p.mask_mode = pr.mask_mode;
+    p.mask_shift = (int)pr.mask_shift;
+    p.scale2 = 1.4426950408889634f / pr.tau;
+    p.inv_tau = 1.f / pr.tau;
+    const float batch = (float)(pr.b_total > 0 ? pr.b_total : pr.B);
+    p.out_scale = 1.f / (batch * pr.tau);          // planes are scaled by the reduce kernel
+    p.out_scale_q = yt == 1 ? p.out_scale : 1.f;
+    p.out_scale_p = xt == 1 ? p.out_scale : 1.f;
+    p.pos_idx = pr.pos_idx;
+    p.row_lse_in = row_lse;
+    p.dQ = dQ; p.lddq = lddq; p.dP = dP; p.lddp = lddp;
+    p.tiled = 1;
+    p.plane_q = yt > 1; p.plane_p = xt > 1;
+    p.dev_status = dev_status;
+    const dim3 grid((unsigned)((pr.d + 63) / 64), (unsigned)xt, (unsigned)yt);
+    return launch_small_t<true>(mq, mp, mdq, mdp, p, grid, st);
 }
 
 }  // namespace gc

@@ -112,3 +112,39 @@ def test_bad_positive_indices_raise_the_device_flags(binding):
     torch.cuda.synchronize()
     assert int(out.dev_status.item()) & 1           # GC_DEV_POS_RANGE
     assert bool(torch.isfinite(out.dQ).all()) and bool(torch.isfinite(out.dP).all())
+
+
+# fp32 batches of a few tiles: the same kernel once per tile pair and column slice
+TILED_F32 = [(129, 257, 72), (130, 130, 128), (200, 513, 192), (257, 1, 64), (65, 300, 768),
+             (300, 200, 320), (140, 270, 448), (129, 300, 1024), (260, 131, 1536), (70, 140, 4096),
+             (1000, 900, 64), (128, 129, 8), (129, 128, 8)]
+
+
+@pytest.mark.parametrize("B,N,d", TILED_F32)
+def test_fp32_batches_of_a_few_tiles(binding, oracle, B, N, d):
+    assert binding.gc_plan_name(binding.GC_OP_BUILD, B, N, d, binding.GC_F32) == "tcgen05-tiles"
+    prob = inputs.random_problem(B, N, d, "f32", seed=B * 1000 + N, tau=0.5, scale=0.5)
+    ref = _oracle_full(oracle, prob)
+    out = run_build(prob)
+    check_against_oracle(prob, out, ref)
+    again = run_build(prob)
+    assert torch.equal(out.dQ, again.dQ) and torch.equal(out.dP, again.dP)
+    # forward and backward as separate calls
+    Q, P, pos = to_device(prob)
+    b = binding.Outputs(prob.B, prob.N, prob.d, binding.GC_F32)
+    b.dQ.fill_(float("nan"))
+    b.dP.fill_(float("nan"))
+    binding.gc_loss_fwd(Q, P, pos, prob.tau, prob.mask_mode, b.loss, b.row_lse, b.pos_logit, b.ws,
+                        b.dev_status)
+    binding.gc_loss_bwd(Q, P, pos, prob.tau, prob.mask_mode, b.row_lse, b.dQ, b.dP, b.ws,
+                        b.dev_status)
+    torch.cuda.synchronize()
+    check_against_oracle(prob, b, ref)
+
+
+@pytest.mark.parametrize("n,d,tau", [(130, 64, 0.1), (257, 128, 0.1), (400, 72, 0.5)])
+def test_fp32_tiles_self_mask(binding, oracle, n, d, tau):
+    prob = inputs.random_problem(n, n, d, "f32", seed=n, tau=tau, mask_mode=inputs.MASK_SELF,
+                                 scale=d ** -0.5, shared=True)
+    out = run_build(prob)
+    check_against_oracle(prob, out, _oracle_full(oracle, prob))

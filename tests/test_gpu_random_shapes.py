@@ -1,7 +1,7 @@
 """Seeded random problem shapes through gc_build_cache against the CPU oracle, element by element:
 sizes drawn so that every plan is met (one-tile batches in bf16 and fp32, narrow and wide bf16
-rows with ragged tiles and split ranges, the four-CTA sweeps, the FMA-tile plan for fp32 beyond
-one tile and for widths that are not a multiple of 64), both mask modes, several temperatures.
+rows with ragged tiles and split ranges, the four-CTA sweeps, fp32 batches of a few tiles, the
+FMA-tile plan for widths that are not a multiple of 8), both mask modes, several temperatures.
 The shapes are fixed by the seed: the same forty-odd cases every run."""
 import numpy as np
 import pytest
@@ -65,8 +65,8 @@ def test_random_shape(binding, oracle, kind, dtype, B, N, d, mask, tau, seed):
     plan = binding.gc_plan_name(binding.GC_OP_BUILD, prob.B, prob.N, prob.d, code)
     if kind == "one-tile":
         assert plan == "tcgen05-one-tile"
-    if kind == "fma":
-        assert plan == "simt"
+    if kind == "fma":            # fp32 beyond one tile: tcgen05 per tile pair, or FMA tiles
+        assert plan == ("tcgen05-tiles" if prob.d % 8 == 0 else "simt")
     out = run_build(prob)
     ref = oracle.build_cache(prob.Q, prob.P, prob.pos_idx, prob.tau, prob.mask_mode)
     check_against_oracle(prob, out, ref)
