@@ -45,7 +45,8 @@ Plan make_plan(int64_t B, int64_t N, int d, int dtype, bool stored) {
     // fp32 batches of a few tiles: the one-tile tcgen05 kernel per tile pair (gc_small.cu); its
     // slots and partial planes share the regions of the plan it replaces
     pl.tiles = small_tiled_applicable(B, N, d, dtype) ? 1 : 0;
-    const int tiles_x = pl.tiles ? small_tiles_x(B) : 0, tiles_y = pl.tiles ? small_tiles_y(N) : 0;
+    pl.tiles_y = pl.tiles ? small_tiles_y(N, dtype) : 0;
+    const int tiles_x = pl.tiles ? small_tiles_x(B) : 0, tiles_y = pl.tiles ? small_tiles_y(N, dtype) : 0;
     pl.fused = (pl.tc && tc_fused_applicable(d)) ? 1 : 0;
     // 1: four-CTA sweeps (rows of two column halves); 2: narrow rows (two S buffers)
     pl.anchored = (pl.fused && quad_applicable(B, d)) ? 1
@@ -549,7 +550,7 @@ int run_tiles_fwd(const Problem& p, const Plan& pl, char* ws, float* loss, float
         e = launch_small_tiled_fwd(p, part_m, part_l, pos_ws, red, dev_status, st);
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
-    e = launch_lse_combine(part_m, part_l, pos_ws, p.pos_idx, small_tiles_y(p.N), p.B, p.N,
+    e = launch_lse_combine(part_m, part_l, pos_ws, p.pos_idx, small_tiles_y(p.N, p.dtype), p.B, p.N,
                            p.mask_mode, row_lse, pos_logit, loss, red, dev_status, kOpen, st,
                            p.b_total, p.mask_shift);
     return e == cudaSuccess ? GC_OK : GC_ERR_CUDA;
@@ -566,7 +567,7 @@ int run_tiles_bwd(const Problem& p, const Plan& pl, char* ws, const float* row_l
                                    st);
     }
     if (e != cudaSuccess) return GC_ERR_CUDA;
-    const int tx = small_tiles_x(p.B), ty = small_tiles_y(p.N);
+    const int tx = small_tiles_x(p.B), ty = small_tiles_y(p.N, p.dtype);
     if (dQ && ty > 1 &&
         launch_partial_reduce(partial_q, ty, p.B, p.d, grad_scale(p), dQ, lddq, kOpen, st) != cudaSuccess)
         return GC_ERR_CUDA;
@@ -589,7 +590,7 @@ namespace {
 // other calls reserves the slots of the widest build plan) and returns the bytes they take.
 size_t forward_layout(Plan* pl, int64_t B, int64_t N) {
     size_t slots = (size_t)pl->g_fwd;
-    if (pl->tiles && (size_t)small_tiles_y(N) > slots) slots = (size_t)small_tiles_y(N);
+    if (pl->tiles && (size_t)pl->tiles_y > slots) slots = (size_t)pl->tiles_y;
     size_t off = 0;
     pl->off_m = off;    off += align256(sizeof(float) * slots * (size_t)B);
     pl->off_l = off;    off += align256(sizeof(float) * slots * (size_t)B);
@@ -641,7 +642,7 @@ int gc_kernel_launches(int op, int64_t B, int64_t N, int d, int dtype) {
     if (B <= 0 || N <= 0 || d <= 0) return 0;
     if (op >= GC_OP_FWD && op <= GC_OP_BUILD && small_applicable(B, N, d, dtype)) return 1;
     if (op >= GC_OP_FWD && op <= GC_OP_BUILD && small_tiled_applicable(B, N, d, dtype)) {
-        const int reduces = (small_tiles_y(N) > 1 ? 1 : 0) + (small_tiles_x(B) > 1 ? 1 : 0);
+        const int reduces = (small_tiles_y(N, dtype) > 1 ? 1 : 0) + (small_tiles_x(B) > 1 ? 1 : 0);
         if (op == GC_OP_FWD) return 2;                  // tile kernel, combine
         if (op == GC_OP_BWD) return 2 + reduces;        // pos_idx validation, tile kernel, reduces
         return 3 + reduces;

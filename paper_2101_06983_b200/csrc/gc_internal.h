@@ -111,7 +111,8 @@ struct FwdArgs {
 // How one call is carried out for given sizes on the current device.
 struct Plan {
     int tc;                 // 1: tcgen05 kernels, 0: SIMT kernels
-    int tiles;              // 1: fp32 batch of a few tiles on the one-tile tcgen05 kernel
+    int tiles;              // 1: batch of a few tiles on the one-tile tcgen05 kernel
+    int tiles_y;            // its passage tiles (slots per row of its forward)
     int g_fwd, g_dq, g_dp;  // split factors of the streamed range
     size_t off_m, off_l, off_pos, off_red, off_accq, off_accp;
     size_t total;           // workspace bytes (multiple of 256)
@@ -197,7 +198,7 @@ cudaError_t launch_small(int op, const Problem& pr, const float* row_lse_in, flo
 
 bool small_tiled_applicable(int64_t B, int64_t N, int d, int dtype);
 int small_tiles_x(int64_t B);
-int small_tiles_y(int64_t N);
+int small_tiles_y(int64_t N, int dtype);
 cudaError_t launch_small_tiled_fwd(const Problem& pr, float* part_m, float* part_l, float* pos_ws,
                                    float* red, int* dev_status, cudaStream_t st);
 cudaError_t launch_small_tiled_bwd(const Problem& pr, const float* row_lse, float* dQ, int64_t lddq,

@@ -670,28 +670,44 @@ cudaError_t launch_small(int op, const Problem& pr, const float* row_lse_in, flo
                : launch_small_t<false>(mq, mp, mdq, mdp, p, grid, st);
 }
 
-// fp32 batches of a few tiles (query tiles of 128 x passage tiles of 128) run the same kernel
-// once per tile pair and column slice: the forward launch leaves one (max, sum) slot per passage
-// tile and row for the combine kernel, the gradient launch (row_lse given) writes every tile
-// pair's slices as planes of partial sums that a reduce kernel adds in index order.  Every CTA
-// of a tile pair forms that pair's logits, so the work grows with d / 64: a plan for batches
-// where launches, not arithmetic, set the time.
+// Batches of a few tiles (query tiles of 128 x passage tiles of 128 for fp32, of 256 for bf16) run
+// the same kernel once per tile pair and column slice: the forward launch leaves one (max, sum)
+// slot per passage tile and row for the combine kernel, the gradient launch (row_lse given)
+// writes every tile pair's slices as planes of partial sums that a reduce kernel adds in index
+// order.  Every CTA of a tile pair forms that pair's logits, so the work grows with d / 64: a plan
+// for batches where launches, not arithmetic, set the time.  fp32: up to 64 tile pairs; bf16:
+// widths that are not a multiple of 64, one wave of CTAs (what serves these cases otherwise is
+// the FMA-tile plan; bf16 rows of whole 64-column chunks belong to the sweeps, although this
+// plan is faster up to one wave of CTAs: 37-42 us against 58-71 us at 300 x 520 x 640 or
+// 1000 x 1000 x 128, measured).
 bool small_tiled_applicable(int64_t B, int64_t N, int d, int dtype) {
-    if (dtype != GC_F32 || d % 8 != 0 || d > 4096 || small_applicable(B, N, d, dtype)) return false;
-    const int64_t xt = (B + 127) / 128, yt = (N + 127) / 128;
-    return xt * yt <= 64 && xt * yt * ((d + 63) / 64) <= 2048;
+    if (d % 8 != 0 || d > 4096 || small_applicable(B, N, d, dtype)) return false;
+    const int64_t xt = small_tiles_x(B), yt = small_tiles_y(N, dtype);
+    const int64_t ctas = xt * yt * ((d + 63) / 64);
+    if (dtype == GC_F32) return xt * yt <= 64 && ctas <= 2048;
+    // bf16: only the widths the sweeps do not take (d not a multiple of 64), and only while the
+    // gradient launch is one wave of CTAs
+    return dtype == GC_BF16 && d % 64 != 0 && xt * yt <= 64 && ctas <= sm_count();
 }
 int small_tiles_x(int64_t B) { return (int)((B + 127) / 128); }
-int small_tiles_y(int64_t N) { return (int)((N + 127) / 128); }
+int small_tiles_y(int64_t N, int dtype) {
+    return dtype == GC_F32 ? (int)((N + 127) / 128) : (int)((N + 255) / 256);
+}
+namespace {
+bool small_in_maps(const Problem& pr, CUtensorMap* mq, CUtensorMap* mp) {
+    return pr.dtype == GC_F32 ? make_map_f32(mq, pr.Q, pr.B, pr.d, pr.ldq, 128) &&
+                                    make_map_f32(mp, pr.P, pr.N, pr.d, pr.ldp, 128)
+                              : make_map(mq, pr.Q, pr.B, pr.d, pr.ldq, 128) &&
+                                    make_map(mp, pr.P, pr.N, pr.d, pr.ldp, 128);
+}
+}  // namespace
 
 // Forward of the tiled plan: slots part_m / part_l [tiles_y][B], pos_ws [B]; `red` is the scratch
 // of the combine kernel that follows.
 cudaError_t launch_small_tiled_fwd(const Problem& pr, float* part_m, float* part_l, float* pos_ws,
                                    float* red, int* dev_status, cudaStream_t st) {
     CUtensorMap mq, mp;
-    if (!make_map_f32(&mq, pr.Q, pr.B, pr.d, pr.ldq, 128) ||
-        !make_map_f32(&mp, pr.P, pr.N, pr.d, pr.ldp, 128))
-        return cudaErrorInvalidValue;
+    if (!small_in_maps(pr, &mq, &mp)) return cudaErrorInvalidValue;
     SmallParams p{};
     p.B = (int)pr.B; p.N = (int)pr.N; p.d = pr.d;
     p.op = GC_OP_FWD;
@@ -704,8 +720,9 @@ cudaError_t launch_small_tiled_fwd(const Problem& pr, float* part_m, float* part
     p.part_m = part_m; p.part_l = part_l; p.pos_ws = pos_ws;
     p.zero_me = reinterpret_cast<int*>(red);
     p.dev_status = dev_status;
-    const dim3 grid(1u, (unsigned)small_tiles_x(pr.B), (unsigned)small_tiles_y(pr.N));
-    return launch_small_t<true>(mq, mp, mq, mp, p, grid, st);
+    const dim3 grid(1u, (unsigned)small_tiles_x(pr.B), (unsigned)small_tiles_y(pr.N, pr.dtype));
+    return pr.dtype == GC_F32 ? launch_small_t<true>(mq, mp, mq, mp, p, grid, st)
+                              : launch_small_t<false>(mq, mp, mq, mp, p, grid, st);
 }
 
 // Gradients of the tiled plan from row_lse.  With one passage tile dQ is final (scaled) in dQ,
@@ -714,11 +731,9 @@ cudaError_t launch_small_tiled_fwd(const Problem& pr, float* part_m, float* part
 cudaError_t launch_small_tiled_bwd(const Problem& pr, const float* row_lse, float* dQ, int64_t lddq,
                                    float* partial_q, float* dP, int64_t lddp, float* partial_p,
                                    int* dev_status, cudaStream_t st) {
-    const int xt = small_tiles_x(pr.B), yt = small_tiles_y(pr.N);
+    const int xt = small_tiles_x(pr.B), yt = small_tiles_y(pr.N, pr.dtype);
     CUtensorMap mq, mp;
-    if (!make_map_f32(&mq, pr.Q, pr.B, pr.d, pr.ldq, 128) ||
-        !make_map_f32(&mp, pr.P, pr.N, pr.d, pr.ldp, 128))
-        return cudaErrorInvalidValue;
+    if (!small_in_maps(pr, &mq, &mp)) return cudaErrorInvalidValue;
     CUtensorMap mdq = mq, mdp = mp;
     if (dQ) {
         const bool ok = yt == 1 ? make_out_map(&mdq, dQ, pr.B, pr.d, lddq, 1)
@@ -748,7 +763,8 @@ cudaError_t launch_small_tiled_bwd(const Problem& pr, const float* row_lse, floa
     p.plane_q = yt > 1; p.plane_p = xt > 1;
     p.dev_status = dev_status;
     const dim3 grid((unsigned)((pr.d + 63) / 64), (unsigned)xt, (unsigned)yt);
-    return launch_small_t<true>(mq, mp, mdq, mdp, p, grid, st);
+    return pr.dtype == GC_F32 ? launch_small_t<true>(mq, mp, mdq, mdp, p, grid, st)
+                              : launch_small_t<false>(mq, mp, mdq, mdp, p, grid, st);
 }
 
 }  // namespace gc

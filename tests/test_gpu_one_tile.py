@@ -148,3 +148,25 @@ def test_fp32_tiles_self_mask(binding, oracle, n, d, tau):
                                  scale=d ** -0.5, shared=True)
     out = run_build(prob)
     check_against_oracle(prob, out, _oracle_full(oracle, prob))
+
+
+# bf16 rows that are not whole 64-column chunks: a few tiles per batch run on the tensor cores too
+TILED_BF16 = [(129, 257, 72), (300, 520, 200), (200, 513, 136), (130, 130, 520), (1000, 1000, 40),
+              (257, 1, 8), (129, 300, 1000)]
+
+
+@pytest.mark.parametrize("B,N,d", TILED_BF16)
+def test_bf16_odd_widths_in_a_few_tiles(binding, oracle, B, N, d):
+    assert binding.gc_plan_name(binding.GC_OP_BUILD, B, N, d, binding.GC_BF16) == "tcgen05-tiles"
+    prob = inputs.random_problem(B, N, d, "bf16", seed=B + N + d, tau=0.5, scale=d ** -0.5)
+    ref = _oracle_full(oracle, prob)
+    out = run_build(prob)
+    check_against_oracle(prob, out, ref)
+    Q, P, pos = to_device(prob)
+    b = binding.Outputs(prob.B, prob.N, prob.d, binding.GC_BF16)
+    binding.gc_loss_fwd(Q, P, pos, prob.tau, prob.mask_mode, b.loss, b.row_lse, b.pos_logit, b.ws,
+                        b.dev_status)
+    binding.gc_loss_bwd(Q, P, pos, prob.tau, prob.mask_mode, b.row_lse, b.dQ, b.dP, b.ws,
+                        b.dev_status)
+    torch.cuda.synchronize()
+    check_against_oracle(prob, b, ref)
