@@ -43,10 +43,10 @@ NOMINAL_BF16_TFLOPS = 2250.0      # public dense bf16 figure for B200, context o
 SWEEP_SOURCES = ['gc_api.cu', 'gc_combine.cu', 'gc_internal.h', 'gc_quad.cu', 'gc_tc.cu', 'tc_common.cuh']
 ONE_TILE_SOURCES = ['gc_api.cu', 'gc_internal.h', 'gc_small.cu', 'tc_common.cuh']
 NCU_STEP_TRAFFIC = {
-    "cfg2_": (82.9e6, SWEEP_SOURCES, "68b658840b8ea1eeb4ae303c1ff4ffd9c7d09a6e"),
-    "cfg4_": (4.80e9, SWEEP_SOURCES, "68b658840b8ea1eeb4ae303c1ff4ffd9c7d09a6e"),
-    "cfg1_": (0.629e6, ONE_TILE_SOURCES, "a4c6433ab8554374787bd385eb26294c2258724e"),
-    "cfg0_": (0.640e6, ONE_TILE_SOURCES, "a4c6433ab8554374787bd385eb26294c2258724e"),
+    "cfg2_": (82.9e6, SWEEP_SOURCES, "adfba88f67b9304c594a699db5c0fd060aefa432"),
+    "cfg4_": (4.80e9, SWEEP_SOURCES, "adfba88f67b9304c594a699db5c0fd060aefa432"),
+    "cfg1_": (0.629e6, ONE_TILE_SOURCES, "b0165c68436f42c275884d8cccfdc22715ae2119"),
+    "cfg0_": (0.640e6, ONE_TILE_SOURCES, "b0165c68436f42c275884d8cccfdc22715ae2119"),
 }
 FP32_LANES_PER_SM = 128           # fp32 FMA lanes of one SM (2 FLOP per lane and clock)
 
