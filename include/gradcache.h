@@ -76,15 +76,15 @@ size_t gc_workspace_bytes(int op, int64_t B, int64_t N, int d, int dtype);
 /* Name of the kernel plan the library will use for these sizes:
  *   "tcgen05-one-tile"  one launch for a batch of one tile: B <= 128, N <= 256 (bf16) or N <= 128
  *                       (fp32, on the tensor cores as three bf16 terms), d a multiple of 8 up to 1024
- *   "tcgen05-tiles"     fp32 batches of at most 64 tile pairs of 128 x 128 (d a multiple of 8 up
- *                       to 4096), and bf16 batches of a few tile pairs of 128 x 256 whose width is
- *                       a multiple of 8 but not of 64: the same kernel per tile pair, then
- *                       combine and reduce kernels
+ *   "tcgen05-tiles"     fp32 batches of at most 64 tile pairs of 128 x 128 and bf16 batches of
+ *                       tile pairs of 128 x 256 that make one wave of CTAs (d a multiple of 8 up
+ *                       to 4096): the same kernel per tile pair, then combine and reduce kernels
  *   "tcgen05"           TMA + tcgen05 MMA sweeps with TMEM accumulators; bf16, d a multiple of 64
  *                       up to 4096; one CTA, a CTA pair or a cluster of four per tile, by shape
  *   "simt"              fp32 FMA tiles: every other case (larger fp32 batches, other widths)
  * "invalid" for an unknown op, non-positive sizes, or a problem GC_OP_BUILD_STORED refuses.
- * Static string. */
+ * Static string.  With GRADCACHE_PLAN=sweeps in the environment (read at every call; a
+ * diagnostic switch) the first two plans are not chosen. */
 const char* gc_plan_name(int op, int64_t B, int64_t N, int d, int dtype);
 
 /* Number of kernels one call launches for these sizes (for launch accounting). */

@@ -17,6 +17,9 @@
 // in fp32 accumulation (spread over three accumulators, see the MMA warp), the weights are kept
 // as two terms and the gradient products take w1 (t1 + t2 + t3) + w2 (t1 + t2).  Every mbarrier
 // wait is bounded.
+#include <stdlib.h>
+#include <string.h>
+
 #include "tc_common.cuh"
 
 namespace gc {
@@ -628,7 +631,16 @@ cudaError_t launch_small_t(const CUtensorMap& mq, const CUtensorMap& mp, const C
 
 }  // namespace
 
+// GRADCACHE_PLAN=sweeps in the environment (read at every call) keeps every problem on the sweep
+// kernels (or the FMA tiles): a diagnostic switch, so that small shapes can still exercise the
+// kernels that large ones run.
+static bool small_plans_enabled() {
+    const char* e = getenv("GRADCACHE_PLAN");
+    return !(e && strcmp(e, "sweeps") == 0);
+}
+
 bool small_applicable(int64_t B, int64_t N, int d, int dtype) {
+    if (!small_plans_enabled()) return false;
     if (B > 128 || d % 8 != 0 || d > 1024) return false;
     return dtype == GC_BF16 ? N <= 256 : N <= 128;
 }
@@ -675,19 +687,17 @@ cudaError_t launch_small(int op, const Problem& pr, const float* row_lse_in, flo
 // slot per passage tile and row for the combine kernel, the gradient launch (row_lse given)
 // writes every tile pair's slices as planes of partial sums that a reduce kernel adds in index
 // order.  Every CTA of a tile pair forms that pair's logits, so the work grows with d / 64: a plan
-// for batches where launches, not arithmetic, set the time.  fp32: up to 64 tile pairs; bf16:
-// widths that are not a multiple of 64, one wave of CTAs (what serves these cases otherwise is
-// the FMA-tile plan; bf16 rows of whole 64-column chunks belong to the sweeps, although this
-// plan is faster up to one wave of CTAs: 37-42 us against 58-71 us at 300 x 520 x 640 or
-// 1000 x 1000 x 128, measured).
+// for batches where launches, not arithmetic, set the time.  fp32: up to 64 tile pairs (what
+// serves fp32 otherwise is the FMA-tile plan); bf16: while the gradient launch is one wave of
+// CTAs (37-42 us against 58-71 us for the sweeps at 300 x 520 x 640 or 1000 x 1000 x 128,
+// measured; beyond one wave the sweeps are faster).
 bool small_tiled_applicable(int64_t B, int64_t N, int d, int dtype) {
+    if (!small_plans_enabled()) return false;
     if (d % 8 != 0 || d > 4096 || small_applicable(B, N, d, dtype)) return false;
     const int64_t xt = small_tiles_x(B), yt = small_tiles_y(N, dtype);
     const int64_t ctas = xt * yt * ((d + 63) / 64);
     if (dtype == GC_F32) return xt * yt <= 64 && ctas <= 2048;
-    // bf16: only the widths the sweeps do not take (d not a multiple of 64), and only while the
-    // gradient launch is one wave of CTAs
-    return dtype == GC_BF16 && d % 64 != 0 && xt * yt <= 64 && ctas <= sm_count();
+    return dtype == GC_BF16 && xt * yt <= 64 && ctas <= sm_count();
 }
 int small_tiles_x(int64_t B) { return (int)((B + 127) / 128); }
 int small_tiles_y(int64_t N, int dtype) {

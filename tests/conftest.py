@@ -27,3 +27,20 @@ def _library_present():
     from paper_2101_06983_b200 import _build
     if _build.stale():
         _build.build()
+
+
+@pytest.fixture(params=["auto", "sweeps"])
+def plan_mode(request, monkeypatch):
+    """Runs a test twice: with the library choosing its plan, and with GRADCACHE_PLAN=sweeps in
+    the environment, which keeps small problems on the sweep kernels (or the FMA tiles), the
+    kernels that large problems run."""
+    if request.param == "sweeps":
+        monkeypatch.setenv("GRADCACHE_PLAN", "sweeps")
+    else:
+        monkeypatch.delenv("GRADCACHE_PLAN", raising=False)
+    return request.param
+
+
+@pytest.fixture
+def sweeps_only(monkeypatch):
+    monkeypatch.setenv("GRADCACHE_PLAN", "sweeps")

@@ -35,7 +35,7 @@ SHAPES = [
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("B,N,d", SHAPES)
-def test_small_shapes(binding, oracle, B, N, d, dtype):
+def test_small_shapes(binding, oracle, B, N, d, dtype, plan_mode):
     if dtype == "bf16" and d % 8:
         d = (d + 7) // 8 * 8            # rows must start on 16-byte boundaries
     prob = inputs.random_problem(B, N, d, dtype, seed=B * 1000 + N, tau=0.5, scale=0.5)
@@ -45,7 +45,7 @@ def test_small_shapes(binding, oracle, B, N, d, dtype):
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("n,d,tau", [(130, 64, 0.1), (257, 128, 0.1), (96, 768, 1.0)])
-def test_self_mask_shared_rows(binding, oracle, n, d, tau, dtype):
+def test_self_mask_shared_rows(binding, oracle, n, d, tau, dtype, plan_mode):
     prob = inputs.random_problem(n, n, d, dtype, seed=n, tau=tau, mask_mode=inputs.MASK_SELF,
                                  scale=d ** -0.5, shared=True)
     out = run_build(prob)
@@ -62,7 +62,7 @@ QUAD_SHAPES = [
 
 
 @pytest.mark.parametrize("B,N,d", QUAD_SHAPES)
-def test_four_cta_cluster_sweeps(binding, oracle, B, N, d):
+def test_four_cta_cluster_sweeps(binding, oracle, B, N, d, plan_mode):
     prob = inputs.random_problem(B, N, d, "bf16", seed=B + N + d, tau=0.3, scale=d ** -0.5)
     out = run_build(prob)
     ref = _oracle_full(oracle, prob)
@@ -78,7 +78,7 @@ def test_four_cta_cluster_sweeps(binding, oracle, B, N, d):
     check_against_oracle(prob, b, ref)
 
 
-def test_four_cta_cluster_sweeps_self_mask(binding, oracle):
+def test_four_cta_cluster_sweeps_self_mask(binding, oracle, plan_mode):
     prob = inputs.random_problem(700, 700, 768, "bf16", seed=77, tau=0.2,
                                  mask_mode=inputs.MASK_SELF, scale=768 ** -0.5, shared=True)
     out = run_build(prob)
@@ -105,7 +105,7 @@ def test_streamed_matrix_larger_than_l2_uses_cta_pairs(binding, oracle, B, N):
     check_against_oracle(prob, b, ref)
 
 
-def test_fwd_then_bwd_equals_build(binding, oracle):
+def test_fwd_then_bwd_equals_build(binding, oracle, plan_mode):
     """The separate forward and backward calls reproduce gc_build_cache: bit for bit where both
     run the same kernels (fp32 inputs), within rounding where gc_build_cache fuses the forward
     into the dQ sweep (bf16 rows)."""
@@ -136,7 +136,7 @@ def test_fwd_then_bwd_equals_build(binding, oracle):
         assert torch.equal(c.dP, a.dP) and bool((c.dQ == 7.0).all())
 
 
-def test_strided_rows(binding, oracle):
+def test_strided_rows(binding, oracle, plan_mode):
     """Leading dimensions larger than d on inputs and outputs."""
     prob = inputs.random_problem(70, 140, 64, "f32", seed=4, tau=1.0, scale=0.3)
     Qb = torch.zeros(70, 80, device="cuda")
@@ -158,7 +158,7 @@ def test_strided_rows(binding, oracle):
 
 # ---- the named workloads ------------------------------------------------------------------------
 @pytest.mark.parametrize("index", [0, 1])
-def test_config_small(binding, oracle, index):
+def test_config_small(binding, oracle, index, plan_mode):
     prob = inputs.config(index)
     out = run_build(prob)
     check_against_oracle(prob, out, _oracle_full(oracle, prob))
@@ -256,7 +256,7 @@ def test_config4_extreme_batch_never_stores_S(binding, oracle):
 
 # ---- bit-exact index and mask behaviour ------------------------------------------------------------
 @pytest.mark.parametrize("dtype,d", [("f32", 64), ("bf16", 64), ("bf16", 768)])
-def test_positive_gather_is_bit_exact(binding, dtype, d):
+def test_positive_gather_is_bit_exact(binding, dtype, d, plan_mode):
     """Q_i = e_0 and P_j[0] = code(j), all other entries 0: S_ij = code(j) exactly, so
     pos_logit[i] must equal code(pos_idx[i]) bit for bit wherever the positive sits."""
     B, N = 300, 1000
@@ -283,7 +283,7 @@ def test_positive_gather_is_bit_exact(binding, dtype, d):
 
 
 @pytest.mark.parametrize("dtype,d", [("f32", 320), ("bf16", 320), ("bf16", 768)])
-def test_self_mask_is_exact_zero(binding, dtype, d):
+def test_self_mask_is_exact_zero(binding, dtype, d, plan_mode):
     """Row i has a private coordinate c_i = i.  dP_i[c_i] = G_ii Q_i[c_i] / tau must be exactly
     +0 under the self mask, and is non-zero without it."""
     n = 300
@@ -306,7 +306,7 @@ def test_self_mask_is_exact_zero(binding, dtype, d):
 
 
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
-def test_mask_does_not_leak(binding, oracle, dtype):
+def test_mask_does_not_leak(binding, oracle, dtype, plan_mode):
     """Rows of norm 8 in random directions, shared between Q and P: every diagonal logit is 64
     while the off-diagonal ones stay below about 30, so a single unmasked diagonal entry would
     move that row's lse by tens.  Sizes are not multiples of any tile."""
@@ -321,7 +321,7 @@ def test_mask_does_not_leak(binding, oracle, dtype):
 
 
 @pytest.mark.parametrize("B,N,d,tau", [(200, 300, 128, 0.01), (300, 520, 768, 0.004)])
-def test_logits_far_above_the_positive(binding, oracle, B, N, d, tau):
+def test_logits_far_above_the_positive(binding, oracle, B, N, d, tau, plan_mode):
     """Rows whose largest logit lies hundreds of powers of two above their positive logit: the
     wide-row build scales its weights by the positive logit and must hand such inputs to the
     kernels that track the running row maximum."""
@@ -332,7 +332,7 @@ def test_logits_far_above_the_positive(binding, oracle, B, N, d, tau):
     check_against_oracle(prob, out, ref)
 
 
-def test_bad_positives_are_flagged_not_fatal(binding, oracle):
+def test_bad_positives_are_flagged_not_fatal(binding, oracle, plan_mode):
     prob = inputs.random_problem(40, 50, 64, "f32", seed=1, tau=1.0, scale=0.3,
                                  mask_mode=inputs.MASK_SELF)
     pos = prob.pos_idx.copy()
@@ -358,7 +358,7 @@ def test_bad_positives_are_flagged_not_fatal(binding, oracle):
 
 
 @pytest.mark.parametrize("d", [128, 768])
-def test_bad_positives_with_a_fixed_row_scale(binding, oracle, d):
+def test_bad_positives_with_a_fixed_row_scale(binding, oracle, d, plan_mode):
     """The bf16 builds that scale each row's weights by its positive logit (narrow rows, and rows
     of two column halves): a row whose pos_idx is unusable has no positive logit to scale by; it
     is flagged, gets no one-hot term, and every other row still matches the oracle."""
@@ -394,7 +394,7 @@ def test_deterministic(binding, index):
         assert torch.equal(getattr(a, name), getattr(b, name)), name
 
 
-def test_workspace_canaries(binding):
+def test_workspace_canaries(binding, plan_mode):
     """Nothing is written outside the reported workspace size or outside the output rows."""
     prob = inputs.config(1)
     Q, P, pos = to_device(prob)
@@ -411,7 +411,7 @@ def test_workspace_canaries(binding):
     assert bool((buf[:off] == 0xA5).all()) and bool((buf[off + need:] == 0xA5).all())
 
 
-def test_per_call_kernel_timing(binding):
+def test_per_call_kernel_timing(binding, sweeps_only):
     """gc_profile_enable(n) keeps one event set per call: n queued calls can be read afterwards,
     each with positive sweep durations; a call that was never made is refused."""
     prob = inputs.random_problem(300, 520, 768, "bf16", seed=2, tau=0.5, scale=768 ** -0.5)
@@ -442,7 +442,7 @@ def _guarded(need, pad=4096):
 
 
 @pytest.mark.parametrize("B,N,d", [(300, 500, 128), (300, 520, 768), (130, 90, 1024)])
-def test_workspace_canaries_of_every_bf16_plan(binding, B, N, d):
+def test_workspace_canaries_of_every_bf16_plan(binding, B, N, d, plan_mode):
     """Narrow rows with a fixed row scale, four-CTA sweeps, paired wide rows: gc_build_cache,
     the rank-local calls and gc_cache_apply stay inside the workspace sizes they report."""
     prob = inputs.random_problem(B, N, d, "bf16", seed=B, tau=0.5, scale=d ** -0.5)

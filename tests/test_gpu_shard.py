@@ -115,8 +115,9 @@ def test_sharded_step_object_on_one_gpu(binding, oracle):
     assert set(step.timings) == {"gather_reps_s", "fwd_dq_s", "lse_and_loss_s", "dp_s"}
 
 
-def test_one_rank_is_the_whole_batch(binding):
-    """world = 1: the two calls together are gc_loss_fwd + gc_loss_bwd on the same kernels."""
+def test_one_rank_is_the_whole_batch(binding, sweeps_only):
+    """world = 1: the two calls together are gc_loss_fwd + gc_loss_bwd on the same kernels (the
+    rank-local calls always run the sweeps, so the whole-batch call is kept on them too)."""
     prob = inputs.random_problem(140, 270, 64, "bf16", seed=5, tau=0.7, scale=0.125)
     Q, P, pos = to_device(prob)
     a = binding.build_cache(Q, P, pos, prob.tau, prob.mask_mode)

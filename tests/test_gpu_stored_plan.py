@@ -103,7 +103,7 @@ def test_config4_sampled(binding, oracle):
     _check_properties(prob, out, Q, P, units=16)
 
 
-def test_out_of_range_logits_fall_back_to_recomputing(binding, oracle):
+def test_out_of_range_logits_fall_back_to_recomputing(binding, oracle, sweeps_only):
     """Logits far above a row's positive logit (here by thousands of powers of two) cannot be
     stored relative to it; the call must then deliver exactly what gc_build_cache delivers.  On
     an ordinary input the two routes differ in rounding, which shows the flag is what switches."""
