@@ -66,7 +66,8 @@ def test_plan_names(binding):
     assert b.gc_kernel_launches(b.GC_OP_BUILD, 64, 129, 768, b.GC_F32) == 4
     assert b.gc_plan_name(b.GC_OP_BUILD, 300, 200, 320, b.GC_F32) == "tcgen05-tiles"
     assert b.gc_plan_name(b.GC_OP_BUILD, 129, 128, 768, b.GC_BF16) == "tcgen05-tiles"   # 24 CTAs
-    assert b.gc_plan_name(b.GC_OP_BUILD, 385, 900, 768, b.GC_BF16) == "tcgen05"         # 192 CTAs
+    assert b.gc_plan_name(b.GC_OP_BUILD, 385, 900, 768, b.GC_BF16) == "tcgen05-tiles"   # 192 CTAs
+    assert b.gc_plan_name(b.GC_OP_BUILD, 1030, 1300, 768, b.GC_BF16) == "tcgen05"       # 648 CTAs
     assert b.gc_plan_name(b.GC_OP_BUILD, 300, 520, 200, b.GC_BF16) == "tcgen05-tiles"
     # FMA tiles: widths that are not a multiple of 8, large batches of fp32 or of odd bf16 widths
     assert b.gc_plan_name(b.GC_OP_BUILD, 64, 128, 100, b.GC_BF16) == "simt"
