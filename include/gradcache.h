@@ -27,7 +27,10 @@
  *     respect to each role and the caller adds them.  Outputs may not alias inputs.
  *   - dtype is the element type of Q and P; all outputs are float, accumulation is float.
  *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t, may be NULL for the default
- *     stream) and return a gc_status for host-detectable errors only.
+ *     stream) and return a gc_status for host-detectable errors only.  After a first ordinary
+ *     call for the same kernels (it sets kernel attributes and creates the side stream), a call
+ *     on a capturing stream can be captured into a CUDA graph and replayed: work on the
+ *     library's side stream is forked from and joined back into `cuda_stream`.
  *   - Data-dependent errors are OR-ed into *dev_status (may be NULL) on the device:
  *     GC_DEV_POS_RANGE for pos_idx[i] outside [0, N), GC_DEV_POS_MASKED for pos_idx[i] equal
  *     to the masked column.  Such a row contributes pos_logit = 0 and no one-hot term; nothing
