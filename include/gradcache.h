@@ -79,12 +79,14 @@ size_t gc_workspace_bytes(int op, int64_t B, int64_t N, int d, int dtype);
 /* Name of the kernel plan the library will use for these sizes:
  *   "tcgen05-one-tile"  one launch for a batch of one tile: B <= 128, N <= 256 (bf16) or N <= 128
  *                       (fp32, on the tensor cores as three bf16 terms), d a multiple of 8 up to 1024
- *   "tcgen05-tiles"     fp32 batches of at most 64 tile pairs of 128 x 128 and bf16 batches of
- *                       tile pairs of 128 x 256 that make at most two waves of CTAs (d a multiple
- *                       of 8 up to 4096): the same kernel per tile pair, then combine and reduce
+ *   "tcgen05-tiles"     fp32 batches of tile pairs of 128 x 128 whose planes of partial sums,
+ *                       4 d (B ceil(N/128) + N ceil(B/128)) bytes of workspace, stay within 2 GiB,
+ *                       and bf16 batches of tile pairs of 128 x 256 that make at most two waves of
+ *                       CTAs (d a multiple of 8 up to 4096): the same kernel per tile pair, then
+ *                       combine and reduce kernels
  *   "tcgen05"           TMA + tcgen05 MMA sweeps with TMEM accumulators; bf16, d a multiple of 64
  *                       up to 4096; one CTA, a CTA pair or a cluster of four per tile, by shape
- *   "simt"              fp32 FMA tiles: every other case (larger fp32 batches, other widths)
+ *   "simt"              fp32 FMA tiles: every other case (other widths, fp32 batches beyond that)
  * "invalid" for an unknown op, non-positive sizes, or a problem GC_OP_BUILD_STORED refuses.
  * Static string.  With GRADCACHE_PLAN=sweeps in the environment (read at every call; a
  * diagnostic switch) the first two plans are not chosen. */

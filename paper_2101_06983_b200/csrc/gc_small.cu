@@ -687,8 +687,8 @@ cudaError_t launch_small(int op, const Problem& pr, const float* row_lse_in, flo
 // slot per passage tile and row for the combine kernel, the gradient launch (row_lse given)
 // writes every tile pair's slices as planes of partial sums that a reduce kernel adds in index
 // order.  Every CTA of a tile pair forms that pair's logits, so the work grows with d / 64: a plan
-// for batches where launches, not arithmetic, set the time.  fp32: up to 64 tile pairs (what
-// serves fp32 otherwise is the FMA-tile plan); bf16: while the gradient launch is at most two
+// for batches where launches, not arithmetic, set the time.  fp32: whatever its partial planes
+// allow (what serves fp32 otherwise is the FMA-tile plan, which is slower at every size); bf16: while the gradient launch is at most two
 // waves of CTAs (measured: 37-42 us against 58-71 us for the sweeps at 300 x 520 x 640 or
 // 1000 x 1000 x 128, 48-51 us against 68-70 us at 385 x 900 x 768 or 512 x 1024 x 768 with 192
 // CTAs; at 1030 x 1300 x 768, 648 CTAs, 87 us against 69 us: there the sweeps are faster).
@@ -697,7 +697,12 @@ bool small_tiled_applicable(int64_t B, int64_t N, int d, int dtype) {
     if (d % 8 != 0 || d > 4096 || small_applicable(B, N, d, dtype)) return false;
     const int64_t xt = small_tiles_x(B), yt = small_tiles_y(N, dtype);
     const int64_t ctas = xt * yt * ((d + 63) / 64);
-    if (dtype == GC_F32) return xt * yt <= 64 && ctas <= 2048;
+    if (dtype == GC_F32) {
+        // as long as the planes of partial sums stay within 2 GiB: the alternative for fp32 is
+        // the FMA-tile plan, which this plan outruns about five times at every size measured
+        const double plane_bytes = ((double)yt * (double)B + (double)xt * (double)N) * d * 4.0;
+        return xt <= 65535 && yt <= 65535 && plane_bytes <= 2147483648.0;
+    }
     return dtype == GC_BF16 && xt * yt <= 64 && ctas <= 2 * sm_count();
 }
 int small_tiles_x(int64_t B) { return (int)((B + 127) / 128); }

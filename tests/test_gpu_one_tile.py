@@ -117,7 +117,7 @@ def test_bad_positive_indices_raise_the_device_flags(binding):
 # fp32 batches of a few tiles: the same kernel once per tile pair and column slice
 TILED_F32 = [(129, 257, 72), (130, 130, 128), (200, 513, 192), (257, 1, 64), (65, 300, 768),
              (300, 200, 320), (140, 270, 448), (129, 300, 1024), (260, 131, 1536), (70, 140, 4096),
-             (1000, 900, 64), (128, 129, 8), (129, 128, 8)]
+             (1000, 900, 64), (128, 129, 8), (129, 128, 8), (1100, 2300, 136), (2100, 1500, 64)]
 
 
 @pytest.mark.parametrize("B,N,d", TILED_F32)

@@ -69,12 +69,14 @@ def test_plan_names(binding):
     assert b.gc_plan_name(b.GC_OP_BUILD, 385, 900, 768, b.GC_BF16) == "tcgen05-tiles"   # 192 CTAs
     assert b.gc_plan_name(b.GC_OP_BUILD, 1030, 1300, 768, b.GC_BF16) == "tcgen05"       # 648 CTAs
     assert b.gc_plan_name(b.GC_OP_BUILD, 300, 520, 200, b.GC_BF16) == "tcgen05-tiles"
-    # FMA tiles: widths that are not a multiple of 8, large batches of fp32 or of odd bf16 widths
+    # FMA tiles: widths that are not a multiple of 8, very large fp32 batches, large batches of
+    # odd bf16 widths
     assert b.gc_plan_name(b.GC_OP_BUILD, 64, 128, 100, b.GC_BF16) == "simt"
     assert b.gc_plan_name(b.GC_OP_BUILD, 4096, 8192, 200, b.GC_BF16) == "simt"
     assert b.gc_plan_name(b.GC_OP_BUILD, 64, 129, 100, b.GC_F32) == "simt"
-    assert b.gc_plan_name(b.GC_OP_BUILD, 4096, 8192, 768, b.GC_F32) == "simt"
-    assert b.gc_kernel_launches(b.GC_OP_BUILD, 4096, 8192, 768, b.GC_F32) >= 4
+    assert b.gc_plan_name(b.GC_OP_BUILD, 4096, 8192, 768, b.GC_F32) == "tcgen05-tiles"
+    assert b.gc_plan_name(b.GC_OP_BUILD, 65536, 131072, 768, b.GC_F32) == "simt"   # planes > 2 GiB
+    assert b.gc_kernel_launches(b.GC_OP_BUILD, 65536, 131072, 768, b.GC_F32) >= 4
 
 
 def _call_fwd(lib, **over):
