@@ -45,8 +45,8 @@ ONE_TILE_SOURCES = ['gc_api.cu', 'gc_internal.h', 'gc_small.cu', 'tc_common.cuh'
 NCU_STEP_TRAFFIC = {
     "cfg2_": (82.9e6, SWEEP_SOURCES, "adfba88f67b9304c594a699db5c0fd060aefa432"),
     "cfg4_": (4.80e9, SWEEP_SOURCES, "adfba88f67b9304c594a699db5c0fd060aefa432"),
-    "cfg1_": (0.629e6, ONE_TILE_SOURCES, "7cacc3ab23ffb6a83e2a0faa23584005bf3bdbc1"),
-    "cfg0_": (0.640e6, ONE_TILE_SOURCES, "7cacc3ab23ffb6a83e2a0faa23584005bf3bdbc1"),
+    "cfg1_": (0.629e6, ONE_TILE_SOURCES, "aba4388866b186f5857ff7690980676530fc42c3"),
+    "cfg0_": (0.640e6, ONE_TILE_SOURCES, "aba4388866b186f5857ff7690980676530fc42c3"),
 }
 FP32_LANES_PER_SM = 128           # fp32 FMA lanes of one SM (2 FLOP per lane and clock)
 
