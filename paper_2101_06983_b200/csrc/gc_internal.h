@@ -185,6 +185,12 @@ cudaError_t tc_launch_fwd_store(const FwdArgs& a, void* weights, int64_t ldw, co
 
 // gc_quad.cu
 bool quad_applicable(int64_t nx, int d);
+// gc_narrow.cu: the gradient sweeps of rows of 64 or 128 bf16 values
+bool narrow_applicable(int d, int dtype);
+cudaError_t narrow_launch_anchored_dq(const FwdArgs& a, float* partial, int groups,
+                                      const float* row_ref, int* range_flag, cudaStream_t st,
+                                      bool overlap_prev);
+cudaError_t narrow_launch_sweep(const SweepArgs& a, cudaStream_t st);
 int quad_groups(int64_t nx, int64_t ny);
 cudaError_t quad_launch_sweep(const SweepArgs& a, cudaStream_t st);
 cudaError_t quad_launch_fused_dq(const FwdArgs& a, float* partial, int groups, const float* row_ref,

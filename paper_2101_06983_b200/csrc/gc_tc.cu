@@ -779,7 +779,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
             }
         } else {
             // per-row constants (DQ: the row is a query)
-            float lse2_x = 0.f, l_sum = 0.f, wmax = 0.f;
+            float lse2_x = 0.f, l_sum = 0.f;
             int32_t pos_x = -1;
             // DA may have been launched ahead of the anchor kernel's completion
             if (MODE == MODE_DA) dep_wait();
@@ -870,9 +870,16 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                                 if (c == rel) sp = __uint_as_float(v[c]);
                             p.pos_logit[x] = sp * p.inv_tau;
                         }
+                        // exponents two at a time (one issue slot per pair)
+                        const uint64_t c1_2 = pack2(p.c1, p.c1), nref_2 = pack2(-lse2_x, -lse2_x);
 #pragma unroll
-                        for (int c = 0; c < 32; ++c)
-                            w[c] = ex2(fmaf(__uint_as_float(v[c]), p.c1, -lse2_x));
+                        for (int c = 0; c < 32; c += 2) {
+                            float e0, e1;
+                            unpack2(fma2(pack2(__uint_as_float(v[c]), __uint_as_float(v[c + 1])),
+                                         c1_2, nref_2), e0, e1);
+                            w[c] = ex2(e0);
+                            w[c + 1] = ex2(e1);
+                        }
                         if (yb + 32 > p.ny) {
 #pragma unroll
                             for (int c = 0; c < 32; ++c)
@@ -884,15 +891,16 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                             for (int c = 0; c < 32; ++c)
                                 if (c == rel) w[c] = 0.f;
                         }
-                        float s0 = 0.f, s1 = 0.f, m0 = 0.f;
+                        // the weights are positive, so the row sum bounds the largest of them
+                        uint64_t sa = pack2(0.f, 0.f), sb = pack2(0.f, 0.f);
 #pragma unroll
-                        for (int c = 0; c < 32; c += 2) {
-                            s0 += w[c];
-                            s1 += w[c + 1];
-                            m0 = fmaxf(m0, fmaxf(w[c], w[c + 1]));
+                        for (int c = 0; c < 32; c += 4) {
+                            sa = add2(sa, pack2(w[c], w[c + 1]));
+                            sb = add2(sb, pack2(w[c + 2], w[c + 3]));
                         }
+                        float s0, s1;
+                        unpack2(add2(sa, sb), s0, s1);
                         l_sum += s0 + s1;
-                        wmax = fmaxf(wmax, m0);
                         if (pos_x >= yb && pos_x < yb + 32) {      // positive: fp32, in the finalize
                             const int rel = (int)(pos_x - yb);
 #pragma unroll
@@ -948,7 +956,7 @@ tc_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUte
                 p.part_m[slot] = lse2_x * 0.69314718055994531f;
                 p.part_l[slot] = l_sum;
                 // weights beyond 2^100 (or not finite) cannot be accumulated safely
-                if (!(wmax <= 1.2676506e30f)) *p.range_flag = 1;
+                if (!(l_sum <= 1.2676506e30f)) *p.range_flag = 1;
             }
             // epilogue: accumulator columns of this part -> global memory (32-column blocks are
             // dealt alternately to the two warps of a lane quarter); final values are scaled,
@@ -1229,6 +1237,8 @@ cudaError_t tc_launch_anchored_dq(const FwdArgs& a, float* partial, int groups,
                                   const float* row_ref, int* range_flag, cudaStream_t st,
                                   bool overlap_prev) {
     const Problem& pr = a.p;
+    if (narrow_applicable(pr.d, GC_BF16))
+        return narrow_launch_anchored_dq(a, partial, groups, row_ref, range_flag, st, overlap_prev);
     constexpr int SN = 128;
     const int kc = pr.d / 64;
     CUtensorMap mx, my, myh, mo;
@@ -1260,6 +1270,7 @@ cudaError_t tc_launch_anchored_dq(const FwdArgs& a, float* partial, int groups,
 
 cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     if (quad_applicable(a.nx, a.d)) return quad_launch_sweep(a, st);
+    if (narrow_applicable(a.d, GC_BF16)) return narrow_launch_sweep(a, st);
     const int kc = a.d / 64;
     constexpr int SN = 128;
     CUtensorMap mx, my, myh;
