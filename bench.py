@@ -42,11 +42,13 @@ NOMINAL_BF16_TFLOPS = 2250.0      # public dense bf16 figure for B200, context o
 # sources its kernels come from still have the hash they had when the counters were taken.
 SWEEP_SOURCES = ['gc_api.cu', 'gc_combine.cu', 'gc_internal.h', 'gc_quad.cu', 'gc_tc.cu', 'tc_common.cuh']
 ONE_TILE_SOURCES = ['gc_api.cu', 'gc_internal.h', 'gc_small.cu', 'tc_common.cuh']
+NARROW_SOURCES = SWEEP_SOURCES + ['gc_narrow.cu']
 NCU_STEP_TRAFFIC = {
-    "cfg2_": (82.9e6, SWEEP_SOURCES, "adfba88f67b9304c594a699db5c0fd060aefa432"),
-    "cfg4_": (4.80e9, SWEEP_SOURCES, "adfba88f67b9304c594a699db5c0fd060aefa432"),
-    "cfg1_": (0.629e6, ONE_TILE_SOURCES, "aba4388866b186f5857ff7690980676530fc42c3"),
-    "cfg0_": (0.640e6, ONE_TILE_SOURCES, "aba4388866b186f5857ff7690980676530fc42c3"),
+    "cfg2_": (82.9e6, SWEEP_SOURCES, "b8d876d88310b6e351a5579d0ac6ebc2fc8b8b7e"),
+    "cfg4_": (4.80e9, SWEEP_SOURCES, "b8d876d88310b6e351a5579d0ac6ebc2fc8b8b7e"),
+    "cfg3_": (26.4e6, NARROW_SOURCES, "25639b36dbf2b6732256b1340a264160eddf8760"),
+    "cfg1_": (0.629e6, ONE_TILE_SOURCES, "42794198880e3035735ceb1c20a53113fbce4c0e"),
+    "cfg0_": (0.640e6, ONE_TILE_SOURCES, "42794198880e3035735ceb1c20a53113fbce4c0e"),
 }
 FP32_LANES_PER_SM = 128           # fp32 FMA lanes of one SM (2 FLOP per lane and clock)
 

@@ -400,7 +400,8 @@ int run_anchored_build(const Problem& p, const Plan& pl, char* ws, float* loss, 
     if (e != cudaSuccess) return GC_ERR_CUDA;
     // Wide rows: a sweep step is long enough to hide the slot merge of the streamed queries,
     // so the dP sweep does not wait for the combine.  Narrow rows have short steps: there the
-    // combine stays on the caller's stream and the dP sweep reads row_lse.
+    // combine stays on the caller's stream and the dP sweep reads row_lse (8192 x 8192 x 128:
+    // 0.100 ms per call against 0.114 with the merge inside the dP sweep).
     const bool dp_merges = side && pl.anchored == 1 && want_dp;
     cudaStream_t comb = dp_merges ? aux : st;
     if (dp_merges && (cudaEventRecord(side->ev[0], st) != cudaSuccess ||
