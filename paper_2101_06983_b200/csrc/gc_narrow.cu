@@ -20,11 +20,10 @@
 // S tile or with X as a tensor-memory operand; 16-column pieces with the next piece's load in
 // flight 0.103.)
 //
-// Warp roles (576 threads; 704 in DP): warp 0 = TMA producer, warp 1 = MMA issuer and
-// tensor-memory allocator, warps 2..17 = softmax / epilogue: per group two warps per
-// tensor-memory lane quarter, each owning half of the tile's columns, one thread per tile row;
-// in DP warps 18..21 prepare, per streamed tile, the 128 column constants -lse2_y and pos_y in
-// shared memory, one column per thread.
+// Warp roles (576 threads): warp 0 = TMA producer (in DP it also writes, per streamed tile, the
+// 128 column constants -lse2_y and the tile row of pos_y to shared memory), warp 1 = MMA issuer
+// and tensor-memory allocator, warps 2..17 = softmax / epilogue: per group two warps per
+// tensor-memory lane quarter, each owning half of the tile's columns, one thread per tile row.
 // Every wait is bounded: on a timeout the CTA raises GC_DEV_WAIT_LIMIT, drains and exits.
 #include "tc_common.cuh"
 
@@ -36,11 +35,7 @@ enum { NMODE_DQ = 0, NMODE_DP = 1, NMODE_DA = 2 };
 
 constexpr int NW_STAGES = 5;                 // streamed tiles in flight
 constexpr int NW_SOFT = 16;                  // softmax warps: two groups of eight
-constexpr int NW_COLW = 4;                   // DP: warps that prepare the column constants
-template <int MODE>
-__host__ __device__ constexpr int nw_threads() {
-    return 32 * (2 + NW_SOFT + (MODE == 1 ? NW_COLW : 0));
-}
+constexpr int NW_THREADS = 32 * (2 + NW_SOFT);
 constexpr uint32_t NCOL_ACC = 0, NCOL_W = 128, NCOL_S = 256;
 constexpr int NW_SBUF = 2;                   // S tiles in tensor memory
 
@@ -61,9 +56,6 @@ struct NarrowParams {
     float* pos_logit;
     const float* row_ref;     // DA: per-query anchor of the weights, log2 domain
     int* range_flag;          // DA: set to 1 when a row sum leaves the range the anchor allows
-    const float* slot_m;      // DP with nslots > 0: forward slots [nslots][ny] to merge instead of
-    const float* slot_l;      //   reading row_lse
-    int nslots;
     int* dev_status;
     Gate gate;                // closed: the kernel returns at once
     int* zero_me;             // DA: the ticket word of the reduction that follows
@@ -82,7 +74,7 @@ struct NBars {
 };
 
 template <int MODE>
-__global__ void __launch_bounds__((nw_threads<MODE>()), 1)
+__global__ void __launch_bounds__(NW_THREADS, 1)
 narrow_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapY,
               const __grid_constant__ CUtensorMap mapO, const NarrowParams p) {
     // All shared memory is dynamic: X and the ring (1024-byte aligned for the
@@ -126,7 +118,7 @@ narrow_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ 
         for (int s = 0; s < NW_STAGES; ++s) {
             mbar_init(smem_u32(&bars.y_full[s]), 1);
             mbar_init(smem_u32(&bars.y_empty[s]), 1);
-            mbar_init(smem_u32(&bars.c_full[s]), NW_COLW);
+            mbar_init(smem_u32(&bars.c_full[s]), 1);
         }
         for (int b = 0; b < NW_SBUF; ++b) {
             mbar_init(smem_u32(&bars.s_full[b]), 1);
@@ -169,6 +161,30 @@ narrow_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ 
                 for (int c = 0; c < p.kc; ++c)
                     tma_load_2d(y_smem + stage * stage_bytes + c * CHUNK_BYTES, &mapY, c * 64,
                                 (int)y0, full);
+            }
+            if (MODE == NMODE_DP) {   // the column constants of the tile: four per lane
+                float nl[4];
+                int rel[4];
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int64_t y = y0 + lane + 32 * k;
+                    float lse_y = INFINITY;
+                    int32_t pos_y = -1;
+                    if (y < p.ny) {
+                        lse_y = p.row_lse[y];
+                        pos_y = p.pos_idx[y];
+                    }
+                    nl[k] = -lse_y * 1.4426950408889634f;
+                    const int64_t r = (int64_t)pos_y - x0;
+                    rel[k] = (pos_y >= 0 && r >= 0 && r < XROWS) ? (int)r : -1;
+                }
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    col_nlse[stage][lane + 32 * k] = nl[k];
+                    col_rel[stage][lane + 32 * k] = (int8_t)rel[k];
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars.c_full[stage]));
             }
             if (++stage == NW_STAGES) { stage = 0; phase ^= 1u; }
         }
@@ -234,31 +250,6 @@ narrow_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ 
             }
         }
         if (ok && elect_one()) tc_commit(smem_u32(&bars.acc_full));
-    } else if (MODE == NMODE_DP && warp >= 2 + NW_SOFT) {
-        // ------------------------------ column constants (DP) -----------------------------------
-        // the streamed rows are queries: their logsumexp (merged from the forward slots where
-        // the call has not combined them yet) and positives, one column per thread and tile
-        const int i = (warp - (2 + NW_SOFT)) * 32 + lane;
-        int stage = 0;
-        uint32_t phase = 0;
-        for (int t = 0; t < T; ++t) {
-            // the softmax warps have read the constants of the tile that used this stage
-            if (!mbar_wait(smem_u32(&bars.y_empty[stage]), phase ^ 1u, abort_flag)) break;
-            const int64_t y = (lo + t) * 128 + i;
-            float lse_y = INFINITY;
-            int32_t pos_y = -1;
-            if (y < p.ny) {
-                lse_y = p.nslots > 0 ? combined_lse(p.slot_m, p.slot_l, p.nslots, p.ny, y)
-                                     : p.row_lse[y];
-                pos_y = p.pos_idx[y];
-            }
-            col_nlse[stage][i] = -lse_y * 1.4426950408889634f;
-            const int64_t rel = (int64_t)pos_y - x0;
-            col_rel[stage][i] = (pos_y >= 0 && rel >= 0 && rel < XROWS) ? (int8_t)rel : (int8_t)-1;
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars.c_full[stage]));
-            if (++stage == NW_STAGES) { stage = 0; phase ^= 1u; }
-        }
     } else {
         // ------------------------------ softmax / epilogue warps --------------------------------
         const int sw = warp - 2;                       // 0..15
@@ -491,7 +482,7 @@ cudaError_t launch_narrow(const CUtensorMap& mx, const CUtensorMap& my, const CU
     const int64_t ctas = ((p.nx + XROWS - 1) / XROWS) * p.groups;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)ctas);
-    cfg.blockDim = dim3(nw_threads<MODE>());
+    cfg.blockDim = dim3(NW_THREADS);
     cfg.dynamicSmemBytes = dynamic_bytes;
     cfg.stream = st;
     cudaLaunchAttribute attr[1];
@@ -554,7 +545,6 @@ cudaError_t narrow_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     p.row_lse = a.row_lse; p.pos_idx = a.pos_idx;
     p.dev_status = a.dev_status;
     p.gate = a.gate;
-    if (a.mode == SWEEP_DP && a.slot_l) { p.slot_m = a.slot_m; p.slot_l = a.slot_l; p.nslots = a.slots; }
     if (a.mode == SWEEP_DQ) return launch_narrow<NMODE_DQ>(mx, my, mo, p, st, false);
     return launch_narrow<NMODE_DP>(mx, my, mo, p, st, false);
 }

@@ -1270,7 +1270,9 @@ cudaError_t tc_launch_anchored_dq(const FwdArgs& a, float* partial, int groups,
 
 cudaError_t tc_launch_sweep(const SweepArgs& a, cudaStream_t st) {
     if (quad_applicable(a.nx, a.d)) return quad_launch_sweep(a, st);
-    if (narrow_applicable(a.d, GC_BF16)) return narrow_launch_sweep(a, st);
+    // (a dP sweep that merges forward slots itself stays on the kernels below)
+    if (narrow_applicable(a.d, GC_BF16) && !(a.mode == SWEEP_DP && a.slot_l))
+        return narrow_launch_sweep(a, st);
     const int kc = a.d / 64;
     constexpr int SN = 128;
     CUtensorMap mx, my, myh;
