@@ -44,9 +44,9 @@ SWEEP_SOURCES = ['gc_api.cu', 'gc_combine.cu', 'gc_internal.h', 'gc_quad.cu', 'g
 ONE_TILE_SOURCES = ['gc_api.cu', 'gc_internal.h', 'gc_small.cu', 'tc_common.cuh']
 NARROW_SOURCES = SWEEP_SOURCES + ['gc_narrow.cu']
 NCU_STEP_TRAFFIC = {
-    "cfg2_": (82.9e6, SWEEP_SOURCES, "b8d876d88310b6e351a5579d0ac6ebc2fc8b8b7e"),
-    "cfg4_": (4.80e9, SWEEP_SOURCES, "b8d876d88310b6e351a5579d0ac6ebc2fc8b8b7e"),
-    "cfg3_": (26.4e6, NARROW_SOURCES, "25639b36dbf2b6732256b1340a264160eddf8760"),
+    "cfg2_": (82.9e6, SWEEP_SOURCES, "984da4d026488e42db1a380f3e3a5b542047d09f"),
+    "cfg4_": (4.80e9, SWEEP_SOURCES, "984da4d026488e42db1a380f3e3a5b542047d09f"),
+    "cfg3_": (26.4e6, NARROW_SOURCES, "f2a7221c737232af76998eac5dcd430faf9adb86"),
     "cfg1_": (0.629e6, ONE_TILE_SOURCES, "42794198880e3035735ceb1c20a53113fbce4c0e"),
     "cfg0_": (0.640e6, ONE_TILE_SOURCES, "42794198880e3035735ceb1c20a53113fbce4c0e"),
 }
