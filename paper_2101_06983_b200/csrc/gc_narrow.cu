@@ -298,14 +298,22 @@ narrow_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ 
                 const int rel_row = col_rel[stage][c0 + (lane & (NE - 1))];
                 const bool mine = lane < NE && rel_row >= q * 32 && rel_row < q * 32 + 32;
                 unsigned hits = __ballot_sync(0xffffffffu, mine);
-                while (hits) {
-                    const int col = __ffs(hits) - 1;
-                    hits &= hits - 1;
-                    const int target = __shfl_sync(0xffffffffu, rel_row, col) - q * 32;
-                    if (lane == target) {
+                if (__popc(hits) > 3) {
+                    // many positives in this block (the tile where streamed queries meet their
+                    // own positives): every column in turn, three instructions each
 #pragma unroll
-                        for (int c = 0; c < NE; ++c)
-                            if (c == col) w[c] -= 1.f;
+                    for (int c = 0; c < NE; ++c)
+                        if (__shfl_sync(0xffffffffu, rel_row, c) == row) w[c] -= 1.f;
+                } else {
+                    while (hits) {
+                        const int col = __ffs(hits) - 1;
+                        hits &= hits - 1;
+                        const int target = __shfl_sync(0xffffffffu, rel_row, col) - q * 32;
+                        if (lane == target) {
+#pragma unroll
+                            for (int c = 0; c < NE; ++c)
+                                if (c == col) w[c] -= 1.f;
+                        }
                     }
                 }
             } else {
