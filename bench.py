@@ -46,7 +46,7 @@ NARROW_SOURCES = SWEEP_SOURCES + ['gc_narrow.cu']
 NCU_STEP_TRAFFIC = {
     "cfg2_": (82.9e6, SWEEP_SOURCES, "984da4d026488e42db1a380f3e3a5b542047d09f"),
     "cfg4_": (4.80e9, SWEEP_SOURCES, "984da4d026488e42db1a380f3e3a5b542047d09f"),
-    "cfg3_": (26.4e6, NARROW_SOURCES, "f2a7221c737232af76998eac5dcd430faf9adb86"),
+    "cfg3_": (26.4e6, NARROW_SOURCES, "44a0d1324795e9d77b5ed87232933502e92ce031"),
     "cfg1_": (0.629e6, ONE_TILE_SOURCES, "42794198880e3035735ceb1c20a53113fbce4c0e"),
     "cfg0_": (0.640e6, ONE_TILE_SOURCES, "42794198880e3035735ceb1c20a53113fbce4c0e"),
 }
